@@ -1,0 +1,141 @@
+/*
+ * bfq — butterfly rotation + low-bit quantization for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The library computes, on one GPU, the data-parallel hot path of ButterflyQuant:
+ *
+ *   Q = B_L ... B_2 B_1,  L = log2 n,  B_i = n/2 Givens rotations G(theta_{i,j}) on index
+ *   pairs at stride 2^{i-1}  (paper Sec. 3.2.1 "Structure and Parameterization"; the
+ *   appendix example for n = 8 prints B_1, B_2, B_3 entry by entry).
+ *
+ * Conventions used by every entry point
+ *   stage s = i - 1 = 0..L-1, stride h = 2^s; theta is stage-major [L][n/2] fp32;
+ *   pair j of stage s (pairs listed by increasing low index) couples
+ *       lo = ((j >> s) << (s+1)) | (j & (h-1)),   hi = lo + h
+ *   and maps (a, b) = (z[lo], z[hi]) to (cos*a - sin*b, sin*a + cos*b).
+ *   y = Q x applies stage 0 (stride 1) first.  There is no input or output permutation.
+ *
+ * Memory: every data pointer below is a DEVICE pointer owned by the caller, 16-byte
+ * aligned; rows are contiguous, row-major, with a leading dimension in elements
+ * (ld >= n, ld * sizeof(element) a multiple of 16).  `stream` is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  Calls validate their arguments on the host,
+ * enqueue work on `stream` and return without synchronising (bfq_plan_create,
+ * bfq_plan_destroy and bfq_device_status synchronise).  No compute call allocates memory.
+ * The plan owns the twiddle tables, the per-CTA d-theta partial sums and a device status
+ * word.  A plan may be used from one host thread at a time; calls on one plan must be
+ * issued to streams that serialise them (they share the plan's workspace).
+ *
+ * Errors: every function returns a bfq_status (0 = OK, negative = error); nothing throws.
+ * rows == 0 is a successful no-op.
+ */
+#ifndef BFQ_H_
+#define BFQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bfq_plan bfq_plan; /* opaque */
+
+typedef enum { BFQ_F32 = 0, BFQ_BF16 = 1 } bfq_dtype;
+
+typedef enum {
+    BFQ_OK = 0,
+    BFQ_ERR_NULL = -1,           /* a required pointer is NULL */
+    BFQ_ERR_UNSUPPORTED_N = -2,  /* n is not a power of two in [BFQ_MIN_N, BFQ_MAX_N] */
+    BFQ_ERR_BITS = -3,           /* bits not in {2, 4, 8} */
+    BFQ_ERR_ALIGN = -4,          /* a pointer is not 16-byte aligned */
+    BFQ_ERR_STRIDE = -5,         /* ld < n, or ld * element size not a multiple of 16, or rows < 0 */
+    BFQ_ERR_DTYPE = -6,          /* dtype not BFQ_F32 / BFQ_BF16 */
+    BFQ_ERR_WORKSPACE = -7,      /* angles not set yet, or plan workspace too small */
+    BFQ_ERR_CUDA = -8,           /* a CUDA runtime call failed; see bfq_last_cuda_error */
+    BFQ_ERR_DEVICE_TIMEOUT = -9  /* a bounded device-side wait gave up (reported by bfq_device_status) */
+} bfq_status;
+
+#define BFQ_MIN_N 16
+#define BFQ_MAX_N 8192
+
+/*
+ * Create a plan for row length n on CUDA device `device` (allocates: twiddle tables,
+ * d-theta partial sums, a status word).  max_rows is a sizing hint (>= 0, may be 0); no call
+ * is limited by it.  Paper: theta is the only learnable state, n log2 n / 2 angles
+ * (Sec. 3.2.1, "Parameters").
+ */
+int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device);
+int bfq_plan_destroy(bfq_plan* plan);
+
+/*
+ * Load the angles: builds the per-stage twiddle tables (cos theta, sin theta) in fp32 on the
+ * device (paper "Inference Efficiency": pre-computed twiddle factors in a lookup table of
+ * n log2 n / 2 entries).  theta: device, fp32, [log2 n][n/2], stage 0 = stride 1.
+ * Enqueued on `stream`; later calls on the same stream see the new tables.
+ */
+int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream);
+
+/*
+ * y = Q x for every row (Sec. 3.2.1: B = prod B_i; stage order as stated at the top).
+ * x: [rows][ldx] of xt; y: [rows][ldy] of yt; fp32 arithmetic.  x and y may be the same buffer
+ * only if xt == yt and ldx == ldy.
+ */
+int bfq_forward(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx,
+                void* y, bfq_dtype yt, int64_t ldy, void* stream);
+
+/*
+ * y = Q x fused with the per-row (per-token) symmetric quantizer of Sec. 3.4:
+ *     qmax = 2^(bits-1) - 1;  s = max_k |y_k| / qmax, stored as IEEE fp16 (round to nearest
+ *     even, saturating at 65504);  code_k = clip(round(y_k / s), -2^(bits-1), qmax),
+ *     round-half-to-even, using the fp16-rounded s.  A row whose fp16 scale is 0 gets codes 0.
+ * codes: [rows][n*bits/8] bytes, two's complement; element k sits in bits
+ *     [bits*(k mod 8/bits), +bits) of byte k*bits/8 (INT4: even element = low nibble).
+ * scales_f16: [rows] fp16 bit patterns.  Dequant(q) = s * q.
+ */
+int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx,
+                      int bits, uint8_t* codes, uint16_t* scales_f16, void* stream);
+
+/*
+ * x = Q^T y (= Q^{-1} y: Q is orthogonal by construction, Sec. 3.2.1): stages L-1..0, each
+ * pair mapped by G(theta)^T.  Also dL/dx = Q^T g.
+ */
+int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64_t ldy,
+                void* x, bfq_dtype xt, int64_t ldx, void* stream);
+
+/*
+ * Backward of y = Q x for an upstream gradient g = dL/dy (Sec. 3.5.1, dG/dtheta):
+ *     dx = Q^T g  per row;   dtheta[s][j] = sum over rows of  gbar^T (dG/dtheta) z  on pair j of
+ *     stage s, z the stage input and gbar the gradient at the stage output.
+ * x, g: [rows][ld]; dx: [rows][ld] of dxt (may be NULL to skip); dtheta: device fp32
+ * [log2 n][n/2], overwritten.  The sum over rows has a fixed order (per-CTA partial sums over a
+ * static row assignment, then CTAs in index order): results are bit-identical run to run on the
+ * same device.  The quantizer is not differentiated here; g is the caller's.
+ */
+int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq_dtype gt,
+                 int64_t rows, int64_t ld, void* dx, bfq_dtype dxt, float* dtheta, void* stream);
+
+/*
+ * Weight folding W' = W Q^T (Sec. 3.1, computational invariance y = W x = (W Q^T)(Q x)):
+ * row i of W Q^T is (Q w_i)^T, so Q is applied to each of the m rows of W, followed by
+ * per-row (per-output-channel) quantization exactly as in bfq_forward_quant.
+ * WQt (optional, may be NULL): the unquantized rotated rows, [m][n] of type ot, ld = n.
+ */
+int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int64_t ldw,
+                     int bits, uint8_t* codes, uint16_t* scales_f16, void* WQt, bfq_dtype ot,
+                     void* stream);
+
+/* Synchronises the device and returns BFQ_OK, or BFQ_ERR_DEVICE_TIMEOUT if a kernel of this plan
+ * reported a bounded wait that ran out, or BFQ_ERR_CUDA.  (No counterpart in the paper.) */
+int bfq_device_status(bfq_plan* plan);
+
+/* Last cudaError_t seen by this plan (0 = cudaSuccess).  (No counterpart in the paper.) */
+int bfq_last_cuda_error(const bfq_plan* plan);
+
+/* Static string for a status code. */
+const char* bfq_status_string(int status);
+
+/* Number of CTAs the backward pass uses (= number of d-theta partial sums); informational. */
+int bfq_backward_partials(const bfq_plan* plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BFQ_H_ */

@@ -1,0 +1,174 @@
+"""ctypes binding of libbfq.so: the same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the CUDA kernels behind these calls.  There is no CPU
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbfq.so")
+
+BFQ_F32, BFQ_BF16 = 0, 1
+BFQ_OK = 0
+STATUS_NAMES = {
+    0: "BFQ_OK", -1: "BFQ_ERR_NULL", -2: "BFQ_ERR_UNSUPPORTED_N", -3: "BFQ_ERR_BITS", -4: "BFQ_ERR_ALIGN",
+    -5: "BFQ_ERR_STRIDE", -6: "BFQ_ERR_DTYPE", -7: "BFQ_ERR_WORKSPACE", -8: "BFQ_ERR_CUDA",
+    -9: "BFQ_ERR_DEVICE_TIMEOUT",
+}
+
+# name -> (restype, argtypes); must list every symbol include/bfq.h declares
+_i, _i64, _p = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p
+SIGNATURES = {
+    "bfq_plan_create": (_i, [ctypes.POINTER(_p), _i, _i64, _i]),
+    "bfq_plan_destroy": (_i, [_p]),
+    "bfq_set_angles": (_i, [_p, _p, _p]),
+    "bfq_forward": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
+    "bfq_forward_quant": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p]),
+    "bfq_inverse": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
+    "bfq_backward": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _p, _i, _p, _p]),
+    "bfq_fold_weights": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p, _i, _p]),
+    "bfq_device_status": (_i, [_p]),
+    "bfq_last_cuda_error": (_i, [_p]),
+    "bfq_status_string": (ctypes.c_char_p, [_i]),
+    "bfq_backward_partials": (_i, [_p]),
+}
+
+_lib = None
+
+
+class BfqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().bfq_status_string(status).decode()
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({msg})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libbfq.so (raises if it has not been built: there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: run `python -m paper_2509_09679_b200.build` "
+                               "(the CUDA library is the only implementation)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != BFQ_OK:
+        raise BfqError(status, where)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return BFQ_F32
+    if t.dtype == torch.bfloat16:
+        return BFQ_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _rows(t: torch.Tensor, n: int):
+    if t.dim() != 2 or t.shape[1] != n or t.stride(1) != 1:
+        raise ValueError(f"expected a [rows][{n}] tensor with unit inner stride, got {tuple(t.shape)}")
+    return t.shape[0], (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), n))
+
+
+def _stream(t: torch.Tensor):
+    return ctypes.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+class Plan:
+    """Owns a bfq_plan for row length n on one CUDA device."""
+
+    def __init__(self, n: int, device=None, max_rows: int = 0):
+        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        if dev.type != "cuda":
+            raise ValueError("bfq runs on CUDA devices only")
+        self.n = int(n)
+        self.L = self.n.bit_length() - 1
+        self.device = torch.device("cuda", dev.index if dev.index is not None else torch.cuda.current_device())
+        self._h = ctypes.c_void_p()
+        _check(lib().bfq_plan_create(ctypes.byref(self._h), self.n, int(max_rows), self.device.index),
+               "bfq_plan_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().bfq_plan_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the C ABI, one method per entry point ------------------------------------------------------
+    def set_angles(self, theta: torch.Tensor):
+        if theta.dtype != torch.float32 or tuple(theta.shape) != (self.L, self.n // 2) or not theta.is_contiguous():
+            raise ValueError(f"theta must be a contiguous fp32 [{self.L}][{self.n // 2}] tensor")
+        _check(lib().bfq_set_angles(self._h, theta.data_ptr(), _stream(theta)), "bfq_set_angles")
+
+    def forward(self, x: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
+        rows, ldx = _rows(x, self.n)
+        y = out if out is not None else torch.empty((rows, self.n), dtype=out_dtype or x.dtype, device=x.device)
+        _, ldy = _rows(y, self.n)
+        _check(lib().bfq_forward(self._h, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(), _dt(y), ldy, _stream(x)),
+               "bfq_forward")
+        return y
+
+    def forward_quant(self, x: torch.Tensor, bits: int, codes=None, scales=None):
+        rows, ldx = _rows(x, self.n)
+        if codes is None:
+            codes = torch.empty((rows, self.n * bits // 8), dtype=torch.uint8, device=x.device)
+        if scales is None:
+            scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        _check(lib().bfq_forward_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
+                                       scales.data_ptr(), _stream(x)), "bfq_forward_quant")
+        return codes, scales
+
+    def inverse(self, y: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
+        rows, ldy = _rows(y, self.n)
+        x = out if out is not None else torch.empty((rows, self.n), dtype=out_dtype or y.dtype, device=y.device)
+        _, ldx = _rows(x, self.n)
+        _check(lib().bfq_inverse(self._h, y.data_ptr(), _dt(y), rows, ldy, x.data_ptr(), _dt(x), ldx, _stream(y)),
+               "bfq_inverse")
+        return x
+
+    def backward(self, x: torch.Tensor, g: torch.Tensor, dx_dtype=None, want_dx: bool = True, dx=None, dtheta=None):
+        rows, ld = _rows(x, self.n)
+        rows_g, ld_g = _rows(g, self.n)
+        if rows_g != rows or ld_g != ld:
+            raise ValueError("x and g must have the same shape and row stride")
+        if want_dx and dx is None:
+            dx = torch.empty_strided((rows, self.n), (ld, 1), dtype=dx_dtype or x.dtype, device=x.device)
+        if dtheta is None:
+            dtheta = torch.empty((self.L, self.n // 2), dtype=torch.float32, device=x.device)
+        _check(lib().bfq_backward(self._h, x.data_ptr(), _dt(x), g.data_ptr(), _dt(g), rows, ld,
+                                  dx.data_ptr() if want_dx else None, _dt(dx) if want_dx else BFQ_F32,
+                                  dtheta.data_ptr(), _stream(x)), "bfq_backward")
+        return (dx if want_dx else None), dtheta
+
+    def fold_weights(self, W: torch.Tensor, bits: int, want_rotated: bool = False, rotated_dtype=None):
+        m, ldw = _rows(W, self.n)
+        codes = torch.empty((m, self.n * bits // 8), dtype=torch.uint8, device=W.device)
+        scales = torch.empty((m,), dtype=torch.float16, device=W.device)
+        rot = torch.empty((m, self.n), dtype=rotated_dtype or W.dtype, device=W.device) if want_rotated else None
+        _check(lib().bfq_fold_weights(self._h, W.data_ptr(), _dt(W), m, ldw, int(bits), codes.data_ptr(),
+                                      scales.data_ptr(), rot.data_ptr() if rot is not None else None,
+                                      _dt(rot) if rot is not None else BFQ_F32, _stream(W)), "bfq_fold_weights")
+        return codes, scales, rot
+
+    def device_status(self) -> int:
+        return int(lib().bfq_device_status(self._h))
+
+    def backward_partials(self) -> int:
+        return int(lib().bfq_backward_partials(self._h))

@@ -1,0 +1,355 @@
+// C ABI of the bfq library: plan management, argument validation, kernel dispatch.
+// See include/bfq.h for the contract of every entry point.
+#include "../../include/bfq.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <new>
+
+#include "bfq_generic.cuh"
+#include "bfq_plan.h"
+
+namespace bfq {
+
+static bool env_flag(const char* name) {
+    const char* v = std::getenv(name);
+    return v != nullptr && v[0] != '\0' && v[0] != '0';
+}
+
+static int ilog2_exact(int64_t n) {
+    int L = 0;
+    while ((int64_t(1) << L) < n) ++L;
+    return (int64_t(1) << L) == n ? L : -1;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int device) {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != device) {
+            err = cudaSetDevice(device);
+            switched = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+static int cuda_fail(bfq_plan* plan, cudaError_t e) {
+    if (plan != nullptr) plan->last_cuda_error = static_cast<int>(e);
+    if (env_flag("BFQ_LOG")) std::fprintf(stderr, "[bfq] CUDA error %d: %s\n", int(e), cudaGetErrorString(e));
+    return BFQ_ERR_CUDA;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static int esize(int dt) { return dt == BFQ_F32 ? 4 : 2; }
+static bool dtype_ok(int dt) { return dt == BFQ_F32 || dt == BFQ_BF16; }
+
+static int check_rows(const void* p, int dt, int64_t rows, int64_t ld, int n) {
+    if (p == nullptr && rows != 0) return BFQ_ERR_NULL;  // an empty batch may come with a null pointer
+    if (!dtype_ok(dt)) return BFQ_ERR_DTYPE;
+    if (rows < 0 || ld < n || ((ld * esize(dt)) & 15) != 0) return BFQ_ERR_STRIDE;
+    if (!aligned16(p)) return BFQ_ERR_ALIGN;
+    return BFQ_OK;
+}
+
+// ---- generic kernel dispatch ------------------------------------------------------------------------
+template <int LOG_N, int R, int MODE>
+static cudaError_t launch_generic_t(const bfq_plan* plan, const GenericParams& p, cudaStream_t st) {
+    using G = Geo<LOG_N>;
+    constexpr size_t smem = sizeof(float) * (size_t(G::kGroups) * R * G::kN + size_t(R) * G::kGroups * G::kWarpsPerRow);
+    static int blocks_per_sm[kMaxDevices] = {0};
+    auto kern = k_generic<LOG_N, R, MODE>;
+    int& occ = blocks_per_sm[plan->device];
+    if (occ == 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, G::kThreads, smem);
+        if (e != cudaSuccess) return e;
+        occ = o > 0 ? o : 1;
+    }
+    constexpr int rows_per_tile = G::kGroups * R;
+    const int64_t tiles = (p.rows + rows_per_tile - 1) / rows_per_tile;
+    const int64_t cap = int64_t(plan->sm_count) * occ;
+    const int grid = int(tiles < cap ? tiles : cap);
+    kern<<<grid, G::kThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <int MODE>
+static cudaError_t launch_generic(const bfq_plan* plan, const GenericParams& p, cudaStream_t st) {
+    switch (plan->log_n) {
+        case 4: return launch_generic_t<4, 2, MODE>(plan, p, st);
+        case 5: return launch_generic_t<5, 2, MODE>(plan, p, st);
+        case 6: return launch_generic_t<6, 2, MODE>(plan, p, st);
+        case 7: return launch_generic_t<7, 2, MODE>(plan, p, st);
+        case 8: return launch_generic_t<8, 2, MODE>(plan, p, st);
+        case 9: return launch_generic_t<9, 2, MODE>(plan, p, st);
+        case 10: return launch_generic_t<10, 2, MODE>(plan, p, st);
+        case 11: return launch_generic_t<11, 2, MODE>(plan, p, st);
+        case 12: return launch_generic_t<12, 2, MODE>(plan, p, st);
+        case 13: return launch_generic_t<13, 2, MODE>(plan, p, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+template <int LOG_N, int R>
+static cudaError_t launch_backward_t(bfq_plan* plan, BackwardParams p, float* dtheta, cudaStream_t st) {
+    using G = Geo<LOG_N>;
+    constexpr size_t smem = sizeof(float) * size_t(G::kGroups) * R * G::kN;
+    static int blocks_per_sm[kMaxDevices] = {0};
+    auto kern = k_backward_generic<LOG_N, R>;
+    int& occ = blocks_per_sm[plan->device];
+    if (occ == 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+        int o = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, G::kThreads, smem);
+        if (e != cudaSuccess) return e;
+        occ = o > 0 ? o : 1;
+    }
+    constexpr int rows_per_tile = G::kGroups * R;
+    const int64_t tiles = (p.rows + rows_per_tile - 1) / rows_per_tile;
+    int64_t cap = int64_t(plan->sm_count) * (occ < kBackwardCtasPerSm ? occ : kBackwardCtasPerSm);
+    if (cap * G::kGroups > plan->partial_slots) cap = plan->partial_slots / G::kGroups;
+    if (cap < 1) return cudaErrorInvalidValue;
+    const int grid = int(tiles < cap ? tiles : cap);
+    p.partial = plan->partial;
+    kern<<<grid, G::kThreads, smem, st>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int count = LOG_N * G::kHalf;
+    k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid * G::kGroups, count, dtheta);
+    plan->last_backward_partials = grid * G::kGroups;
+    return cudaGetLastError();
+}
+
+static cudaError_t launch_backward(bfq_plan* plan, const BackwardParams& p, float* dtheta, cudaStream_t st) {
+    switch (plan->log_n) {
+        case 4: return launch_backward_t<4, 1>(plan, p, dtheta, st);
+        case 5: return launch_backward_t<5, 1>(plan, p, dtheta, st);
+        case 6: return launch_backward_t<6, 1>(plan, p, dtheta, st);
+        case 7: return launch_backward_t<7, 1>(plan, p, dtheta, st);
+        case 8: return launch_backward_t<8, 1>(plan, p, dtheta, st);
+        case 9: return launch_backward_t<9, 1>(plan, p, dtheta, st);
+        case 10: return launch_backward_t<10, 1>(plan, p, dtheta, st);
+        case 11: return launch_backward_t<11, 1>(plan, p, dtheta, st);
+        case 12: return launch_backward_t<12, 1>(plan, p, dtheta, st);
+        case 13: return launch_backward_t<13, 1>(plan, p, dtheta, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+// slots needed by the generic backward for this n: CTAs * row groups per CTA
+static int64_t backward_slots(int log_n, int sm_count) {
+    const int n = 1 << log_n;
+    const int tpr = n / 16;
+    const int threads = tpr > 256 ? tpr : 256;
+    return int64_t(sm_count) * kBackwardCtasPerSm * (threads / tpr);
+}
+
+}  // namespace bfq
+
+using namespace bfq;
+
+extern "C" {
+
+int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
+    if (out == nullptr) return BFQ_ERR_NULL;
+    *out = nullptr;
+    if (n < BFQ_MIN_N || n > BFQ_MAX_N || ilog2_exact(n) < 0) return BFQ_ERR_UNSUPPORTED_N;
+    if (max_rows < 0) return BFQ_ERR_STRIDE;
+    if (device < 0 || device >= kMaxDevices) return BFQ_ERR_CUDA;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (device >= count) return BFQ_ERR_CUDA;
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) return cuda_fail(nullptr, guard.err);
+
+    bfq_plan* plan = new (std::nothrow) bfq_plan();
+    if (plan == nullptr) return BFQ_ERR_WORKSPACE;
+    plan->n = n;
+    plan->log_n = ilog2_exact(n);
+    plan->device = device;
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) {
+        delete plan;
+        return cuda_fail(nullptr, e);
+    }
+    plan->sm_count = prop.multiProcessorCount;
+    plan->cc_major = prop.major;
+    const size_t angles = size_t(plan->log_n) * (n / 2);
+    plan->partial_slots = backward_slots(plan->log_n, plan->sm_count);
+    e = cudaMalloc(&plan->tw, angles * sizeof(float2));
+    if (e == cudaSuccess) e = cudaMalloc(&plan->partial, size_t(plan->partial_slots) * angles * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        cudaFree(plan->tw);
+        cudaFree(plan->partial);
+        cudaFree(plan->status_word);
+        delete plan;
+        return cuda_fail(nullptr, e);
+    }
+    *out = plan;
+    return BFQ_OK;
+}
+
+int bfq_plan_destroy(bfq_plan* plan) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    DeviceGuard guard(plan->device);
+    cudaDeviceSynchronize();
+    cudaFree(plan->tw);
+    cudaFree(plan->partial);
+    cudaFree(plan->status_word);
+    delete plan;
+    return BFQ_OK;
+}
+
+int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
+    if (plan == nullptr || theta == nullptr) return BFQ_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(theta) & 3u) != 0) return BFQ_ERR_ALIGN;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    const int count = plan->log_n * (plan->n / 2);
+    k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    plan->angles_set = true;
+    return BFQ_OK;
+}
+
+int bfq_forward(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, void* y, bfq_dtype yt,
+                int64_t ldy, void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    int rc = check_rows(x, xt, rows, ldx, plan->n);
+    if (rc == BFQ_OK) rc = check_rows(y, yt, rows, ldy, plan->n);
+    if (rc != BFQ_OK) return rc;
+    if (!plan->angles_set) return BFQ_ERR_WORKSPACE;
+    if (rows == 0) return BFQ_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    GenericParams p{};
+    p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = ldy, p.rows = rows;
+    cudaError_t e = launch_generic<kModeForward>(plan, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t rows, int64_t ldx, int bits,
+                              uint8_t* codes, uint16_t* scales, void* y, int yt, void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    int rc = check_rows(x, xt, rows, ldx, plan->n);
+    if (rc != BFQ_OK) return rc;
+    if ((codes == nullptr || scales == nullptr) && rows != 0) return BFQ_ERR_NULL;
+    if (bits != 2 && bits != 4 && bits != 8) return BFQ_ERR_BITS;
+    if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 1u) != 0) return BFQ_ERR_ALIGN;
+    if (y != nullptr) {
+        rc = check_rows(y, yt, rows, plan->n, plan->n);
+        if (rc != BFQ_OK) return rc;
+    }
+    if (!plan->angles_set) return BFQ_ERR_WORKSPACE;
+    if (rows == 0) return BFQ_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    GenericParams p{};
+    p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = plan->n;
+    p.codes = codes, p.scales = scales, p.bits = bits, p.rows = rows;
+    cudaError_t e = launch_generic<kModeForwardQuant>(plan, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
+                      uint8_t* codes, uint16_t* scales_f16, void* stream) {
+    return forward_quant_impl(plan, x, xt, rows, ldx, bits, codes, scales_f16, nullptr, BFQ_F32, stream);
+}
+
+int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int64_t ldw, int bits, uint8_t* codes,
+                     uint16_t* scales_f16, void* WQt, bfq_dtype ot, void* stream) {
+    return forward_quant_impl(plan, W, wt, m, ldw, bits, codes, scales_f16, WQt, ot, stream);
+}
+
+int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64_t ldy, void* x, bfq_dtype xt,
+                int64_t ldx, void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    int rc = check_rows(y, yt, rows, ldy, plan->n);
+    if (rc == BFQ_OK) rc = check_rows(x, xt, rows, ldx, plan->n);
+    if (rc != BFQ_OK) return rc;
+    if (!plan->angles_set) return BFQ_ERR_WORKSPACE;
+    if (rows == 0) return BFQ_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    GenericParams p{};
+    p.tw = plan->tw, p.x = y, p.xt = yt, p.ldx = ldy, p.y = x, p.yt = xt, p.ldy = ldx, p.rows = rows;
+    cudaError_t e = launch_generic<kModeInverse>(plan, p, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq_dtype gt, int64_t rows, int64_t ld,
+                 void* dx, bfq_dtype dxt, float* dtheta, void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    int rc = check_rows(x, xt, rows, ld, plan->n);
+    if (rc == BFQ_OK) rc = check_rows(g, gt, rows, ld, plan->n);
+    if (rc == BFQ_OK && dx != nullptr) rc = check_rows(dx, dxt, rows, ld, plan->n);
+    if (rc != BFQ_OK) return rc;
+    if (dtheta == nullptr) return BFQ_ERR_NULL;
+    if (!aligned16(dtheta)) return BFQ_ERR_ALIGN;
+    if (!plan->angles_set) return BFQ_ERR_WORKSPACE;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (rows == 0) {
+        cudaError_t e = cudaMemsetAsync(dtheta, 0, sizeof(float) * size_t(plan->log_n) * (plan->n / 2), st);
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
+    BackwardParams p{};
+    p.tw = plan->tw, p.x = x, p.xt = xt, p.g = g, p.gt = gt, p.ld = ld, p.dx = dx, p.dxt = dxt, p.rows = rows;
+    cudaError_t e = launch_backward(plan, p, dtheta, st);
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+int bfq_device_status(bfq_plan* plan) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    int word = 0;
+    e = cudaMemcpy(&word, plan->status_word, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    if (word != 0) {
+        cudaMemset(plan->status_word, 0, sizeof(int));
+        return BFQ_ERR_DEVICE_TIMEOUT;
+    }
+    return BFQ_OK;
+}
+
+int bfq_last_cuda_error(const bfq_plan* plan) { return plan == nullptr ? 0 : plan->last_cuda_error; }
+
+int bfq_backward_partials(const bfq_plan* plan) { return plan == nullptr ? 0 : plan->last_backward_partials; }
+
+const char* bfq_status_string(int status) {
+    switch (status) {
+        case BFQ_OK: return "ok";
+        case BFQ_ERR_NULL: return "null pointer";
+        case BFQ_ERR_UNSUPPORTED_N: return "unsupported n (power of two in [16, 8192] required)";
+        case BFQ_ERR_BITS: return "bits must be 2, 4 or 8";
+        case BFQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case BFQ_ERR_STRIDE: return "bad rows / leading dimension";
+        case BFQ_ERR_DTYPE: return "dtype must be BFQ_F32 or BFQ_BF16";
+        case BFQ_ERR_WORKSPACE: return "angles not set or workspace too small";
+        case BFQ_ERR_CUDA: return "CUDA runtime error";
+        case BFQ_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,24 @@
+// Internal layout of a plan (opaque to callers of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bfq {
+constexpr int kMaxDevices = 64;
+constexpr int kBackwardCtasPerSm = 2;  // upper bound on resident backward CTAs per SM (sizes the partial sums)
+}  // namespace bfq
+
+struct bfq_plan {
+    int n = 0;
+    int log_n = 0;
+    int device = 0;
+    int sm_count = 0;
+    int cc_major = 0;
+    bool angles_set = false;
+    float2* tw = nullptr;        // [log_n][n/2] (cos, sin), fp32
+    float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
+    int64_t partial_slots = 0;
+    int* status_word = nullptr;  // device: non-zero when a bounded wait gave up
+    int last_cuda_error = 0;
+    int last_backward_partials = 0;
+};

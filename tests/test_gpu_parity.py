@@ -1,0 +1,219 @@
+"""GPU parity: every entry point of the C ABI against the CPU oracle, element by element,
+on seeded inputs.  Sizes span several tiles and ragged tails; the rules are in parity.py."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_09679_b200 import BfqError, Plan, synth
+from parity import Guarded, check_dtheta, check_quant, check_rows_close, to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def make(n, rows, dtype, dist="student_t3", angle_kind="normal", seed=1, outliers=4, oscale=20.0):
+    theta = synth.angles(n, angle_kind, seed)
+    x = synth.rows(rows, n, dist, seed + 1, outliers=min(outliers, n // 4), outlier_scale=oscale, dtype=dtype)
+    return theta, x
+
+
+def plan_for(n, theta):
+    p = Plan(n, DEV)
+    p.set_angles(theta.to(DEV))
+    return p
+
+
+def absmax_rows(x):
+    return np.abs(to_f64(x)).max(axis=1) if x.shape[0] else np.zeros(0)
+
+
+# ---- the tiny correctness configuration: n = 256, 1024 fp32 rows, angles U[-pi, pi) ------------------
+def test_tiny256_all_entry_points():
+    wl = synth.WORKLOADS["tiny256"]
+    theta, x, g = wl.theta(), wl.x(), wl.g()
+    th64, x64, g64 = to_f64(theta), to_f64(x), to_f64(g)
+    p = plan_for(wl.n, theta)
+    xd, gd = x.to(DEV), g.to(DEV)
+    y_ref = oracle.forward(th64, x64)
+    y = p.forward(xd)
+    check_rows_close(y, y_ref, absmax_rows(x), "forward")
+    xr = p.inverse(y)
+    check_rows_close(xr, oracle.inverse(th64, to_f64(y)), absmax_rows(y), "inverse")
+    check_rows_close(xr, x64, np.sqrt(wl.n) * absmax_rows(x), "round trip")
+    codes, scales = p.forward_quant(xd, 4)
+    stats = check_quant(codes, scales, y_ref, 4, "forward_quant")
+    assert stats["scale_ulp_rows"] <= 16
+    dx, dth = p.backward(xd, gd)
+    dx_ref, dth_ref = oracle.backward(th64, x64, g64)
+    check_rows_close(dx, dx_ref, absmax_rows(g), "dx")
+    check_dtheta(dth, dth_ref, "dtheta")
+    assert p.device_status() == 0
+
+
+# ---- every supported n, both dtypes, ragged row counts, padded leading dimension ----------------------
+@pytest.mark.parametrize("n", [16, 32, 64, 128, 256, 512, 1024, 2048, 4096, 8192])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_forward_inverse_every_n(n, dtype):
+    rows = 67 if n >= 2048 else 333
+    theta, x = make(n, rows, dtype, angle_kind="uniform", seed=n)
+    th64 = to_f64(theta)
+    p = plan_for(n, theta)
+    ld = n + 24
+    xpad = torch.zeros((rows, ld), dtype=dtype, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    xv = xpad[:, :n]
+    y_ref = oracle.forward(th64, to_f64(x))
+    for out_dtype in (torch.float32, torch.bfloat16):
+        out = Guarded((rows, n), out_dtype, DEV)
+        p.forward(xv, out=out.view)
+        check_rows_close(out.view, y_ref, absmax_rows(x), f"forward n={n} {dtype}->{out_dtype}")
+        assert out.intact()
+    xi_ref = oracle.inverse(th64, to_f64(x))
+    out = Guarded((rows, n), torch.float32, DEV)
+    p.inverse(xv, out=out.view)
+    check_rows_close(out.view, xi_ref, absmax_rows(x), f"inverse n={n}")
+    assert out.intact()
+    assert p.device_status() == 0
+
+
+@pytest.mark.parametrize("n,rows", [(16, 5), (64, 1), (128, 1000), (256, 129), (1024, 77), (4096, 130), (8192, 35)])
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_forward_quant_every_width(n, rows, bits):
+    theta, x = make(n, rows, torch.bfloat16, seed=7 * n + bits)
+    p = plan_for(n, theta)
+    y_ref = oracle.forward(to_f64(theta), to_f64(x))
+    codes = Guarded((rows, n * bits // 8), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.forward_quant(x.to(DEV), bits, codes=codes.view, scales=scales.view)
+    check_quant(codes.view, scales.view, y_ref, bits, f"n={n} bits={bits}")
+    assert codes.intact() and scales.intact()
+
+
+@pytest.mark.parametrize("n,rows", [(16, 9), (128, 300), (512, 70), (2048, 45), (4096, 40), (8192, 20)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_backward_every_n(n, rows, dtype):
+    theta, x = make(n, rows, dtype, angle_kind="uniform", seed=3 * n)
+    g = synth.rows(rows, n, "normal", 99 + n, dtype=dtype)
+    p = plan_for(n, theta)
+    dx_ref, dth_ref = oracle.backward(to_f64(theta), to_f64(x), to_f64(g))
+    dx = Guarded((rows, n), dtype, DEV)
+    dth = Guarded((p.L, n // 2), torch.float32, DEV)
+    p.backward(x.to(DEV), g.to(DEV), dx=dx.view, dtheta=dth.view)
+    check_rows_close(dx.view, dx_ref, absmax_rows(g), f"dx n={n}")
+    check_dtheta(dth.view, dth_ref, f"dtheta n={n}")
+    assert dx.intact() and dth.intact()
+    # dtheta only
+    _, dth2 = p.backward(x.to(DEV), g.to(DEV), want_dx=False)
+    assert torch.equal(dth2, dth.view)
+
+
+def test_backward_is_bit_reproducible():
+    n, rows = 4096, 3000
+    theta, x = make(n, rows, torch.bfloat16, seed=5)
+    g = synth.rows(rows, n, "normal", 6, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    xd, gd = x.to(DEV), g.to(DEV)
+    dx1, d1 = p.backward(xd, gd)
+    dx2, d2 = p.backward(xd, gd)
+    assert torch.equal(d1, d2) and torch.equal(dx1.view(torch.int16), dx2.view(torch.int16))
+    assert p.backward_partials() > 0
+
+
+# ---- special angle sets ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("n", [256, 4096])
+def test_identity_and_hadamard_angles(n):
+    x = synth.rows(50, n, "normal", 3, dtype=torch.float32)
+    p = plan_for(n, synth.angles(n, "zero", 0))
+    assert torch.equal(p.forward(x.to(DEV)).cpu(), x)  # theta = 0: exact identity
+    p.set_angles(synth.angles(n, "hadamard", 0).to(DEV))
+    eye = torch.zeros((64, n), dtype=torch.float32)
+    eye[torch.arange(64), torch.arange(64) * (n // 64)] = 1.0
+    y = p.forward(eye.to(DEV)).cpu()
+    assert torch.allclose(y.abs(), torch.full_like(y, 1 / math.sqrt(n)), rtol=0, atol=1e-6)  # coherence 1/sqrt(n)
+    np.testing.assert_allclose(np.linalg.norm(to_f64(p.forward(x.to(DEV))), axis=1),
+                               np.linalg.norm(to_f64(x), axis=1), rtol=1e-5)
+
+
+# ---- degenerate rows ---------------------------------------------------------------------------------------
+def test_zero_rows_tiny_rows_and_saturating_rows():
+    n = 512
+    theta, x = make(n, 8, torch.float32, seed=11)
+    x[0] = 0.0
+    x[1] = x[1] * 1e-12   # scale underflows fp16: codes must be all zero
+    x[2] = x[2] * 1e5     # amax/qmax above 65504 for INT2: scale saturates, codes clip
+    x[3] = x[3] * 1e-6    # subnormal fp16 scale
+    p = plan_for(n, theta)
+    y_ref = oracle.forward(to_f64(theta), to_f64(x))
+    for bits in (2, 4, 8):
+        codes, scales = p.forward_quant(x.to(DEV), bits)
+        check_quant(codes, scales, y_ref, bits, f"degenerate bits={bits}")
+        assert not codes[0].any() and scales[0].item() == 0
+
+
+def test_zero_row_count_and_single_row():
+    n = 1024
+    theta, x = make(n, 1, torch.bfloat16, seed=12)
+    p = plan_for(n, theta)
+    empty = torch.empty((0, n), dtype=torch.bfloat16, device=DEV)
+    assert p.forward(empty).shape == (0, n)
+    c, s = p.forward_quant(empty, 4)
+    assert c.shape == (0, n // 2) and s.shape == (0,)
+    dx, dth = p.backward(empty, empty)
+    assert not dth.any()
+    y = p.forward(x.to(DEV), out_dtype=torch.float32)
+    check_rows_close(y, oracle.forward(to_f64(theta), to_f64(x)), absmax_rows(x), "single row")
+
+
+# ---- argument validation (host side, before any launch) ----------------------------------------------------
+def test_argument_validation_codes():
+    n = 256
+    theta, x = make(n, 4, torch.float32)
+    with pytest.raises(BfqError) as e:
+        Plan(100, DEV)
+    assert e.value.status == -2
+    p = Plan(n, DEV)
+    xd = x.to(DEV)
+    with pytest.raises(BfqError) as e:  # angles not set
+        p.forward(xd)
+    assert e.value.status == -7
+    p.set_angles(theta.to(DEV))
+    with pytest.raises(BfqError) as e:
+        p.forward_quant(xd, 3)
+    assert e.value.status == -3
+    mis = torch.empty(4 * n + 1, dtype=torch.float32, device=DEV)[1:].view(4, n)
+    with pytest.raises(BfqError) as e:
+        p.forward(mis)
+    assert e.value.status == -4
+    with pytest.raises(TypeError):
+        p.forward(xd.to(torch.float16))
+    bad_ld = torch.empty((4, n + 1), dtype=torch.float32, device=DEV)[:, :n]
+    with pytest.raises(BfqError) as e:
+        p.forward(bad_ld)
+    assert e.value.status == -5
+    assert p.device_status() == 0
+
+
+# ---- weight folding: (W Q^T)(Q x) = W x ---------------------------------------------------------------------
+def test_fold_weights_small():
+    n, m = 1024, 96
+    theta = synth.angles(n, "normal", 21)
+    W = synth.rows(m, n, "normal", 22, scale=0.02, dtype=torch.bfloat16)
+    x = synth.rows(32, n, "laplace", 23, outliers=4, outlier_scale=100.0, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    th64 = to_f64(theta)
+    codes, scales, rot = p.fold_weights(W.to(DEV), 2, want_rotated=True, rotated_dtype=torch.float32)
+    WQt_ref = oracle.forward(th64, to_f64(W))
+    check_rows_close(rot, WQt_ref, absmax_rows(W), "W Q^T")
+    check_quant(codes, scales, WQt_ref, 2, "fold codes")
+    Qx = to_f64(p.forward(x.to(DEV), out_dtype=torch.float32))
+    ref = to_f64(W) @ to_f64(x).T
+    np.testing.assert_allclose(to_f64(rot) @ Qx.T, ref, atol=1e-4 * np.abs(ref).max())
+    # quantized product: same error level as the oracle's own quantized product
+    o_codes, o_scales = oracle.quantize(WQt_ref, 2)
+    err_ref = np.linalg.norm(oracle.dequantize(o_codes, o_scales) @ oracle.forward(th64, to_f64(x)).T - ref)
+    deq = oracle.dequantize(oracle.unpack(codes.cpu().numpy(), 2), scales.cpu().view(torch.int16).numpy().view(np.uint16))
+    err_gpu = np.linalg.norm(deq @ Qx.T - ref)
+    assert abs(err_gpu - err_ref) <= 1e-3 * err_ref
