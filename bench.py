@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the butterfly-rotation + INT4 quantization hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = load the angles (twiddle-table build) + rotate and quantize every row of the
+LLaMA-7B-shaped workload (32768 bf16 rows of n = 4096, INT4 codes + fp16 scales).  Prints
+one JSON line (rank 0).  The other operations (backward on the 128 x 2048-token learning
+batch, inverse, n = 8192 INT2, weight folding) are timed after the K steps and reported
+in the same line under "others".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "butterfly+INT4-quant rows/s at n=4096"
+UNIT = "rows/s"
+WORKLOAD = "act4096_int4"
+
+# Algorithmic work per row (n = 4096, L = 12): bytes = bf16 row + packed INT4 codes + fp16 scale;
+# FP32 issue slots = 2 MUL + 2 FMA per pair (paper's FLOP table: 3 n log2 n flops) + n for the scale.
+BYTES_PER_ROW = 4096 * 2 + 4096 // 2 + 2
+SLOTS_PER_ROW = 4 * (4096 // 2) * 12 + 4096
+FP32_LANES_PER_SM = 128
+# dram bytes per launch of the forward+quant kernel from the committed ncu capture (profiles/);
+# None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES_PER_ROW = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        for line in rows:
+            f = [p.strip() for p in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def time_oracle(fn, min_seconds=0.0):
+    t0 = time.perf_counter()
+    fn()
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(sample_rows=32768):
+    """The fp64 oracle, as it stands, on the host cores: forward + INT4 quantize on the first
+    `sample_rows` rows of the workload."""
+    import oracle
+    from paper_2509_09679_b200 import synth
+
+    wl = synth.WORKLOADS[WORKLOAD]
+    theta = wl.theta().double().numpy()
+    x = wl.x(n_rows=sample_rows).double().numpy()
+    oracle.forward_quant(theta, x[:64], wl.bits)  # load the library, warm caches
+    dt = time_oracle(lambda: oracle.forward_quant(theta, x, wl.bits))
+    return {"value": sample_rows / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {sample_rows} of {wl.n_rows} rows of {WORKLOAD} (fp64 C oracle, OpenMP over rows), {dt:.2f} s"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2509_09679_b200 import synth
+
+    wl = synth.WORKLOADS[WORKLOAD]
+    sample_rows = 2048
+    theta = wl.theta().double().numpy()
+    x = wl.x(n_rows=sample_rows).double().numpy()
+    for _ in range(args.warmup):
+        oracle.forward_quant(theta, x, wl.bits)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.forward_quant(theta, x, wl.bits)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sample_rows / dt
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "n": wl.n, "rows_per_step": sample_rows, "bits": wl.bits},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": f"{sample_rows} rows of {WORKLOAD} per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def event_time_ms(torch, fn, iters):
+    """Average device time of fn() over `iters` back-to-back calls on the current stream."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="bfq", choices=["bfq", "reference"])
+    ap.add_argument("--no-others", action="store_true", help="skip the secondary operations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "bfq" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2509_09679_b200 import Plan, lib, synth
+
+    lib()  # fail loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v: float) -> float:
+        if dist is None:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    wl = synth.WORKLOADS[WORKLOAD]
+    # replicas only: every rank runs the whole workload on its own GPU with its own seed
+    theta = wl.theta(device=dev, seed=wl.seed)
+    x = wl.x(device=dev, seed=wl.seed + 100 * rank)
+    plan = Plan(wl.n, dev)
+    codes = torch.empty((wl.n_rows, wl.n * wl.bits // 8), dtype=torch.uint8, device=dev)
+    scales = torch.empty((wl.n_rows,), dtype=torch.float16, device=dev)
+
+    def step():
+        plan.set_angles(theta)
+        plan.forward_quant(x, wl.bits, codes=codes, scales=scales)
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    # per-launch events for the dominant kernel (forward+quant) inside the timed region
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record()
+    for k in range(args.steps):
+        plan.set_angles(theta)
+        kev[k][0].record()
+        plan.forward_quant(x, wl.bits, codes=codes, scales=scales)
+        kev[k][1].record()
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_step = ms_total / args.steps
+    kernel_ms = [a.elapsed_time(b) for a, b in kev]
+    kernel_ms_avg = max_over_ranks(sum(kernel_ms) / len(kernel_ms))
+    status = plan.device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}")
+    value = world * wl.n_rows / (ms_step * 1e-3)
+
+    # ---- end-to-end through the public API with host buffers --------------------------------------
+    x_host = x.to("cpu").pin_memory()
+    codes_host = torch.empty(codes.shape, dtype=codes.dtype).pin_memory()
+    scales_host = torch.empty(scales.shape, dtype=scales.dtype).pin_memory()
+    x_dev = torch.empty_like(x)
+
+    def e2e_step():
+        x_dev.copy_(x_host, non_blocking=True)
+        plan.set_angles(theta)
+        plan.forward_quant(x_dev, wl.bits, codes=codes, scales=scales)
+        codes_host.copy_(codes, non_blocking=True)
+        scales_host.copy_(scales, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    ms_e2e = max_over_ranks(event_time_ms(torch, e2e_step, e2e_steps))
+    e2e = {"value": world * wl.n_rows / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
+           "d2h_bytes_per_step": codes_host.numel() + scales_host.numel() * 2}
+
+    # ---- secondary operations (single rank, after the headline) -------------------------------------
+    others = {}
+    if rank == 0 and not args.no_others:
+        others = time_others(torch, synth, Plan, dev)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    props = torch.cuda.get_device_properties(dev)
+    alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6  # slots/s
+    t_kernel = kernel_ms_avg * 1e-3
+    slots_per_s = SLOTS_PER_ROW * wl.n_rows / t_kernel
+    gbs = BYTES_PER_ROW * wl.n_rows / t_kernel / 1e9
+    t_alu = SLOTS_PER_ROW * wl.n_rows / alu_peak
+    t_hbm = BYTES_PER_ROW * wl.n_rows / (peaks["hbm_gbs"] * 1e9)
+    bound = "alu" if t_alu >= t_hbm else "hbm"
+    roofline = {
+        "bound": bound,
+        "achieved": slots_per_s / 1e12 if bound == "alu" else gbs,
+        "peak": alu_peak / 1e12 if bound == "alu" else peaks["hbm_gbs"],
+        "unit": "Tslot/s (FP32 issue slots: MUL or FMA per lane)" if bound == "alu" else "GB/s",
+        "frac": max(t_alu, t_hbm) / t_kernel,
+        "traffic": None if NCU_TRAFFIC_BYTES_PER_ROW is None else NCU_TRAFFIC_BYTES_PER_ROW * wl.n_rows,
+        "kernel": "forward+quant", "kernel_ms": kernel_ms_avg,
+        "algorithmic_bytes": BYTES_PER_ROW * wl.n_rows, "algorithmic_slots": SLOTS_PER_ROW * wl.n_rows,
+        "hbm_achieved_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"], "hbm_peak_gbs": peaks["hbm_gbs"],
+        "peaks": f"HBM {peaks['source']}; ALU = SMs x 128 lanes x {peaks['sm_max_mhz']:.0f} MHz",
+    }
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "n": wl.n, "rows": wl.n_rows, "bits": wl.bits, "input": "bf16",
+                   "l2": "inputs larger than L2 (268 MB per step)", "parallelism": "replicas only",
+                   "x_checksum": f"{synth.checksum64(x[:256]):016x}"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps, "roofline": roofline,
+        "gbs": gbs, "others": others,
+    }
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def time_others(torch, synth, Plan, dev):
+    """Backward (learning batch), inverse, n = 8192 INT2 and weight folding: device-timed,
+    inputs resident, 3 warm-up + a few timed launches each."""
+    res = {}
+    alu_peak = torch.cuda.get_device_properties(dev).multi_processor_count * FP32_LANES_PER_SM * 1.965e9
+
+    def record(name, rows, n, L, slots_per_pair, bytes_per_row, fn, iters):
+        for _ in range(3):
+            fn()
+        ms = event_time_ms(torch, fn, iters)
+        slots = slots_per_pair * (n // 2) * L * rows
+        res[name] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": bytes_per_row * rows / (ms * 1e-3) / 1e9,
+                     "alu_frac": slots / alu_peak / (ms * 1e-3), "rows": rows, "n": n}
+
+    # angle-learning step: forward + backward on 128 x 2048 rows of n = 4096
+    wl = synth.WORKLOADS["learn4096"]
+    theta = wl.theta(device=dev)
+    plan = Plan(wl.n, dev)
+    plan.set_angles(theta)
+    x = wl.x(device=dev)
+    g = wl.g(device=dev)
+    dx = torch.empty_like(x)
+    dth = torch.empty((wl.L, wl.n // 2), dtype=torch.float32, device=dev)
+    record("backward_n4096", wl.n_rows, wl.n, wl.L, 14, 3 * 2 * wl.n,
+           lambda: plan.backward(x, g, dx=dx, dtheta=dth), 3)
+    record("inverse_n4096", wl.n_rows, wl.n, wl.L, 4, 2 * 2 * wl.n, lambda: plan.inverse(g, out=dx), 3)
+    del x, g, dx
+    torch.cuda.empty_cache()
+    # n = 8192 INT2
+    wl = synth.WORKLOADS["act8192_int2"]
+    plan8 = Plan(wl.n, dev)
+    plan8.set_angles(wl.theta(device=dev))
+    x = wl.x(device=dev)
+    codes = torch.empty((wl.n_rows, wl.n // 4), dtype=torch.uint8, device=dev)
+    scales = torch.empty((wl.n_rows,), dtype=torch.float16, device=dev)
+    record("forward_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
+           lambda: plan8.forward_quant(x, 2, codes=codes, scales=scales), 5)
+    del x
+    wl = synth.WORKLOADS["fold8192_int2"]
+    W = wl.x(device=dev)
+    record("fold_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
+           lambda: plan8.fold_weights(W, 2), 5)
+    return res
+
+
+if __name__ == "__main__":
+    main()

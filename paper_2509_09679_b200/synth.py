@@ -170,7 +170,7 @@ WORKLOADS = {
 
 def checksum64(t: torch.Tensor) -> int:
     """Order-dependent 64-bit checksum of a tensor's raw bytes (for bench records)."""
-    b = t.detach().contiguous().view(torch.uint8).to("cpu")
+    b = t.detach().contiguous().view(torch.uint8).reshape(-1).to("cpu")
     pad = (-b.numel()) % 8
     if pad:
         b = torch.cat([b, torch.zeros(pad, dtype=torch.uint8)])
