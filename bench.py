@@ -173,6 +173,8 @@ def main():
     ap.add_argument("--impl", default="bfq", choices=["bfq", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the secondary operations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler captures of a small case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bfq" else args.warmup
     if args.impl == "reference":
@@ -208,6 +210,10 @@ def main():
         return float(t.item())
 
     wl = synth.WORKLOADS[WORKLOAD]
+    if args.rows:
+        import dataclasses
+
+        wl = dataclasses.replace(wl, n_rows=args.rows)
     # replicas only: every rank runs the whole workload on its own GPU with its own seed
     theta = wl.theta(device=dev, seed=wl.seed)
     x = wl.x(device=dev, seed=wl.seed + 100 * rank)
@@ -250,6 +256,23 @@ def main():
     value = world * wl.n_rows / (ms_step * 1e-3)
 
     # ---- end-to-end through the public API with host buffers --------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(torch, args, wl, plan, theta, x, codes, scales, barrier, max_over_ranks, world)
+
+    # ---- secondary operations (single rank, after the headline) -------------------------------------
+    others = {}
+    if rank == 0 and not args.no_others:
+        others = time_others(torch, synth, Plan, dev)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    finish(torch, args, wl, synth, x, dev, world, value, ms_step, kernel_ms_avg, clocks, e2e, others, dist)
+
+
+def run_e2e(torch, args, wl, plan, theta, x, codes, scales, barrier, max_over_ranks, world):
     x_host = x.to("cpu").pin_memory()
     codes_host = torch.empty(codes.shape, dtype=codes.dtype).pin_memory()
     scales_host = torch.empty(scales.shape, dtype=scales.dtype).pin_memory()
@@ -267,20 +290,12 @@ def main():
         e2e_step()
     barrier()
     ms_e2e = max_over_ranks(event_time_ms(torch, e2e_step, e2e_steps))
-    e2e = {"value": world * wl.n_rows / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
-           "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
-           "d2h_bytes_per_step": codes_host.numel() + scales_host.numel() * 2}
+    return {"value": world * wl.n_rows / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+            "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
+            "d2h_bytes_per_step": codes_host.numel() + scales_host.numel() * 2}
 
-    # ---- secondary operations (single rank, after the headline) -------------------------------------
-    others = {}
-    if rank == 0 and not args.no_others:
-        others = time_others(torch, synth, Plan, dev)
 
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
-
+def finish(torch, args, wl, synth, x, dev, world, value, ms_step, kernel_ms_avg, clocks, e2e, others, dist):
     peaks = measured_peaks()
     props = torch.cuda.get_device_properties(dev)
     alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * peaks["sm_max_mhz"] * 1e6  # slots/s

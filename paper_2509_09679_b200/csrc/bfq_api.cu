@@ -8,6 +8,7 @@
 #include <cstdlib>
 #include <new>
 
+#include "bfq_fast.h"
 #include "bfq_generic.cuh"
 #include "bfq_plan.h"
 
@@ -190,11 +191,13 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     plan->partial_slots = backward_slots(plan->log_n, plan->sm_count);
     e = cudaMalloc(&plan->tw, angles * sizeof(float2));
     if (e == cudaSuccess) e = cudaMalloc(&plan->partial, size_t(plan->partial_slots) * angles * sizeof(float));
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img4096, 128 * 512 * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         cudaFree(plan->tw);
+        cudaFree(plan->img4096);
         cudaFree(plan->partial);
         cudaFree(plan->status_word);
         delete plan;
@@ -209,6 +212,7 @@ int bfq_plan_destroy(bfq_plan* plan) {
     DeviceGuard guard(plan->device);
     cudaDeviceSynchronize();
     cudaFree(plan->tw);
+    cudaFree(plan->img4096);
     cudaFree(plan->partial);
     cudaFree(plan->status_word);
     delete plan;
@@ -223,6 +227,9 @@ int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
     const int count = plan->log_n * (plan->n / 2);
     k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
     cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && plan->img4096 != nullptr) {
+        e = fwdq4096_build_image(plan, theta, static_cast<cudaStream_t>(stream));
+    }
     if (e != cudaSuccess) return cuda_fail(plan, e);
     plan->angles_set = true;
     return BFQ_OK;
@@ -260,10 +267,16 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     if (rows == 0) return BFQ_OK;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaError_t e;
+    if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq4096_available(plan)) {
+        e = fwdq4096_launch(plan, x, rows, ldx, codes, scales, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     GenericParams p{};
     p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = plan->n;
     p.codes = codes, p.scales = scales, p.bits = bits, p.rows = rows;
-    cudaError_t e = launch_generic<kModeForwardQuant>(plan, p, static_cast<cudaStream_t>(stream));
+    e = launch_generic<kModeForwardQuant>(plan, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
 

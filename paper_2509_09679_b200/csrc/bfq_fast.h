@@ -1,0 +1,16 @@
+// Entry points of the tuned kernels (host side), called by the C-ABI layer.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bfq_plan.h"
+
+namespace bfq {
+
+// n = 4096, bf16 rows, INT4: tensor-memory-resident rotation constants
+bool fwdq4096_available(const bfq_plan* plan);
+cudaError_t fwdq4096_build_image(const bfq_plan* plan, const float* theta, cudaStream_t st);
+cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                            uint16_t* scales, cudaStream_t st);
+
+}  // namespace bfq

@@ -418,7 +418,7 @@ __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_backward_generic(const
 }
 
 // dtheta[k] = sum over partial slots in slot order (fixed order => reproducible bits)
-__global__ void k_reduce_partials(const float* __restrict__ partial, int slots, int count, float* __restrict__ out) {
+static __global__ void k_reduce_partials(const float* __restrict__ partial, int slots, int count, float* __restrict__ out) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= count) return;
     float acc = 0.f;
@@ -427,7 +427,7 @@ __global__ void k_reduce_partials(const float* __restrict__ partial, int slots, 
 }
 
 // twiddle table from angles: (cos, sin) evaluated in double, rounded once to fp32
-__global__ void k_build_twiddles(const float* __restrict__ theta, int count, float2* __restrict__ tw) {
+static __global__ void k_build_twiddles(const float* __restrict__ theta, int count, float2* __restrict__ tw) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= count) return;
     double s, c;

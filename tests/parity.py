@@ -7,6 +7,10 @@ codes / scales: the fp16 scale equals the oracle's or differs by exactly one fp1
                 boundary); for such rows the oracle re-quantises with the GPU's scale.  Codes
                 are then bit-exact except for off-by-one codes where the oracle's pre-rounding
                 value lies within 1e-4 of a rounding boundary, at most 1e-4 of all elements.
+                An exact tie (pre-rounding value exactly k + 1/2, which happens in bulk only for
+                degenerate inputs such as theta = 0 on bf16 rows) has two nearest integers and the
+                paper's round() names no tie rule: either neighbour is accepted and such elements
+                do not count against the 1e-4 budget.
 d-theta:        per stage  max_j |d - ref| <= 1e-4 * max_j |ref[s]|,  and  |d - ref|_2 <= 1e-4 |ref|_2.
 """
 from __future__ import annotations
@@ -58,7 +62,9 @@ def check_quant(codes_packed: torch.Tensor, scales: torch.Tensor, y_ref: np.ndar
         frac = pre[bad] - np.floor(pre[bad])
         dist = np.abs(frac - 0.5)
         assert np.all(dist < 1e-4), f"{what}: code mismatch away from a rounding boundary (dist {dist.max():.3e})"
-        assert nbad <= max(1, int(1e-4 * rows * n)), f"{what}: {nbad} boundary mismatches of {rows * n}"
+        exact_tie = dist < 1e-12
+        near = int(nbad - exact_tie.sum())
+        assert near <= max(1, int(1e-4 * rows * n)), f"{what}: {near} boundary mismatches of {rows * n}"
     return {"rows": rows, "scale_ulp_rows": int(shifted.size), "boundary_codes": nbad}
 
 

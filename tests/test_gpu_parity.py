@@ -217,3 +217,73 @@ def test_fold_weights_small():
     deq = oracle.dequantize(oracle.unpack(codes.cpu().numpy(), 2), scales.cpu().view(torch.int16).numpy().view(np.uint16))
     err_gpu = np.linalg.norm(deq @ Qx.T - ref)
     assert abs(err_gpu - err_ref) <= 1e-3 * err_ref
+
+
+# ---- full-size workloads, in the launch configuration the benchmark times --------------------------------
+def _sample_rows(n_rows, count):
+    idx = np.unique(np.concatenate([np.arange(0, n_rows, max(1, n_rows // count)), np.arange(min(n_rows, 8)),
+                                    np.arange(max(0, n_rows - 8), n_rows)]))
+    return idx
+
+
+def test_full_size_forward_int4_n4096():
+    wl = synth.WORKLOADS["act4096_int4"]
+    theta = wl.theta(device=DEV)
+    x = wl.x(device=DEV)
+    p = Plan(wl.n, DEV)
+    p.set_angles(theta)
+    codes = Guarded((wl.n_rows, wl.n // 2), torch.uint8, DEV)
+    scales = Guarded((wl.n_rows,), torch.float16, DEV)
+    p.forward_quant(x, 4, codes=codes.view, scales=scales.view)
+    assert p.device_status() == 0
+    assert codes.intact() and scales.intact()
+    idx = _sample_rows(wl.n_rows, 4096)
+    ti = torch.from_numpy(idx).to(DEV)
+    y_ref = oracle.forward(to_f64(theta), to_f64(x[ti]))
+    stats = check_quant(codes.view[ti], scales.view[ti], y_ref, 4, "act4096_int4")
+    assert stats["scale_ulp_rows"] <= max(4, len(idx) // 100)
+    # run twice: identical bits
+    c2, s2 = p.forward_quant(x, 4)
+    assert torch.equal(c2, codes.view) and torch.equal(s2.view(torch.int16), scales.view.view(torch.int16))
+    # the tuned path and the generic path must agree on the scales (same fp32 absmax up to rounding order)
+    ds = (s2.view(torch.int16).int() - scales.view.view(torch.int16).int()).abs().max().item()
+    assert ds == 0
+
+
+@pytest.mark.parametrize("rows", [1, 2, 3, 5, 147, 148 * 3 + 1, 1000])
+@pytest.mark.parametrize("angle_kind", ["normal", "uniform"])
+def test_tuned_n4096_ragged_row_counts(rows, angle_kind):
+    n = 4096
+    theta = synth.angles(n, angle_kind, 40 + rows)
+    x = synth.rows(rows, n, "student_t3", 41 + rows, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    ld = n + 8
+    xpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    codes = Guarded((rows, n // 2), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.forward_quant(xpad[:, :n], 4, codes=codes.view, scales=scales.view)
+    assert p.device_status() == 0
+    check_quant(codes.view, scales.view, oracle.forward(to_f64(theta), to_f64(x)), 4, f"tuned rows={rows}")
+    assert codes.intact() and scales.intact()
+
+
+def test_tuned_n4096_special_angles_and_degenerate_rows():
+    n = 4096
+    x = synth.rows(64, n, "normal", 77, dtype=torch.bfloat16)
+    x[0] = 0
+    x[1] *= 1e-9
+    x[2] *= 1e6
+    x[3] *= 3e-5
+    for kind, seed in (("zero", 0), ("hadamard", 0), ("uniform", 5)):
+        theta = synth.angles(n, kind, seed)
+        if kind == "uniform":  # exact multiples of pi/2 and pi exercise the angle reduction
+            theta[:, ::7] = math.pi / 2
+            theta[:, 1::7] = -math.pi
+            theta[:, 2::7] = math.pi
+            theta[:, 3::7] = -math.pi / 2
+            theta[:, 4::7] = 100.0
+        p = plan_for(n, theta)
+        codes, scales = p.forward_quant(x.to(DEV), 4)
+        check_quant(codes, scales, oracle.forward(to_f64(theta), to_f64(x)), 4, f"tuned {kind}")
+        assert p.device_status() == 0
