@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-One step = load the angles (twiddle-table build) + rotate and quantize every row of the
+One step = load the angles (two table-build kernels) + rotate and quantize every row of the
 LLaMA-7B-shaped workload (32768 bf16 rows of n = 4096, INT4 codes + fp16 scales).  Prints
 one JSON line (rank 0).  The other operations (backward on the 128 x 2048-token learning
 batch, inverse, n = 8192 INT2, weight folding) are timed after the K steps and reported
@@ -33,9 +33,9 @@ WORKLOAD = "act4096_int4"
 BYTES_PER_ROW = 4096 * 2 + 4096 // 2 + 2
 SLOTS_PER_ROW = 4 * (4096 // 2) * 12 + 4096
 FP32_LANES_PER_SM = 128
-# dram bytes per launch of the forward+quant kernel from the committed ncu capture (profiles/);
-# None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_ROW = None
+# dram bytes (read + write) per row of the forward+quant kernel, from the committed ncu capture of the
+# current kernel on this workload; set back to None whenever that kernel changes.
+NCU_TRAFFIC_BYTES_PER_ROW = (268.678144e6 + 50.600960e6) / 32768  # profiles/fwdq4096_act4096_int4.md
 
 
 def measured_peaks():
@@ -168,7 +168,7 @@ def event_time_ms(torch, fn, iters):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="bfq", choices=["bfq", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the secondary operations")
@@ -324,7 +324,7 @@ def finish(torch, args, wl, synth, x, dev, world, value, ms_step, kernel_ms_avg,
         "config": {"workload": WORKLOAD, "n": wl.n, "rows": wl.n_rows, "bits": wl.bits, "input": "bf16",
                    "l2": "inputs larger than L2 (268 MB per step)", "parallelism": "replicas only",
                    "x_checksum": f"{synth.checksum64(x[:256]):016x}"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * args.steps, "roofline": roofline,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * args.steps, "roofline": roofline,
         "gbs": gbs, "others": others,
     }
     if not args.no_cpu_baseline:

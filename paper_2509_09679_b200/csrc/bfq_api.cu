@@ -191,13 +191,15 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     plan->partial_slots = backward_slots(plan->log_n, plan->sm_count);
     e = cudaMalloc(&plan->tw, angles * sizeof(float2));
     if (e == cudaSuccess) e = cudaMalloc(&plan->partial, size_t(plan->partial_slots) * angles * sizeof(float));
-    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img4096, 128 * 512 * sizeof(float));
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img4096, fwdq4096_image_bytes());
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->prep4096, fwdq4096_prep_bytes());
     if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         cudaFree(plan->tw);
         cudaFree(plan->img4096);
+        cudaFree(plan->prep4096);
         cudaFree(plan->partial);
         cudaFree(plan->status_word);
         delete plan;
@@ -213,6 +215,7 @@ int bfq_plan_destroy(bfq_plan* plan) {
     cudaDeviceSynchronize();
     cudaFree(plan->tw);
     cudaFree(plan->img4096);
+    cudaFree(plan->prep4096);
     cudaFree(plan->partial);
     cudaFree(plan->status_word);
     delete plan;
@@ -224,11 +227,13 @@ int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
     if ((reinterpret_cast<uintptr_t>(theta) & 3u) != 0) return BFQ_ERR_ALIGN;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
-    const int count = plan->log_n * (plan->n / 2);
-    k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
-    cudaError_t e = cudaGetLastError();
-    if (e == cudaSuccess && plan->img4096 != nullptr) {
-        e = fwdq4096_build_image(plan, theta, static_cast<cudaStream_t>(stream));
+    cudaError_t e;
+    if (plan->img4096 != nullptr) {
+        e = fwdq4096_set_angles(plan, theta, static_cast<cudaStream_t>(stream));
+    } else {
+        const int count = plan->log_n * (plan->n / 2);
+        k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
+        e = cudaGetLastError();
     }
     if (e != cudaSuccess) return cuda_fail(plan, e);
     plan->angles_set = true;

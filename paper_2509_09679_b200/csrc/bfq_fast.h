@@ -9,7 +9,10 @@ namespace bfq {
 
 // n = 4096, bf16 rows, INT4: tensor-memory-resident rotation constants
 bool fwdq4096_available(const bfq_plan* plan);
-cudaError_t fwdq4096_build_image(const bfq_plan* plan, const float* theta, cudaStream_t st);
+size_t fwdq4096_image_bytes();
+size_t fwdq4096_prep_bytes();
+// builds the plan's (cos, sin) table and the tensor-memory image from the angles
+cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st);
 cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st);
 

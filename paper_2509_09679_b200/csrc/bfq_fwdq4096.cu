@@ -1,24 +1,31 @@
 // Tuned forward + INT4 quantization for n = 4096 bf16 rows on sm_100a.
 //
-// Design (one persistent CTA per SM, 12 warps):
-//  * The 12 stages are split into phase A (stages 0-5, pair strides 1..32) and phase B (stages
-//    6-11, strides 64..2048).  In either phase a thread owns 64 elements of a row whose pair
-//    partners are all among them, so a whole phase runs in registers.
+// Design (one persistent CTA per SM, G row groups of 128 threads):
+//  * A row is owned by one group of four warps, one warp per scheduler and per tensor-memory lane
+//    quarter.  The 12 stages run as three phases of four stages.  In each phase a thread holds 32
+//    elements of the row as 16 packed fp32x2 registers: four index bits are the phase's stage bits
+//    (so all partners are in the thread's own registers) and the fifth selects the half of the
+//    packed register and is never a stage bit of that phase, so every rotation is a packed FMA.
+//        phase 1: stage bits 0-3, packed along bit 8     (two runs of 16 consecutive elements)
+//        phase 2: stage bits 4-7, packed along bit 8
+//        phase 3: stage bits 8-11, packed along bit 0    (adjacent elements -> one code byte)
+//    Between phases the row is regrouped through shared memory.  The first regrouping swaps bits
+//    0-3 with bits 4-7 among the 16 lanes of a half-warp: 64-bit stores and loads of whole packed
+//    registers and a warp-level sync only.  The second crosses warps: scalar stores, 64-bit loads,
+//    one named barrier.  The buffer layouts are additive in the index bits (padded, not
+//    XOR-swizzled) so that every access is base + immediate and bank-conflict free.
 //  * Rotations use the three-shear (lifting) form  a += -t*b; b += s*a; a += -t*b  with
-//    t = tan(phi/2), s = sin(phi): three FMAs and two constants per pair instead of two MULs, two
-//    FMAs and a negation.  Angles are reduced to |phi| <= pi/2 (so |t| <= 1); the sign flips that
-//    reduction introduces are tracked per element when the tables are built and are absorbed by
-//    later stages' angles; the last stage uses a general 2x2 form whose constants restore the true
-//    signs.  All of this is table preparation: the kernel sees only constants.
-//  * The constants (53248 words) live in tensor memory (TMEM), one private 384/448-word strip per
-//    thread role, and are streamed into registers with tcgen05.ld one 32-word chunk ahead of use.
-//    TMEM lanes are tied to warp id mod 4, so warps 0,1 (mod 4) are phase-A teams and warps 2,3
-//    (mod 4) are phase-B teams: a row flows  TMA -> A team -> shared-memory transpose -> B team.
-//    Three such pipelines run per SM.
-//  * Rows arrive by TMA (128-byte swizzled tiles, 3-deep ring per pipeline, mbarrier completion);
-//    the A->B hand-off is double buffered with named barriers; the per-row absmax is a warp
-//    reduction plus one cross-warp step inside the B team; INT4 codes are produced with the
-//    magic-number rounding trick, transposed across 8 lanes with shuffles and stored as 32-bit words.
+//    t = tan(phi/2), s = sin(phi): three FMAs and two constants per pair.  Angles are reduced to
+//    |phi| <= pi/2 (so |t| <= 1); the sign flips that the reduction introduces are tracked per
+//    element when the tables are built and are absorbed by later stages' angles; the last stage
+//    uses a general 2x2 form whose constants restore the true signs.  All of this is table
+//    preparation: the kernel sees only constants.
+//  * The constants (416 words per thread role, 53248 in all) live in tensor memory, one strip per
+//    lane; every group reads the same strips.  They are streamed into registers with tcgen05.ld,
+//    one chunk ahead of use.
+//  * Rows arrive by TMA (128-byte swizzled tiles, two-deep ring per group, mbarrier completion).
+//    The per-row absmax is a warp reduction plus one step across the group's four warps; INT4
+//    codes are produced with the magic-number rounding trick, one byte per packed register.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -31,70 +38,92 @@ namespace f4k {
 using namespace ptx;
 
 constexpr int kN = 4096;
-constexpr int kPipes = 3;
-constexpr int kThreads = kPipes * 128;
-constexpr int kInStages = 3;
-constexpr uint32_t kRowBytes = kN * 2;   // one bf16 row
-constexpr uint32_t kTBufBytes = kN * 4;  // one fp32 row
-constexpr uint32_t kInOff = 0;
-constexpr uint32_t kTOff = kInOff + kPipes * kInStages * kRowBytes;
-constexpr uint32_t kMiscOff = kTOff + kPipes * 2 * kTBufBytes;
-constexpr uint32_t kBarOff = kMiscOff;          // mbarriers [kPipes][kInStages], 8 bytes each
-constexpr uint32_t kAmaxOff = kMiscOff + 128;   // float [kPipes][2 parities][2 warps]
-constexpr uint32_t kTmemOff = kMiscOff + 192;   // tensor-memory base address
-constexpr uint32_t kSmemUsed = kMiscOff + 256;
-constexpr uint32_t kSmemBytes = kSmemUsed + 1024;  // slack for 1024-byte alignment of the TMA tiles
+constexpr int kGroupThreads = 128;
+constexpr int kInSlots = 2;                  // TMA ring depth per group
+constexpr uint32_t kRowBytes = kN * 2;       // one bf16 row
+constexpr uint32_t kExWords = 4128;          // padded fp32 row (see the layouts below)
+constexpr uint32_t kExBytes = kExWords * 4;
+constexpr int kCols = 416;                   // tensor-memory columns in use
 
-constexpr int kChunksA = 12;  // 6 stages x 64 words / 32
-constexpr int kChunksB = 14;  // 5 stages x 64 words + 128 words (general last stage)
+// G row groups per CTA; XB regrouping buffers per group (2: one per regrouping; 1: shared, at the
+// price of one more barrier per row)
+template <int G, int XB>
+struct Smem {
+    static constexpr uint32_t kInOff = 0;  // [G][kInSlots][kRowBytes], 1024-byte aligned tiles
+    static constexpr uint32_t kExOff = kInOff + G * kInSlots * kRowBytes;  // [G][XB][kExBytes]
+    static constexpr uint32_t kBarOff = kExOff + G * XB * kExBytes;       // mbarriers [G][kInSlots]
+    static constexpr uint32_t kAmaxOff = kBarOff + 8 * G * kInSlots;      // float [G][2 parities][4 warps]
+    static constexpr uint32_t kTmemOff = kAmaxOff + 32 * G;               // tensor-memory base address
+    static constexpr uint32_t kUsed = kTmemOff + 16;
+    static constexpr uint32_t kBytes = kUsed + 1024;  // slack for the 1024-byte alignment of the TMA tiles
+};
 
 __device__ __forceinline__ uint4 lds128(uint32_t a) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
     return v;
 }
+__device__ __forceinline__ u64 lds64(uint32_t a) {
+    u64 v;
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(a));
+    return v;
+}
 __device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
 }
+__device__ __forceinline__ void sts64(uint32_t a, u64 v) {
+    asm volatile("st.shared.b64 [%0], %1;" ::"r"(a), "l"(v) : "memory");
+}
+
+// ---- element held by role t, packed register m, half h in each phase -----------------------------------
+//   phase 1: i = m | (t & 15) << 4 | h << 8 | (t >> 4) << 9
+//   phase 2: i = (t & 15) | m << 4 | h << 8 | (t >> 4) << 9
+//   phase 3: i = h | t << 1 | m << 8
+// ---- shared-memory layouts of the two regroupings (word addresses; i = element index bits) -----------
+// first:   A1 = i8 + 2*(i4..i7) + 32*(i9 + 2*i10 + 4*i11) + 258*(i0..i3)
+// second:  A2 = (i0..i4) + 16*i9 + 32*(i5 + 2*i6 + 4*i7 + 8*i8 + 16*i10 + 32*i11 + 64*i9)
+// Both are injective into [0, kExWords); a half-warp's 16 64-bit accesses and a warp's 32 scalar
+// stores each cover the 32 banks exactly once.  In the first, the words a thread writes are read by
+// the 16 lanes of its own half-warp only.
+__device__ __forceinline__ constexpr uint32_t ex1_wr_local(int m) { return 4u * 258u * m; }
+__device__ __forceinline__ constexpr uint32_t ex1_rd_local(int m) { return 4u * 2u * m; }
+__device__ __forceinline__ constexpr uint32_t ex2_wr_local(int m, int h) {
+    return 4u * (16u * (m & 1) + 32u * (m >> 1) + 256u * h);
+}
+__device__ __forceinline__ constexpr uint32_t ex2_rd_local(int m) {
+    return 4u * (256u * (m & 1) + 2064u * ((m >> 1) & 1) + 512u * ((m >> 2) & 1) + 1024u * ((m >> 3) & 1));
+}
 
 // ---- one stage on the registers of a thread ---------------------------------------------------------
-// P[m] packs local elements (2m, 2m+1).  Local bit 0 pairs the two halves of one register (scalar
-// lifting); local bit K >= 1 pairs registers m and m | 2^(K-1) (packed lifting, both lanes at once).
-template <int H>
-__device__ __forceinline__ void stage_bit0(u64 (&P)[32], const uint32_t (&T)[32]) {
+// Local stage K pairs packed registers m and m | 2^K; both fp32 lanes rotate at once.  T holds
+// (nt, nt', sn, sn') for NU consecutive pairs starting at pair U0.  The three shears are issued level
+// by level so that dependent instructions are NU apart.
+template <int K, int U0, int NU, int CW>
+__device__ __forceinline__ void stage_lift(u64 (&P)[16], const uint32_t (&T)[CW]) {
+    static_assert(4 * NU <= CW, "chunk too small");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const int m = 16 * H + i;
-        float a, b;
-        unpack2(P[m], a, b);
-        const float nt = __uint_as_float(T[2 * i]), sn = __uint_as_float(T[2 * i + 1]);
-        const float a1 = fmaf(nt, b, a);
-        const float b2 = fmaf(sn, a1, b);
-        const float a2 = fmaf(nt, b2, a1);
-        P[m] = pack2(a2, b2);
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), P[m_hi], P[m_lo]);
+    }
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        P[m_hi] = fma2(pack2u(T[4 * i + 2], T[4 * i + 3]), P[m_lo], P[m_hi]);
+    }
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), P[m_hi], P[m_lo]);
     }
 }
-template <int K, int H>
-__device__ __forceinline__ void stage_lift(u64 (&P)[32], const uint32_t (&T)[32]) {
+// last stage (local bit 3 of phase 3): out_lo = k1*a + k2*b, out_hi = k3*a + k4*b for pairs U0..U0+NU-1
+template <int U0, int NU, int CW>
+__device__ __forceinline__ void stage_general(u64 (&P)[16], const uint32_t (&T)[CW]) {
+    static_assert(8 * NU <= CW, "chunk too small");
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int u = 8 * H + i;
-        const int m_lo = ((u >> (K - 1)) << K) | (u & ((1 << (K - 1)) - 1));
-        const int m_hi = m_lo | (1 << (K - 1));
-        const u64 NT = pack2u(T[4 * i], T[4 * i + 1]);
-        const u64 SN = pack2u(T[4 * i + 2], T[4 * i + 3]);
-        const u64 a1 = fma2(NT, P[m_hi], P[m_lo]);
-        const u64 b2 = fma2(SN, a1, P[m_hi]);
-        P[m_lo] = fma2(NT, b2, a1);
-        P[m_hi] = b2;
-    }
-}
-// last stage (local bit 5 of phase B): out_lo = k1*a + k2*b, out_hi = k3*a + k4*b
-template <int Q>
-__device__ __forceinline__ void stage_general5(u64 (&P)[32], const uint32_t (&T)[32]) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int m_lo = 4 * Q + i, m_hi = m_lo | 16;
+    for (int i = 0; i < NU; ++i) {
+        const int m_lo = U0 + i, m_hi = m_lo | 8;
         const u64 K1 = pack2u(T[8 * i], T[8 * i + 1]), K2 = pack2u(T[8 * i + 2], T[8 * i + 3]);
         const u64 K3 = pack2u(T[8 * i + 4], T[8 * i + 5]), K4 = pack2u(T[8 * i + 6], T[8 * i + 7]);
         const u64 a = P[m_lo], b = P[m_hi];
@@ -103,90 +132,113 @@ __device__ __forceinline__ void stage_general5(u64 (&P)[32], const uint32_t (&T)
     }
 }
 
-template <int PHASE, int C>
-__device__ __forceinline__ void run_chunk(u64 (&P)[32], const uint32_t (&T)[32]) {
-    if constexpr (C < 2) {
-        stage_bit0<C>(P, T);
-    } else if constexpr (PHASE == 1 && C >= 10) {
-        stage_general5<C - 10>(P, T);
+struct ExAddr {
+    uint32_t w1, r1, w2, r2;  // per-thread byte addresses of the two regroupings (write / read side)
+    int bar;                  // named barrier of the group
+};
+
+// chunk C of CW words: columns [C*CW, C*CW + CW) of the thread's strip
+template <int CW>
+struct Chunks {
+    static constexpr int kPerStage = 32 / CW;             // chunks per lifting stage
+    static constexpr int kLift = 11 * kPerStage;          // chunks of the 11 lifting stages
+    static constexpr int kCount = kLift + 64 / CW;        // + the general last stage
+    static constexpr int kAfterPhase1 = 4 * kPerStage - 1;  // last chunk of stage 3
+    static constexpr int kAfterPhase2 = 8 * kPerStage - 1;  // last chunk of stage 7
+};
+
+template <int C, int CW>
+__device__ __forceinline__ void run_chunk(u64 (&P)[16], const uint32_t (&T)[CW]) {
+    using CH = Chunks<CW>;
+    constexpr int NU = CW / 4;
+    if constexpr (C < CH::kLift) {
+        stage_lift<(C / CH::kPerStage) & 3, (C % CH::kPerStage) * NU, NU, CW>(P, T);
     } else {
-        stage_lift<C / 2, C % 2>(P, T);
+        stage_general<(C - CH::kLift) * (CW / 8), CW / 8, CW>(P, T);
     }
 }
-// chunk C is in Tcur (load already issued); the load of chunk C+1 is issued right after the wait so
-// that exactly one tensor-memory load is in flight while chunk C is being used.
-template <int PHASE, int C, int NC>
-__device__ __forceinline__ void run_chunks(u64 (&P)[32], uint32_t (&Tcur)[32], uint32_t (&Tnext)[32], uint32_t tbase) {
-    tmem_wait_ld32(Tcur);
-    if constexpr (C + 1 < NC) tmem_ld32(tbase + 32 * (C + 1), Tnext);
-    run_chunk<PHASE, C>(P, Tcur);
-    if constexpr (C + 1 < NC) run_chunks<PHASE, C + 1, NC>(P, Tnext, Tcur, tbase);
-}
-template <int PHASE>
-__device__ __forceinline__ void run_phase(u64 (&P)[32], uint32_t tbase) {
-    uint32_t T0[32], T1[32];
-    tmem_ld32(tbase, T0);
-    run_chunks<PHASE, 0, (PHASE == 0 ? kChunksA : kChunksB)>(P, T0, T1, tbase);
-}
 
-// 8x8 transpose of 4-bit fields across lanes l, l^1, .., l^7 (field k of lane r <-> field r of lane k)
-__device__ __forceinline__ uint32_t xpose_nibbles8(uint32_t w, int lane) {
-    uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, w, 4);
-    w = __byte_perm(w, o, (lane & 4) ? 0x3276 : 0x5410);
-    o = __shfl_xor_sync(0xFFFFFFFFu, w, 2);
-    w = __byte_perm(w, o, (lane & 2) ? 0x3715 : 0x6240);
-    const uint32_t snd = __funnelshift_l(w, w, (lane & 1) ? 4 : 28);
-    o = __shfl_xor_sync(0xFFFFFFFFu, snd, 1);
-    const uint32_t keep = (lane & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu;
-    return (w & keep) | (o & ~keep);
+__device__ __forceinline__ void regroup1(u64 (&P)[16], const ExAddr& ex) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) sts64(ex.w1 + ex1_wr_local(m), P[m]);
+    __syncwarp();
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r1 + ex1_rd_local(m));
+}
+template <int XB>
+__device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
+    // with one shared buffer, every warp of the group must be past its reads of the first layout
+    if constexpr (XB == 1) bar_sync(ex.bar, kGroupThreads);
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+        uint32_t lo, hi;
+        unpack2u(P[m], lo, hi);
+        sts32(ex.w2 + ex2_wr_local(m, 0), lo);
+        sts32(ex.w2 + ex2_wr_local(m, 1), hi);
+    }
+    bar_sync(ex.bar, kGroupThreads);
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r2 + ex2_rd_local(m));
 }
 
-constexpr uint32_t kMagicBits = 0x4B400000u;  // 1.5 * 2^23
-// sum over k of (kMagicBits << 4k) mod 2^32: what eight stacked magic bit patterns add up to
-constexpr uint32_t kHornerConst = kMagicBits + (kMagicBits << 4) + (kMagicBits << 8) + (kMagicBits << 12) +
-                                  (kMagicBits << 16) + (kMagicBits << 20) + (kMagicBits << 24) + (kMagicBits << 28);
-static_assert(kHornerConst == 0x3F400000u, "stacked magic constant");
+// Chunk C is in Tcur (load already issued); the load of chunk C+1 is issued right after the wait so
+// that exactly one tensor-memory load is in flight while chunk C is being used.  `issue_next` runs
+// once per row, after the second regrouping's barrier (all reads of the input slot are done by then).
+template <int C, int CW, int XB, class F>
+__device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[CW], uint32_t (&Tnext)[CW], uint32_t tbase,
+                                           const ExAddr& ex, F&& issue_next) {
+    using CH = Chunks<CW>;
+    tmem_wait_ld(Tcur);
+    if constexpr (C + 1 < CH::kCount) tmem_ld(tbase + CW * (C + 1), Tnext);
+    run_chunk<C, CW>(P, Tcur);
+    if constexpr (C == CH::kAfterPhase1) regroup1(P, ex);
+    if constexpr (C == CH::kAfterPhase2) {
+        regroup2<XB>(P, ex);
+        issue_next();
+    }
+    if constexpr (C + 1 < CH::kCount) run_chunks<C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, issue_next);
+}
 
-__global__ void __launch_bounds__(kThreads, 1)
+template <int G, int CW, int XB>
+__global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, uint8_t* __restrict__ codes,
            uint16_t* __restrict__ scales, int rows, int* __restrict__ status) {
+    using S = Smem<G, XB>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int q = warp & 3, p = warp >> 2;
-    const bool is_a = q < 2;
-    const int t = (q & 1) * 32 + lane;  // role within the team: 0..63
+    const int q = warp & 3, g = warp >> 2;
+    const int t = q * 32 + lane;  // role within the group: 0..127
 
-    if (warp == 0) tmem_alloc512(sbase + kTmemOff);
-    if (threadIdx.x < kPipes * kInStages) {
-        mbar_init(sbase + kBarOff + 8 * threadIdx.x, 1);
+    if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
+    if (threadIdx.x < G * kInSlots) {
+        mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
         mbar_init_fence();
     }
     tmem_fence_before();
     __syncthreads();
     tmem_fence_after();
     uint32_t tmem_base;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + kTmemOff));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
     const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 
-    const int first = blockIdx.x * kPipes + p;
-    const int stride = gridDim.x * kPipes;
+    const int first = blockIdx.x * G + g;
+    const int stride = gridDim.x * G;
     const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
-    const uint32_t in_base = sbase + kInOff + p * kInStages * kRowBytes;
-    const uint32_t bar_base = sbase + kBarOff + 8 * p * kInStages;
+    const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
+    const uint32_t bar_base = sbase + S::kBarOff + 8 * g * kInSlots;
 
-    // first rows of this pipeline: issued before the table fill so that HBM latency overlaps it
-    if (is_a && t == 0) {
-        for (int k = 0; k < kInStages && k < count; ++k) {
+    // first rows of this group: issued before the table fill so that HBM latency overlaps it
+    if (t == 0) {
+        for (int k = 0; k < kInSlots && k < count; ++k) {
             mbar_expect_tx(bar_base + 8 * k, kRowBytes);
             tma_load_3d(in_base + k * kRowBytes, &tmap, 0, 0, first + k * stride, bar_base + 8 * k);
         }
     }
-    // fill tensor memory: the four warps of pipeline 0 cover the four lane quarters
-    if (p == 0) {
-        const float4* src = reinterpret_cast<const float4*>(img + (q * 32 + lane) * 512);
-        const int ncols = q < 2 ? 32 * kChunksA : 32 * kChunksB;
-        for (int c = 0; c < ncols; c += 16) {
+    // fill tensor memory: the G warps of a lane quarter share its 26 blocks of 16 columns
+    {
+        const float4* src = reinterpret_cast<const float4*>(img + (q * 32 + lane) * kCols);
+        for (int c = 16 * g; c < kCols; c += 16 * G) {
             uint32_t v[16];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -202,125 +254,107 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     __syncthreads();
     tmem_fence_after();
 
-    const int bar_full = 1 + p * 5, bar_empty = 3 + p * 5, bar_team = 5 + p * 5;
-    const uint32_t tb_base = sbase + kTOff + p * 2 * kTBufBytes;
-    u64 P[32];
+    ExAddr ex;
+    {
+        const uint32_t eb1 = sbase + S::kExOff + g * XB * kExBytes;
+        const uint32_t eb2 = eb1 + (XB - 1) * kExBytes;
+        const uint32_t t4 = (t >> 4) & 1, t5 = (t >> 5) & 1, t6 = (t >> 6) & 1;
+        ex.w1 = eb1 + 4u * (2u * (t & 15) + 32u * (t >> 4));
+        ex.r1 = eb1 + 4u * (258u * (t & 15) + 32u * (t >> 4));
+        ex.w2 = eb2 + 4u * ((t & 15) + 2064u * t4 + 512u * t5 + 1024u * t6);
+        ex.r2 = eb2 + 4u * (2u * (t & 15) + 32u * (t >> 4));
+        ex.bar = 1 + g;
+    }
+    // input tile: thread t owns two runs of 32 bytes, at byte 32 (t & 15) + 1024 (t >> 4) + 512 h of the
+    // row, i.e. 16-byte chunks 2 (t & 3) + c of 128-byte line ((t >> 2) & 3) + 8 (t >> 4) + 4 h; the TMA
+    // swizzle stores chunk j of line l at position j ^ (l & 7)
+    const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+    const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+    const uint32_t amax_base = sbase + S::kAmaxOff + g * 32;
+    uint8_t* const out_t = codes + t;
 
-    if (is_a) {
-        uint32_t st_off[8];
+    u64 P[16];
+    uint32_t T0[CW], T1[CW];
+
+    for (int k = 0; k < count; ++k) {
+        const int row = first + k * stride;
+        const int slot = k & 1;
+        tmem_ld(tlane, T0);
+        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+        const uint32_t src = in_base + slot * kRowBytes + in_line;
+        {
+            // run (h, c) holds elements 8c..8c+7 of half h; element m of half h is half h of P[m]
+            uint4 w[2][2];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) st_off[c] = 4 * (t ^ (c << 2));
-        const uint32_t in_line = t * 128, in_x = (t & 7) << 4;
-        for (int k = 0; k < count; ++k) {
-            const int bi = k % kInStages;
-            const uint32_t parity = (k / kInStages) & 1;
-            mbar_wait_bounded(bar_base + 8 * bi, parity, status);
-            const uint32_t src = in_base + bi * kRowBytes;
+            for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint4 w = lds128(src + in_line + ((c << 4) ^ in_x));
-                P[4 * c + 0] = pack2u(w.x << 16, w.x & 0xFFFF0000u);
-                P[4 * c + 1] = pack2u(w.y << 16, w.y & 0xFFFF0000u);
-                P[4 * c + 2] = pack2u(w.z << 16, w.z & 0xFFFF0000u);
-                P[4 * c + 3] = pack2u(w.w << 16, w.w & 0xFFFF0000u);
-            }
-            run_phase<0>(P, tlane);
-            const int bt = k & 1;
-            bar_sync(bar_empty + bt, 128);  // B team has drained transpose buffer bt
-            if (t == 0 && k + kInStages < count) {  // every A thread is past its reads of ring slot bi
-                mbar_expect_tx(bar_base + 8 * bi, kRowBytes);
-                tma_load_3d(src, &tmap, 0, 0, first + (k + kInStages) * stride, bar_base + 8 * bi);
-            }
-            const uint32_t dst = tb_base + bt * kTBufBytes;
+                for (int c = 0; c < 2; ++c) w[h][c] = lds128(src + 512u * h + (in_x ^ ((c | (h << 2)) << 4)));
 #pragma unroll
-            for (int m = 0; m < 32; ++m) {
-                uint32_t lo, hi;
-                unpack2u(P[m], lo, hi);
-                sts32(dst + (2 * m) * 256 + st_off[(2 * m) & 7], lo);
-                sts32(dst + (2 * m + 1) * 256 + st_off[(2 * m + 1) & 7], hi);
+            for (int c = 0; c < 2; ++c) {
+                const uint32_t a[4] = {w[0][c].x, w[0][c].y, w[0][c].z, w[0][c].w};
+                const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    P[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
+                    P[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
+                }
             }
-            __threadfence_block();
-            bar_arrive(bar_full + bt, 128);
         }
-        // pair off the B team's two priming arrivals
-        bar_sync(bar_empty + 0, 128);
-        bar_sync(bar_empty + 1, 128);
-    } else {
-        const uint32_t ld_line = t * 256, ld_x = (t & 7) << 4;
-        bar_arrive(bar_empty + 0, 128);
-        bar_arrive(bar_empty + 1, 128);
-        const uint32_t amax_base = sbase + kAmaxOff + p * 16;
-        for (int k = 0; k < count; ++k) {
-            const int row = first + k * stride;
-            const int bt = k & 1;
-            bar_sync(bar_full + bt, 128);
-            const uint32_t src = tb_base + bt * kTBufBytes;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const uint4 w = lds128(src + ld_line + ((c << 4) ^ ld_x));
-                P[2 * c + 0] = pack2u(w.x, w.y);
-                P[2 * c + 1] = pack2u(w.z, w.w);
+        run_chunks<0, CW, XB>(P, T0, T1, tlane, ex, [&]() {
+            if (t == 0 && k + kInSlots < count) {
+                mbar_expect_tx(bar_base + 8 * slot, kRowBytes);
+                tma_load_3d(in_base + slot * kRowBytes, &tmap, 0, 0, first + (k + kInSlots) * stride,
+                            bar_base + 8 * slot);
             }
-            bar_arrive(bar_empty + bt, 128);
-            run_phase<1>(P, tlane);
+        });
 
-            // per-row absmax: thread, warp, then the team's two warps
-            float m0 = 0.f, m1 = 0.f;
+        // per-row absmax: thread, warp, then the group's four warps
+        float m0 = 0.f, m1 = 0.f;
 #pragma unroll
-            for (int m = 0; m < 32; ++m) {
-                float a, b;
-                unpack2(P[m], a, b);
-                m0 = fmaxf(m0, fabsf(a));
-                m1 = fmaxf(m1, fabsf(b));
-            }
-            float amax = fmaxf(m0, m1);
+        for (int m = 0; m < 16; ++m) {
+            float a, b;
+            unpack2(P[m], a, b);
+            m0 = fmaxf(m0, fabsf(a));
+            m1 = fmaxf(m1, fabsf(b));
+        }
+        float amax = fmaxf(m0, m1);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
-            const uint32_t slot = amax_base + (k & 1) * 8;
-            if (lane == 0) sts32(slot + (q & 1) * 4, __float_as_uint(amax));
-            bar_sync(bar_team, 64);
-            {
-                uint32_t o0, o1;
-                asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(o0), "=r"(o1) : "r"(slot));
-                amax = fmaxf(__uint_as_float(o0), __uint_as_float(o1));
-            }
-            float inv;
-            const uint16_t s16 = row_scale(amax, 7, &inv);
-            if (t == 0) scales[row] = s16;
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+        const uint32_t aslot = amax_base + (k & 1) * 16;
+        if (lane == 0) sts32(aslot + q * 4, __float_as_uint(amax));
+        bar_sync(ex.bar, kGroupThreads);
+        {
+            const uint4 o = lds128(aslot);
+            amax = fmaxf(fmaxf(__uint_as_float(o.x), __uint_as_float(o.y)),
+                         fmaxf(__uint_as_float(o.z), __uint_as_float(o.w)));
+        }
+        float inv;
+        const uint16_t s16 = row_scale(amax, 7, &inv);
+        if (t == 0) scales[row] = s16;
 
-            // codes: q + 8 lands in the low nibble of the fp32 bit pattern of v*inv + (1.5*2^23 + 8)
-            const uint32_t e16 = (s16 >> 10) & 31u;
-            const bool plain = (e16 != 0u) && (s16 != 0x7BFFu);  // normal fp16 scale: |v*inv| <= 7.004, no clipping
-            uint32_t* out = reinterpret_cast<uint32_t*>(codes + static_cast<size_t>(row) * (kN / 2) + 32 * (t & 7) +
-                                                        4 * (t >> 3));
+        // codes: thread t holds elements 2t + 256m (+1) = byte t + 128m of the row's packed codes
+        const uint32_t e16 = (s16 >> 10) & 31u;
+        const bool plain = (e16 != 0u) && (s16 != 0x7BFFu);  // normal fp16 scale: |v*inv| <= 7.004, no clipping
+        uint8_t* out = out_t + static_cast<size_t>(row) * (kN / 2);
+        if (plain) {
+            // q + 8 lands in the low nibble of the fp32 bit pattern of v*inv + (1.5*2^23 + 8), whose other
+            // low bits are zero: hi*16 + lo has (q_hi + 8) << 4 | (q_lo + 8) in its low byte
             const u64 inv2 = pack2(inv, inv);
             const u64 magic2 = pack2(12582920.0f, 12582920.0f);
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                uint32_t w;
-                if (plain) {
-                    uint32_t bits[8];
+            for (int m = 0; m < 16; ++m) {
+                uint32_t lo, hi;
+                unpack2u(fma2(P[m], inv2, magic2), lo, hi);
+                out[128 * m] = static_cast<uint8_t>((hi * 16u + lo) ^ 0x88u);  // offset-binary -> two's complement
+            }
+        } else {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) unpack2u(fma2(P[4 * g + i], inv2, magic2), bits[2 * i], bits[2 * i + 1]);
-                    uint32_t acc = bits[7];
-#pragma unroll
-                    for (int i = 6; i >= 0; --i) acc = acc * 16u + bits[i];
-                    w = acc - kHornerConst;
-                } else {
-                    w = 0u;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float a, b;
-                        unpack2(P[4 * g + i], a, b);
-                        const int qa = static_cast<int>(fminf(fmaxf(rintf(a * inv), -8.f), 7.f)) + 8;
-                        const int qb = static_cast<int>(fminf(fmaxf(rintf(b * inv), -8.f), 7.f)) + 8;
-                        w |= static_cast<uint32_t>(qa) << (8 * i);
-                        w |= static_cast<uint32_t>(qb) << (8 * i + 4);
-                    }
-                }
-                w ^= 0x88888888u;  // offset-binary -> two's complement
-                w = xpose_nibbles8(w, lane);
-                out[g * 64] = w;   // 8 consecutive columns of element group e = 8g + (t & 7)
+            for (int m = 0; m < 16; ++m) {
+                float a, b;
+                unpack2(P[m], a, b);
+                const int qa = static_cast<int>(fminf(fmaxf(rintf(a * inv), -8.f), 7.f));
+                const int qb = static_cast<int>(fminf(fmaxf(rintf(b * inv), -8.f), 7.f));
+                out[128 * m] = static_cast<uint8_t>((qa & 0xF) | ((qb & 0xF) << 4));
             }
         }
     }
@@ -331,61 +365,74 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
 }
 
 // ---- table preparation -----------------------------------------------------------------------------------
-// One CTA walks the stages in order, tracking the sign each element carries, and writes the
-// tensor-memory image: img[lane][col], lanes 0..63 = phase-A roles, 64..127 = phase-B roles.
-__global__ void __launch_bounds__(1024) k_build_image4096(const float* __restrict__ theta, float* __restrict__ img) {
-    __shared__ signed char sg[kN];
-    for (int i = threadIdx.x; i < kN; i += blockDim.x) sg[i] = 1;
-    for (int i = threadIdx.x; i < 128 * 512; i += blockDim.x) img[i] = 0.f;
-    __syncthreads();
+// Step 1 (one thread per angle): the generic (cos, sin) table entry, the reduced-angle lifting
+// constants and whether the reduction negates the pair.  With r = theta mod 2 pi in [-pi, pi], the pair
+// is negated iff |r| > pi/2, and phi = r -+ pi in that case; tan(phi/2) and sin(phi) are odd in phi,
+// so the constants for the mirrored rotation G(-theta) are the negatives of the stored ones.
+__global__ void __launch_bounds__(256) k_prep_angles4096(const float* __restrict__ theta, float2* __restrict__ tw,
+                                                          float4* __restrict__ prep, uint8_t* __restrict__ flip) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 12 * (kN / 2)) return;
     const double kPi = 3.14159265358979323846;
-    for (int s = 0; s < 12; ++s) {
-        for (int j = threadIdx.x; j < kN / 2; j += blockDim.x) {
-            const int lo = ((j >> s) << (s + 1)) | (j & ((1 << s) - 1));
-            const int hi = lo + (1 << s);
-            const double th = static_cast<double>(theta[s * (kN / 2) + j]);
-            int sa = sg[lo], sb = sg[hi];
-            int role, e, k;
-            if (s <= 5) {
-                role = lo >> 6, e = lo & 63, k = s;
-            } else {
-                role = 64 + (lo & 63), e = lo >> 6, k = s - 6;
-            }
-            float* strip = img + role * 512;
-            if (s < 11) {
-                double te = remainder(sa == sb ? th : -th, 2.0 * kPi);  // [-pi, pi]
-                bool flip = false;
-                if (te > 0.5 * kPi) {
-                    te -= kPi, flip = true;
-                } else if (te < -0.5 * kPi) {
-                    te += kPi, flip = true;
-                }
-                const float nt = static_cast<float>(-tan(0.5 * te));
-                const float sn = static_cast<float>(sin(te));
-                if (flip) sa = -sa, sb = -sb;
-                sg[lo] = static_cast<signed char>(sa);
-                sg[hi] = static_cast<signed char>(sb);
-                if (k == 0) {
-                    strip[2 * (e >> 1)] = nt;
-                    strip[2 * (e >> 1) + 1] = sn;
-                } else {
-                    const int u = ((e >> (k + 1)) << (k - 1)) | ((e & ((1 << k) - 1)) >> 1);
-                    const int col = 64 * k + 4 * u + (e & 1);
-                    strip[col] = nt;
-                    strip[col + 2] = sn;
-                }
-            } else {
-                double sn, c;
-                sincos(th, &sn, &c);
-                const int u = e >> 1;
-                const int col = 320 + 8 * u + (e & 1);
-                strip[col + 0] = static_cast<float>(c * sa);
-                strip[col + 2] = static_cast<float>(-sn * sb);
-                strip[col + 4] = static_cast<float>(sn * sa);
-                strip[col + 6] = static_cast<float>(c * sb);
-            }
-        }
-        __syncthreads();
+    const double th = static_cast<double>(theta[k]);
+    double sn, c;
+    sincos(th, &sn, &c);
+    tw[k] = make_float2(static_cast<float>(c), static_cast<float>(sn));
+    double te = remainder(th, 2.0 * kPi);
+    bool f = false;
+    if (te > 0.5 * kPi) {
+        te -= kPi, f = true;
+    } else if (te < -0.5 * kPi) {
+        te += kPi, f = true;
+    }
+    flip[k] = f ? 1 : 0;
+    prep[k] = make_float4(static_cast<float>(-tan(0.5 * te)), static_cast<float>(sin(te)), static_cast<float>(c),
+                          static_cast<float>(sn));
+}
+
+// sign carried by element i when it enters stage s: the product of the negations of the pairs it
+// belonged to in stages 0..s-1
+__device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int i, int s) {
+    int f = 0;
+    for (int sp = 0; sp < s; ++sp) {
+        const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
+        f ^= flip[sp * (kN / 2) + j];
+    }
+    return f ? -1 : 1;
+}
+
+// Step 2 (one thread per angle): place the constants of pair (s, j) in the tensor-memory image
+// img[role][column], with the role / register / half of the pair's low element in its phase.
+__global__ void __launch_bounds__(256) k_build_image4096(const float4* __restrict__ prep,
+                                                          const uint8_t* __restrict__ flip, float* __restrict__ img) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 12 * (kN / 2)) return;
+    const int s = k / (kN / 2), j = k % (kN / 2);
+    const int lo = ((j >> s) << (s + 1)) | (j & ((1 << s) - 1));
+    const int hi = lo + (1 << s);
+    const int sa = sign_before(flip, lo, s), sb = sign_before(flip, hi, s);
+    const int kk = s & 3;
+    int r, m, h;
+    if (s < 4) {
+        r = ((lo >> 4) & 15) | ((lo >> 9) << 4), m = lo & 15, h = (lo >> 8) & 1;
+    } else if (s < 8) {
+        r = (lo & 15) | ((lo >> 9) << 4), m = (lo >> 4) & 15, h = (lo >> 8) & 1;
+    } else {
+        r = (lo >> 1) & 127, m = lo >> 8, h = lo & 1;
+    }
+    const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
+    const float4 p = prep[k];
+    float* strip = img + r * kCols;
+    if (s < 11) {
+        const float sg = (sa == sb) ? 1.f : -1.f;
+        strip[32 * s + 4 * u + h] = sg * p.x;
+        strip[32 * s + 4 * u + h + 2] = sg * p.y;
+    } else {
+        const int col = 352 + 8 * u + h;
+        strip[col + 0] = p.z * sa;
+        strip[col + 2] = -p.w * sb;
+        strip[col + 4] = p.w * sa;
+        strip[col + 6] = p.z * sb;
     }
 }
 
@@ -411,8 +458,18 @@ static EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-cudaError_t fwdq4096_build_image(const bfq_plan* plan, const float* theta, cudaStream_t st) {
-    f4k::k_build_image4096<<<1, 1024, 0, st>>>(theta, plan->img4096);
+size_t fwdq4096_image_bytes() { return size_t(128) * f4k::kCols * sizeof(float); }
+size_t fwdq4096_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1); }
+
+// Builds the generic (cos, sin) table and the tensor-memory image from the angles (two launches).
+cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st) {
+    const int count = 12 * (f4k::kN / 2);
+    float4* prep = reinterpret_cast<float4*>(plan->prep4096);
+    uint8_t* flip = reinterpret_cast<uint8_t*>(prep + count);
+    f4k::k_prep_angles4096<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, flip);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    f4k::k_build_image4096<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img4096);
     return cudaGetLastError();
 }
 
@@ -420,15 +477,26 @@ bool fwdq4096_available(const bfq_plan* plan) {
     return plan->n == f4k::kN && plan->cc_major == 10 && plan->img4096 != nullptr && encode_tiled() != nullptr;
 }
 
-cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                            uint16_t* scales, cudaStream_t st) {
+template <int G, int CW, int XB>
+static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap, int64_t rows, uint8_t* codes,
+                                  uint16_t* scales, cudaStream_t st) {
+    using S = f4k::Smem<G, XB>;
     static bool attr_set[kMaxDevices] = {false};
+    auto kern = f4k::k_fwdq4096<G, CW, XB>;
     if (!attr_set[plan->device]) {
-        cudaError_t e = cudaFuncSetAttribute(f4k::k_fwdq4096, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             int(f4k::kSmemBytes));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
         if (e != cudaSuccess) return e;
         attr_set[plan->device] = true;
     }
+    const int64_t want = (rows + G - 1) / G;
+    const int grid = int(want < plan->sm_count ? want : plan->sm_count);
+    kern<<<grid, G * f4k::kGroupThreads, S::kBytes, st>>>(tmap, plan->img4096, codes, scales, int(rows),
+                                                          plan->status_word);
+    return cudaGetLastError();
+}
+
+cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                            uint16_t* scales, cudaStream_t st) {
     CUtensorMap tmap;
     const cuuint64_t dims[3] = {64, 64, static_cast<cuuint64_t>(rows)};
     const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ldx) * 2};
@@ -438,11 +506,9 @@ cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, i
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    const int64_t want = (rows + f4k::kPipes - 1) / f4k::kPipes;
-    const int grid = int(want < plan->sm_count ? want : plan->sm_count);
-    f4k::k_fwdq4096<<<grid, f4k::kThreads, f4k::kSmemBytes, st>>>(tmap, plan->img4096, codes, scales, int(rows),
-                                                                   plan->status_word);
-    return cudaGetLastError();
+    // four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest
+    // among the configurations that compile without spills; more groups did not help)
+    return launch_variant<4, 32, 2>(plan, tmap, rows, codes, scales, st);
 }
 
 }  // namespace bfq

@@ -16,7 +16,8 @@ struct bfq_plan {
     int cc_major = 0;
     bool angles_set = false;
     float2* tw = nullptr;        // [log_n][n/2] (cos, sin), fp32
-    float* img4096 = nullptr;    // [128][512] tensor-memory image of the rotation constants (n = 4096 only)
+    float* img4096 = nullptr;    // [128][416] tensor-memory image of the rotation constants (n = 4096 only)
+    void* prep4096 = nullptr;    // staging for the image build: per-angle constants and negation flags (n = 4096 only)
     float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
     int64_t partial_slots = 0;
     int* status_word = nullptr;  // device: non-zero when a bounded wait gave up
