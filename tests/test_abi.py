@@ -1,0 +1,55 @@
+"""Host-side checks of the C ABI that need no GPU: the library builds for sm_100a, loads, exports
+every function include/bfq.h declares, the binding lists the same set, and the entry points that
+can answer without a device (status strings, argument validation that precedes any CUDA call) do."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2509_09679_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "bfq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bfq_[a-z0-9_]+)\s*\(", text)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def test_header_functions_are_exported_and_bound(lib):
+    names = declared_functions()
+    for required in ("bfq_forward_quant", "bfq_inverse", "bfq_backward", "bfq_fold_weights"):
+        assert required in names
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in bfq.h but not exported by libbfq.so"
+    assert sorted(binding.SIGNATURES) == names
+
+
+def test_status_strings(lib):
+    codes = sorted(binding.STATUS_NAMES)
+    assert codes == list(range(min(codes), 1))
+    seen = {lib.bfq_status_string(c).decode() for c in codes}
+    assert len(seen) == len(codes) and "unknown status" not in seen
+    assert lib.bfq_status_string(-99).decode() == "unknown status"
+
+
+def test_validation_that_precedes_any_cuda_call(lib):
+    h = ctypes.c_void_p()
+    assert lib.bfq_plan_create(None, 256, 0, 0) == -1                      # BFQ_ERR_NULL
+    assert lib.bfq_plan_create(ctypes.byref(h), 100, 0, 0) == -2           # not a power of two
+    assert lib.bfq_plan_create(ctypes.byref(h), 8, 0, 0) == -2             # below BFQ_MIN_N
+    assert lib.bfq_plan_create(ctypes.byref(h), 16384, 0, 0) == -2         # above BFQ_MAX_N
+    assert lib.bfq_plan_create(ctypes.byref(h), 256, -1, 0) == -5          # negative max_rows
+    assert h.value is None
+    assert lib.bfq_plan_destroy(None) == -1
+    assert lib.bfq_last_cuda_error(None) == 0
+    assert lib.bfq_backward_partials(None) == 0
+    assert lib.bfq_forward_quant(None, None, 0, 0, 0, 4, None, None, None) == -1
