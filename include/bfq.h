@@ -50,11 +50,13 @@ typedef enum {
     BFQ_ERR_DTYPE = -6,          /* dtype not BFQ_F32 / BFQ_BF16 */
     BFQ_ERR_WORKSPACE = -7,      /* angles not set yet, or plan workspace too small */
     BFQ_ERR_CUDA = -8,           /* a CUDA runtime call failed; see bfq_last_cuda_error */
-    BFQ_ERR_DEVICE_TIMEOUT = -9  /* a bounded device-side wait gave up (reported by bfq_device_status) */
+    BFQ_ERR_DEVICE_TIMEOUT = -9, /* a bounded device-side wait gave up (reported by bfq_device_status) */
+    BFQ_ERR_TOO_LARGE = -10      /* bfq_backward_noalloc: n exceeds BFQ_NOALLOC_MAX_N */
 } bfq_status;
 
 #define BFQ_MIN_N 16
 #define BFQ_MAX_N 8192
+#define BFQ_NOALLOC_MAX_N 1024 /* largest row length bfq_backward_noalloc accepts */
 
 /*
  * Create a plan for row length n on CUDA device `device` (allocates: twiddle tables,
@@ -121,6 +123,30 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
 int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int64_t ldw,
                      int bits, uint8_t* codes, uint16_t* scales_f16, void* WQt, bfq_dtype ot,
                      void* stream);
+
+/*
+ * bfq_backward without any device-memory allocation.  (No counterpart in the paper: this exists for
+ * the library's hosts, not for the method.)
+ *
+ * For callers that must not allocate on the GPU -- a process whose device memory belongs entirely to
+ * a framework's caching allocator, or a latency-critical loop that cannot take the device-wide
+ * synchronisation of cudaMalloc / cudaFree -- and therefore cannot create a plan.  Same result as
+ * bfq_set_angles + bfq_backward (d-theta may differ in rounding: the rows are summed over a different
+ * number of CTAs), same argument meaning, but no plan: theta (device, fp32 [log2 n][n/2]) is passed
+ * directly and the work runs on the CURRENT device.  The cos/sin table and the partial sums live in
+ * an 8 MiB array in the library's device data segment, which every GPU that loads the library holds
+ * until the process exits.  Limits and rules that follow from that:
+ *   - n <= BFQ_NOALLOC_MAX_N (power of two >= BFQ_MIN_N), else BFQ_ERR_TOO_LARGE; rows is unlimited;
+ *   - all calls share the one array: calls that may overlap on a GPU (different streams, different
+ *     threads) race with each other -- serialise them; contents left by an earlier call are harmless
+ *     (each call rewrites the table and zeroes the partial sums it reads);
+ *   - the first call on each device resolves the array's address (cudaGetSymbolAddress) and sets a
+ *     kernel attribute; make that first call before any stream capture begins.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  d-theta is bit-reproducible from call
+ * to call on the same device.
+ */
+int bfq_backward_noalloc(int n, const float* theta, const void* x, bfq_dtype xt, const void* g, bfq_dtype gt,
+                         int64_t rows, int64_t ld, void* dx, bfq_dtype dxt, float* dtheta, void* stream);
 
 /* Synchronises the device and returns BFQ_OK, or BFQ_ERR_DEVICE_TIMEOUT if a kernel of this plan
  * reported a bounded wait that ran out, or BFQ_ERR_CUDA.  (No counterpart in the paper.) */

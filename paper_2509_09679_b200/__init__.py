@@ -5,4 +5,4 @@ draws the seeded synthetic workloads.  Importing the package does not load the
 library; the first call does, and fails loudly if it has not been built.
 """
 from . import synth  # noqa: F401
-from .binding import BFQ_BF16, BFQ_F32, BfqError, Plan, lib  # noqa: F401
+from .binding import BFQ_BF16, BFQ_F32, BfqError, Plan, backward_noalloc, lib  # noqa: F401

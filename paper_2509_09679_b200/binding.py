@@ -18,7 +18,7 @@ BFQ_OK = 0
 STATUS_NAMES = {
     0: "BFQ_OK", -1: "BFQ_ERR_NULL", -2: "BFQ_ERR_UNSUPPORTED_N", -3: "BFQ_ERR_BITS", -4: "BFQ_ERR_ALIGN",
     -5: "BFQ_ERR_STRIDE", -6: "BFQ_ERR_DTYPE", -7: "BFQ_ERR_WORKSPACE", -8: "BFQ_ERR_CUDA",
-    -9: "BFQ_ERR_DEVICE_TIMEOUT",
+    -9: "BFQ_ERR_DEVICE_TIMEOUT", -10: "BFQ_ERR_TOO_LARGE",
 }
 
 # name -> (restype, argtypes); must list every symbol include/bfq.h declares
@@ -36,6 +36,7 @@ SIGNATURES = {
     "bfq_last_cuda_error": (_i, [_p]),
     "bfq_status_string": (ctypes.c_char_p, [_i]),
     "bfq_backward_partials": (_i, [_p]),
+    "bfq_backward_noalloc": (_i, [_i, _p, _p, _i, _p, _i, _i64, _i64, _p, _i, _p, _p]),
 }
 
 _lib = None
@@ -172,3 +173,24 @@ class Plan:
 
     def backward_partials(self) -> int:
         return int(lib().bfq_backward_partials(self._h))
+
+
+def backward_noalloc(theta: torch.Tensor, x: torch.Tensor, g: torch.Tensor, dx: torch.Tensor | None,
+                     dtheta: torch.Tensor):
+    """bfq_backward_noalloc: the backward pass without a plan and without any device allocation by the
+    library (for hosts that must not call cudaMalloc; row length at most 1024).  Every buffer,
+    outputs included, is the caller's; pass dx=None to skip dL/dx.  Runs on x's device, which is
+    made current for the call.  Calls share one fixed scratch array per GPU: do not overlap them."""
+    n = x.shape[1]
+    rows, ld = _rows(x, n)
+    rows_g, ld_g = _rows(g, n)
+    if rows_g != rows or ld_g != ld:
+        raise ValueError("x and g must have the same shape and row stride")
+    if dx is not None and _rows(dx, n) != (rows, ld):
+        raise ValueError("dx must have the shape and row stride of x")
+    with torch.cuda.device(x.device):
+        _check(lib().bfq_backward_noalloc(n, theta.data_ptr(), x.data_ptr(), _dt(x), g.data_ptr(), _dt(g), rows, ld,
+                                          dx.data_ptr() if dx is not None else None,
+                                          _dt(dx) if dx is not None else BFQ_F32, dtheta.data_ptr(), _stream(x)),
+               "bfq_backward_noalloc")
+    return dx, dtheta

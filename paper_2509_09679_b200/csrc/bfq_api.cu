@@ -366,6 +366,7 @@ const char* bfq_status_string(int status) {
         case BFQ_ERR_WORKSPACE: return "angles not set or workspace too small";
         case BFQ_ERR_CUDA: return "CUDA runtime error";
         case BFQ_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
+        case BFQ_ERR_TOO_LARGE: return "row length exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
