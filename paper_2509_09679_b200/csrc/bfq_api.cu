@@ -193,6 +193,9 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess) e = cudaMalloc(&plan->partial, size_t(plan->partial_slots) * angles * sizeof(float));
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img4096, fwdq4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->prep4096, fwdq4096_prep_bytes());
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_b4096, bwd4096_image_bytes());
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->dsign4096, bwd4096_dsign_bytes());
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->gsign4096, bwd4096_gsign_bytes());
     if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -200,6 +203,9 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
         cudaFree(plan->tw);
         cudaFree(plan->img4096);
         cudaFree(plan->prep4096);
+        cudaFree(plan->img_b4096);
+        cudaFree(plan->dsign4096);
+        cudaFree(plan->gsign4096);
         cudaFree(plan->partial);
         cudaFree(plan->status_word);
         delete plan;
@@ -216,6 +222,9 @@ int bfq_plan_destroy(bfq_plan* plan) {
     cudaFree(plan->tw);
     cudaFree(plan->img4096);
     cudaFree(plan->prep4096);
+    cudaFree(plan->img_b4096);
+    cudaFree(plan->dsign4096);
+    cudaFree(plan->gsign4096);
     cudaFree(plan->partial);
     cudaFree(plan->status_word);
     delete plan;
@@ -237,6 +246,7 @@ int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
     }
     if (e != cudaSuccess) return cuda_fail(plan, e);
     plan->angles_set = true;
+    plan->bwd_tables_valid = false;
     return BFQ_OK;
 }
 
@@ -326,6 +336,16 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (rows == 0) {
         cudaError_t e = cudaMemsetAsync(dtheta, 0, sizeof(float) * size_t(plan->log_n) * (plan->n / 2), st);
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
+    if (xt == BFQ_BF16 && gt == BFQ_BF16 && (dx == nullptr || dxt == BFQ_BF16) && rows < (int64_t(1) << 31) - 1 &&
+        !env_flag("BFQ_GENERIC_ONLY") && bwd4096_available(plan)) {
+        cudaError_t e = cudaSuccess;
+        if (!plan->bwd_tables_valid) {  // built on first use after bfq_set_angles, on the caller's stream
+            e = bwd4096_build_tables(plan, st);
+            plan->bwd_tables_valid = (e == cudaSuccess);
+        }
+        if (e == cudaSuccess) e = bwd4096_launch(plan, x, g, rows, ld, dx, dtheta, st);
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     BackwardParams p{};

@@ -1,0 +1,549 @@
+// Tuned backward pass for n = 4096 bf16 rows on sm_100a:  dx = Q^T g  and  d-theta summed over rows.
+//
+// One persistent CTA of 128 threads per SM works on two rows at a time (row pair p of the CTA is rows
+// 2p, 2p+1).  The thread roles, phases and regrouping layouts are those of the forward kernel
+// (bfq_n4096.cuh).  Per row pair:
+//   1. y = Q x with the three-shear constants, all 12 stages, in the tracked-sign basis sigma.
+//   2. y and g are moved to the basis sigma * (-1)^popcount(index).  Any two indices that a stage pairs
+//      differ in one bit, so in this basis the high element of every pair of every stage is negated
+//      relative to the low one, and there the inverse of a stage's rotation is the SAME three shears
+//      with the SAME constants.  The reverse walk therefore reuses the forward tables unchanged.
+//   3. for s = 11..0:  d[s][pair] += g_hi*y_lo - g_lo*y_hi on the stage's outputs (the stage-output
+//      form of g^T (dG/dtheta) z; its sign in this basis is fixed per pair and applied when the sums
+//      are written out), then y and g are both un-rotated.  After stage 0, g is dx up to the parity sign.
+// d-theta accumulators are owned by thread role (no atomics): stages 0-7 in the tensor-memory columns the
+// constants leave free, stages 8-11 in shared memory.  Each CTA walks its row pairs in a fixed order and
+// writes its sums to its own slot; a second kernel adds the slots in index order: bit-reproducible.
+#include "bfq_fast.h"
+#include "bfq_generic.cuh"
+#include "bfq_n4096.cuh"
+
+namespace bfq {
+namespace b4k {
+using namespace ptx;
+using namespace f4k;
+
+constexpr int kThreads = 128;
+constexpr int kSlots = 2;                    // TMA ring depth (row pairs)
+constexpr int kConstCols = 384;              // 12 stages x 32 words
+constexpr int kAccCol = 384;                 // accumulators of stages 0..7: 16 columns each
+constexpr uint32_t kPairBytes = 4 * kRowBytes;  // x0, x1, g0, g1
+
+struct Smem {
+    static constexpr uint32_t kInOff = 0;                                  // [kSlots][4][kRowBytes]
+    static constexpr uint32_t kExOff = kInOff + kSlots * kPairBytes;       // [4][kExBytes]: y0, y1, g0, g1
+    static constexpr uint32_t kAccOff = kExOff + 4 * kExBytes;             // [16][128] float4: stages 8..11
+    static constexpr uint32_t kSgnOff = kAccOff + 16 * kThreads * 16;      // [4][128] uint4: sign words of g
+    static constexpr uint32_t kBarOff = kSgnOff + 4 * kThreads * 16;       // mbarriers [kSlots]
+    static constexpr uint32_t kTmemOff = kBarOff + 8 * kSlots;
+    static constexpr uint32_t kUsed = kTmemOff + 16;
+    static constexpr uint32_t kBytes = kUsed + 1024;
+};
+
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+struct Addr {
+    uint32_t w1, r1, w2, r2;  // per-thread byte offsets inside a regrouping buffer (forward write / read sides)
+    uint32_t ex;              // base of the four regrouping buffers
+};
+
+// ---- regroupings: forward direction (phase 1 -> 2 -> 3) and back, one row array at a time -------------
+__device__ __forceinline__ void fwd1_store(const u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) sts64(buf + a.w1 + ex1_wr_local(m), P[m]);
+}
+__device__ __forceinline__ void fwd1_load(u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(buf + a.r1 + ex1_rd_local(m));
+}
+__device__ __forceinline__ void fwd2_store(const u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+        uint32_t lo, hi;
+        unpack2u(P[m], lo, hi);
+        sts32(buf + a.w2 + ex2_wr_local(m, 0), lo);
+        sts32(buf + a.w2 + ex2_wr_local(m, 1), hi);
+    }
+}
+__device__ __forceinline__ void fwd2_load(u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(buf + a.r2 + ex2_rd_local(m));
+}
+// back from phase 3 to phase 2: the phase-3 owner stores whole packed registers where it read them,
+// the phase-2 owner reads scalars where it wrote them
+__device__ __forceinline__ void rev2_store(const u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) sts64(buf + a.r2 + ex2_rd_local(m), P[m]);
+}
+__device__ __forceinline__ void rev2_load(u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m)
+        P[m] = pack2u(lds32(buf + a.w2 + ex2_wr_local(m, 0)), lds32(buf + a.w2 + ex2_wr_local(m, 1)));
+}
+__device__ __forceinline__ void rev1_store(const u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) sts64(buf + a.r1 + ex1_rd_local(m), P[m]);
+}
+__device__ __forceinline__ void rev1_load(u64 (&P)[16], uint32_t buf, const Addr& a) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(buf + a.w1 + ex1_wr_local(m));
+}
+
+// ---- d-theta of four pairs (U0..U0+3) of local stage K, both rows:  A[i] += g_hi*y_lo - g_lo*y_hi ------
+template <int K, int U0>
+__device__ __forceinline__ void dtheta4(u64 (&A)[4], const u64 (&Y0)[16], const u64 (&Y1)[16], const u64 (&G0)[16],
+                                        const u64 (&G1)[16]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        u64 neg = mul2(G0[m_lo], Y0[m_hi]);
+        neg = fma2(G1[m_lo], Y1[m_hi], neg);
+        u64 pos = fma2(G0[m_hi], Y0[m_lo], A[i]);
+        pos = fma2(G1[m_hi], Y1[m_lo], pos);
+        A[i] = sub2(pos, neg);
+    }
+}
+
+struct Ctx {
+    Addr a;
+    uint32_t tlane;     // tensor-memory address of this thread's lane, column 0
+    uint32_t acc_smem;  // this thread's first float4 of the shared-memory accumulators
+};
+
+// ---- forward recompute: 24 chunks of 16 constants (two per stage), both rows ---------------------------
+// Chunk C is in Tcur; the next chunk (or, after the last one, the first chunk of the reverse walk) is
+// requested right after the wait.
+template <int C>
+__device__ __forceinline__ void fwd_chunks(u64 (&X0)[16], u64 (&X1)[16], uint32_t (&Tcur)[16], uint32_t (&Tnext)[16],
+                                           const Ctx& cx) {
+    constexpr int s = C / 2, K = s & 3, U0 = 4 * (C & 1);
+    tmem_wait_ld16(Tcur);
+    if constexpr (C + 1 < 24) {
+        tmem_ld16(cx.tlane + 16 * (C + 1), Tnext);
+    } else {
+        tmem_ld16(cx.tlane + 32 * 11, Tnext);
+    }
+    stage_lift<K, U0, 4, 16>(X0, Tcur);
+    stage_lift<K, U0, 4, 16>(X1, Tcur);
+    if constexpr (C == 7) {
+        __syncwarp();  // the half-warp's reads of the previous row pair's last regrouping are done
+        fwd1_store(X0, cx.a.ex + 0 * kExBytes, cx.a);
+        fwd1_store(X1, cx.a.ex + 1 * kExBytes, cx.a);
+        __syncwarp();
+        fwd1_load(X0, cx.a.ex + 0 * kExBytes, cx.a);
+        fwd1_load(X1, cx.a.ex + 1 * kExBytes, cx.a);
+    }
+    if constexpr (C == 15) {
+        bar_sync(1, kThreads);  // every warp is past its reads of buffers 2 and 3 for the previous row pair
+        fwd2_store(X0, cx.a.ex + 2 * kExBytes, cx.a);
+        fwd2_store(X1, cx.a.ex + 3 * kExBytes, cx.a);
+        bar_sync(1, kThreads);
+        fwd2_load(X0, cx.a.ex + 2 * kExBytes, cx.a);
+        fwd2_load(X1, cx.a.ex + 3 * kExBytes, cx.a);
+    }
+    if constexpr (C + 1 < 24) fwd_chunks<C + 1>(X0, X1, Tnext, Tcur, cx);
+}
+
+// ---- reverse walk: step I handles half c = I & 1 of stage s = 11 - I / 2 ---------------------------------
+template <int I>
+struct RevStep {
+    static constexpr int s = 11 - I / 2, c = I & 1, K = s & 3, U0 = 4 * c;
+    static constexpr uint32_t kTCol = 32 * s + 16 * c;
+    static constexpr bool kAccInTmem = s < 8;
+    static constexpr uint32_t kAccCol = b4k::kAccCol + 16 * s + 8 * c;       // stages 0..7
+    static constexpr uint32_t kAccSmem = ((s - 8) * 4 + 2 * c) * kThreads * 16;  // stages 8..11: two float4
+};
+
+template <int I, class F>
+__device__ __forceinline__ void rev_steps(u64 (&Y0)[16], u64 (&Y1)[16], u64 (&G0)[16], u64 (&G1)[16],
+                                          uint32_t (&Tcur)[16], uint32_t (&Tnext)[16], uint32_t (&Acur)[8],
+                                          uint32_t (&Anext)[8], const Ctx& cx, F&& after_phase3) {
+    using S = RevStep<I>;
+    if constexpr (S::kAccInTmem) {
+        tmem_wait_ld16_8(Tcur, Acur);
+    } else {
+        tmem_wait_ld16(Tcur);
+        const uint4 a0 = lds128(cx.acc_smem + S::kAccSmem), a1 = lds128(cx.acc_smem + S::kAccSmem + kThreads * 16);
+        Acur[0] = a0.x, Acur[1] = a0.y, Acur[2] = a0.z, Acur[3] = a0.w;
+        Acur[4] = a1.x, Acur[5] = a1.y, Acur[6] = a1.z, Acur[7] = a1.w;
+    }
+    if constexpr (I + 1 < 24) {
+        using N = RevStep<I + 1>;
+        tmem_ld16(cx.tlane + N::kTCol, Tnext);
+        if constexpr (N::kAccInTmem) tmem_ld8(cx.tlane + N::kAccCol, Anext);
+    }
+    {
+        u64 A[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) A[i] = pack2u(Acur[2 * i], Acur[2 * i + 1]);
+        dtheta4<S::K, S::U0>(A, Y0, Y1, G0, G1);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack2u(A[i], Acur[2 * i], Acur[2 * i + 1]);
+    }
+    if constexpr (S::kAccInTmem) {
+        tmem_st8(cx.tlane + S::kAccCol, Acur);
+    } else {
+        sts128(cx.acc_smem + S::kAccSmem, make_uint4(Acur[0], Acur[1], Acur[2], Acur[3]));
+        sts128(cx.acc_smem + S::kAccSmem + kThreads * 16, make_uint4(Acur[4], Acur[5], Acur[6], Acur[7]));
+    }
+    if constexpr (S::s > 0) {  // y below stage 0 is x again: not needed
+        stage_lift<S::K, S::U0, 4, 16>(Y0, Tcur);
+        stage_lift<S::K, S::U0, 4, 16>(Y1, Tcur);
+    }
+    stage_lift<S::K, S::U0, 4, 16>(G0, Tcur);
+    stage_lift<S::K, S::U0, 4, 16>(G1, Tcur);
+    if constexpr (I == 7) {  // phase 3 -> phase 2, across warps
+        bar_sync(1, kThreads);  // every warp is past its forward reads of buffers 2 and 3
+        rev2_store(Y0, cx.a.ex + 0 * kExBytes, cx.a);
+        rev2_store(Y1, cx.a.ex + 1 * kExBytes, cx.a);
+        rev2_store(G0, cx.a.ex + 2 * kExBytes, cx.a);
+        rev2_store(G1, cx.a.ex + 3 * kExBytes, cx.a);
+        bar_sync(1, kThreads);
+        after_phase3();  // all reads of the input slot are done: the next row pair may be requested
+        rev2_load(Y0, cx.a.ex + 0 * kExBytes, cx.a);
+        rev2_load(Y1, cx.a.ex + 1 * kExBytes, cx.a);
+        rev2_load(G0, cx.a.ex + 2 * kExBytes, cx.a);
+        rev2_load(G1, cx.a.ex + 3 * kExBytes, cx.a);
+    }
+    if constexpr (I == 15) {  // phase 2 -> phase 1, inside each half-warp, but the buffers were read across warps
+        bar_sync(1, kThreads);
+        rev1_store(Y0, cx.a.ex + 0 * kExBytes, cx.a);
+        rev1_store(Y1, cx.a.ex + 1 * kExBytes, cx.a);
+        rev1_store(G0, cx.a.ex + 2 * kExBytes, cx.a);
+        rev1_store(G1, cx.a.ex + 3 * kExBytes, cx.a);
+        __syncwarp();
+        rev1_load(Y0, cx.a.ex + 0 * kExBytes, cx.a);
+        rev1_load(Y1, cx.a.ex + 1 * kExBytes, cx.a);
+        rev1_load(G0, cx.a.ex + 2 * kExBytes, cx.a);
+        rev1_load(G1, cx.a.ex + 3 * kExBytes, cx.a);
+    }
+    if constexpr (I + 1 < 24) rev_steps<I + 1>(Y0, Y1, G0, G1, Tnext, Tcur, Anext, Acur, cx, after_phase3);
+}
+
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// element index of (phase P, role t, packed register m, half h)
+__device__ __forceinline__ int elem_of(int P, int t, int m, int h) {
+    if (P == 0) return m | ((t & 15) << 4) | (h << 8) | ((t >> 4) << 9);
+    if (P == 1) return (t & 15) | (m << 4) | (h << 8) | ((t >> 4) << 9);
+    return h | (t << 1) | (m << 8);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap gmap,
+          const float* __restrict__ img, const uint32_t* __restrict__ gsign, const int8_t* __restrict__ dsign,
+          __nv_bfloat16* __restrict__ dx, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status) {
+    using S = Smem;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = threadIdx.x;  // role 0..127; warp = tensor-memory lane quarter
+
+    if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
+    if (threadIdx.x < kSlots) {
+        mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
+        mbar_init_fence();
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
+
+    Ctx cx;
+    cx.tlane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    cx.acc_smem = sbase + S::kAccOff + t * 16;
+    {
+        const uint32_t t4 = (t >> 4) & 1, t5 = (t >> 5) & 1, t6 = (t >> 6) & 1;
+        cx.a.ex = sbase + S::kExOff;
+        cx.a.w1 = 4u * (2u * (t & 15) + 32u * (t >> 4));
+        cx.a.r1 = 4u * (258u * (t & 15) + 32u * (t >> 4));
+        cx.a.w2 = 4u * ((t & 15) + 2064u * t4 + 512u * t5 + 1024u * t6);
+        cx.a.r2 = 4u * (2u * (t & 15) + 32u * (t >> 4));
+    }
+
+    const int pairs = (rows + 1) / 2;
+    const int first = blockIdx.x;
+    const int stride = gridDim.x;
+    const int count = first < pairs ? (pairs - first + stride - 1) / stride : 0;
+    const uint32_t in_base = sbase + S::kInOff;
+    const uint32_t bar_base = sbase + S::kBarOff;
+
+    // a row index past the end is legal for the tensor map: the tile is filled with zeros
+    auto request = [&](int k) {
+        const int slot = k & 1;
+        const int r0 = 2 * (first + k * stride);
+        const uint32_t dst = in_base + slot * kPairBytes, bar = bar_base + 8 * slot;
+        mbar_expect_tx(bar, kPairBytes);
+        tma_load_3d(dst + 0 * kRowBytes, &xmap, 0, 0, r0, bar);
+        tma_load_3d(dst + 1 * kRowBytes, &xmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(dst + 2 * kRowBytes, &gmap, 0, 0, r0, bar);
+        tma_load_3d(dst + 3 * kRowBytes, &gmap, 0, 0, r0 + 1, bar);
+    };
+    if (t == 0) {
+        for (int k = 0; k < kSlots && k < count; ++k) request(k);
+    }
+    // constants into tensor memory, accumulators to zero, sign words of g into shared memory
+    {
+        const float4* src = reinterpret_cast<const float4*>(img + t * kConstCols);
+        for (int c = 0; c < kConstCols; c += 16) {
+            uint32_t v[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 f = __ldg(src + (c >> 2) + i);
+                v[4 * i + 0] = __float_as_uint(f.x), v[4 * i + 1] = __float_as_uint(f.y);
+                v[4 * i + 2] = __float_as_uint(f.z), v[4 * i + 3] = __float_as_uint(f.w);
+            }
+            tmem_st16(cx.tlane + c, v);
+        }
+        uint32_t z[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) z[i] = 0u;
+        for (int c = kAccCol; c < 512; c += 16) tmem_st16(cx.tlane + c, z);
+        tmem_wait_st();
+        for (int q = 0; q < 16; ++q) sts128(cx.acc_smem + q * kThreads * 16, make_uint4(0u, 0u, 0u, 0u));
+        const uint4* gs = reinterpret_cast<const uint4*>(gsign);
+        for (int q = 0; q < 4; ++q) sts128(sbase + S::kSgnOff + (q * kThreads + t) * 16, __ldg(gs + q * kThreads + t));
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+
+    // x tile, phase-1 ownership (as in the forward kernel)
+    const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+    const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+    // g tile, phase-3 ownership: the 32-bit word of elements 2t + 256m, 2t + 256m + 1 is word t & 3 of 16-byte
+    // chunk (t & 31) >> 2 of 128-byte line (t >> 5) + 4m; the swizzle moves the chunk to chunk ^ (line & 7)
+    const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
+    const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
+    const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
+    // parity of the role: popcount(t) & 1
+    const uint32_t par_t = __popc(t) & 1;
+    const uint32_t sgn_a = par_t ? 0x80000000u : 0u, sgn_b = par_t ? 0u : 0x80000000u;
+
+    u64 Y0[16], Y1[16], G0[16], G1[16];
+    uint32_t T0[16], T1[16], A0[8], A1[8];
+
+    for (int k = 0; k < count; ++k) {
+        const int slot = k & 1;
+        const int r0 = 2 * (first + k * stride);
+        tmem_ld16(cx.tlane, T0);
+        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+        const uint32_t tile = in_base + slot * kPairBytes;
+        // ---- x rows -> packed fp32, phase 1 ----
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            u64(&X)[16] = r == 0 ? Y0 : Y1;
+            const uint32_t src = tile + r * kRowBytes + in_line;
+            uint4 w[2][2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) w[h][c] = lds128(src + 512u * h + (in_x ^ ((c | (h << 2)) << 4)));
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const uint32_t a[4] = {w[0][c].x, w[0][c].y, w[0][c].z, w[0][c].w};
+                const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    X[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
+                    X[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
+                }
+            }
+        }
+        fwd_chunks<0>(Y0, Y1, T0, T1, cx);  // leaves the first reverse chunk requested in T0
+
+        // ---- y to the parity basis; g rows -> packed fp32 in the same basis, phase 3 ----
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+            const bool odd = (__builtin_popcount(m) & 1) != 0;  // compile-time after unrolling
+            const u64 mask = odd ? pack2u(sgn_b, sgn_a) : pack2u(sgn_a, sgn_b);
+            Y0[m] ^= mask;
+            Y1[m] ^= mask;
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            u64(&G)[16] = r == 0 ? G0 : G1;
+            const uint32_t src = tile + (2 + r) * kRowBytes;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 sw = lds128(sbase + S::kSgnOff + (q * kThreads + t) * 16);
+                const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int m = 4 * q + i;
+                    const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
+                    G[m] = pack2u(w << 16, w & 0xFFFF0000u);
+                }
+            }
+        }
+        rev_steps<0>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [&]() {
+            if (t == 0 && k + kSlots < count) request(k + kSlots);
+        });
+
+        // ---- dx = parity sign * g, bf16, phase-1 ownership: two runs of 16 elements per row ----
+        if (dx != nullptr) {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                if (r0 + r < rows) {
+                    const u64(&G)[16] = r == 0 ? G0 : G1;
+                    __nv_bfloat16* row = dx + static_cast<int64_t>(r0 + r) * ld + 16 * (t & 15) + 512 * (t >> 4);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            uint32_t lo0, hi0, lo1, hi1;
+                            unpack2u(G[2 * j], lo0, hi0);
+                            unpack2u(G[2 * j + 1], lo1, hi1);
+                            const float e0 = __uint_as_float(h ? hi0 : lo0), e1 = __uint_as_float(h ? hi1 : lo1);
+                            // elements m = 2j, 2j+1 of half h: parity popcount(2j) ^ h ^ popcount(t), opposite for 2j+1
+                            const bool odd_c = ((__builtin_popcount(2 * j) + h) & 1) != 0;
+                            const uint32_t neg_lo = odd_c ? (sgn_b >> 16) : (sgn_a >> 16);  // bit 15: element 2j
+                            const uint32_t neg_hi = odd_c ? sgn_a : sgn_b;                  // bit 31: element 2j+1
+                            w[j] = cvt_bf16x2(e0, e1) ^ (neg_lo | neg_hi);
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(row + 256 * h);
+                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    }
+                }
+            }
+        }
+        tmem_wait_st();  // this row pair's accumulator stores land before the next pair reloads them
+    }
+
+    // ---- this CTA's sums -> its slot of the partial sums, with the sign of the basis undone ----
+    {
+        float* out = partial + static_cast<int64_t>(blockIdx.x) * (12 * (kN / 2));
+        for (int s = 0; s < 12; ++s) {
+            const int K = s & 3, P = s >> 2;
+            for (int c = 0; c < 2; ++c) {
+                uint32_t a[8];
+                if (s < 8) {
+                    tmem_ld8(cx.tlane + kAccCol + 16 * s + 8 * c, a);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                } else {
+                    const uint32_t base = cx.acc_smem + ((s - 8) * 4 + 2 * c) * kThreads * 16;
+                    const uint4 v0 = lds128(base), v1 = lds128(base + kThreads * 16);
+                    a[0] = v0.x, a[1] = v0.y, a[2] = v0.z, a[3] = v0.w, a[4] = v1.x, a[5] = v1.y, a[6] = v1.z, a[7] = v1.w;
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int u = 4 * c + (e >> 1), h = e & 1;
+                    const int m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1));
+                    const int lo = elem_of(P, t, m_lo, h);
+                    const int j = ((lo >> (s + 1)) << s) | (lo & ((1 << s) - 1));
+                    out[s * (kN / 2) + j] = __uint_as_float(a[e]) * static_cast<float>(dsign[s * (kN / 2) + j]);
+                }
+            }
+        }
+    }
+    tmem_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc512(tmem_base);
+}
+
+// ---- tables ---------------------------------------------------------------------------------------------------
+// One thread per angle: the three-shear constants of pair (s, j), negated when its two elements carry
+// opposite signs, at the place the owning role reads them; and the sign that turns the accumulated
+// g_hi*y_lo - g_lo*y_hi of the parity basis into d-theta.
+__global__ void __launch_bounds__(256) k_build_image_bwd4096(const float4* __restrict__ prep,
+                                                              const uint8_t* __restrict__ flip,
+                                                              float* __restrict__ img, int8_t* __restrict__ dsign) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 12 * (kN / 2)) return;
+    const int s = k / (kN / 2), j = k % (kN / 2);
+    const int lo = ((j >> s) << (s + 1)) | (j & ((1 << s) - 1));
+    const int hi = lo + (1 << s);
+    const int sa = sign_before(flip, lo, s), sb = sign_before(flip, hi, s);
+    const int kk = s & 3;
+    int r, m, h;
+    if (s < 4) {
+        r = ((lo >> 4) & 15) | ((lo >> 9) << 4), m = lo & 15, h = (lo >> 8) & 1;
+    } else if (s < 8) {
+        r = (lo & 15) | ((lo >> 9) << 4), m = (lo >> 4) & 15, h = (lo >> 8) & 1;
+    } else {
+        r = (lo >> 1) & 127, m = lo >> 8, h = lo & 1;
+    }
+    const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
+    const float4 p = prep[k];
+    const float sg = (sa == sb) ? 1.f : -1.f;
+    float* strip = img + r * kConstCols;
+    strip[32 * s + 4 * u + h] = sg * p.x;
+    strip[32 * s + 4 * u + h + 2] = sg * p.y;
+    dsign[k] = static_cast<int8_t>(-(sa * sb));
+}
+
+// One thread per 32-bit word of a bf16 g row in phase-3 ownership (role t, register m): bit 15 / bit 31 set
+// when element 2t + 256m / its neighbour must be negated to enter the basis sigma(after stage 11) * parity.
+__global__ void __launch_bounds__(256) k_build_gsign4096(const uint8_t* __restrict__ flip, uint32_t* __restrict__ gsign) {
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w >= 16 * kThreads) return;
+    const int m = (w / (4 * kThreads)) * 4 + (w & 3), t = (w >> 2) % kThreads;  // layout [m / 4][t][m % 4]
+    const int e = 2 * t + 256 * m;
+    const int s0 = sign_before(flip, e, 12) * ((__popc(e) & 1) ? -1 : 1);
+    const int s1 = sign_before(flip, e + 1, 12) * ((__popc(e + 1) & 1) ? -1 : 1);
+    gsign[w] = (s0 < 0 ? 0x00008000u : 0u) | (s1 < 0 ? 0x80000000u : 0u);
+}
+
+}  // namespace b4k
+
+// ---- host side ---------------------------------------------------------------------------------------------
+size_t bwd4096_image_bytes() { return size_t(128) * b4k::kConstCols * sizeof(float); }
+size_t bwd4096_dsign_bytes() { return size_t(12) * (f4k::kN / 2); }
+size_t bwd4096_gsign_bytes() { return size_t(16) * b4k::kThreads * sizeof(uint32_t); }
+
+bool bwd4096_available(const bfq_plan* plan) {
+    return plan->n == f4k::kN && plan->cc_major == 10 && plan->img_b4096 != nullptr && plan->prep4096 != nullptr &&
+           plan->partial_slots >= plan->sm_count && encode_tiled() != nullptr;
+}
+
+// Builds the backward tables from the staging area bfq_set_angles filled (two launches).
+cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st) {
+    const int count = 12 * (f4k::kN / 2);
+    const float4* prep = reinterpret_cast<const float4*>(plan->prep4096);
+    const uint8_t* flip = reinterpret_cast<const uint8_t*>(prep + count);
+    b4k::k_build_image_bwd4096<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img_b4096, plan->dsign4096);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    b4k::k_build_gsign4096<<<(16 * b4k::kThreads + 255) / 256, 256, 0, st>>>(flip, plan->gsign4096);
+    return cudaGetLastError();
+}
+
+cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
+                           float* dtheta, cudaStream_t st) {
+    static bool attr_set[kMaxDevices] = {false};
+    if (!attr_set[plan->device]) {
+        cudaError_t e = cudaFuncSetAttribute(b4k::k_bwd4096, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             int(b4k::Smem::kBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[plan->device] = true;
+    }
+    CUtensorMap xmap, gmap;
+    if (!encode_row_map(&xmap, x, rows, ld) || !encode_row_map(&gmap, g, rows, ld)) return cudaErrorInvalidValue;
+    const int64_t pairs = (rows + 1) / 2;
+    const int grid = int(pairs < plan->sm_count ? pairs : plan->sm_count);
+    b4k::k_bwd4096<<<grid, b4k::kThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
+                                                                   plan->dsign4096, static_cast<__nv_bfloat16*>(dx), ld,
+                                                                   plan->partial, int(rows), plan->status_word);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int count = 12 * (f4k::kN / 2);
+    k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid, count, dtheta);
+    plan->last_backward_partials = grid;
+    return cudaGetLastError();
+}
+
+}  // namespace bfq

@@ -16,4 +16,13 @@ cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaSt
 cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st);
 
+// n = 4096, bf16 x / g / dx: backward with tensor-memory constants and accumulators
+size_t bwd4096_image_bytes();
+size_t bwd4096_dsign_bytes();
+size_t bwd4096_gsign_bytes();
+bool bwd4096_available(const bfq_plan* plan);
+cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st);
+cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
+                           float* dtheta, cudaStream_t st);
+
 }  // namespace bfq

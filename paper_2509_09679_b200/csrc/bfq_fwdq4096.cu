@@ -26,24 +26,12 @@
 //  * Rows arrive by TMA (128-byte swizzled tiles, two-deep ring per group, mbarrier completion).
 //    The per-row absmax is a warp reduction plus one step across the group's four warps; INT4
 //    codes are produced with the magic-number rounding trick, one byte per packed register.
-#include <cuda.h>
-#include <cuda_runtime.h>
-
 #include "bfq_fast.h"
 #include "bfq_generic.cuh"
-#include "bfq_ptx.cuh"
+#include "bfq_n4096.cuh"
 
 namespace bfq {
 namespace f4k {
-using namespace ptx;
-
-constexpr int kN = 4096;
-constexpr int kGroupThreads = 128;
-constexpr int kInSlots = 2;                  // TMA ring depth per group
-constexpr uint32_t kRowBytes = kN * 2;       // one bf16 row
-constexpr uint32_t kExWords = 4128;          // padded fp32 row (see the layouts below)
-constexpr uint32_t kExBytes = kExWords * 4;
-constexpr int kCols = 416;                   // tensor-memory columns in use
 
 // G row groups per CTA; XB regrouping buffers per group (2: one per regrouping; 1: shared, at the
 // price of one more barrier per row)
@@ -58,65 +46,6 @@ struct Smem {
     static constexpr uint32_t kBytes = kUsed + 1024;  // slack for the 1024-byte alignment of the TMA tiles
 };
 
-__device__ __forceinline__ uint4 lds128(uint32_t a) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ u64 lds64(uint32_t a) {
-    u64 v;
-    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-__device__ __forceinline__ void sts64(uint32_t a, u64 v) {
-    asm volatile("st.shared.b64 [%0], %1;" ::"r"(a), "l"(v) : "memory");
-}
-
-// ---- element held by role t, packed register m, half h in each phase -----------------------------------
-//   phase 1: i = m | (t & 15) << 4 | h << 8 | (t >> 4) << 9
-//   phase 2: i = (t & 15) | m << 4 | h << 8 | (t >> 4) << 9
-//   phase 3: i = h | t << 1 | m << 8
-// ---- shared-memory layouts of the two regroupings (word addresses; i = element index bits) -----------
-// first:   A1 = i8 + 2*(i4..i7) + 32*(i9 + 2*i10 + 4*i11) + 258*(i0..i3)
-// second:  A2 = (i0..i4) + 16*i9 + 32*(i5 + 2*i6 + 4*i7 + 8*i8 + 16*i10 + 32*i11 + 64*i9)
-// Both are injective into [0, kExWords); a half-warp's 16 64-bit accesses and a warp's 32 scalar
-// stores each cover the 32 banks exactly once.  In the first, the words a thread writes are read by
-// the 16 lanes of its own half-warp only.
-__device__ __forceinline__ constexpr uint32_t ex1_wr_local(int m) { return 4u * 258u * m; }
-__device__ __forceinline__ constexpr uint32_t ex1_rd_local(int m) { return 4u * 2u * m; }
-__device__ __forceinline__ constexpr uint32_t ex2_wr_local(int m, int h) {
-    return 4u * (16u * (m & 1) + 32u * (m >> 1) + 256u * h);
-}
-__device__ __forceinline__ constexpr uint32_t ex2_rd_local(int m) {
-    return 4u * (256u * (m & 1) + 2064u * ((m >> 1) & 1) + 512u * ((m >> 2) & 1) + 1024u * ((m >> 3) & 1));
-}
-
-// ---- one stage on the registers of a thread ---------------------------------------------------------
-// Local stage K pairs packed registers m and m | 2^K; both fp32 lanes rotate at once.  T holds
-// (nt, nt', sn, sn') for NU consecutive pairs starting at pair U0.  The three shears are issued level
-// by level so that dependent instructions are NU apart.
-template <int K, int U0, int NU, int CW>
-__device__ __forceinline__ void stage_lift(u64 (&P)[16], const uint32_t (&T)[CW]) {
-    static_assert(4 * NU <= CW, "chunk too small");
-#pragma unroll
-    for (int i = 0; i < NU; ++i) {
-        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
-        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), P[m_hi], P[m_lo]);
-    }
-#pragma unroll
-    for (int i = 0; i < NU; ++i) {
-        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
-        P[m_hi] = fma2(pack2u(T[4 * i + 2], T[4 * i + 3]), P[m_lo], P[m_hi]);
-    }
-#pragma unroll
-    for (int i = 0; i < NU; ++i) {
-        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
-        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), P[m_hi], P[m_lo]);
-    }
-}
 // last stage (local bit 3 of phase 3): out_lo = k1*a + k2*b, out_hi = k3*a + k4*b for pairs U0..U0+NU-1
 template <int U0, int NU, int CW>
 __device__ __forceinline__ void stage_general(u64 (&P)[16], const uint32_t (&T)[CW]) {
@@ -390,17 +319,6 @@ __global__ void __launch_bounds__(256) k_prep_angles4096(const float* __restrict
                           static_cast<float>(sn));
 }
 
-// sign carried by element i when it enters stage s: the product of the negations of the pairs it
-// belonged to in stages 0..s-1
-__device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int i, int s) {
-    int f = 0;
-    for (int sp = 0; sp < s; ++sp) {
-        const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
-        f ^= flip[sp * (kN / 2) + j];
-    }
-    return f ? -1 : 1;
-}
-
 // Step 2 (one thread per angle): place the constants of pair (s, j) in the tensor-memory image
 // img[role][column], with the role / register / half of the pair's low element in its phase.
 __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restrict__ prep,
@@ -439,25 +357,6 @@ __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restric
 }  // namespace f4k
 
 // ---- host side ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess) {
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-        }
-    }
-    return fn;
-}
-
 size_t fwdq4096_image_bytes() { return size_t(128) * f4k::kCols * sizeof(float); }
 size_t fwdq4096_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1); }
 
@@ -498,14 +397,7 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
 cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st) {
     CUtensorMap tmap;
-    const cuuint64_t dims[3] = {64, 64, static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ldx) * 2};
-    const cuuint32_t box[3] = {64, 64, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = encode_tiled()(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box,
-                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
     // four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest
     // among the configurations that compile without spills; more groups did not help)
     return launch_variant<4, 32, 2>(plan, tmap, rows, codes, scales, st);

@@ -1,0 +1,128 @@
+// Pieces shared by the tuned n = 4096 kernels: the thread-role layouts of the three 4-stage phases,
+// the shared-memory regrouping layouts, the packed three-shear stage, and the tensor-map encoder.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bfq_ptx.cuh"
+
+namespace bfq {
+namespace f4k {
+using namespace ptx;
+
+constexpr int kN = 4096;
+constexpr int kGroupThreads = 128;
+constexpr int kInSlots = 2;                  // TMA ring depth per group
+constexpr uint32_t kRowBytes = kN * 2;       // one bf16 row
+constexpr uint32_t kExWords = 4128;          // padded fp32 row (see the layouts below)
+constexpr uint32_t kExBytes = kExWords * 4;
+constexpr int kCols = 416;                   // tensor-memory columns in use
+
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ u64 lds64(uint32_t a) {
+    u64 v;
+    asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t a, u64 v) {
+    asm volatile("st.shared.b64 [%0], %1;" ::"r"(a), "l"(v) : "memory");
+}
+
+// ---- element held by role t, packed register m, half h in each phase -----------------------------------
+//   phase 1: i = m | (t & 15) << 4 | h << 8 | (t >> 4) << 9
+//   phase 2: i = (t & 15) | m << 4 | h << 8 | (t >> 4) << 9
+//   phase 3: i = h | t << 1 | m << 8
+// ---- shared-memory layouts of the two regroupings (word addresses; i = element index bits) -----------
+// first:   A1 = i8 + 2*(i4..i7) + 32*(i9 + 2*i10 + 4*i11) + 258*(i0..i3)
+// second:  A2 = (i0..i4) + 16*i9 + 32*(i5 + 2*i6 + 4*i7 + 8*i8 + 16*i10 + 32*i11 + 64*i9)
+// Both are injective into [0, kExWords); a half-warp's 16 64-bit accesses and a warp's 32 scalar
+// stores each cover the 32 banks exactly once.  In the first, the words a thread writes are read by
+// the 16 lanes of its own half-warp only.
+__device__ __forceinline__ constexpr uint32_t ex1_wr_local(int m) { return 4u * 258u * m; }
+__device__ __forceinline__ constexpr uint32_t ex1_rd_local(int m) { return 4u * 2u * m; }
+__device__ __forceinline__ constexpr uint32_t ex2_wr_local(int m, int h) {
+    return 4u * (16u * (m & 1) + 32u * (m >> 1) + 256u * h);
+}
+__device__ __forceinline__ constexpr uint32_t ex2_rd_local(int m) {
+    return 4u * (256u * (m & 1) + 2064u * ((m >> 1) & 1) + 512u * ((m >> 2) & 1) + 1024u * ((m >> 3) & 1));
+}
+
+// ---- one stage on the registers of a thread ---------------------------------------------------------
+// Local stage K pairs packed registers m and m | 2^K; both fp32 lanes rotate at once.  T holds
+// (nt, nt', sn, sn') for NU consecutive pairs starting at pair U0.  The three shears are issued level
+// by level so that dependent instructions are NU apart.
+template <int K, int U0, int NU, int CW>
+__device__ __forceinline__ void stage_lift(u64 (&P)[16], const uint32_t (&T)[CW]) {
+    static_assert(4 * NU <= CW, "chunk too small");
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), P[m_hi], P[m_lo]);
+    }
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        P[m_hi] = fma2(pack2u(T[4 * i + 2], T[4 * i + 3]), P[m_lo], P[m_hi]);
+    }
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), P[m_hi], P[m_lo]);
+    }
+}
+
+// sign carried by element i when it enters stage s: the product of the negations (flip = 1) of the pairs
+// it belonged to in stages 0..s-1
+__device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int i, int s) {
+    int f = 0;
+    for (int sp = 0; sp < s; ++sp) {
+        const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
+        f ^= flip[sp * (kN / 2) + j];
+    }
+    return f ? -1 : 1;
+}
+
+}  // namespace f4k
+
+// ---- host side: cuTensorMapEncodeTiled through the runtime's driver entry point ------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static inline EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess) {
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+        }
+    }
+    return fn;
+}
+
+
+// 3-D map over bf16 rows of 4096: {64 elements, 64 lines, rows}, box = one row, 128-byte swizzle
+static inline bool encode_row_map(CUtensorMap* tmap, const void* x, int64_t rows, int64_t ld) {
+    const cuuint64_t dims[3] = {64, 64, static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ld) * 2};
+    const cuuint32_t box[3] = {64, 64, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return encode_tiled()(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace bfq

@@ -287,3 +287,78 @@ def test_tuned_n4096_special_angles_and_degenerate_rows():
         codes, scales = p.forward_quant(x.to(DEV), 4)
         check_quant(codes, scales, oracle.forward(to_f64(theta), to_f64(x)), 4, f"tuned {kind}")
         assert p.device_status() == 0
+
+
+# ---- tuned backward for n = 4096 bf16 rows ------------------------------------------------------------------
+@pytest.mark.parametrize("rows", [1, 2, 3, 295, 296, 297, 1001])
+@pytest.mark.parametrize("angle_kind", ["normal", "uniform"])
+def test_tuned_backward_n4096_ragged_row_counts(rows, angle_kind):
+    n = 4096
+    theta = synth.angles(n, angle_kind, 60 + rows)
+    if angle_kind == "uniform":  # exact multiples of pi/2 and pi exercise the angle reduction and its sign tracking
+        theta[:, ::7] = math.pi / 2
+        theta[:, 1::7] = -math.pi
+        theta[:, 2::7] = math.pi
+        theta[:, 3::7] = -math.pi / 2
+        theta[:, 4::7] = 100.0
+    x = synth.rows(rows, n, "student_t3", 61 + rows, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
+    g = synth.rows(rows, n, "normal", 62 + rows, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    ld = n + 8
+    xpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    gpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    gpad[:, :n] = g.to(DEV)
+    dxbuf = Guarded((rows, ld), torch.bfloat16, DEV)
+    dth = Guarded((p.L, n // 2), torch.float32, DEV)
+    p.backward(xpad[:, :n], gpad[:, :n], dx=dxbuf.view[:, :n], dtheta=dth.view)
+    assert p.device_status() == 0
+    dx_ref, dth_ref = oracle.backward(to_f64(theta), to_f64(x), to_f64(g))
+    check_rows_close(dxbuf.view[:, :n], dx_ref, absmax_rows(g), f"tuned dx rows={rows}")
+    check_dtheta(dth.view, dth_ref, f"tuned dtheta rows={rows}")
+    assert dxbuf.intact() and dth.intact()
+    assert (dxbuf.view[:, n:].view(torch.int16) == torch.tensor(0xA5A5, dtype=torch.uint16).view(torch.int16)).all()
+    assert p.backward_partials() == min((rows + 1) // 2, torch.cuda.get_device_properties(0).multi_processor_count)
+    # d-theta only, and again: same bits
+    _, dth2 = p.backward(xpad[:, :n], gpad[:, :n], want_dx=False)
+    assert torch.equal(dth2, dth.view)
+
+
+def test_tuned_backward_follows_new_angles_and_agrees_with_the_generic_kernels(monkeypatch):
+    n, rows = 4096, 500
+    x = synth.rows(rows, n, "student_t3", 71, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16).to(DEV)
+    g = synth.rows(rows, n, "normal", 72, dtype=torch.bfloat16).to(DEV)
+    p = Plan(n, DEV)
+    for seed in (73, 74):  # the backward tables are rebuilt after every bfq_set_angles
+        theta = synth.angles(n, "uniform", seed).to(DEV)
+        p.set_angles(theta)
+        dx, dth = p.backward(x, g)
+        monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+        dx_gen, dth_gen = p.backward(x, g, dx_dtype=torch.float32)  # fp32 dx: one bf16 rounding between the two
+        monkeypatch.delenv("BFQ_GENERIC_ONLY")
+        check_rows_close(dx, to_f64(dx_gen), absmax_rows(g), "tuned vs generic dx")
+        check_dtheta(dth, to_f64(dth_gen), "tuned vs generic dtheta")
+
+
+def test_full_size_backward_n4096_sampled():
+    wl = synth.WORKLOADS["learn4096"]
+    rows = 65536  # a quarter of the learning batch keeps the oracle's share of the test to seconds
+    theta = wl.theta(device=DEV)
+    x = wl.x(device=DEV, n_rows=rows)
+    g = wl.g(device=DEV, n_rows=rows)
+    p = Plan(wl.n, DEV)
+    p.set_angles(theta)
+    dx = Guarded((rows, wl.n), torch.bfloat16, DEV)
+    dth = Guarded((wl.L, wl.n // 2), torch.float32, DEV)
+    p.backward(x, g, dx=dx.view, dtheta=dth.view)
+    assert p.device_status() == 0 and dx.intact() and dth.intact()
+    idx = _sample_rows(rows, 1024)
+    ti = torch.from_numpy(idx).to(DEV)
+    dx_ref, _ = oracle.backward(to_f64(theta), to_f64(x[ti]), to_f64(g[ti]))
+    check_rows_close(dx.view[ti], dx_ref, absmax_rows(g[ti]), "learn4096 dx")
+    # d-theta over all rows: linear in the rows, so the oracle's sum over 8 row blocks must match
+    th64 = to_f64(theta)
+    acc = np.zeros((wl.L, wl.n // 2))
+    for r0 in range(0, rows, 8192):
+        acc += oracle.backward(th64, to_f64(x[r0:r0 + 8192]), to_f64(g[r0:r0 + 8192]))[1]
+    check_dtheta(dth.view, acc, "learn4096 dtheta")
