@@ -175,6 +175,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler captures of a small case)")
+    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward"],
+                    help="backward: time only bfq_backward on the learning batch (for profiler captures; "
+                         "prints a short JSON line, not the benchmark line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bfq" else args.warmup
     if args.impl == "reference":
@@ -209,6 +212,8 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
+    if args.op == "backward":
+        return run_backward_only(torch, args, synth, Plan, dev)
     wl = synth.WORKLOADS[WORKLOAD]
     if args.rows:
         import dataclasses
@@ -270,6 +275,22 @@ def main():
             dist.destroy_process_group()
         return
     finish(torch, args, wl, synth, x, dev, world, value, ms_step, kernel_ms_avg, clocks, e2e, others, dist)
+
+
+def run_backward_only(torch, args, synth, Plan, dev):
+    """bfq_backward alone on (a prefix of) the learning batch: warm-up, then `steps` timed launches."""
+    wl = synth.WORKLOADS["learn4096"]
+    rows = args.rows or wl.n_rows
+    plan = Plan(wl.n, dev)
+    plan.set_angles(wl.theta(device=dev))
+    x, g = wl.x(device=dev, n_rows=rows), wl.g(device=dev, n_rows=rows)
+    dx = torch.empty_like(x)
+    dth = torch.empty((wl.L, wl.n // 2), dtype=torch.float32, device=dev)
+    for _ in range(args.warmup):
+        plan.backward(x, g, dx=dx, dtheta=dth)
+    ms = event_time_ms(torch, lambda: plan.backward(x, g, dx=dx, dtheta=dth), args.steps)
+    print(json.dumps({"op": "backward", "workload": "learn4096", "rows": rows, "ms": ms,
+                      "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
 
 
 def run_e2e(torch, args, wl, plan, theta, x, codes, scales, barrier, max_over_ranks, world):
