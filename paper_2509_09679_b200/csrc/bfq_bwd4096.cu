@@ -1,7 +1,9 @@
 // Tuned backward pass for n = 4096 bf16 rows on sm_100a:  dx = Q^T g  and  d-theta summed over rows.
 //
-// One persistent CTA of 128 threads per SM works on two rows at a time (row pair p of the CTA is rows
-// 2p, 2p+1).  The thread roles, phases and regrouping layouts are those of the forward kernel
+// One persistent CTA per SM works on two rows at a time (row pair p of the CTA is rows 2p, 2p+1) with two
+// groups of 128 threads: the forward group recomputes y for pair k+1 while the reverse group walks pair k
+// down; y changes hands through one shared-memory buffer.  Only the reverse group touches the d-theta
+// accumulators.  The thread roles, phases and regrouping layouts are those of the forward kernel
 // (bfq_n4096.cuh).  Per row pair:
 //   1. y = Q x with the three-shear constants, all 12 stages, in the tracked-sign basis sigma.
 //   2. y and g are moved to the basis sigma * (-1)^popcount(index).  Any two indices that a stage pairs
@@ -23,22 +25,27 @@ namespace b4k {
 using namespace ptx;
 using namespace f4k;
 
-constexpr int kThreads = 128;
-constexpr int kSlots = 2;                    // TMA ring depth (row pairs)
+constexpr int kThreads = 128;                // one group; the CTA has two (reverse = threads 0..127, forward = 128..255)
+constexpr int kCtaThreads = 2 * kThreads;
+constexpr int kSlots = 2;                    // TMA ring depth (row pairs), x and g rings separately
+constexpr int kBarRev = 1, kBarFwd = 2, kBarFull = 3, kBarEmpty = 4;  // named barriers
 constexpr int kConstCols = 384;              // 12 stages x 32 words
 constexpr int kAccCol = 384;                 // accumulators of stages 0..7: 16 columns each
-constexpr uint32_t kPairBytes = 4 * kRowBytes;  // x0, x1, g0, g1
+constexpr uint32_t kPairBytes = 2 * kRowBytes;  // two bf16 rows
 
 struct Smem {
-    static constexpr uint32_t kInOff = 0;                                  // [kSlots][4][kRowBytes]
-    static constexpr uint32_t kExOff = kInOff + kSlots * kPairBytes;       // [4][kExBytes]: y0, y1, g0, g1
-    static constexpr uint32_t kAccOff = kExOff + 4 * kExBytes;             // [16][128] float4: stages 8..11
-    static constexpr uint32_t kSgnOff = kAccOff + 16 * kThreads * 16;      // [4][128] uint4: sign words of g
-    static constexpr uint32_t kBarOff = kSgnOff + 4 * kThreads * 16;       // mbarriers [kSlots]
-    static constexpr uint32_t kTmemOff = kBarOff + 8 * kSlots;
+    static constexpr uint32_t kXOff = 0;                                   // [kSlots][2][kRowBytes]
+    static constexpr uint32_t kGOff = kXOff + kSlots * kPairBytes;         // [kSlots][2][kRowBytes]
+    static constexpr uint32_t kExFOff = kGOff + kSlots * kPairBytes;       // forward group: [2][kExBytes]
+    static constexpr uint32_t kExROff = kExFOff + 2 * kExBytes;            // reverse group: [4][kExBytes]: y0, y1, g0, g1
+    static constexpr uint32_t kHandOff = kExROff + 4 * kExBytes;           // y hand-off: [2 rows][16][128] packed pairs
+    static constexpr uint32_t kAccOff = kHandOff + 2 * 16 * kThreads * 8;  // [16][128] float4: stages 8..11
+    static constexpr uint32_t kBarOff = kAccOff + 16 * kThreads * 16;      // mbarriers: x ring, g ring
+    static constexpr uint32_t kTmemOff = kBarOff + 8 * 2 * kSlots;
     static constexpr uint32_t kUsed = kTmemOff + 16;
     static constexpr uint32_t kBytes = kUsed + 1024;
 };
+static_assert(Smem::kBytes <= 232448, "shared memory budget of one CTA");
 
 __device__ __forceinline__ uint32_t lds32(uint32_t a) {
     uint32_t v;
@@ -51,7 +58,8 @@ __device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
 
 struct Addr {
     uint32_t w1, r1, w2, r2;  // per-thread byte offsets inside a regrouping buffer (forward write / read sides)
-    uint32_t ex;              // base of the four regrouping buffers
+    uint32_t ex;              // base of the group's regrouping buffers
+    int bar;                  // the group's named barrier
 };
 
 // ---- regroupings: forward direction (phase 1 -> 2 -> 3) and back, one row array at a time -------------
@@ -118,22 +126,17 @@ struct Ctx {
 };
 
 // ---- forward recompute: 24 chunks of 16 constants (two per stage), both rows ---------------------------
-// Chunk C is in Tcur; the next chunk (or, after the last one, the first chunk of the reverse walk) is
-// requested right after the wait.
+// Chunk C is in Tcur; the next chunk is requested right after the wait.
 template <int C>
 __device__ __forceinline__ void fwd_chunks(u64 (&X0)[16], u64 (&X1)[16], uint32_t (&Tcur)[16], uint32_t (&Tnext)[16],
                                            const Ctx& cx) {
     constexpr int s = C / 2, K = s & 3, U0 = 4 * (C & 1);
     tmem_wait_ld16(Tcur);
-    if constexpr (C + 1 < 24) {
-        tmem_ld16(cx.tlane + 16 * (C + 1), Tnext);
-    } else {
-        tmem_ld16(cx.tlane + 32 * 11, Tnext);
-    }
+    if constexpr (C + 1 < 24) tmem_ld16(cx.tlane + 16 * (C + 1), Tnext);
     stage_lift<K, U0, 4, 16>(X0, Tcur);
     stage_lift<K, U0, 4, 16>(X1, Tcur);
-    if constexpr (C == 7) {
-        __syncwarp();  // the half-warp's reads of the previous row pair's last regrouping are done
+    if constexpr (C == 7) {  // inside each half-warp; the group-wide hand-off barrier of the previous row pair
+                             // has put every other warp past its reads of these buffers
         fwd1_store(X0, cx.a.ex + 0 * kExBytes, cx.a);
         fwd1_store(X1, cx.a.ex + 1 * kExBytes, cx.a);
         __syncwarp();
@@ -141,12 +144,12 @@ __device__ __forceinline__ void fwd_chunks(u64 (&X0)[16], u64 (&X1)[16], uint32_
         fwd1_load(X1, cx.a.ex + 1 * kExBytes, cx.a);
     }
     if constexpr (C == 15) {
-        bar_sync(1, kThreads);  // every warp is past its reads of buffers 2 and 3 for the previous row pair
-        fwd2_store(X0, cx.a.ex + 2 * kExBytes, cx.a);
-        fwd2_store(X1, cx.a.ex + 3 * kExBytes, cx.a);
-        bar_sync(1, kThreads);
-        fwd2_load(X0, cx.a.ex + 2 * kExBytes, cx.a);
-        fwd2_load(X1, cx.a.ex + 3 * kExBytes, cx.a);
+        bar_sync(cx.a.bar, kThreads);  // every warp of the group is past its reads of the first layout
+        fwd2_store(X0, cx.a.ex + 0 * kExBytes, cx.a);
+        fwd2_store(X1, cx.a.ex + 1 * kExBytes, cx.a);
+        bar_sync(cx.a.bar, kThreads);
+        fwd2_load(X0, cx.a.ex + 0 * kExBytes, cx.a);
+        fwd2_load(X1, cx.a.ex + 1 * kExBytes, cx.a);
     }
     if constexpr (C + 1 < 24) fwd_chunks<C + 1>(X0, X1, Tnext, Tcur, cx);
 }
@@ -200,12 +203,12 @@ __device__ __forceinline__ void rev_steps(u64 (&Y0)[16], u64 (&Y1)[16], u64 (&G0
     stage_lift<S::K, S::U0, 4, 16>(G0, Tcur);
     stage_lift<S::K, S::U0, 4, 16>(G1, Tcur);
     if constexpr (I == 7) {  // phase 3 -> phase 2, across warps
-        bar_sync(1, kThreads);  // every warp is past its forward reads of buffers 2 and 3
+        bar_sync(cx.a.bar, kThreads);  // every warp is past its half-warp reads for the previous row pair
         rev2_store(Y0, cx.a.ex + 0 * kExBytes, cx.a);
         rev2_store(Y1, cx.a.ex + 1 * kExBytes, cx.a);
         rev2_store(G0, cx.a.ex + 2 * kExBytes, cx.a);
         rev2_store(G1, cx.a.ex + 3 * kExBytes, cx.a);
-        bar_sync(1, kThreads);
+        bar_sync(cx.a.bar, kThreads);
         after_phase3();  // all reads of the input slot are done: the next row pair may be requested
         rev2_load(Y0, cx.a.ex + 0 * kExBytes, cx.a);
         rev2_load(Y1, cx.a.ex + 1 * kExBytes, cx.a);
@@ -213,7 +216,7 @@ __device__ __forceinline__ void rev_steps(u64 (&Y0)[16], u64 (&Y1)[16], u64 (&G0
         rev2_load(G1, cx.a.ex + 3 * kExBytes, cx.a);
     }
     if constexpr (I == 15) {  // phase 2 -> phase 1, inside each half-warp, but the buffers were read across warps
-        bar_sync(1, kThreads);
+        bar_sync(cx.a.bar, kThreads);
         rev1_store(Y0, cx.a.ex + 0 * kExBytes, cx.a);
         rev1_store(Y1, cx.a.ex + 1 * kExBytes, cx.a);
         rev1_store(G0, cx.a.ex + 2 * kExBytes, cx.a);
@@ -240,18 +243,20 @@ __device__ __forceinline__ int elem_of(int P, int t, int m, int h) {
     return h | (t << 1) | (m << 8);
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kCtaThreads, 1)
 k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap gmap,
           const float* __restrict__ img, const uint32_t* __restrict__ gsign, const int8_t* __restrict__ dsign,
           __nv_bfloat16* __restrict__ dx, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status) {
     using S = Smem;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = threadIdx.x;  // role 0..127; warp = tensor-memory lane quarter
+    const int warp = threadIdx.x >> 5;
+    const int t = threadIdx.x & (kThreads - 1);      // role 0..127
+    const bool is_fwd = threadIdx.x >= kThreads;     // warps 4..7 recompute y, warps 0..3 walk back
+    const int quarter = warp & 3;                    // tensor-memory lane quarter of this warp
 
     if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
-    if (threadIdx.x < kSlots) {
+    if (threadIdx.x < 2 * kSlots) {
         mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
         mbar_init_fence();
     }
@@ -262,11 +267,12 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
 
     Ctx cx;
-    cx.tlane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    cx.tlane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     cx.acc_smem = sbase + S::kAccOff + t * 16;
     {
         const uint32_t t4 = (t >> 4) & 1, t5 = (t >> 5) & 1, t6 = (t >> 6) & 1;
-        cx.a.ex = sbase + S::kExOff;
+        cx.a.ex = sbase + (is_fwd ? S::kExFOff : S::kExROff);
+        cx.a.bar = is_fwd ? kBarFwd : kBarRev;
         cx.a.w1 = 4u * (2u * (t & 15) + 32u * (t >> 4));
         cx.a.r1 = 4u * (258u * (t & 15) + 32u * (t >> 4));
         cx.a.w2 = 4u * ((t & 15) + 2064u * t4 + 512u * t5 + 1024u * t6);
@@ -277,27 +283,26 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     const int first = blockIdx.x;
     const int stride = gridDim.x;
     const int count = first < pairs ? (pairs - first + stride - 1) / stride : 0;
-    const uint32_t in_base = sbase + S::kInOff;
-    const uint32_t bar_base = sbase + S::kBarOff;
+    const uint32_t ring = sbase + (is_fwd ? S::kXOff : S::kGOff);                 // this group's input ring
+    const uint32_t bar_base = sbase + S::kBarOff + (is_fwd ? 0 : 8 * kSlots);     // and its mbarriers
+    const CUtensorMap* tmap = is_fwd ? &xmap : &gmap;
 
     // a row index past the end is legal for the tensor map: the tile is filled with zeros
     auto request = [&](int k) {
         const int slot = k & 1;
         const int r0 = 2 * (first + k * stride);
-        const uint32_t dst = in_base + slot * kPairBytes, bar = bar_base + 8 * slot;
+        const uint32_t dst = ring + slot * kPairBytes, bar = bar_base + 8 * slot;
         mbar_expect_tx(bar, kPairBytes);
-        tma_load_3d(dst + 0 * kRowBytes, &xmap, 0, 0, r0, bar);
-        tma_load_3d(dst + 1 * kRowBytes, &xmap, 0, 0, r0 + 1, bar);
-        tma_load_3d(dst + 2 * kRowBytes, &gmap, 0, 0, r0, bar);
-        tma_load_3d(dst + 3 * kRowBytes, &gmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(dst, tmap, 0, 0, r0, bar);
+        tma_load_3d(dst + kRowBytes, tmap, 0, 0, r0 + 1, bar);
     };
     if (t == 0) {
         for (int k = 0; k < kSlots && k < count; ++k) request(k);
     }
-    // constants into tensor memory, accumulators to zero, sign words of g into shared memory
+    // constants into tensor memory (each group fills half of the columns), accumulators to zero
     {
         const float4* src = reinterpret_cast<const float4*>(img + t * kConstCols);
-        for (int c = 0; c < kConstCols; c += 16) {
+        for (int c = is_fwd ? 16 : 0; c < kConstCols; c += 32) {
             uint32_t v[16];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -307,125 +312,153 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
             }
             tmem_st16(cx.tlane + c, v);
         }
-        uint32_t z[16];
+        if (!is_fwd) {
+            uint32_t z[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) z[i] = 0u;
-        for (int c = kAccCol; c < 512; c += 16) tmem_st16(cx.tlane + c, z);
+            for (int i = 0; i < 16; ++i) z[i] = 0u;
+            for (int c = kAccCol; c < 512; c += 16) tmem_st16(cx.tlane + c, z);
+            for (int q = 0; q < 16; ++q) sts128(cx.acc_smem + q * kThreads * 16, make_uint4(0u, 0u, 0u, 0u));
+        }
         tmem_wait_st();
-        for (int q = 0; q < 16; ++q) sts128(cx.acc_smem + q * kThreads * 16, make_uint4(0u, 0u, 0u, 0u));
-        const uint4* gs = reinterpret_cast<const uint4*>(gsign);
-        for (int q = 0; q < 4; ++q) sts128(sbase + S::kSgnOff + (q * kThreads + t) * 16, __ldg(gs + q * kThreads + t));
     }
     tmem_fence_before();
     __syncthreads();
     tmem_fence_after();
 
-    // x tile, phase-1 ownership (as in the forward kernel)
-    const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
-    const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
-    // g tile, phase-3 ownership: the 32-bit word of elements 2t + 256m, 2t + 256m + 1 is word t & 3 of 16-byte
-    // chunk (t & 31) >> 2 of 128-byte line (t >> 5) + 4m; the swizzle moves the chunk to chunk ^ (line & 7)
-    const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
-    const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
-    const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
     // parity of the role: popcount(t) & 1
     const uint32_t par_t = __popc(t) & 1;
     const uint32_t sgn_a = par_t ? 0x80000000u : 0u, sgn_b = par_t ? 0u : 0x80000000u;
+    const uint32_t hand = sbase + S::kHandOff + t * 8;  // + (row * 16 + m) * 1024: conflict free, same role both sides
 
-    u64 Y0[16], Y1[16], G0[16], G1[16];
-    uint32_t T0[16], T1[16], A0[8], A1[8];
-
-    for (int k = 0; k < count; ++k) {
-        const int slot = k & 1;
-        const int r0 = 2 * (first + k * stride);
-        tmem_ld16(cx.tlane, T0);
-        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
-        const uint32_t tile = in_base + slot * kPairBytes;
-        // ---- x rows -> packed fp32, phase 1 ----
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            u64(&X)[16] = r == 0 ? Y0 : Y1;
-            const uint32_t src = tile + r * kRowBytes + in_line;
-            uint4 w[2][2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int c = 0; c < 2; ++c) w[h][c] = lds128(src + 512u * h + (in_x ^ ((c | (h << 2)) << 4)));
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const uint32_t a[4] = {w[0][c].x, w[0][c].y, w[0][c].z, w[0][c].w};
-                const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    X[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
-                    X[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
-                }
-            }
-        }
-        fwd_chunks<0>(Y0, Y1, T0, T1, cx);  // leaves the first reverse chunk requested in T0
-
-        // ---- y to the parity basis; g rows -> packed fp32 in the same basis, phase 3 ----
-#pragma unroll
-        for (int m = 0; m < 16; ++m) {
-            const bool odd = (__builtin_popcount(m) & 1) != 0;  // compile-time after unrolling
-            const u64 mask = odd ? pack2u(sgn_b, sgn_a) : pack2u(sgn_a, sgn_b);
-            Y0[m] ^= mask;
-            Y1[m] ^= mask;
-        }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            u64(&G)[16] = r == 0 ? G0 : G1;
-            const uint32_t src = tile + (2 + r) * kRowBytes;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint4 sw = lds128(sbase + S::kSgnOff + (q * kThreads + t) * 16);
-                const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int m = 4 * q + i;
-                    const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
-                    G[m] = pack2u(w << 16, w & 0xFFFF0000u);
-                }
-            }
-        }
-        rev_steps<0>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [&]() {
-            if (t == 0 && k + kSlots < count) request(k + kSlots);
-        });
-
-        // ---- dx = parity sign * g, bf16, phase-1 ownership: two runs of 16 elements per row ----
-        if (dx != nullptr) {
+    if (is_fwd) {
+        // =============================== forward group: y = Q x ===============================
+        // x tile, phase-1 ownership (as in the forward kernel)
+        const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+        const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+        u64 X0[16], X1[16];
+        uint32_t T0[16], T1[16];
+        for (int k = 0; k < count; ++k) {
+            const int slot = k & 1;
+            tmem_ld16(cx.tlane, T0);
+            mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+            const uint32_t tile = ring + slot * kPairBytes;
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-                if (r0 + r < rows) {
-                    const u64(&G)[16] = r == 0 ? G0 : G1;
-                    __nv_bfloat16* row = dx + static_cast<int64_t>(r0 + r) * ld + 16 * (t & 15) + 512 * (t >> 4);
+                u64(&X)[16] = r == 0 ? X0 : X1;
+                const uint32_t src = tile + r * kRowBytes + in_line;
+                uint4 w[2][2];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t w[8];
+                for (int h = 0; h < 2; ++h)
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            uint32_t lo0, hi0, lo1, hi1;
-                            unpack2u(G[2 * j], lo0, hi0);
-                            unpack2u(G[2 * j + 1], lo1, hi1);
-                            const float e0 = __uint_as_float(h ? hi0 : lo0), e1 = __uint_as_float(h ? hi1 : lo1);
-                            // elements m = 2j, 2j+1 of half h: parity popcount(2j) ^ h ^ popcount(t), opposite for 2j+1
-                            const bool odd_c = ((__builtin_popcount(2 * j) + h) & 1) != 0;
-                            const uint32_t neg_lo = odd_c ? (sgn_b >> 16) : (sgn_a >> 16);  // bit 15: element 2j
-                            const uint32_t neg_hi = odd_c ? sgn_a : sgn_b;                  // bit 31: element 2j+1
-                            w[j] = cvt_bf16x2(e0, e1) ^ (neg_lo | neg_hi);
-                        }
-                        uint4* dst = reinterpret_cast<uint4*>(row + 256 * h);
-                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    for (int c = 0; c < 2; ++c) w[h][c] = lds128(src + 512u * h + (in_x ^ ((c | (h << 2)) << 4)));
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const uint32_t a[4] = {w[0][c].x, w[0][c].y, w[0][c].z, w[0][c].w};
+                    const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        X[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
+                        X[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
                     }
                 }
             }
+            fwd_chunks<0>(X0, X1, T0, T1, cx);
+            // every thread of the group read its part of the x tile before the barriers inside fwd_chunks
+            if (t == 0 && k + kSlots < count) request(k + kSlots);
+            // y to the parity basis, then hand it over once the reverse group has taken the previous pair
+            bar_sync(kBarEmpty, kCtaThreads);
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                const bool odd = (__builtin_popcount(m) & 1) != 0;  // compile-time after unrolling
+                const u64 mask = odd ? pack2u(sgn_b, sgn_a) : pack2u(sgn_a, sgn_b);
+                sts64(hand + (0 * 16 + m) * 1024u, X0[m] ^ mask);
+                sts64(hand + (1 * 16 + m) * 1024u, X1[m] ^ mask);
+            }
+            __threadfence_block();
+            bar_arrive(kBarFull, kCtaThreads);
         }
-        tmem_wait_st();  // this row pair's accumulator stores land before the next pair reloads them
+    } else {
+        // =============================== reverse group: d-theta and dx ===============================
+        // g tile, phase-3 ownership: the 32-bit word of elements 2t + 256m, 2t + 256m + 1 is word t & 3 of
+        // 16-byte chunk (t & 31) >> 2 of 128-byte line (t >> 5) + 4m; the swizzle moves the chunk to
+        // chunk ^ (line & 7)
+        const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
+        const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
+        const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
+        uint32_t gs[16];  // sign words of this role's 16 words of a g row
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(gsign);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 v = __ldg(src + q * kThreads + t);
+                gs[4 * q] = v.x, gs[4 * q + 1] = v.y, gs[4 * q + 2] = v.z, gs[4 * q + 3] = v.w;
+            }
+        }
+        u64 Y0[16], Y1[16], G0[16], G1[16];
+        uint32_t T0[16], T1[16], A0[8], A1[8];
+        if (count > 0) bar_arrive(kBarEmpty, kCtaThreads);  // the hand-off buffer starts empty
+        for (int k = 0; k < count; ++k) {
+            const int slot = k & 1;
+            const int r0 = 2 * (first + k * stride);
+            tmem_ld16(cx.tlane + 32 * 11, T0);
+            mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+            const uint32_t tile = ring + slot * kPairBytes;
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                u64(&G)[16] = r == 0 ? G0 : G1;
+                const uint32_t src = tile + r * kRowBytes;
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ gs[m];
+                    G[m] = pack2u(w << 16, w & 0xFFFF0000u);
+                }
+            }
+            bar_sync(kBarFull, kCtaThreads);
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                Y0[m] = lds64(hand + (0 * 16 + m) * 1024u);
+                Y1[m] = lds64(hand + (1 * 16 + m) * 1024u);
+            }
+            if (k + 1 < count) bar_arrive(kBarEmpty, kCtaThreads);  // each thread re-reads only its own words
+            rev_steps<0>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [&]() {
+                if (t == 0 && k + kSlots < count) request(k + kSlots);
+            });
+
+            // ---- dx = parity sign * g, bf16, phase-1 ownership: two runs of 16 elements per row ----
+            if (dx != nullptr) {
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    if (r0 + r < rows) {
+                        const u64(&G)[16] = r == 0 ? G0 : G1;
+                        __nv_bfloat16* row = dx + static_cast<int64_t>(r0 + r) * ld + 16 * (t & 15) + 512 * (t >> 4);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            uint32_t w[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                uint32_t lo0, hi0, lo1, hi1;
+                                unpack2u(G[2 * j], lo0, hi0);
+                                unpack2u(G[2 * j + 1], lo1, hi1);
+                                const float e0 = __uint_as_float(h ? hi0 : lo0), e1 = __uint_as_float(h ? hi1 : lo1);
+                                // elements m = 2j, 2j+1 of half h: parity popcount(2j) ^ h ^ popcount(t), opposite for 2j+1
+                                const bool odd_c = ((__builtin_popcount(2 * j) + h) & 1) != 0;
+                                const uint32_t neg_lo = odd_c ? (sgn_b >> 16) : (sgn_a >> 16);  // bit 15: element 2j
+                                const uint32_t neg_hi = odd_c ? sgn_a : sgn_b;                  // bit 31: element 2j+1
+                                w[j] = cvt_bf16x2(e0, e1) ^ (neg_lo | neg_hi);
+                            }
+                            uint4* dst = reinterpret_cast<uint4*>(row + 256 * h);
+                            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        }
+                    }
+                }
+            }
+            tmem_wait_st();  // this row pair's accumulator stores land before the next pair reloads them
+        }
     }
 
     // ---- this CTA's sums -> its slot of the partial sums, with the sign of the basis undone ----
-    {
+    if (!is_fwd) {
         float* out = partial + static_cast<int64_t>(blockIdx.x) * (12 * (kN / 2));
         for (int s = 0; s < 12; ++s) {
             const int K = s & 3, P = s >> 2;
@@ -535,7 +568,7 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
     if (!encode_row_map(&xmap, x, rows, ld) || !encode_row_map(&gmap, g, rows, ld)) return cudaErrorInvalidValue;
     const int64_t pairs = (rows + 1) / 2;
     const int grid = int(pairs < plan->sm_count ? pairs : plan->sm_count);
-    b4k::k_bwd4096<<<grid, b4k::kThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
+    b4k::k_bwd4096<<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
                                                                    plan->dsign4096, static_cast<__nv_bfloat16*>(dx), ld,
                                                                    plan->partial, int(rows), plan->status_word);
     cudaError_t e = cudaGetLastError();
