@@ -175,9 +175,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler captures of a small case)")
-    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward"],
-                    help="backward: time only bfq_backward on the learning batch (for profiler captures; "
-                         "prints a short JSON line, not the benchmark line)")
+    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward", "int2_8192"],
+                    help="backward / int2_8192: time only bfq_backward on the learning batch / bfq_forward_quant "
+                         "(INT2) on the n = 8192 activations (for profiler captures; prints a short JSON line, "
+                         "not the benchmark line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bfq" else args.warmup
     if args.impl == "reference":
@@ -214,6 +215,8 @@ def main():
 
     if args.op == "backward":
         return run_backward_only(torch, args, synth, Plan, dev)
+    if args.op == "int2_8192":
+        return run_int2_8192_only(torch, args, synth, Plan, dev)
     wl = synth.WORKLOADS[WORKLOAD]
     if args.rows:
         import dataclasses
@@ -290,6 +293,22 @@ def run_backward_only(torch, args, synth, Plan, dev):
         plan.backward(x, g, dx=dx, dtheta=dth)
     ms = event_time_ms(torch, lambda: plan.backward(x, g, dx=dx, dtheta=dth), args.steps)
     print(json.dumps({"op": "backward", "workload": "learn4096", "rows": rows, "ms": ms,
+                      "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
+
+
+def run_int2_8192_only(torch, args, synth, Plan, dev):
+    """bfq_forward_quant (INT2) alone on (a prefix of) the n = 8192 activations."""
+    wl = synth.WORKLOADS["act8192_int2"]
+    rows = args.rows or wl.n_rows
+    plan = Plan(wl.n, dev)
+    plan.set_angles(wl.theta(device=dev))
+    x = wl.x(device=dev, n_rows=rows)
+    codes = torch.empty((rows, wl.n // 4), dtype=torch.uint8, device=dev)
+    scales = torch.empty((rows,), dtype=torch.float16, device=dev)
+    for _ in range(args.warmup):
+        plan.forward_quant(x, 2, codes=codes, scales=scales)
+    ms = event_time_ms(torch, lambda: plan.forward_quant(x, 2, codes=codes, scales=scales), args.steps)
+    print(json.dumps({"op": "int2_8192", "workload": "act8192_int2", "rows": rows, "ms": ms,
                       "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
 
 

@@ -93,9 +93,9 @@ static cudaError_t launch_generic(const bfq_plan* plan, const GenericParams& p, 
         case 8: return launch_generic_t<8, 2, MODE>(plan, p, st);
         case 9: return launch_generic_t<9, 2, MODE>(plan, p, st);
         case 10: return launch_generic_t<10, 2, MODE>(plan, p, st);
-        case 11: return launch_generic_t<11, 2, MODE>(plan, p, st);
-        case 12: return launch_generic_t<12, 2, MODE>(plan, p, st);
-        case 13: return launch_generic_t<13, 2, MODE>(plan, p, st);
+        case 11: return launch_generic_t<11, 4, MODE>(plan, p, st);
+        case 12: return launch_generic_t<12, 4, MODE>(plan, p, st);
+        case 13: return launch_generic_t<13, 4, MODE>(plan, p, st);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -193,6 +193,8 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess) e = cudaMalloc(&plan->partial, size_t(plan->partial_slots) * angles * sizeof(float));
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img4096, fwdq4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->prep4096, fwdq4096_prep_bytes());
+    if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->img8192, fwdq8192_image_bytes());
+    if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->prep8192, fwdq8192_prep_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_b4096, bwd4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->dsign4096, bwd4096_dsign_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->gsign4096, bwd4096_gsign_bytes());
@@ -204,6 +206,10 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
         cudaFree(plan->img4096);
         cudaFree(plan->prep4096);
         cudaFree(plan->img_b4096);
+    cudaFree(plan->img8192);
+    cudaFree(plan->prep8192);
+        cudaFree(plan->img8192);
+        cudaFree(plan->prep8192);
         cudaFree(plan->dsign4096);
         cudaFree(plan->gsign4096);
         cudaFree(plan->partial);
@@ -223,6 +229,8 @@ int bfq_plan_destroy(bfq_plan* plan) {
     cudaFree(plan->img4096);
     cudaFree(plan->prep4096);
     cudaFree(plan->img_b4096);
+    cudaFree(plan->img8192);
+    cudaFree(plan->prep8192);
     cudaFree(plan->dsign4096);
     cudaFree(plan->gsign4096);
     cudaFree(plan->partial);
@@ -239,6 +247,8 @@ int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
     cudaError_t e;
     if (plan->img4096 != nullptr) {
         e = fwdq4096_set_angles(plan, theta, static_cast<cudaStream_t>(stream));
+    } else if (plan->img8192 != nullptr) {
+        e = fwdq8192_set_angles(plan, theta, static_cast<cudaStream_t>(stream));
     } else {
         const int count = plan->log_n * (plan->n / 2);
         k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
@@ -286,6 +296,11 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq4096_available(plan)) {
         e = fwdq4096_launch(plan, x, rows, ldx, codes, scales, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
+    if (xt == BFQ_BF16 && bits == 2 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq8192_available(plan)) {
+        e = fwdq8192_launch(plan, x, rows, ldx, codes, scales, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     GenericParams p{};

@@ -16,6 +16,14 @@ cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaSt
 cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st);
 
+// n = 8192, bf16 rows, INT2: two-CTA clusters, one 4096-point half per CTA
+size_t fwdq8192_image_bytes();
+size_t fwdq8192_prep_bytes();
+bool fwdq8192_available(const bfq_plan* plan);
+cudaError_t fwdq8192_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st);
+cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                            uint16_t* scales, cudaStream_t st);
+
 // n = 4096, bf16 x / g / dx: backward with tensor-memory constants and accumulators
 size_t bwd4096_image_bytes();
 size_t bwd4096_dsign_bytes();

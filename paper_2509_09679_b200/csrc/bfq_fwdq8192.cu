@@ -1,0 +1,432 @@
+// Tuned forward + INT2 quantization for n = 8192 bf16 rows on sm_100a.
+//
+// Stages 0-11 of the 13-stage transform never leave a half of the row (their pair strides are at most
+// 2048), so a row is two independent 4096-point transforms, each with its own angles, followed by one
+// stage that pairs element i of the lower half with element i of the upper half.  The 13 stages of
+// rotation constants (425984 bytes) do not fit the tensor memory of one SM, but each half's twelve
+// stages do.  So the kernel runs as clusters of two CTAs on the two SMs of a processor cluster:
+// CTA rank h holds the constants of half h in its tensor memory and runs the 12-stage pipeline of the
+// n = 4096 kernel (same thread roles, phases, regroupings: bfq_n4096.cuh) on half h of every row the
+// cluster owns.  For stage 12 the two CTAs swap half of their registers through distributed shared
+// memory (rank 0 finishes packed registers 0-7 of both halves, rank 1 registers 8-15), rotate with a
+// general 2x2 form that also restores the signs the angle reduction tracked, exchange their absmax,
+// and each writes the INT2 codes of the elements it finished.  Every cross-CTA wait is a bounded
+// mbarrier wait; the cluster-wide barriers at entry and exit involve every thread unconditionally.
+#include "bfq_fast.h"
+#include "bfq_generic.cuh"
+#include "bfq_n4096.cuh"
+
+namespace bfq {
+namespace f8k {
+using namespace ptx;
+using namespace f4k;
+
+constexpr int kN8 = 8192;
+constexpr int kCols8 = 384 + 64;  // 12 three-shear stages of this half + this rank's share of stage 12
+
+template <int G>
+struct Smem {
+    static constexpr uint32_t kInOff = 0;                                  // [G][kInSlots][kRowBytes]
+    static constexpr uint32_t kExOff = kInOff + G * kInSlots * kRowBytes;  // [G][2][kExBytes]
+    static constexpr uint32_t kPeerOff = kExOff + G * 2 * kExBytes;        // [G][8][128] packed pairs from the peer
+    static constexpr uint32_t kAmaxOff = kPeerOff + G * 8 * kGroupThreads * 8;  // float [G][2 parities][8]
+    static constexpr uint32_t kBarOff = kAmaxOff + 64 * G;                 // mbarriers [G][kInSlots + 2]
+    static constexpr uint32_t kTmemOff = kBarOff + 8 * G * (kInSlots + 2);
+    static constexpr uint32_t kUsed = kTmemOff + 16;
+    static constexpr uint32_t kBytes = kUsed + 1024;
+};
+
+struct ExAddr {
+    uint32_t w1, r1, w2, r2;
+    int bar;
+};
+
+__device__ __forceinline__ void regroup1(u64 (&P)[16], const ExAddr& ex) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) sts64(ex.w1 + ex1_wr_local(m), P[m]);
+    __syncwarp();
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r1 + ex1_rd_local(m));
+}
+__device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+        uint32_t lo, hi;
+        unpack2u(P[m], lo, hi);
+        sts32(ex.w2 + ex2_wr_local(m, 0), lo);
+        sts32(ex.w2 + ex2_wr_local(m, 1), hi);
+    }
+    bar_sync(ex.bar, kGroupThreads);
+#pragma unroll
+    for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r2 + ex2_rd_local(m));
+}
+
+// 12 three-shear stages in chunks of 32 constants; chunk C is in Tcur, chunk C+1 (after the last stage:
+// the first half of this rank's stage-12 constants) is requested right after the wait
+template <int C, class F>
+__device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[32], uint32_t (&Tnext)[32], uint32_t tbase,
+                                           const ExAddr& ex, F&& issue_next) {
+    tmem_wait_ld32(Tcur);
+    tmem_ld32(tbase + 32 * (C + 1), Tnext);
+    stage_lift<C & 3, 0, 8, 32>(P, Tcur);
+    if constexpr (C == 3) regroup1(P, ex);
+    if constexpr (C == 7) {
+        regroup2(P, ex);
+        issue_next();
+    }
+    if constexpr (C + 1 < 12) run_chunks<C + 1>(P, Tnext, Tcur, tbase, ex, issue_next);
+}
+
+// stage 12 on four (lower-half, upper-half) register pairs: out_lo = k1*a + k2*b, out_hi = k3*a + k4*b
+template <int I0>
+__device__ __forceinline__ void stage12_quad(u64 (&A)[8], u64 (&B)[8], const uint32_t (&T)[32]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const u64 K1 = pack2u(T[8 * i], T[8 * i + 1]), K2 = pack2u(T[8 * i + 2], T[8 * i + 3]);
+        const u64 K3 = pack2u(T[8 * i + 4], T[8 * i + 5]), K4 = pack2u(T[8 * i + 6], T[8 * i + 7]);
+        const u64 a = A[I0 + i], b = B[I0 + i];
+        A[I0 + i] = fma2(K2, b, mul2(K1, a));
+        B[I0 + i] = fma2(K4, b, mul2(K3, a));
+    }
+}
+
+// two INT2 codes of a packed pair (elements e, e+1) as a nibble: bits 0-1 = code(e), bits 2-3 = code(e+1)
+__device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool plain) {
+    if (plain) {
+        // |v * inv| <= 1.0005: v*inv + 1.5*2^23 has q in {-1, 0, 1} (mod 4) in its two low bits
+        uint32_t lo, hi;
+        unpack2u(fma2(v, inv2, pack2(12582912.0f, 12582912.0f)), lo, hi);
+        return (lo & 3u) | ((hi & 3u) << 2);
+    }
+    float a, b;
+    unpack2(v, a, b);
+    const int qa = static_cast<int>(fminf(fmaxf(rintf(a * inv), -2.f), 1.f));
+    const int qb = static_cast<int>(fminf(fmaxf(rintf(b * inv), -2.f), 1.f));
+    return (static_cast<uint32_t>(qa) & 3u) | ((static_cast<uint32_t>(qb) & 3u) << 2);
+}
+
+template <int G>
+__global__ void __launch_bounds__(G * kGroupThreads, 1)
+k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
+           const float* __restrict__ img, uint8_t* __restrict__ codes, uint16_t* __restrict__ scales, int rows,
+           int* __restrict__ status) {
+    using S = Smem<G>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q = warp & 3, g = warp >> 2;
+    const int t = q * 32 + lane;                  // role within the group: 0..127
+    const uint32_t rank = cluster_ctarank();      // which half of every row this CTA transforms
+    const uint32_t peer = rank ^ 1u;
+
+    const uint32_t bar_in = sbase + S::kBarOff + 8 * g * (kInSlots + 2);  // [kInSlots] TMA, then swap, then absmax
+    const uint32_t bar_swap = bar_in + 8 * kInSlots, bar_amax = bar_swap + 8;
+    if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
+    if (t == 0) {
+        for (int k = 0; k < kInSlots; ++k) mbar_init(bar_in + 8 * k, 1);
+        mbar_init(bar_swap, 1);  // per row: this thread's arrive.expect_tx + the peer's 8 KB of asynchronous stores
+        mbar_init(bar_amax, 1);
+        mbar_init_fence();
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+    cluster_sync_all();  // the peer's barriers exist before anything arrives on them
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
+    const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+
+    const int n_clusters = gridDim.x >> 1;
+    const int first = (blockIdx.x >> 1) * G + g;
+    const int stride = n_clusters * G;
+    const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
+    const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
+    const CUtensorMap* tmap = rank == 0 ? &map_lo : &map_hi;
+
+    if (t == 0) {
+        for (int k = 0; k < kInSlots && k < count; ++k) {
+            mbar_expect_tx(bar_in + 8 * k, kRowBytes);
+            tma_load_3d(in_base + k * kRowBytes, tmap, 0, 0, first + k * stride, bar_in + 8 * k);
+        }
+    }
+    {
+        const float4* src = reinterpret_cast<const float4*>(img + (static_cast<size_t>(rank) * 128 + q * 32 + lane) * kCols8);
+        for (int c = 16 * g; c < kCols8; c += 16 * G) {
+            uint32_t v[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 f = __ldg(src + (c >> 2) + i);
+                v[4 * i + 0] = __float_as_uint(f.x), v[4 * i + 1] = __float_as_uint(f.y);
+                v[4 * i + 2] = __float_as_uint(f.z), v[4 * i + 3] = __float_as_uint(f.w);
+            }
+            tmem_st16(tlane + c, v);
+        }
+        tmem_wait_st();
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+
+    ExAddr ex;
+    {
+        const uint32_t eb1 = sbase + S::kExOff + g * 2 * kExBytes, eb2 = eb1 + kExBytes;
+        const uint32_t t4 = (t >> 4) & 1, t5 = (t >> 5) & 1, t6 = (t >> 6) & 1;
+        ex.w1 = eb1 + 4u * (2u * (t & 15) + 32u * (t >> 4));
+        ex.r1 = eb1 + 4u * (258u * (t & 15) + 32u * (t >> 4));
+        ex.w2 = eb2 + 4u * ((t & 15) + 2064u * t4 + 512u * t5 + 1024u * t6);
+        ex.r2 = eb2 + 4u * (2u * (t & 15) + 32u * (t >> 4));
+        ex.bar = 1 + g;
+    }
+    const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+    const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+    const uint32_t my_box = sbase + S::kPeerOff + (g * 8 * kGroupThreads + t) * 8;  // + i * 1024: register i from the peer
+    const uint32_t peer_box = map_to_cta(my_box, peer);
+    const uint32_t amax_base = sbase + S::kAmaxOff + g * 64;                         // [2][8] floats
+    const uint32_t peer_amax = map_to_cta(amax_base, peer);
+    const uint32_t peer_bar_swap = map_to_cta(bar_swap, peer), peer_bar_amax = map_to_cta(bar_amax, peer);
+    // INT2 codes: elements 2t + 256m, +1 are a nibble of byte (t >> 1) + 64m; lanes t, t^1 share the byte.  The
+    // even lane stores the bytes of the lower half of the row, the odd lane those of the upper half.
+    uint8_t* const out_t = codes + (t >> 1) + 64 * 8 * rank + ((t & 1) ? 1024 : 0);
+
+    u64 P[16];
+    uint32_t T0[32], T1[32];
+
+    for (int k = 0; k < count; ++k) {
+        const int row = first + k * stride;
+        const int slot = k & 1;
+        tmem_ld32(tlane, T0);
+        mbar_wait_bounded(bar_in + 8 * slot, (k >> 1) & 1, status);
+        const uint32_t src = in_base + slot * kRowBytes + in_line;
+        {
+            uint4 w[2][2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) w[h][c] = lds128(src + 512u * h + (in_x ^ ((c | (h << 2)) << 4)));
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const uint32_t a[4] = {w[0][c].x, w[0][c].y, w[0][c].z, w[0][c].w};
+                const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    P[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
+                    P[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
+                }
+            }
+        }
+        run_chunks<0>(P, T0, T1, tlane, ex, [&]() {
+            if (t == 0 && k + kInSlots < count) {
+                mbar_expect_tx(bar_in + 8 * slot, kRowBytes);
+                tma_load_3d(in_base + slot * kRowBytes, tmap, 0, 0, first + (k + kInSlots) * stride, bar_in + 8 * slot);
+            }
+        });  // the first 32 of this rank's stage-12 constants are now requested in T0
+
+        // ---- stage 12: rank 0 finishes registers 0-7 of both halves, rank 1 registers 8-15 ----
+        u64 A[8], B[8];  // lower-half / upper-half values of the registers this rank finishes
+        if (t == 0) {  // this row's incoming bytes: 8 registers from each of the peer's 128 threads, then its absmax
+            mbar_expect_tx(bar_swap, 8 * 8 * kGroupThreads);
+            mbar_expect_tx(bar_amax, 4);
+        }
+        if (rank == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) st_async_b64(peer_box + i * 1024u, P[8 + i], peer_bar_swap);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) st_async_b64(peer_box + i * 1024u, P[i], peer_bar_swap);
+        }
+        mbar_wait_cluster_bounded(bar_swap, k & 1, status);
+        if (rank == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) A[i] = P[i], B[i] = lds64(my_box + i * 1024u);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) A[i] = lds64(my_box + i * 1024u), B[i] = P[8 + i];
+        }
+        tmem_wait_ld32(T0);
+        tmem_ld32(tlane + 416, T1);
+        stage12_quad<0>(A, B, T0);
+        tmem_wait_ld32(T1);
+        stage12_quad<4>(A, B, T1);
+
+        // ---- absmax of the whole row: thread, warp, group, then the peer's half ----
+        float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float a0, a1, b0, b1;
+            unpack2(A[i], a0, a1);
+            unpack2(B[i], b0, b1);
+            m0 = fmaxf(m0, fmaxf(fabsf(a0), fabsf(b0)));
+            m1 = fmaxf(m1, fmaxf(fabsf(a1), fabsf(b1)));
+        }
+        float amax = fmaxf(m0, m1);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+        const uint32_t aslot = amax_base + (k & 1) * 32;
+        if (lane == 0) sts32(aslot + q * 4, __float_as_uint(amax));
+        bar_sync(ex.bar, kGroupThreads);
+        {
+            const uint4 o = lds128(aslot);
+            amax = fmaxf(fmaxf(__uint_as_float(o.x), __uint_as_float(o.y)),
+                         fmaxf(__uint_as_float(o.z), __uint_as_float(o.w)));
+        }
+        if (t == 0) {
+            st_async_b32(peer_amax + (k & 1) * 32 + 16, __float_as_uint(amax), peer_bar_amax);
+        }
+        mbar_wait_cluster_bounded(bar_amax, k & 1, status);
+        amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
+        float inv;
+        const uint16_t s16 = row_scale(amax, 1, &inv);
+        if (rank == 0 && t == 0) scales[row] = s16;
+
+        const uint32_t e16 = (s16 >> 10) & 31u;
+        const bool plain = (e16 != 0u) && (s16 != 0x7BFFu);  // normal fp16 scale: |v*inv| <= 1.0005, no clipping
+        const u64 inv2 = pack2(inv, inv);
+        uint8_t* out = out_t + static_cast<size_t>(row) * (kN8 / 4);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t nl = nibble_int2(A[i], inv2, inv, plain), nh = nibble_int2(B[i], inv2, inv, plain);
+            const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (t & 1) ? nl : nh, 1);
+            // even lane: its lower-half nibble + the odd lane's; odd lane: the even lane's upper-half nibble + its own
+            out[64 * i] = static_cast<uint8_t>((t & 1) ? (got | (nh << 4)) : (nl | (got << 4)));
+        }
+    }
+
+    tmem_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc512(tmem_base);
+    cluster_sync_all();  // neither CTA leaves while the other may still write into its shared memory
+}
+
+// ---- table preparation -----------------------------------------------------------------------------------
+// Step 1 (one thread per angle): cos/sin table entry, reduced-angle three-shear constants and whether the
+// reduction negates the pair (as for n = 4096: r = theta mod 2 pi, negated iff |r| > pi/2).
+__global__ void __launch_bounds__(256) k_prep_angles8192(const float* __restrict__ theta, float2* __restrict__ tw,
+                                                          float4* __restrict__ prep, uint8_t* __restrict__ flip) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 13 * (kN8 / 2)) return;
+    const double kPi = 3.14159265358979323846;
+    const double th = static_cast<double>(theta[k]);
+    double sn, c;
+    sincos(th, &sn, &c);
+    tw[k] = make_float2(static_cast<float>(c), static_cast<float>(sn));
+    double te = remainder(th, 2.0 * kPi);
+    bool f = false;
+    if (te > 0.5 * kPi) {
+        te -= kPi, f = true;
+    } else if (te < -0.5 * kPi) {
+        te += kPi, f = true;
+    }
+    flip[k] = f ? 1 : 0;
+    prep[k] = make_float4(static_cast<float>(-tan(0.5 * te)), static_cast<float>(sin(te)), static_cast<float>(c),
+                          static_cast<float>(sn));
+}
+
+// sign carried by element i (0..4095) of half `half` when it enters stage s <= 12: stages 0..11 pair inside
+// the half, and pair j of such a stage belongs to the upper half iff j >= 2048
+__device__ __forceinline__ int sign_before8(const uint8_t* __restrict__ flip, int half, int i, int s) {
+    int f = 0;
+    for (int sp = 0; sp < s; ++sp) {
+        const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
+        f ^= flip[sp * (kN8 / 2) + half * (kN / 2) + j];
+    }
+    return f ? -1 : 1;
+}
+
+// Step 2 (one thread per angle): constants of pair (s, j) into the image of the CTA rank that uses them,
+// img[rank][role][column]
+__global__ void __launch_bounds__(256) k_build_image8192(const float4* __restrict__ prep,
+                                                          const uint8_t* __restrict__ flip, float* __restrict__ img) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 13 * (kN8 / 2)) return;
+    const int s = k / (kN8 / 2), j = k % (kN8 / 2);
+    const float4 p = prep[k];
+    if (s < 12) {
+        const int half = j >> 11, jj = j & 2047;
+        const int lo = ((jj >> s) << (s + 1)) | (jj & ((1 << s) - 1));  // inside the half
+        const int hi = lo + (1 << s);
+        const int sa = sign_before8(flip, half, lo, s), sb = sign_before8(flip, half, hi, s);
+        const int kk = s & 3;
+        int r, m, h;
+        if (s < 4) {
+            r = ((lo >> 4) & 15) | ((lo >> 9) << 4), m = lo & 15, h = (lo >> 8) & 1;
+        } else if (s < 8) {
+            r = (lo & 15) | ((lo >> 9) << 4), m = (lo >> 4) & 15, h = (lo >> 8) & 1;
+        } else {
+            r = (lo >> 1) & 127, m = lo >> 8, h = lo & 1;
+        }
+        const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
+        const float sg = (sa == sb) ? 1.f : -1.f;
+        float* strip = img + (static_cast<size_t>(half) * 128 + r) * kCols8;
+        strip[32 * s + 4 * u + h] = sg * p.x;
+        strip[32 * s + 4 * u + h + 2] = sg * p.y;
+    } else {
+        // stage 12: element j of the lower half with element j of the upper half, in phase-3 ownership;
+        // registers 0-7 are finished by rank 0, 8-15 by rank 1
+        const int sa = sign_before8(flip, 0, j, 12), sb = sign_before8(flip, 1, j, 12);
+        const int r = (j >> 1) & 127, m = j >> 8, h = j & 1;
+        float* strip = img + (static_cast<size_t>(m >> 3) * 128 + r) * kCols8;
+        const int col = 384 + 8 * (m & 7) + h;
+        strip[col + 0] = p.z * sa;
+        strip[col + 2] = -p.w * sb;
+        strip[col + 4] = p.w * sa;
+        strip[col + 6] = p.z * sb;
+    }
+}
+
+}  // namespace f8k
+
+// ---- host side ---------------------------------------------------------------------------------------------
+size_t fwdq8192_image_bytes() { return size_t(2) * 128 * f8k::kCols8 * sizeof(float); }
+size_t fwdq8192_prep_bytes() { return size_t(13) * (f8k::kN8 / 2) * (sizeof(float4) + 1); }
+
+cudaError_t fwdq8192_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st) {
+    const int count = 13 * (f8k::kN8 / 2);
+    float4* prep = reinterpret_cast<float4*>(plan->prep8192);
+    uint8_t* flip = reinterpret_cast<uint8_t*>(prep + count);
+    f8k::k_prep_angles8192<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, flip);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    f8k::k_build_image8192<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img8192);
+    return cudaGetLastError();
+}
+
+bool fwdq8192_available(const bfq_plan* plan) {
+    return plan->n == f8k::kN8 && plan->cc_major == 10 && plan->img8192 != nullptr && plan->sm_count >= 2 &&
+           encode_tiled() != nullptr;
+}
+
+cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                            uint16_t* scales, cudaStream_t st) {
+    constexpr int G = 4;
+    using S = f8k::Smem<G>;
+    auto kern = f8k::k_fwdq8192<G>;
+    static bool attr_set[kMaxDevices] = {false};
+    if (!attr_set[plan->device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[plan->device] = true;
+    }
+    CUtensorMap map_lo, map_hi;
+    const uint16_t* xb = static_cast<const uint16_t*>(x);
+    if (!encode_row_map(&map_lo, xb, rows, ldx) || !encode_row_map(&map_hi, xb + f4k::kN, rows, ldx))
+        return cudaErrorInvalidValue;
+    const int64_t want = (rows + G - 1) / G;
+    const int max_clusters = plan->sm_count / 2;
+    const int clusters = int(want < max_clusters ? want : max_clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * clusters, 1, 1);
+    cfg.blockDim = dim3(G * f4k::kGroupThreads, 1, 1);
+    cfg.dynamicSmemBytes = S::kBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192), codes, scales,
+                              int(rows), plan->status_word);
+}
+
+}  // namespace bfq

@@ -30,6 +30,11 @@ __device__ __forceinline__ u64 lds64(uint32_t a) {
     asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(a));
     return v;
 }
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
 __device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
 }

@@ -22,6 +22,8 @@ struct bfq_plan {
     int8_t* dsign4096 = nullptr; // [12][2048] sign applied to the accumulated d-theta (n = 4096 only)
     uint32_t* gsign4096 = nullptr;  // [16 * 128] sign words applied to bf16 g rows (n = 4096 only)
     bool bwd_tables_valid = false;  // the three above match the current angles
+    float* img8192 = nullptr;    // [2][128][448] constants of the n = 8192 forward kernel, one image per CTA rank
+    void* prep8192 = nullptr;    // staging for that image build
     float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
     int64_t partial_slots = 0;
     int* status_word = nullptr;  // device: non-zero when a bounded wait gave up

@@ -98,6 +98,64 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int 
         : "memory");
 }
 
+// ---- thread-block clusters: rank, peer shared-memory addresses, remote stores and mbarrier arrivals -------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the peer CTA's copy of a shared::cta address of this CTA
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_b64(uint32_t cluster_addr, u64 v) {
+    asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(cluster_addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_b32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// asynchronous store into another CTA's shared memory; its bytes are counted on that CTA's mbarrier
+__device__ __forceinline__ void st_async_b64(uint32_t cluster_addr, u64 v, uint32_t cluster_bar) {
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];" ::"r"(cluster_addr), "l"(v),
+                 "r"(cluster_bar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_b32(uint32_t cluster_addr, uint32_t v, uint32_t cluster_bar) {
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(cluster_addr), "r"(v),
+                 "r"(cluster_bar)
+                 : "memory");
+}
+// arrive (count 1) on an mbarrier of another CTA of the cluster; releases this thread's earlier stores
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded like mbar_wait_bounded, for barriers that a peer CTA arrives on
+__device__ __forceinline__ void mbar_wait_cluster_bounded(uint32_t bar, uint32_t parity, int* status,
+                                                          int limit = 1 << 22) {
+    for (int i = 0; i < limit; ++i) {
+        if (mbar_try_wait_cluster(bar, parity)) return;
+    }
+    atomicExch(status, 2);
+}
+// all threads of all CTAs of the cluster
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // ---- tensor memory -------------------------------------------------------------------------------------
 // All 512 columns of the SM's tensor memory; executed by one full warp.  The base address is written
 // to *smem_dst.

@@ -362,3 +362,55 @@ def test_full_size_backward_n4096_sampled():
     for r0 in range(0, rows, 8192):
         acc += oracle.backward(th64, to_f64(x[r0:r0 + 8192]), to_f64(g[r0:r0 + 8192]))[1]
     check_dtheta(dth.view, acc, "learn4096 dtheta")
+
+
+# ---- tuned forward + INT2 for n = 8192 bf16 rows (two-CTA clusters) ---------------------------------------------
+@pytest.mark.parametrize("rows", [1, 2, 3, 5, 73, 74 * 4 + 1, 1000])
+@pytest.mark.parametrize("angle_kind", ["normal", "uniform"])
+def test_tuned_n8192_int2_ragged_row_counts(rows, angle_kind):
+    n = 8192
+    theta = synth.angles(n, angle_kind, 80 + rows)
+    if angle_kind == "uniform":
+        theta[:, ::7] = math.pi / 2
+        theta[:, 1::7] = -math.pi
+        theta[:, 2::7] = math.pi
+        theta[:, 3::7] = -math.pi / 2
+        theta[:, 4::7] = 100.0
+    x = synth.rows(rows, n, "laplace", 81 + rows, outliers=16, outlier_scale=100.0, dtype=torch.bfloat16)
+    if rows >= 5:  # degenerate rows: zero, fp16-underflowing, fp16-saturating and subnormal scales
+        x[0] = 0
+        x[1] *= 1e-9
+        x[2] *= 1e4
+        x[3] *= 3e-8
+    p = plan_for(n, theta)
+    ld = n + 8
+    xpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    codes = Guarded((rows, n // 4), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.forward_quant(xpad[:, :n], 2, codes=codes.view, scales=scales.view)
+    assert p.device_status() == 0
+    check_quant(codes.view, scales.view, oracle.forward(to_f64(theta), to_f64(x)), 2, f"tuned 8192 rows={rows}")
+    assert codes.intact() and scales.intact()
+    c2, s2 = p.forward_quant(xpad[:, :n], 2)
+    assert torch.equal(c2, codes.view) and torch.equal(s2.view(torch.int16), scales.view.view(torch.int16))
+
+
+def test_full_size_int2_n8192_and_fold_sampled():
+    for name in ("act8192_int2", "fold8192_int2"):
+        wl = synth.WORKLOADS[name]
+        theta = wl.theta(device=DEV)
+        x = wl.x(device=DEV)
+        p = Plan(wl.n, DEV)
+        p.set_angles(theta)
+        if name.startswith("fold"):
+            codes, scales, _ = p.fold_weights(x, 2)
+        else:
+            codes, scales = p.forward_quant(x, 2)
+        assert p.device_status() == 0
+        idx = _sample_rows(wl.n_rows, 1024)
+        ti = torch.from_numpy(idx).to(DEV)
+        y_ref = oracle.forward(to_f64(theta), to_f64(x[ti]))
+        stats = check_quant(codes[ti], scales[ti], y_ref, 2, name)
+        assert stats["scale_ulp_rows"] <= max(4, len(idx) // 100)
+        del x, codes, scales
