@@ -330,6 +330,16 @@ int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64
     if (rows == 0) return BFQ_OK;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    if (yt == BFQ_BF16 && rows < (int64_t(1) << 31) && x != y && !env_flag("BFQ_GENERIC_ONLY") && bwd4096_available(plan)) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        cudaError_t e = cudaSuccess;
+        if (!plan->bwd_tables_valid) {  // shared with bfq_backward: built on first use after bfq_set_angles
+            e = bwd4096_build_tables(plan, st);
+            plan->bwd_tables_valid = (e == cudaSuccess);
+        }
+        if (e == cudaSuccess) e = inv4096_launch(plan, y, rows, ldy, x, xt == BFQ_BF16, ldx, st);
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     GenericParams p{};
     p.tw = plan->tw, p.x = y, p.xt = yt, p.ldx = ldy, p.y = x, p.yt = xt, p.ldy = ldx, p.rows = rows;
     cudaError_t e = launch_generic<kModeInverse>(plan, p, static_cast<cudaStream_t>(stream));

@@ -526,6 +526,178 @@ __global__ void __launch_bounds__(256) k_build_gsign4096(const uint8_t* __restri
     gsign[w] = (s0 < 0 ? 0x00008000u : 0u) | (s1 < 0 ? 0x80000000u : 0u);
 }
 
+
+// =================================================================================================================
+// Inverse / transpose for n = 4096 bf16 rows:  x = Q^T y.  The reverse walk of the backward kernel on one array,
+// organised like the forward kernel: four row groups of 128 threads per CTA, 32 constants per tensor-memory chunk.
+// =================================================================================================================
+template <int G>
+struct InvSmem {
+    static constexpr uint32_t kInOff = 0;                                  // [G][kInSlots][kRowBytes]
+    static constexpr uint32_t kExOff = kInOff + G * kInSlots * kRowBytes;  // [G][2][kExBytes]
+    static constexpr uint32_t kBarOff = kExOff + G * 2 * kExBytes;         // mbarriers [G][kInSlots]
+    static constexpr uint32_t kTmemOff = kBarOff + 8 * G * kInSlots;
+    static constexpr uint32_t kUsed = kTmemOff + 16;
+    static constexpr uint32_t kBytes = kUsed + 1024;
+};
+
+// stage S (11..0) is in Tcur; stage S-1 is requested right after the wait
+template <int S, class F>
+__device__ __forceinline__ void inv_stages(u64 (&P)[16], uint32_t (&Tcur)[32], uint32_t (&Tnext)[32], uint32_t tlane,
+                                           const Addr& a, uint32_t buf2, uint32_t buf1, F&& after_phase3) {
+    tmem_wait_ld32(Tcur);
+    if constexpr (S > 0) tmem_ld32(tlane + 32 * (S - 1), Tnext);
+    stage_lift<S & 3, 0, 8, 32>(P, Tcur);
+    if constexpr (S == 8) {
+        bar_sync(a.bar, kThreads);  // every warp is past its scalar reads of the previous row
+        rev2_store(P, buf2, a);
+        bar_sync(a.bar, kThreads);
+        after_phase3();
+        rev2_load(P, buf2, a);
+    }
+    if constexpr (S == 4) {
+        __syncwarp();
+        rev1_store(P, buf1, a);
+        __syncwarp();
+        rev1_load(P, buf1, a);
+    }
+    if constexpr (S > 0) inv_stages<S - 1>(P, Tnext, Tcur, tlane, a, buf2, buf1, after_phase3);
+}
+
+template <int G, bool OUT_BF16>
+__global__ void __launch_bounds__(G * kThreads, 1)
+k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ img, const uint32_t* __restrict__ gsign,
+          void* __restrict__ xout, int64_t ldx, int rows, int* __restrict__ status) {
+    using S = InvSmem<G>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q = warp & 3, g = warp >> 2;
+    const int t = q * 32 + lane;
+
+    if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
+    if (threadIdx.x < G * kInSlots) {
+        mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
+        mbar_init_fence();
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
+    const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+
+    const int first = blockIdx.x * G + g;
+    const int stride = gridDim.x * G;
+    const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
+    const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
+    const uint32_t bar_base = sbase + S::kBarOff + 8 * g * kInSlots;
+    if (t == 0) {
+        for (int k = 0; k < kInSlots && k < count; ++k) {
+            mbar_expect_tx(bar_base + 8 * k, kRowBytes);
+            tma_load_3d(in_base + k * kRowBytes, &ymap, 0, 0, first + k * stride, bar_base + 8 * k);
+        }
+    }
+    {
+        const float4* src = reinterpret_cast<const float4*>(img + (q * 32 + lane) * kConstCols);
+        for (int c = 16 * g; c < kConstCols; c += 16 * G) {
+            uint32_t v[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 f = __ldg(src + (c >> 2) + i);
+                v[4 * i + 0] = __float_as_uint(f.x), v[4 * i + 1] = __float_as_uint(f.y);
+                v[4 * i + 2] = __float_as_uint(f.z), v[4 * i + 3] = __float_as_uint(f.w);
+            }
+            tmem_st16(tlane + c, v);
+        }
+        tmem_wait_st();
+    }
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+
+    Addr a;
+    {
+        const uint32_t t4 = (t >> 4) & 1, t5 = (t >> 5) & 1, t6 = (t >> 6) & 1;
+        a.ex = sbase + S::kExOff + g * 2 * kExBytes;
+        a.bar = 1 + g;
+        a.w1 = 4u * (2u * (t & 15) + 32u * (t >> 4));
+        a.r1 = 4u * (258u * (t & 15) + 32u * (t >> 4));
+        a.w2 = 4u * ((t & 15) + 2064u * t4 + 512u * t5 + 1024u * t6);
+        a.r2 = 4u * (2u * (t & 15) + 32u * (t >> 4));
+    }
+    const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
+    const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
+    const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
+    const uint32_t par_t = __popc(t) & 1;
+    const uint32_t sgn_a = par_t ? 0x80000000u : 0u, sgn_b = par_t ? 0u : 0x80000000u;
+    const uint4* gsv = reinterpret_cast<const uint4*>(gsign);
+
+    u64 P[16];
+    uint32_t T0[32], T1[32];
+    for (int k = 0; k < count; ++k) {
+        const int row = first + k * stride;
+        const int slot = k & 1;
+        tmem_ld32(tlane + 32 * 11, T0);
+        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+        const uint32_t tile = in_base + slot * kRowBytes;
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) {
+            const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
+            const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int m = 4 * qq + i;
+                const uint32_t w = lds32(tile + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
+                P[m] = pack2u(w << 16, w & 0xFFFF0000u);
+            }
+        }
+        inv_stages<11>(P, T0, T1, tlane, a, a.ex, a.ex + kExBytes, [&]() {
+            if (t == 0 && k + kInSlots < count) {
+                mbar_expect_tx(bar_base + 8 * slot, kRowBytes);
+                tma_load_3d(in_base + slot * kRowBytes, &ymap, 0, 0, first + (k + kInSlots) * stride, bar_base + 8 * slot);
+            }
+        });
+        // phase-1 ownership: two runs of 16 consecutive elements; undo the parity sign
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int64_t off = static_cast<int64_t>(row) * ldx + 16 * (t & 15) + 512 * (t >> 4) + 256 * h;
+            if constexpr (OUT_BF16) {
+                uint32_t w[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t lo0, hi0, lo1, hi1;
+                    unpack2u(P[2 * j], lo0, hi0);
+                    unpack2u(P[2 * j + 1], lo1, hi1);
+                    const float e0 = __uint_as_float(h ? hi0 : lo0), e1 = __uint_as_float(h ? hi1 : lo1);
+                    const bool odd_c = ((__builtin_popcount(2 * j) + h) & 1) != 0;
+                    const uint32_t neg_lo = odd_c ? (sgn_b >> 16) : (sgn_a >> 16);
+                    const uint32_t neg_hi = odd_c ? sgn_a : sgn_b;
+                    w[j] = cvt_bf16x2(e0, e1) ^ (neg_lo | neg_hi);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(xout) + off);
+                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            } else {
+                uint32_t w[16];
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    uint32_t lo, hi;
+                    unpack2u(P[m], lo, hi);
+                    const bool odd_c = ((__builtin_popcount(m) + h) & 1) != 0;  // parity popcount(m) ^ h ^ popcount(t)
+                    w[m] = (h ? hi : lo) ^ (odd_c ? sgn_b : sgn_a);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(xout) + off);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) dst[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+            }
+        }
+    }
+    tmem_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc512(tmem_base);
+}
+
 }  // namespace b4k
 
 // ---- host side ---------------------------------------------------------------------------------------------
@@ -571,6 +743,33 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
     const int count = 12 * (f4k::kN / 2);
     k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid, count, dtheta);
     plan->last_backward_partials = grid;
+    return cudaGetLastError();
+}
+
+cudaError_t inv4096_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, bool x_bf16, int64_t ldx,
+                           cudaStream_t st) {
+    constexpr int G = 4;
+    using S = b4k::InvSmem<G>;
+    static bool attr_set[kMaxDevices] = {false};
+    if (!attr_set[plan->device]) {
+        cudaError_t e = cudaFuncSetAttribute(b4k::k_inv4096<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             int(S::kBytes));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(b4k::k_inv4096<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[plan->device] = true;
+    }
+    CUtensorMap ymap;
+    if (!encode_row_map(&ymap, y, rows, ldy)) return cudaErrorInvalidValue;
+    const int64_t want = (rows + G - 1) / G;
+    const int grid = int(want < plan->sm_count ? want : plan->sm_count);
+    if (x_bf16) {
+        b4k::k_inv4096<G, true><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->gsign4096, x, ldx,
+                                                                            int(rows), plan->status_word);
+    } else {
+        b4k::k_inv4096<G, false><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->gsign4096, x, ldx,
+                                                                             int(rows), plan->status_word);
+    }
     return cudaGetLastError();
 }
 

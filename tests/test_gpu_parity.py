@@ -414,3 +414,33 @@ def test_full_size_int2_n8192_and_fold_sampled():
         stats = check_quant(codes[ti], scales[ti], y_ref, 2, name)
         assert stats["scale_ulp_rows"] <= max(4, len(idx) // 100)
         del x, codes, scales
+
+
+# ---- tuned inverse for n = 4096 bf16 rows ------------------------------------------------------------------------
+@pytest.mark.parametrize("rows", [1, 3, 147, 148 * 4 + 1, 1000])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_tuned_inverse_n4096(rows, out_dtype):
+    n = 4096
+    theta = synth.angles(n, "uniform", 90 + rows)
+    theta[:, ::7] = math.pi / 2
+    theta[:, 1::7] = -math.pi
+    theta[:, 3::7] = -math.pi / 2
+    theta[:, 4::7] = 100.0
+    y = synth.rows(rows, n, "student_t3", 91 + rows, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    ld = n + 8
+    ypad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    ypad[:, :n] = y.to(DEV)
+    out = Guarded((rows, ld), out_dtype, DEV)
+    p.inverse(ypad[:, :n], out=out.view[:, :n])
+    assert p.device_status() == 0
+    check_rows_close(out.view[:, :n], oracle.inverse(to_f64(theta), to_f64(y)), absmax_rows(y), f"tuned inverse rows={rows}")
+    assert out.intact()
+    # new angles on the same plan: the tables follow
+    theta2 = synth.angles(n, "normal", 92 + rows)
+    p.set_angles(theta2.to(DEV))
+    x2 = p.inverse(y.to(DEV), out_dtype=out_dtype)
+    check_rows_close(x2, oracle.inverse(to_f64(theta2), to_f64(y)), absmax_rows(y), "tuned inverse, second angle set")
+    # round trip through the tuned-path forward of the generic kernels
+    back = p.forward(x2.float(), out_dtype=torch.float32)
+    check_rows_close(back, to_f64(y), 64 * absmax_rows(y), "round trip") if out_dtype == torch.float32 else None
