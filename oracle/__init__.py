@@ -40,6 +40,8 @@ def lib() -> ctypes.CDLL:
         P = ctypes.c_void_p
         L.orc_forward.argtypes = [i64, P, P, i64, i64, P, i64]
         L.orc_inverse.argtypes = [i64, P, P, i64, i64, P, i64]
+        L.orc_hadamard.argtypes = [i64, P, i64, i64, P, i64]
+        L.orc_hadamard.restype = i32
         L.orc_dense_stage.argtypes = [i64, i32, P, P]
         L.orc_quantize.argtypes = [i64, i32, P, i64, i64, P, P, P, P]
         L.orc_pack.argtypes = [i64, i32, P, i64, P]
@@ -103,6 +105,16 @@ def inverse(theta, y) -> np.ndarray:
     x = np.empty_like(y2)
     _check(lib().orc_inverse(n, _ptr(th), _ptr(y2), y2.shape[0], n, _ptr(x), n), "inverse")
     return x.reshape(y.shape)
+
+
+def hadamard(x) -> np.ndarray:
+    """y = H_n x per row, H_n the normalised Sylvester-Hadamard matrix of the paper's Sec. 3.1.1."""
+    x = _f64(x)
+    x2 = x.reshape(-1, x.shape[-1])
+    n = x2.shape[1]
+    y = np.empty_like(x2)
+    _check(lib().orc_hadamard(n, _ptr(x2), x2.shape[0], n, _ptr(y), n), "hadamard")
+    return y.reshape(x.shape)
 
 
 def dense_stage(n: int, s: int, theta_s) -> np.ndarray:

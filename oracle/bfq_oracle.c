@@ -30,7 +30,8 @@
  * Kronecker closed form for stage-uniform angles; stage-by-stage == dense product;
  * inverse(forward(x)) = x; d theta == central finite differences; adjoint identity;
  * quantizer closed-form properties and a hand-worked example; fold invariance
- * (W Q^T)(Q x) = W x; fp16 rounding against numpy's float16.
+ * (W Q^T)(Q x) = W x; fp16 rounding against numpy's float16; the Hadamard transform against the
+ * Kronecker power of H_2, |entries| = 1/sqrt(n) and the theta = pi/4 butterfly (Q = H_n D).
  */
 #include <math.h>
 #include <stdint.h>
@@ -168,6 +169,44 @@ int orc_inverse(int64_t n, const double* theta, const double* y, int64_t rows, i
         for (int s = L - 1; s >= 0; --s) stage_transpose(n, s, theta + (int64_t)s * (n / 2), z);
     }
     return 0;
+}
+
+/*
+ * Normalised Walsh-Hadamard transform y = H_n x, the fixed rotation the paper compares against
+ * (Sec. 3.1.1): H_1 = [1], H_2n = 1/sqrt(2) [[H_n, H_n], [H_n, -H_n]].  Written as that recursion:
+ * the first and second halves of x are transformed by H_{n/2}, then combined.
+ */
+static void hadamard_rec(int64_t n, double* z, double* tmp) {
+    if (n == 1) return;
+    const int64_t h = n / 2;
+    hadamard_rec(h, z, tmp);
+    hadamard_rec(h, z + h, tmp);
+    const double r = 1.0 / sqrt(2.0);
+    for (int64_t i = 0; i < h; ++i) {
+        const double a = z[i], b = z[h + i];
+        tmp[i] = r * (a + b);
+        tmp[h + i] = r * (a - b);
+    }
+    memcpy(z, tmp, sizeof(double) * (size_t)n);
+}
+
+int orc_hadamard(int64_t n, const double* x, int64_t rows, int64_t ldx, double* y, int64_t ldy) {
+    if (ilog2_exact(n) < 0) return -1;
+    int64_t r;
+    int fail = 0;
+#pragma omp parallel for schedule(static)
+    for (r = 0; r < rows; ++r) {
+        double* tmp = (double*)malloc(sizeof(double) * (size_t)n);
+        if (!tmp) {
+            fail = 1;
+            continue;
+        }
+        double* z = y + r * ldy;
+        memmove(z, x + r * ldx, sizeof(double) * (size_t)n);
+        hadamard_rec(n, z, tmp);
+        free(tmp);
+    }
+    return fail ? -8 : 0;
 }
 
 /*

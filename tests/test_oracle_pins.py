@@ -353,3 +353,25 @@ def test_bf16_widening_is_exact():
     t = torch.randn(1000, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
     bits = t.view(torch.int16).numpy()
     assert np.array_equal(oracle.bf16_bits_to_f64(bits), t.to(torch.float64).numpy())
+
+
+# ---- Hadamard transform (the fixed rotation of Sec. 3.1.1) -----------------------------------------------
+def test_hadamard_is_the_kronecker_power_of_h2_and_relates_to_the_pi_over_4_butterfly():
+    h2 = np.array([[1.0, 1.0], [1.0, -1.0]]) / math.sqrt(2.0)
+    for n in (2, 4, 8, 64):
+        H = np.array([[1.0]])
+        for _ in range(n.bit_length() - 1):
+            H = np.kron(h2, H)  # H_2n = 1/sqrt(2) [[H, H], [H, -H]]
+        got = oracle.hadamard(np.eye(n)).T  # row i of the result is H e_i, i.e. column i of H
+        np.testing.assert_allclose(got, H, atol=1e-14)
+        np.testing.assert_allclose(np.abs(got), 1.0 / math.sqrt(n), atol=1e-14)  # coherence 1/sqrt(n)
+        np.testing.assert_allclose(got @ got.T, np.eye(n), atol=1e-13)
+        # theorem "Hadamard is a butterfly": all theta = pi/4 gives Q = H_n D, D_jj = (-1)^popcount(j)
+        theta = np.full((n.bit_length() - 1, n // 2), math.pi / 4)
+        x = RNG.standard_normal((5, n))
+        D = np.array([(-1.0) ** bin(j).count("1") for j in range(n)])
+        np.testing.assert_allclose(oracle.forward(theta, x), oracle.hadamard(x * D), atol=1e-13)
+    x = RNG.standard_normal((3, 4096))
+    y = oracle.hadamard(x)
+    np.testing.assert_allclose(np.linalg.norm(y, axis=1), np.linalg.norm(x, axis=1), rtol=1e-13)
+    np.testing.assert_allclose(oracle.hadamard(y), x, atol=1e-12)  # H is symmetric and orthogonal
