@@ -375,8 +375,9 @@ def finish(torch, args, wl, synth, x, dev, world, value, ms_step, kernel_ms_avg,
 
 
 def time_others(torch, synth, Plan, dev):
-    """Backward (learning batch), inverse, n = 8192 INT2 and weight folding: device-timed,
-    inputs resident, 3 warm-up + a few timed launches each."""
+    """Hadamard / unquantized variants of the headline, backward (learning batch), inverse, n = 8192 INT2 and
+    weight folding: device-timed, inputs resident, 3 warm-up + a few timed launches each.  alu_frac uses the
+    paper's FLOP table: 4 slots per pair for the butterfly, 1 (an add or a subtract per element) for Hadamard."""
     res = {}
     alu_peak = torch.cuda.get_device_properties(dev).multi_processor_count * FP32_LANES_PER_SM * 1.965e9
 
@@ -388,6 +389,19 @@ def time_others(torch, synth, Plan, dev):
         res[name] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": bytes_per_row * rows / (ms * 1e-3) / 1e9,
                      "alu_frac": slots / alu_peak / (ms * 1e-3), "rows": rows, "n": n}
 
+    # the fixed Hadamard rotation and the unquantized (16-bit activation) outputs on the headline rows
+    wl = synth.WORKLOADS[WORKLOAD]
+    plan = Plan(wl.n, dev)
+    plan.set_angles(wl.theta(device=dev))
+    x = wl.x(device=dev)
+    codes = torch.empty((wl.n_rows, wl.n // 2), dtype=torch.uint8, device=dev)
+    scales = torch.empty((wl.n_rows,), dtype=torch.float16, device=dev)
+    y = torch.empty_like(x)
+    record("hadamard_int4_n4096", wl.n_rows, wl.n, wl.L, 1, BYTES_PER_ROW,
+           lambda: plan.hadamard_quant(x, 4, codes=codes, scales=scales), 20)
+    record("forward_bf16_n4096", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan.forward(x, out=y), 20)
+    record("hadamard_bf16_n4096", wl.n_rows, wl.n, wl.L, 1, 4 * wl.n, lambda: plan.hadamard(x, out=y), 20)
+    del x, y, codes, scales, plan
     # angle-learning step: forward + backward on 128 x 2048 rows of n = 4096
     wl = synth.WORKLOADS["learn4096"]
     theta = wl.theta(device=dev)

@@ -96,6 +96,19 @@ int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows,
                       int bits, uint8_t* codes, uint16_t* scales_f16, void* stream);
 
 /*
+ * The fixed rotation the paper compares the learned butterfly with (Sec. 3.1.1, Hadamard transform; QuaRot's
+ * x' = H x): y = H_n x per row, H_1 = [1], H_2n = 1/sqrt(2) [[H_n, H_n], [H_n, -H_n]].  Needs no angles
+ * (bfq_set_angles may or may not have been called).  With all theta = pi/4 the butterfly is H_n diag((-1)^popcount(j)).
+ * bfq_hadamard_quant fuses the same per-row quantizer as bfq_forward_quant.  Together with bfq_forward
+ * (unquantized rows, the weight-only "W2A16" setting of the paper's main table) these two let one machine
+ * measure what the learned rotation costs over the fixed one ("Inference Efficiency" / FLOP-comparison table).
+ */
+int bfq_hadamard(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, void* y, bfq_dtype yt,
+                 int64_t ldy, void* stream);
+int bfq_hadamard_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
+                       uint8_t* codes, uint16_t* scales_f16, void* stream);
+
+/*
  * x = Q^T y (= Q^{-1} y: Q is orthogonal by construction, Sec. 3.2.1): stages L-1..0, each
  * pair mapped by G(theta)^T.  Also dL/dx = Q^T g.
  */

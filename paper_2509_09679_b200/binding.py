@@ -30,6 +30,8 @@ SIGNATURES = {
     "bfq_forward": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
     "bfq_forward_quant": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p]),
     "bfq_inverse": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
+    "bfq_hadamard": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
+    "bfq_hadamard_quant": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p]),
     "bfq_backward": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _p, _i, _p, _p]),
     "bfq_fold_weights": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p, _i, _p]),
     "bfq_device_status": (_i, [_p]),
@@ -134,6 +136,24 @@ class Plan:
             scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
         _check(lib().bfq_forward_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
                                        scales.data_ptr(), _stream(x)), "bfq_forward_quant")
+        return codes, scales
+
+    def hadamard(self, x: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
+        rows, ldx = _rows(x, self.n)
+        y = out if out is not None else torch.empty((rows, self.n), dtype=out_dtype or x.dtype, device=x.device)
+        _, ldy = _rows(y, self.n)
+        _check(lib().bfq_hadamard(self._h, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(), _dt(y), ldy, _stream(x)),
+               "bfq_hadamard")
+        return y
+
+    def hadamard_quant(self, x: torch.Tensor, bits: int, codes=None, scales=None):
+        rows, ldx = _rows(x, self.n)
+        if codes is None:
+            codes = torch.empty((rows, self.n * bits // 8), dtype=torch.uint8, device=x.device)
+        if scales is None:
+            scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        _check(lib().bfq_hadamard_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
+                                        scales.data_ptr(), _stream(x)), "bfq_hadamard_quant")
         return codes, scales
 
     def inverse(self, y: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:

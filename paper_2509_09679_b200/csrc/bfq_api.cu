@@ -270,6 +270,12 @@ int bfq_forward(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64
     if (rows == 0) return BFQ_OK;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    if (xt == BFQ_BF16 && yt == BFQ_BF16 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq4096_available(plan)) {
+        cudaError_t e = fwdq4096_launch(plan, x, rows, ldx, false, nullptr, nullptr, y, ldy,
+                                        static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     GenericParams p{};
     p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = ldy, p.rows = rows;
     cudaError_t e = launch_generic<kModeForward>(plan, p, static_cast<cudaStream_t>(stream));
@@ -295,7 +301,7 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     cudaError_t e;
     if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq4096_available(plan)) {
-        e = fwdq4096_launch(plan, x, rows, ldx, codes, scales, static_cast<cudaStream_t>(stream));
+        e = fwdq4096_launch(plan, x, rows, ldx, false, codes, scales, nullptr, 0, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     if (xt == BFQ_BF16 && bits == 2 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
@@ -318,6 +324,53 @@ int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows,
 int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int64_t ldw, int bits, uint8_t* codes,
                      uint16_t* scales_f16, void* WQt, bfq_dtype ot, void* stream) {
     return forward_quant_impl(plan, W, wt, m, ldw, bits, codes, scales_f16, WQt, ot, stream);
+}
+
+int bfq_hadamard(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, void* y, bfq_dtype yt,
+                 int64_t ldy, void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    int rc = check_rows(x, xt, rows, ldx, plan->n);
+    if (rc == BFQ_OK) rc = check_rows(y, yt, rows, ldy, plan->n);
+    if (rc != BFQ_OK) return rc;
+    if (rows == 0) return BFQ_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (xt == BFQ_BF16 && yt == BFQ_BF16 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq4096_available(plan)) {
+        e = fwdq4096_launch(plan, x, rows, ldx, true, nullptr, nullptr, y, ldy, st);
+    } else {
+        GenericParams p{};
+        p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = ldy, p.rows = rows;
+        e = launch_generic<kModeHadamard>(plan, p, st);
+    }
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+int bfq_hadamard_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                       uint16_t* scales_f16, void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    int rc = check_rows(x, xt, rows, ldx, plan->n);
+    if (rc != BFQ_OK) return rc;
+    if ((codes == nullptr || scales_f16 == nullptr) && rows != 0) return BFQ_ERR_NULL;
+    if (bits != 2 && bits != 4 && bits != 8) return BFQ_ERR_BITS;
+    if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(scales_f16) & 1u) != 0) return BFQ_ERR_ALIGN;
+    if (rows == 0) return BFQ_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (xt == BFQ_BF16 && bits == 4 && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq4096_available(plan)) {
+        e = fwdq4096_launch(plan, x, rows, ldx, true, codes, scales_f16, nullptr, 0, st);
+    } else {
+        GenericParams p{};
+        p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = nullptr, p.yt = BFQ_F32, p.ldy = plan->n;
+        p.codes = codes, p.scales = scales_f16, p.bits = bits, p.rows = rows;
+        e = launch_generic<kModeHadamardQuant>(plan, p, st);
+    }
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
 
 int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64_t ldy, void* x, bfq_dtype xt,

@@ -1,4 +1,5 @@
-// Tuned forward + INT4 quantization for n = 4096 bf16 rows on sm_100a.
+// Tuned forward for n = 4096 bf16 rows on sm_100a: learned butterfly or fixed Walsh-Hadamard rotation, fused with
+// INT4 quantization or writing the rotated rows in bf16.  The description below is the butterfly + INT4 case.
 //
 // Design (one persistent CTA per SM, G row groups of 128 threads):
 //  * A row is owned by one group of four warps, one warp per scheduler and per tensor-memory lane
@@ -128,27 +129,59 @@ __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[CW], u
     if constexpr (C + 1 < CH::kCount) run_chunks<C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, issue_next);
 }
 
-template <int G, int CW, int XB>
+// Walsh-Hadamard stages 4*PH .. 4*PH+3 of a phase: (a, b) -> (a + b, a - b), no constants; the 1/sqrt(n) is
+// applied by the epilogue
+template <int K>
+__device__ __forceinline__ void stage_hadamard(u64 (&P)[16]) {
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        const u64 a = P[m_lo], b = P[m_hi];
+        P[m_lo] = add2(a, b);
+        P[m_hi] = sub2(a, b);
+    }
+}
+template <int XB, class F>
+__device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&& issue_next) {
+    stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);
+    regroup1(P, ex);
+    stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);
+    regroup2<XB>(P, ex);
+    issue_next();
+    stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);
+}
+
+enum : int { kButterfly = 0, kHadamard = 1 };  // TRANSFORM
+enum : int { kOutInt4 = 0, kOutBf16 = 1 };     // OUT
+
+// TRANSFORM: learned butterfly (constants in tensor memory) or the fixed Walsh-Hadamard transform (no constants,
+// no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy).
+template <int G, int CW, int XB, int TRANSFORM, int OUT>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, uint8_t* __restrict__ codes,
-           uint16_t* __restrict__ scales, int rows, int* __restrict__ status) {
+           uint16_t* __restrict__ scales, __nv_bfloat16* __restrict__ yout, int64_t ldy, int rows,
+           int* __restrict__ status) {
     using S = Smem<G, XB>;
+    constexpr bool kTmem = TRANSFORM == kButterfly;
+    constexpr float kPost = TRANSFORM == kHadamard ? 1.0f / 64.0f : 1.0f;  // 1/sqrt(4096), exact
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = warp & 3, g = warp >> 2;
     const int t = q * 32 + lane;  // role within the group: 0..127
 
-    if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
+    if constexpr (kTmem) {
+        if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
+    }
     if (threadIdx.x < G * kInSlots) {
         mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
         mbar_init_fence();
     }
-    tmem_fence_before();
+    if constexpr (kTmem) tmem_fence_before();
     __syncthreads();
-    tmem_fence_after();
-    uint32_t tmem_base;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
+    if constexpr (kTmem) tmem_fence_after();
+    uint32_t tmem_base = 0;
+    if constexpr (kTmem) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
     const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 
     const int first = blockIdx.x * G + g;
@@ -165,7 +198,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         }
     }
     // fill tensor memory: the G warps of a lane quarter share its 26 blocks of 16 columns
-    {
+    if constexpr (kTmem) {
         const float4* src = reinterpret_cast<const float4*>(img + (q * 32 + lane) * kCols);
         for (int c = 16 * g; c < kCols; c += 16 * G) {
             uint32_t v[16];
@@ -178,10 +211,10 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             tmem_st16(tlane + c, v);
         }
         tmem_wait_st();
+        tmem_fence_before();
     }
-    tmem_fence_before();
     __syncthreads();
-    tmem_fence_after();
+    if constexpr (kTmem) tmem_fence_after();
 
     ExAddr ex;
     {
@@ -208,7 +241,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
         const int slot = k & 1;
-        tmem_ld(tlane, T0);
+        if constexpr (kTmem) tmem_ld(tlane, T0);
         mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
         const uint32_t src = in_base + slot * kRowBytes + in_line;
         {
@@ -229,13 +262,32 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                 }
             }
         }
-        run_chunks<0, CW, XB>(P, T0, T1, tlane, ex, [&]() {
+        auto issue_next = [&]() {
             if (t == 0 && k + kInSlots < count) {
                 mbar_expect_tx(bar_base + 8 * slot, kRowBytes);
                 tma_load_3d(in_base + slot * kRowBytes, &tmap, 0, 0, first + (k + kInSlots) * stride,
                             bar_base + 8 * slot);
             }
-        });
+        };
+        if constexpr (kTmem) {
+            run_chunks<0, CW, XB>(P, T0, T1, tlane, ex, issue_next);
+        } else {
+            run_hadamard<XB>(P, ex, issue_next);
+        }
+
+        if constexpr (OUT == kOutBf16) {
+            // thread t holds elements 2t + 256m, +1: one 32-bit word of the bf16 row per packed register
+            uint32_t* out = reinterpret_cast<uint32_t*>(yout + static_cast<int64_t>(row) * ldy) + t;
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                float a, b;
+                unpack2(P[m], a, b);
+                const __nv_bfloat162 v = __floats2bfloat162_rn(a * kPost, b * kPost);
+                out[128 * m] = *reinterpret_cast<const uint32_t*>(&v);
+            }
+            bar_sync(ex.bar, kGroupThreads);  // every warp is past its reads of the second regrouping buffer
+            continue;
+        }
 
         // per-row absmax: thread, warp, then the group's four warps
         float m0 = 0.f, m1 = 0.f;
@@ -258,7 +310,8 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                          fmaxf(__uint_as_float(o.z), __uint_as_float(o.w)));
         }
         float inv;
-        const uint16_t s16 = row_scale(amax, 7, &inv);
+        const uint16_t s16 = row_scale(amax * kPost, 7, &inv);
+        inv *= kPost;  // the registers still hold the un-normalised values (kPost is a power of two)
         if (t == 0) scales[row] = s16;
 
         // codes: thread t holds elements 2t + 256m (+1) = byte t + 128m of the row's packed codes
@@ -288,9 +341,11 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         }
     }
 
-    tmem_fence_before();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc512(tmem_base);
+    if constexpr (kTmem) {
+        tmem_fence_before();
+        __syncthreads();
+        if (warp == 0) tmem_dealloc512(tmem_base);
+    }
 }
 
 // ---- table preparation -----------------------------------------------------------------------------------
@@ -376,12 +431,12 @@ bool fwdq4096_available(const bfq_plan* plan) {
     return plan->n == f4k::kN && plan->cc_major == 10 && plan->img4096 != nullptr && encode_tiled() != nullptr;
 }
 
-template <int G, int CW, int XB>
+template <int G, int CW, int XB, int TRANSFORM, int OUT>
 static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap, int64_t rows, uint8_t* codes,
-                                  uint16_t* scales, cudaStream_t st) {
+                                  uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
     using S = f4k::Smem<G, XB>;
     static bool attr_set[kMaxDevices] = {false};
-    auto kern = f4k::k_fwdq4096<G, CW, XB>;
+    auto kern = f4k::k_fwdq4096<G, CW, XB, TRANSFORM, OUT>;
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
         if (e != cudaSuccess) return e;
@@ -389,18 +444,27 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
     }
     const int64_t want = (rows + G - 1) / G;
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
-    kern<<<grid, G * f4k::kGroupThreads, S::kBytes, st>>>(tmap, plan->img4096, codes, scales, int(rows),
+    kern<<<grid, G * f4k::kGroupThreads, S::kBytes, st>>>(tmap, plan->img4096, codes, scales,
+                                                          static_cast<__nv_bfloat16*>(y), ldy, int(rows),
                                                           plan->status_word);
     return cudaGetLastError();
 }
 
-cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                            uint16_t* scales, cudaStream_t st) {
+// Four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest among the
+// configurations that compile without spills; more groups did not help).
+// hadamard: the fixed Walsh-Hadamard transform instead of the plan's butterfly.  y != nullptr: write the rotated
+// rows in bf16 instead of INT4 codes + scales.
+cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, bool hadamard,
+                            uint8_t* codes, uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
     CUtensorMap tmap;
     if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
-    // four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest
-    // among the configurations that compile without spills; more groups did not help)
-    return launch_variant<4, 32, 2>(plan, tmap, rows, codes, scales, st);
+    using namespace f4k;
+    if (!hadamard) {
+        return y == nullptr ? launch_variant<4, 32, 2, kButterfly, kOutInt4>(plan, tmap, rows, codes, scales, y, ldy, st)
+                            : launch_variant<4, 32, 2, kButterfly, kOutBf16>(plan, tmap, rows, codes, scales, y, ldy, st);
+    }
+    return y == nullptr ? launch_variant<4, 32, 2, kHadamard, kOutInt4>(plan, tmap, rows, codes, scales, y, ldy, st)
+                        : launch_variant<4, 32, 2, kHadamard, kOutBf16>(plan, tmap, rows, codes, scales, y, ldy, st);
 }
 
 }  // namespace bfq

@@ -18,7 +18,7 @@
 namespace bfq {
 
 enum : int { kF32 = 0, kBF16 = 1 };
-enum : int { kModeForward = 0, kModeForwardQuant = 1, kModeInverse = 2 };
+enum : int { kModeForward = 0, kModeForwardQuant = 1, kModeInverse = 2, kModeHadamard = 3, kModeHadamardQuant = 4 };
 
 struct GenericParams {
     const float2* tw;  // [L][n/2] (cos, sin)
@@ -133,6 +133,36 @@ __device__ __forceinline__ void forward_from(float (&v)[R][16], const float2* tw
     if constexpr (P + 1 < Geo<LOG_N>::kPhases) {
         exchange<LOG_N, P, P + 1, R>(v, rowbuf, t);
         forward_from<LOG_N, P + 1, R>(v, tw, rowbuf, t);
+    }
+}
+
+// Walsh-Hadamard version of a phase: (a, b) -> (a + b, a - b) on every pair of the phase's stages, no table;
+// the 1/sqrt(n) normalisation is applied once at the end by the caller
+template <int LOG_N, int P, int R>
+__device__ __forceinline__ void phase_hadamard(float (&v)[R][16]) {
+    using PH = Phase<LOG_N, P>;
+#pragma unroll
+    for (int k = 0; k < PH::kNs; ++k) {
+        const int lb = PH::kF + k;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int e_lo = ((q >> lb) << (lb + 1)) | (q & ((1 << lb) - 1));
+            const int e_hi = e_lo | (1 << lb);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float a = v[r][e_lo], bb = v[r][e_hi];
+                v[r][e_lo] = a + bb;
+                v[r][e_hi] = a - bb;
+            }
+        }
+    }
+}
+template <int LOG_N, int P, int R>
+__device__ __forceinline__ void hadamard_from(float (&v)[R][16], float* rowbuf, int t) {
+    phase_hadamard<LOG_N, P, R>(v);
+    if constexpr (P + 1 < Geo<LOG_N>::kPhases) {
+        exchange<LOG_N, P, P + 1, R>(v, rowbuf, t);
+        hadamard_from<LOG_N, P + 1, R>(v, rowbuf, t);
     }
 }
 
@@ -286,6 +316,16 @@ __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_generic(const GenericP
         if constexpr (MODE == kModeInverse) {
             if constexpr (G::kPhases > 1) exchange<LOG_N, 0, G::kPhases - 1, R>(v, rowbuf, t);
             inverse_from<LOG_N, G::kPhases - 1, R>(v, p.tw, rowbuf, t);
+        } else if constexpr (MODE == kModeHadamard || MODE == kModeHadamardQuant) {
+            hadamard_from<LOG_N, 0, R>(v, rowbuf, t);
+            if constexpr (G::kPhases > 1) exchange<LOG_N, G::kPhases - 1, 0, R>(v, rowbuf, t);
+            // 1/sqrt(n): a power of two for even log2 n
+            const float scale = (LOG_N & 1) ? 0.70710678118654752f / static_cast<float>(1 << (LOG_N / 2))
+                                            : 1.0f / static_cast<float>(1 << (LOG_N / 2));
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[r][e] *= scale;
         } else {
             forward_from<LOG_N, 0, R>(v, p.tw, rowbuf, t);
             if constexpr (G::kPhases > 1) exchange<LOG_N, G::kPhases - 1, 0, R>(v, rowbuf, t);
@@ -296,7 +336,7 @@ __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_generic(const GenericP
             for (int r = 0; r < R; ++r)
                 if (row0 + r < p.rows) store16(p.y, p.yt, (row0 + r) * p.ldy + t * 16, v[r]);
         }
-        if constexpr (MODE == kModeForwardQuant) {
+        if constexpr (MODE == kModeForwardQuant || MODE == kModeHadamardQuant) {
             const int qmax = (1 << (p.bits - 1)) - 1;
             const int64_t row_bytes = (static_cast<int64_t>(G::kN) * p.bits) >> 3;
 #pragma unroll

@@ -444,3 +444,50 @@ def test_tuned_inverse_n4096(rows, out_dtype):
     # round trip through the tuned-path forward of the generic kernels
     back = p.forward(x2.float(), out_dtype=torch.float32)
     check_rows_close(back, to_f64(y), 64 * absmax_rows(y), "round trip") if out_dtype == torch.float32 else None
+
+
+# ---- Walsh-Hadamard transform (the fixed rotation the paper compares with) and unquantized bf16 rows ---------------
+@pytest.mark.parametrize("n", [16, 64, 256, 1024, 2048, 4096, 8192])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_hadamard_every_n(n, dtype):
+    rows = 70 if n >= 2048 else 301
+    x = synth.rows(rows, n, "student_t3", 100 + n, outliers=min(4, n // 4), outlier_scale=20.0, dtype=dtype)
+    p = Plan(n, DEV)  # no angles needed
+    ref = oracle.hadamard(to_f64(x))
+    for out_dtype in (torch.float32, torch.bfloat16):
+        out = Guarded((rows, n), out_dtype, DEV)
+        p.hadamard(x.to(DEV), out=out.view)
+        check_rows_close(out.view, ref, absmax_rows(x), f"hadamard n={n} {dtype}->{out_dtype}")
+        assert out.intact()
+    for bits in (2, 4, 8):
+        codes, scales = p.hadamard_quant(x.to(DEV), bits)
+        check_quant(codes, scales, ref, bits, f"hadamard_quant n={n} bits={bits}")
+    assert p.device_status() == 0
+
+
+@pytest.mark.parametrize("rows", [1, 5, 593, 1000])
+def test_tuned_n4096_hadamard_and_bf16_rows(rows):
+    n = 4096
+    theta = synth.angles(n, "uniform", 110 + rows)
+    x = synth.rows(rows, n, "student_t3", 111 + rows, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    ld = n + 8
+    xpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    xv = xpad[:, :n]
+    y_ref, h_ref = oracle.forward(to_f64(theta), to_f64(x)), oracle.hadamard(to_f64(x))
+    # learned butterfly, unquantized bf16 rows (the weight-only setting: activations stay 16-bit)
+    out = Guarded((rows, ld), torch.bfloat16, DEV)
+    p.forward(xv, out=out.view[:, :n])
+    check_rows_close(out.view[:, :n], y_ref, absmax_rows(x), "tuned forward bf16")
+    assert out.intact()
+    # fixed Hadamard rotation, rows and INT4
+    out = Guarded((rows, ld), torch.bfloat16, DEV)
+    p.hadamard(xv, out=out.view[:, :n])
+    check_rows_close(out.view[:, :n], h_ref, absmax_rows(x), "tuned hadamard bf16")
+    assert out.intact()
+    codes = Guarded((rows, n // 2), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.hadamard_quant(xv, 4, codes=codes.view, scales=scales.view)
+    check_quant(codes.view, scales.view, h_ref, 4, "tuned hadamard INT4")
+    assert codes.intact() and scales.intact() and p.device_status() == 0
