@@ -399,6 +399,8 @@ def time_others(torch, synth, Plan, dev):
     y = torch.empty_like(x)
     record("hadamard_int4_n4096", wl.n_rows, wl.n, wl.L, 1, BYTES_PER_ROW,
            lambda: plan.hadamard_quant(x, 4, codes=codes, scales=scales), 20)
+    record("forward_int4_stats_n4096", wl.n_rows, wl.n, wl.L, 4, BYTES_PER_ROW + 8,
+           lambda: plan.forward_quant_stats(x, 4), 10)
     record("forward_bf16_n4096", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan.forward(x, out=y), 20)
     record("hadamard_bf16_n4096", wl.n_rows, wl.n, wl.L, 1, 4 * wl.n, lambda: plan.hadamard(x, out=y), 20)
     del x, y, codes, scales, plan

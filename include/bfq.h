@@ -96,6 +96,18 @@ int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows,
                       int bits, uint8_t* codes, uint16_t* scales_f16, void* stream);
 
 /*
+ * bfq_forward_quant plus two cheap reductions over the rotated rows y = Q x:
+ *   hist     [2^bits] uint64, overwritten: how often each code occurs over all rows, index = code + 2^(bits-1).
+ *            P_bins = hist / (rows * n) is the distribution whose divergence from uniform is the paper's
+ *            uniformity regulariser L_uniform = D_KL(P_bins || U) (Sec. 3.4); the caller forms the value.
+ *   rowstats [rows][2] fp32: sum_k y_k^2 and sum_k y_k^4 of each row (kurtosis n * s4 / s2^2, sigma^2 = s2 / n,
+ *            max|y| / sigma with the row's scale: the diagnostics of the paper's kurtosis / outlier tables).
+ * Counts are exact for the codes written; the sums are taken in a fixed order (bit-reproducible).
+ */
+int bfq_forward_quant_stats(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
+                            uint8_t* codes, uint16_t* scales_f16, uint64_t* hist, float* rowstats, void* stream);
+
+/*
  * The fixed rotation the paper compares the learned butterfly with (Sec. 3.1.1, Hadamard transform; QuaRot's
  * x' = H x): y = H_n x per row, H_1 = [1], H_2n = 1/sqrt(2) [[H_n, H_n], [H_n, -H_n]].  Needs no angles
  * (bfq_set_angles may or may not have been called).  With all theta = pi/4 the butterfly is H_n diag((-1)^popcount(j)).

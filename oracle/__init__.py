@@ -171,6 +171,28 @@ def dequantize(codes, scale_f16) -> np.ndarray:
     return np.asarray(codes, dtype=np.float64) * f16_bits_to_f64(scale_f16)[:, None]
 
 
+def code_histogram(codes, bits: int) -> np.ndarray:
+    """Counts of every code value, index = code + 2^(bits-1) (the bins of the paper's P_bins, Sec. 3.4)."""
+    c = np.asarray(codes, dtype=np.int64).reshape(-1) + (1 << (bits - 1))
+    return np.bincount(c, minlength=1 << bits).astype(np.int64)
+
+
+def uniformity_kl(hist) -> float:
+    """L_uniform = D_KL(P_bins || U) = sum_i p_i log(p_i * number of bins), 0 log 0 = 0 (Sec. 3.4)."""
+    h = np.asarray(hist, dtype=np.float64)
+    p = h / h.sum()
+    nz = p > 0
+    return float(np.sum(p[nz] * np.log(p[nz] * h.size)))
+
+
+def row_moments(y) -> np.ndarray:
+    """[rows][2]: sum y^2 and sum y^4 per row, in float64."""
+    y = _f64(y)
+    y2 = y.reshape(-1, y.shape[-1])
+    sq = y2 * y2
+    return np.stack([sq.sum(axis=1), (sq * sq).sum(axis=1)], axis=1)
+
+
 def backward(theta, x, g):
     """-> (dx float64 [rows][n], dtheta float64 [L][n/2] summed over rows)."""
     x = _f64(x)

@@ -29,6 +29,7 @@ SIGNATURES = {
     "bfq_set_angles": (_i, [_p, _p, _p]),
     "bfq_forward": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
     "bfq_forward_quant": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p]),
+    "bfq_forward_quant_stats": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p, _p, _p]),
     "bfq_inverse": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
     "bfq_hadamard": (_i, [_p, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
     "bfq_hadamard_quant": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p]),
@@ -137,6 +138,18 @@ class Plan:
         _check(lib().bfq_forward_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
                                        scales.data_ptr(), _stream(x)), "bfq_forward_quant")
         return codes, scales
+
+    def forward_quant_stats(self, x: torch.Tensor, bits: int):
+        """-> (codes, scales, hist int64 [2^bits], rowstats fp32 [rows][2] = (sum y^2, sum y^4))."""
+        rows, ldx = _rows(x, self.n)
+        codes = torch.empty((rows, self.n * bits // 8), dtype=torch.uint8, device=x.device)
+        scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        hist = torch.empty((1 << bits,), dtype=torch.int64, device=x.device)
+        rowstats = torch.empty((rows, 2), dtype=torch.float32, device=x.device)
+        _check(lib().bfq_forward_quant_stats(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
+                                             scales.data_ptr(), hist.data_ptr(), rowstats.data_ptr(), _stream(x)),
+               "bfq_forward_quant_stats")
+        return codes, scales, hist, rowstats
 
     def hadamard(self, x: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
         rows, ldx = _rows(x, self.n)

@@ -63,7 +63,9 @@ static int check_rows(const void* p, int dt, int64_t rows, int64_t ld, int n) {
 template <int LOG_N, int R, int MODE>
 static cudaError_t launch_generic_t(const bfq_plan* plan, const GenericParams& p, cudaStream_t st) {
     using G = Geo<LOG_N>;
-    constexpr size_t smem = sizeof(float) * (size_t(G::kGroups) * R * G::kN + size_t(R) * G::kGroups * G::kWarpsPerRow);
+    // rows being regrouped + per-row reduction slots + the 256-bin code histogram of the statistics variant
+    constexpr size_t smem =
+        sizeof(float) * (size_t(G::kGroups) * R * G::kN + size_t(R) * G::kGroups * G::kWarpsPerRow + 256);
     static int blocks_per_sm[kMaxDevices] = {0};
     auto kern = k_generic<LOG_N, R, MODE>;
     int& occ = blocks_per_sm[plan->device];
@@ -283,7 +285,8 @@ int bfq_forward(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64
 }
 
 static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t rows, int64_t ldx, int bits,
-                              uint8_t* codes, uint16_t* scales, void* y, int yt, void* stream) {
+                              uint8_t* codes, uint16_t* scales, void* y, int yt, void* stream,
+                              unsigned long long* hist = nullptr, float* rowstats = nullptr) {
     if (plan == nullptr) return BFQ_ERR_NULL;
     int rc = check_rows(x, xt, rows, ldx, plan->n);
     if (rc != BFQ_OK) return rc;
@@ -299,19 +302,22 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
     cudaError_t e;
-    if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+    if (hist != nullptr) {  // statistics: the histogram starts at zero; the generic kernels carry them
+        e = cudaMemsetAsync(hist, 0, sizeof(unsigned long long) << bits, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(plan, e);
+    } else if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq4096_available(plan)) {
         e = fwdq4096_launch(plan, x, rows, ldx, false, codes, scales, nullptr, 0, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
-    if (xt == BFQ_BF16 && bits == 2 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
-        fwdq8192_available(plan)) {
+    if (hist == nullptr && xt == BFQ_BF16 && bits == 2 && y == nullptr && rows < (int64_t(1) << 31) &&
+        !env_flag("BFQ_GENERIC_ONLY") && fwdq8192_available(plan)) {
         e = fwdq8192_launch(plan, x, rows, ldx, codes, scales, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     GenericParams p{};
     p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = plan->n;
-    p.codes = codes, p.scales = scales, p.bits = bits, p.rows = rows;
+    p.codes = codes, p.scales = scales, p.bits = bits, p.rows = rows, p.hist = hist, p.rowstats = rowstats;
     e = launch_generic<kModeForwardQuant>(plan, p, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
@@ -319,6 +325,20 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
 int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
                       uint8_t* codes, uint16_t* scales_f16, void* stream) {
     return forward_quant_impl(plan, x, xt, rows, ldx, bits, codes, scales_f16, nullptr, BFQ_F32, stream);
+}
+
+int bfq_forward_quant_stats(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
+                            uint8_t* codes, uint16_t* scales_f16, uint64_t* hist, float* rowstats, void* stream) {
+    if (hist == nullptr || (rowstats == nullptr && rows != 0)) return BFQ_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(hist) & 7u) != 0 || (reinterpret_cast<uintptr_t>(rowstats) & 3u) != 0) return BFQ_ERR_ALIGN;
+    if (bits != 2 && bits != 4 && bits != 8) return BFQ_ERR_BITS;
+    if (rows == 0 && plan != nullptr) {
+        DeviceGuard guard(plan->device);
+        cudaError_t e = cudaMemsetAsync(hist, 0, sizeof(uint64_t) << bits, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(plan, e);
+    }
+    return forward_quant_impl(plan, x, xt, rows, ldx, bits, codes, scales_f16, nullptr, BFQ_F32, stream,
+                              reinterpret_cast<unsigned long long*>(hist), rowstats);
 }
 
 int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int64_t ldw, int bits, uint8_t* codes,

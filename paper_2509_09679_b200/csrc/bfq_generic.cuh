@@ -32,6 +32,9 @@ struct GenericParams {
     uint16_t* scales;
     int bits;
     int64_t rows;
+    // optional statistics of the rotated rows (quantizing modes only; both null or both set)
+    unsigned long long* hist;  // [2^bits] counts of every code value over all rows, index = code + 2^(bits-1)
+    float* rowstats;           // [rows][2]: sum of y^2 and sum of y^4 of each rotated row
 };
 
 struct BackwardParams {
@@ -296,11 +299,40 @@ __device__ __forceinline__ float row_max(float m, float* red, int r, int group, 
     }
 }
 
+// sum over the TPR threads of a row in a fixed order (shuffle tree, then warps in index order); red as in row_max
+template <int LOG_N>
+__device__ __forceinline__ float row_sum(float v, float* red, int r, int group, int t) {
+    using G = Geo<LOG_N>;
+    if constexpr (G::kTPR < 32) {
+#pragma unroll
+        for (int o = G::kTPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        return v;
+    } else {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        constexpr int W = G::kWarpsPerRow;
+        float* slot = red + (r * G::kGroups + group) * W;
+        __syncthreads();  // the slot's previous use (a maximum or another sum) has been read by everyone
+        if ((t & 31) == 0) slot[t >> 5] = v;
+        __syncthreads();
+        float acc = slot[0];
+#pragma unroll
+        for (int w = 1; w < W; ++w) acc += slot[w];
+        return acc;
+    }
+}
+
 template <int LOG_N, int R, int MODE>
 __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_generic(const GenericParams p) {
     using G = Geo<LOG_N>;
     extern __shared__ __align__(16) float smem[];
     float* red = smem + G::kGroups * R * G::kN;  // [R][kGroups][warps per row]
+    unsigned int* shist = reinterpret_cast<unsigned int*>(red + R * G::kGroups * G::kWarpsPerRow);  // [256], stats only
+    const bool stats = (MODE == kModeForwardQuant || MODE == kModeHadamardQuant) && p.hist != nullptr;
+    if (stats) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) shist[i] = 0u;
+        __syncthreads();
+    }
     const int group = threadIdx.x / G::kTPR;
     const int t = threadIdx.x % G::kTPR;
     float* rowbuf = smem + group * R * G::kN;
@@ -351,9 +383,34 @@ __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_generic(const GenericP
                     if (t == 0) p.scales[row0 + r] = s16;
                     store_codes16(p.codes + (row0 + r) * row_bytes + t * 2 * p.bits, p.bits, v[r], inv);
                 }
+                if (stats) {  // uniform over the CTA: the barriers inside row_sum are reached by every thread
+                    float s2 = 0.f, s4 = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float sq = v[r][e] * v[r][e];
+                        s2 += sq;
+                        s4 = fmaf(sq, sq, s4);
+                    }
+                    s2 = row_sum<LOG_N>(s2, red, r, group, t);
+                    s4 = row_sum<LOG_N>(s4, red, r, group, t);
+                    if (row0 + r < p.rows) {
+                        if (t == 0) {
+                            p.rowstats[2 * (row0 + r)] = s2;
+                            p.rowstats[2 * (row0 + r) + 1] = s4;
+                        }
+                        const int qmin = -(1 << (p.bits - 1));
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) atomicAdd(&shist[quant1(v[r][e], inv, qmin, qmax) - qmin], 1u);
+                    }
+                }
             }
             if constexpr (G::kTPR >= 32) __syncthreads();  // red[] is reused by the next tile
         }
+    }
+    if (stats) {  // integer counts: the order of the additions does not matter
+        __syncthreads();
+        for (int i = threadIdx.x; i < (1 << p.bits); i += blockDim.x)
+            if (shist[i] != 0u) atomicAdd(&p.hist[i], static_cast<unsigned long long>(shist[i]));
     }
 }
 

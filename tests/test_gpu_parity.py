@@ -491,3 +491,26 @@ def test_tuned_n4096_hadamard_and_bf16_rows(rows):
     p.hadamard_quant(xv, 4, codes=codes.view, scales=scales.view)
     check_quant(codes.view, scales.view, h_ref, 4, "tuned hadamard INT4")
     assert codes.intact() and scales.intact() and p.device_status() == 0
+
+
+# ---- statistics riding on forward + quantize ---------------------------------------------------------------------
+@pytest.mark.parametrize("n,rows,bits,dtype", [(256, 1000, 4, torch.float32), (4096, 333, 4, torch.bfloat16),
+                                               (8192, 70, 2, torch.bfloat16), (1024, 129, 8, torch.bfloat16)])
+def test_forward_quant_stats(n, rows, bits, dtype):
+    theta, x = make(n, rows, dtype, seed=120 + n)
+    p = plan_for(n, theta)
+    y_ref = oracle.forward(to_f64(theta), to_f64(x))
+    codes, scales, hist, rowstats = p.forward_quant_stats(x.to(DEV), bits)
+    check_quant(codes, scales, y_ref, bits, f"stats codes n={n}")
+    # same codes and scales as the plain entry point (which may take a tuned kernel)
+    c0, s0 = p.forward_quant(x.to(DEV), bits)
+    assert torch.equal(s0.view(torch.int16), scales.view(torch.int16))
+    got = oracle.unpack(codes.cpu().numpy(), bits)
+    # the histogram is exact for the codes written, and close to the oracle's own (boundary cases aside)
+    assert np.array_equal(hist.cpu().numpy(), oracle.code_histogram(got, bits))
+    ref_hist = oracle.code_histogram(oracle.quantize(y_ref, bits)[0], bits)
+    assert np.abs(hist.cpu().numpy() - ref_hist).sum() <= 2 * max(1, int(1e-4 * rows * n)) + 2 * n * 16
+    assert oracle.uniformity_kl(hist.cpu().numpy()) == pytest.approx(oracle.uniformity_kl(ref_hist), abs=2e-3)
+    np.testing.assert_allclose(to_f64(rowstats), oracle.row_moments(y_ref), rtol=2e-5)
+    _, _, hist2, rs2 = p.forward_quant_stats(x.to(DEV), bits)
+    assert torch.equal(hist, hist2) and torch.equal(rs2, rowstats)

@@ -375,3 +375,26 @@ def test_hadamard_is_the_kronecker_power_of_h2_and_relates_to_the_pi_over_4_butt
     y = oracle.hadamard(x)
     np.testing.assert_allclose(np.linalg.norm(y, axis=1), np.linalg.norm(x, axis=1), rtol=1e-13)
     np.testing.assert_allclose(oracle.hadamard(y), x, atol=1e-12)  # H is symmetric and orthogonal
+
+
+# ---- statistics of rotated rows: code histogram, uniformity divergence, moments ---------------------------
+def test_uniformity_kl_and_moments_closed_forms():
+    assert oracle.uniformity_kl(np.full(16, 7)) == pytest.approx(0.0, abs=1e-15)          # uniform bins
+    one = np.zeros(16)
+    one[3] = 5
+    assert oracle.uniformity_kl(one) == pytest.approx(math.log(16.0), rel=1e-15)          # all mass in one bin
+    two = np.zeros(4)
+    two[[0, 2]] = 1
+    assert oracle.uniformity_kl(two) == pytest.approx(math.log(2.0), rel=1e-15)           # half of the bins
+    codes = np.array([[-8, 7, 0, 0], [1, -1, 7, -8]])
+    h = oracle.code_histogram(codes, 4)
+    assert h.sum() == 8 and h[0] == 2 and h[15] == 2 and h[8] == 2 and h[9] == 1 and h[7] == 1
+    # moments: +-1 rows have kurtosis exactly 1; a rotation preserves sum y^2
+    pm = np.where(RNG.random((3, 64)) < 0.5, -1.0, 1.0)
+    m = oracle.row_moments(pm)
+    np.testing.assert_allclose(64 * m[:, 1] / m[:, 0] ** 2, 1.0, rtol=1e-15)
+    theta, x = rand_theta(64), RNG.standard_normal((4, 64))
+    np.testing.assert_allclose(oracle.row_moments(oracle.forward(theta, x))[:, 0], (x * x).sum(axis=1), rtol=1e-12)
+    g = RNG.standard_normal((1, 1 << 20))
+    mg = oracle.row_moments(g)[0]
+    assert (1 << 20) * mg[1] / mg[0] ** 2 == pytest.approx(3.0, abs=0.03)                 # Gaussian kurtosis
