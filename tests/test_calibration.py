@@ -1,0 +1,54 @@
+"""The calibration step built on the kernels (reconstruction loss, straight-through quantizers, SGD with a
+cosine schedule from the identity initialisation): one step against a float64 reference composed from the
+oracle's functions, and descent on a synthetic layer with outlier channels."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_09679_b200 import synth
+from paper_2509_09679_b200.calibrate import LayerCalibrator, calibrate, dequantize
+from parity import to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def reference_step(theta, W, x, bits):
+    """float64: loss and d-theta of mean || x W^T - (Q x) Dequant(Quant(W Q^T))^T ||^2, quantizer passed straight through."""
+    y = oracle.forward(theta, x)
+    Wr = oracle.forward(theta, W)                      # row i of W Q^T is Q w_i
+    codes, scales = oracle.quantize(Wr, bits)
+    Wq = oracle.dequantize(codes, scales)
+    err = y @ Wq.T - x @ W.T
+    k = 2.0 / err.size
+    g_y, g_w = (k * err) @ Wq, (k * err).T @ y
+    return float((err * err).mean()), oracle.backward(theta, x, g_y)[1] + oracle.backward(theta, W, g_w)[1]
+
+
+def test_one_step_matches_the_oracle_composition():
+    n, out, tokens, bits = 256, 64, 128, 4
+    theta = synth.angles(n, "uniform", 131) * 0.3
+    W = synth.rows(out, n, "normal", 132, scale=0.02, dtype=torch.float32)
+    x = synth.rows(tokens, n, "student_t3", 133, outliers=4, outlier_scale=20.0, dtype=torch.float32)
+    cal = LayerCalibrator(W.to(DEV), bits, None, theta=theta.to(DEV))
+    loss, grad = cal.loss_and_grad(x.to(DEV))
+    ref_loss, ref_grad = reference_step(to_f64(theta), to_f64(W), to_f64(x), bits)
+    assert float(loss) == pytest.approx(ref_loss, rel=2e-3)
+    rel = np.linalg.norm(to_f64(grad) - ref_grad) / np.linalg.norm(ref_grad)
+    assert rel <= 5e-3, rel
+    # the torch-side dequantizer agrees with the oracle's
+    codes, scales, _ = cal.plan.fold_weights(W.to(DEV), bits)
+    deq = oracle.dequantize(oracle.unpack(codes.cpu().numpy(), bits), scales.cpu().view(torch.int16).numpy().view(np.uint16))
+    np.testing.assert_array_equal(to_f64(dequantize(codes, scales, bits)), deq)
+
+
+@pytest.mark.parametrize("n,dtype,wbits,abits", [(1024, torch.float32, 2, None), (4096, torch.bfloat16, 4, 4)])
+def test_calibration_reduces_the_reconstruction_loss(n, dtype, wbits, abits):
+    out, tokens = n // 4, 2048
+    W = synth.rows(out, n, "normal", 141, scale=0.02, dtype=dtype).to(DEV)
+    X = synth.rows(tokens, n, "student_t3", 142, outliers=8, outlier_scale=20.0, dtype=dtype).to(DEV)
+    cal, losses = calibrate(W, X, steps=30, batch=tokens, weight_bits=wbits, act_bits=abits)  # full batch: no sampling noise
+    assert all(np.isfinite(losses))
+    assert min(losses[-5:]) < 0.9 * losses[0], losses
+    assert cal.plan.device_status() == 0
