@@ -193,6 +193,31 @@ def row_moments(y) -> np.ndarray:
     return np.stack([sq.sum(axis=1), (sq * sq).sum(axis=1)], axis=1)
 
 
+def cayley(params, n1: int) -> np.ndarray:
+    """Q1 = (I - A)(I + A)^{-1}, A skew-symmetric with the n1 (n1 - 1) / 2 parameters in its upper triangle,
+    row by row (paper Sec. 3.3, "Concrete Example for d = 5120")."""
+    p = _f64(params).reshape(-1)
+    if p.size != n1 * (n1 - 1) // 2:
+        raise ValueError("need n1 (n1 - 1) / 2 parameters")
+    A = np.zeros((n1, n1))
+    A[np.triu_indices(n1, 1)] = p
+    A = A - A.T
+    I = np.eye(n1)
+    return np.linalg.solve((I + A).T, (I - A).T).T  # X (I + A) = (I - A)
+
+
+def composite_forward(Q1, theta2, x) -> np.ndarray:
+    """y = (Q1 kron Q2) x per row, Q2 the butterfly of theta2 (Sec. 3.3): with x as an n1 x n2 matrix X,
+    Y = Q1 (X Q2^T): Q2 on every run of n2 consecutive elements, then Q1 across the n1 runs."""
+    Q1 = _f64(Q1)
+    n1 = Q1.shape[0]
+    x = _f64(x)
+    rows = x.reshape(-1, x.shape[-1])
+    n2 = rows.shape[1] // n1
+    inner = forward(theta2, rows.reshape(-1, n2)).reshape(rows.shape[0], n1, n2)
+    return np.einsum("ik,rkj->rij", Q1, inner).reshape(x.shape)
+
+
 def backward(theta, x, g):
     """-> (dx float64 [rows][n], dtheta float64 [L][n/2] summed over rows)."""
     x = _f64(x)

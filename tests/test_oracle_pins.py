@@ -398,3 +398,30 @@ def test_uniformity_kl_and_moments_closed_forms():
     g = RNG.standard_normal((1, 1 << 20))
     mg = oracle.row_moments(g)[0]
     assert (1 << 20) * mg[1] / mg[0] ** 2 == pytest.approx(3.0, abs=0.03)                 # Gaussian kurtosis
+
+
+# ---- composite transform for non-power-of-2 sizes: Cayley factor (x) butterfly (Sec. 3.3) --------------------
+def test_cayley_and_kronecker_composite():
+    # 2 x 2 by hand: A = [[0, a], [-a, 0]]; (I - A)(I + A)^-1 = [[1 - a^2, -2a], [2a, 1 - a^2]] / (1 + a^2),
+    # the rotation by 2 atan(a)
+    a = 0.37
+    Q = oracle.cayley([a], 2)
+    np.testing.assert_allclose(Q, np.array([[1 - a * a, -2 * a], [2 * a, 1 - a * a]]) / (1 + a * a), atol=1e-15)
+    phi = 2.0 * math.atan(a)
+    np.testing.assert_allclose(Q, [[math.cos(phi), -math.sin(phi)], [math.sin(phi), math.cos(phi)]], atol=1e-15)
+    np.testing.assert_allclose(oracle.cayley(np.zeros(780), 40), np.eye(40), atol=0)        # A = 0 gives I
+    p = RNG.standard_normal(780) * 0.2
+    Q1 = oracle.cayley(p, 40)
+    np.testing.assert_allclose(Q1.T @ Q1, np.eye(40), atol=1e-13)                           # orthogonal by construction
+    assert abs(np.linalg.det(Q1) - 1.0) < 1e-12
+    assert 780 + 7 * 64 == 1228 and round(5120 * 5120 / 1228) == 21347                      # the paper's parameter count
+    # (Q1 kron Q2) x by brute force on a small case, and orthogonality of the composite
+    n1, n2 = 5, 8
+    Q1s = oracle.cayley(RNG.standard_normal(n1 * (n1 - 1) // 2), n1)
+    th2 = rand_theta(n2)
+    K = np.kron(Q1s, dense_Q(th2))
+    x = RNG.standard_normal((6, n1 * n2))
+    np.testing.assert_allclose(oracle.composite_forward(Q1s, th2, x), x @ K.T, atol=1e-13)
+    np.testing.assert_allclose(K.T @ K, np.eye(n1 * n2), atol=1e-13)
+    y = oracle.composite_forward(Q1, rand_theta(128), RNG.standard_normal((2, 5120)))
+    assert y.shape == (2, 5120)
