@@ -57,6 +57,8 @@ typedef enum {
 #define BFQ_MIN_N 16
 #define BFQ_MAX_N 8192
 #define BFQ_NOALLOC_MAX_N 1024 /* largest row length bfq_backward_noalloc accepts */
+#define BFQ_MAX_N1 64          /* largest dense factor of the composite transform */
+#define BFQ_COMPOSITE_MAX_D 16384 /* largest composite row length n1 * n2 */
 
 /*
  * Create a plan for row length n on CUDA device `device` (allocates: twiddle tables,
@@ -148,6 +150,30 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
 int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int64_t ldw,
                      int bits, uint8_t* codes, uint16_t* scales_f16, void* WQt, bfq_dtype ot,
                      void* stream);
+
+/*
+ * Composite transform for row lengths d that are not a power of two (Sec. 3.3, Kronecker product construction):
+ * d = n1 * n2, Q = Q1 (x) Q2, with Q2 the plan's butterfly (n2 = the plan's n, angles from bfq_set_angles) and Q1 a
+ * dense orthogonal n1 x n1 factor.  With a row read as an n1 x n2 matrix X (row r = elements [r n2, (r+1) n2)),
+ *     Y = Q1 (X Q2^T):  y[i n2 + j] = sum_k Q1[i][k] (Q2 x_k)[j],  x_k the k-th run of n2 elements.
+ * The paper's example: d = 5120 = 40 x 128, 780 Cayley parameters + 448 angles.
+ *
+ * bfq_cayley builds Q1 = (I - A)(I + A)^{-1} ("Concrete Example for d = 5120"): params = the n1 (n1 - 1) / 2 entries of
+ * the strict upper triangle of the skew-symmetric A, row by row (device, fp32); q1 = device fp32 [n1][n1] row-major,
+ * written.  Solved in float64 on the device.  2 <= n1 <= BFQ_MAX_N1.  The plan only names the device.
+ *
+ * bfq_composite_forward / _quant: x: [rows][ldx] of xt with ldx >= d; y: [rows][ldy]; codes: [rows][d*bits/8] and one
+ * fp16 scale per row over all d elements (the quantizer of bfq_forward_quant).  q1 is read as given: any n1 x n1
+ * matrix works, the caller keeps it orthogonal.  Needs 16 <= n2 <= 1024 and d <= BFQ_COMPOSITE_MAX_D, else
+ * BFQ_ERR_UNSUPPORTED_N.  For n1 = 40, n2 = 128 and bf16 rows the dense factor runs on the tensor cores in TF32
+ * (inputs rounded to 10 mantissa bits, fp32 accumulation): |error| <= 2e-3 max|y| there, fp32 arithmetic everywhere
+ * else.  x and y must not overlap.
+ */
+int bfq_cayley(bfq_plan* plan, const float* params, int n1, float* q1, void* stream);
+int bfq_composite_forward(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,
+                          int64_t ldx, void* y, bfq_dtype yt, int64_t ldy, void* stream);
+int bfq_composite_forward_quant(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,
+                                int64_t ldx, int bits, uint8_t* codes, uint16_t* scales_f16, void* stream);
 
 /*
  * bfq_backward without any device-memory allocation.  (No counterpart in the paper: this exists for

@@ -40,6 +40,9 @@ SIGNATURES = {
     "bfq_status_string": (ctypes.c_char_p, [_i]),
     "bfq_backward_partials": (_i, [_p]),
     "bfq_backward_noalloc": (_i, [_i, _p, _p, _i, _p, _i, _i64, _i64, _p, _i, _p, _p]),
+    "bfq_cayley": (_i, [_p, _p, _i, _p, _p]),
+    "bfq_composite_forward": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
+    "bfq_composite_forward_quant": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _i, _p, _p, _p]),
 }
 
 _lib = None
@@ -137,6 +140,40 @@ class Plan:
             scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
         _check(lib().bfq_forward_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
                                        scales.data_ptr(), _stream(x)), "bfq_forward_quant")
+        return codes, scales
+
+    # -- composite transform Q1 (x) Q2 for d = n1 * n (paper Sec. 3.3); this plan's butterfly is Q2 --------------
+    def cayley(self, params: torch.Tensor, n1: int) -> torch.Tensor:
+        """Q1 = (I - A)(I + A)^-1 from the n1 (n1 - 1) / 2 upper-triangle entries of the skew A -> fp32 [n1][n1]."""
+        if params.dtype != torch.float32 or params.numel() != n1 * (n1 - 1) // 2 or not params.is_contiguous():
+            raise ValueError("params must be a contiguous fp32 tensor of n1 (n1 - 1) / 2 entries")
+        q1 = torch.empty((n1, n1), dtype=torch.float32, device=params.device)
+        _check(lib().bfq_cayley(self._h, params.data_ptr(), int(n1), q1.data_ptr(), _stream(params)), "bfq_cayley")
+        return q1
+
+    def _q1(self, q1: torch.Tensor) -> int:
+        if q1.dtype != torch.float32 or q1.dim() != 2 or q1.shape[0] != q1.shape[1] or not q1.is_contiguous():
+            raise ValueError("q1 must be a contiguous fp32 [n1][n1] tensor")
+        return q1.shape[0]
+
+    def composite_forward(self, q1: torch.Tensor, x: torch.Tensor, out_dtype=None) -> torch.Tensor:
+        n1 = self._q1(q1)
+        d = n1 * self.n
+        rows, ldx = _rows(x, d)
+        y = torch.empty((rows, d), dtype=out_dtype or x.dtype, device=x.device)
+        _check(lib().bfq_composite_forward(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(),
+                                           _dt(y), d, _stream(x)), "bfq_composite_forward")
+        return y
+
+    def composite_forward_quant(self, q1: torch.Tensor, x: torch.Tensor, bits: int):
+        n1 = self._q1(q1)
+        d = n1 * self.n
+        rows, ldx = _rows(x, d)
+        codes = torch.empty((rows, d * bits // 8), dtype=torch.uint8, device=x.device)
+        scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        _check(lib().bfq_composite_forward_quant(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, int(bits),
+                                                 codes.data_ptr(), scales.data_ptr(), _stream(x)),
+               "bfq_composite_forward_quant")
         return codes, scales
 
     def forward_quant_stats(self, x: torch.Tensor, bits: int):

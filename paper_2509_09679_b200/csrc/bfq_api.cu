@@ -452,6 +452,53 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
     return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
 
+int bfq_cayley(bfq_plan* plan, const float* params, int n1, float* q1, void* stream) {
+    if (plan == nullptr || params == nullptr || q1 == nullptr) return BFQ_ERR_NULL;
+    if (n1 < 2 || n1 > BFQ_MAX_N1) return BFQ_ERR_UNSUPPORTED_N;
+    if ((reinterpret_cast<uintptr_t>(params) & 3u) != 0 || (reinterpret_cast<uintptr_t>(q1) & 3u) != 0) return BFQ_ERR_ALIGN;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaError_t e = cayley_launch(params, n1, q1, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+static int composite_impl(bfq_plan* plan, const float* q1, int n1, const void* x, int xt, int64_t rows, int64_t ldx,
+                          void* y, int yt, int64_t ldy, int bits, uint8_t* codes, uint16_t* scales, void* stream) {
+    if (plan == nullptr || q1 == nullptr) return BFQ_ERR_NULL;
+    if (n1 < 2 || n1 > BFQ_MAX_N1 || plan->n > 1024 || int64_t(n1) * plan->n > BFQ_COMPOSITE_MAX_D)
+        return BFQ_ERR_UNSUPPORTED_N;
+    const int d = n1 * plan->n;
+    int rc = check_rows(x, xt, rows, ldx, d);
+    if (rc != BFQ_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(q1) & 3u) != 0) return BFQ_ERR_ALIGN;
+    if (codes != nullptr || y == nullptr) {  // the quantizing entry point
+        if ((codes == nullptr || scales == nullptr) && rows != 0) return BFQ_ERR_NULL;
+        if (bits != 2 && bits != 4 && bits != 8) return BFQ_ERR_BITS;
+        if (!aligned16(codes) || (reinterpret_cast<uintptr_t>(scales) & 1u) != 0) return BFQ_ERR_ALIGN;
+    } else {
+        rc = check_rows(y, yt, rows, ldy, d);
+        if (rc != BFQ_OK) return rc;
+    }
+    if (!plan->angles_set) return BFQ_ERR_WORKSPACE;
+    if (rows == 0) return BFQ_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaError_t e = composite_generic_launch(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, bits, codes, scales,
+                                             static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+}
+
+int bfq_composite_forward(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,
+                          int64_t ldx, void* y, bfq_dtype yt, int64_t ldy, void* stream) {
+    if (y == nullptr && rows != 0) return BFQ_ERR_NULL;
+    return composite_impl(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, 4, nullptr, nullptr, stream);
+}
+
+int bfq_composite_forward_quant(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,
+                                int64_t ldx, int bits, uint8_t* codes, uint16_t* scales_f16, void* stream) {
+    return composite_impl(plan, q1, n1, x, xt, rows, ldx, nullptr, BFQ_F32, 0, bits, codes, scales_f16, stream);
+}
+
 int bfq_device_status(bfq_plan* plan) {
     if (plan == nullptr) return BFQ_ERR_NULL;
     DeviceGuard guard(plan->device);

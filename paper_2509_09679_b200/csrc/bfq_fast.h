@@ -37,4 +37,10 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
 cudaError_t inv4096_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, bool x_bf16, int64_t ldx,
                            cudaStream_t st);
 
+// composite transform Q1 (x) Q2 (n1 <= 64, n2 = the plan's n): Cayley solve and the kernels for every shape
+cudaError_t cayley_launch(const float* params, int n1, float* q1, cudaStream_t st);
+cudaError_t composite_generic_launch(const bfq_plan* plan, const float* q1, int n1, const void* x, int xt, int64_t rows,
+                                     int64_t ldx, void* y, int yt, int64_t ldy, int bits, uint8_t* codes,
+                                     uint16_t* scales, cudaStream_t st);
+
 }  // namespace bfq

@@ -103,6 +103,17 @@ def rows(
     return out
 
 
+def cayley_params(n1: int, seed: int, std: float = 0.1, device="cpu") -> torch.Tensor:
+    """n1 (n1 - 1) / 2 entries N(0, std^2) for the strict upper triangle of a skew-symmetric matrix, row by row
+    (the dense factor of the composite transform; a small std keeps the factor near the identity, as a learned
+    factor initialised at identity would be)."""
+    return std * torch.randn(n1 * (n1 - 1) // 2, generator=_gen(seed ^ 0xCA71E7, device), dtype=torch.float32, device=device)
+
+
+# the composite example of the paper: hidden size 5120 = 40 x 128 (a LLaMA-13B-shaped activation row)
+COMPOSITE_5120 = dict(n1=40, n2=128, n_rows=32768, dist="student_t3", outliers=8, outlier_scale=50.0, seed=6000)
+
+
 @dataclass(frozen=True)
 class Workload:
     """One of the named configurations (shapes and distributions only)."""
