@@ -157,6 +157,24 @@ static int64_t backward_slots(int log_n, int sm_count) {
     return int64_t(sm_count) * kBackwardCtasPerSm * (threads / tpr);
 }
 
+// frees everything a plan owns (every pointer is null or valid) and the plan itself
+static void release_plan(bfq_plan* plan) {
+    cudaFree(plan->tw);
+    cudaFree(plan->img4096);
+    cudaFree(plan->prep4096);
+    cudaFree(plan->img_b4096);
+    cudaFree(plan->img8192);
+    cudaFree(plan->prep8192);
+    cudaFree(plan->dsign4096);
+    cudaFree(plan->gsign4096);
+    cudaFree(plan->partial);
+    cudaFree(plan->status_word);
+    if (plan->theta_host != nullptr) cudaFreeHost(plan->theta_host);
+    if (plan->theta_event != nullptr) cudaEventDestroy(plan->theta_event);
+    std::free(plan->comp5120);
+    delete plan;
+}
+
 }  // namespace bfq
 
 using namespace bfq;
@@ -200,23 +218,19 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_b4096, bwd4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->dsign4096, bwd4096_dsign_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->gsign4096, bwd4096_gsign_bytes());
+    if (e == cudaSuccess && n == 128) {  // the composite kernel's constants are computed on the host from the angles
+        e = cudaMallocHost(&plan->theta_host, angles * sizeof(float));
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->theta_event, cudaEventDisableTiming);
+        if (e == cudaSuccess) {
+            plan->comp5120 = std::calloc(1, comp5120_param_bytes());
+            if (plan->comp5120 == nullptr) e = cudaErrorMemoryAllocation;
+        }
+    }
     if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
-        cudaFree(plan->tw);
-        cudaFree(plan->img4096);
-        cudaFree(plan->prep4096);
-        cudaFree(plan->img_b4096);
-    cudaFree(plan->img8192);
-    cudaFree(plan->prep8192);
-        cudaFree(plan->img8192);
-        cudaFree(plan->prep8192);
-        cudaFree(plan->dsign4096);
-        cudaFree(plan->gsign4096);
-        cudaFree(plan->partial);
-        cudaFree(plan->status_word);
-        delete plan;
+        release_plan(plan);
         return cuda_fail(nullptr, e);
     }
     *out = plan;
@@ -227,17 +241,7 @@ int bfq_plan_destroy(bfq_plan* plan) {
     if (plan == nullptr) return BFQ_ERR_NULL;
     DeviceGuard guard(plan->device);
     cudaDeviceSynchronize();
-    cudaFree(plan->tw);
-    cudaFree(plan->img4096);
-    cudaFree(plan->prep4096);
-    cudaFree(plan->img_b4096);
-    cudaFree(plan->img8192);
-    cudaFree(plan->prep8192);
-    cudaFree(plan->dsign4096);
-    cudaFree(plan->gsign4096);
-    cudaFree(plan->partial);
-    cudaFree(plan->status_word);
-    delete plan;
+    release_plan(plan);
     return BFQ_OK;
 }
 
@@ -255,6 +259,12 @@ int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
         const int count = plan->log_n * (plan->n / 2);
         k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
         e = cudaGetLastError();
+    }
+    if (e == cudaSuccess && plan->theta_host != nullptr) {
+        e = cudaMemcpyAsync(plan->theta_host, theta, sizeof(float) * plan->log_n * (plan->n / 2), cudaMemcpyDeviceToHost,
+                            static_cast<cudaStream_t>(stream));
+        if (e == cudaSuccess) e = cudaEventRecord(plan->theta_event, static_cast<cudaStream_t>(stream));
+        plan->comp5120_valid = false;
     }
     if (e != cudaSuccess) return cuda_fail(plan, e);
     plan->angles_set = true;
@@ -483,8 +493,14 @@ static int composite_impl(bfq_plan* plan, const float* q1, int n1, const void* x
     if (rows == 0) return BFQ_OK;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
-    cudaError_t e = composite_generic_launch(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, bits, codes, scales,
-                                             static_cast<cudaStream_t>(stream));
+    cudaError_t e;
+    if (n1 == 40 && xt == BFQ_BF16 && rows < (int64_t(1) << 31) && (codes == nullptr || bits == 4) &&
+        (y == nullptr || yt == BFQ_BF16) && !env_flag("BFQ_GENERIC_ONLY") && comp5120_available(plan)) {
+        e = comp5120_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
+    e = composite_generic_launch(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, bits, codes, scales,
+                                 static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
 

@@ -43,4 +43,11 @@ cudaError_t composite_generic_launch(const bfq_plan* plan, const float* q1, int 
                                      int64_t ldx, void* y, int yt, int64_t ldy, int bits, uint8_t* codes,
                                      uint16_t* scales, cudaStream_t st);
 
+
+// composite 40 x 128 on bf16 rows: butterfly with kernel-parameter constants + tcgen05 TF32 dense factor
+bool comp5120_available(const bfq_plan* plan);
+size_t comp5120_param_bytes();
+cudaError_t comp5120_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                            uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
+
 }  // namespace bfq

@@ -24,6 +24,11 @@ struct bfq_plan {
     bool bwd_tables_valid = false;  // the three above match the current angles
     float* img8192 = nullptr;    // [2][128][448] constants of the n = 8192 forward kernel, one image per CTA rank
     void* prep8192 = nullptr;    // staging for that image build
+    float* theta_host = nullptr;    // pinned host copy of the angles (n = 128 only: the composite kernel's constants
+                                    // are kernel parameters computed on the host)
+    cudaEvent_t theta_event = nullptr;  // recorded after that copy
+    void* comp5120 = nullptr;       // host: kernel parameters of the 40 x 128 composite kernel
+    bool comp5120_valid = false;    // they match the current angles
     float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
     int64_t partial_slots = 0;
     int* status_word = nullptr;  // device: non-zero when a bounded wait gave up

@@ -88,3 +88,110 @@ def test_composite_argument_validation():
     assert e.value.status == -7
     y = p.composite_forward(torch.eye(40, device=DEV), x[:0])
     assert y.shape == (0, 5120)
+
+
+# ---- 40 x 128 on bf16 rows: the dense factor runs on the tensor cores in TF32 ------------------------------------
+# Tolerance from the arithmetic: both operands of every product are rounded to 11 significant bits (relative error
+# 2^-12 each, round to nearest), the accumulation is fp32, so
+#     |y - y_ref| <= 2^-11 (1 + 2^-13) sum_k |Q1[i][k]| |X'[k][j]|  +  the fp32 error of the butterfly (1e-5 max|x|).
+# The test allows 2^-10 of that sum (twice the bound).
+def _tf32_setup(rows, seed=5, std=0.1, angle_kind="normal", dist="student_t3"):
+    n1, n2 = 40, 128
+    theta2 = synth.angles(n2, angle_kind, seed)
+    params = synth.cayley_params(n1, seed, std)
+    x = synth.rows(rows, n1 * n2, dist, seed + 1, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
+    p = Plan(n2, DEV)
+    p.set_angles(theta2.to(DEV))
+    q1 = p.cayley(params.to(DEV), n1)
+    Q1 = oracle.cayley(to_f64(params), n1)
+    x64 = to_f64(x)
+    inner = oracle.forward(to_f64(theta2), x64.reshape(-1, n2)).reshape(rows, n1, n2)
+    y_ref = np.einsum("ik,rkj->rij", Q1, inner).reshape(rows, -1)
+    assert np.array_equal(y_ref, oracle.composite_forward(Q1, to_f64(theta2), x64))
+    tol = 2.0 ** -10 * np.einsum("ik,rkj->rij", np.abs(Q1), np.abs(inner)).reshape(rows, -1)
+    tol = tol + 1e-5 * np.abs(x64).max(axis=1, keepdims=True)
+    return p, q1, x, y_ref, tol
+
+
+def _check_tf32_rows(y, y_ref, tol, what):
+    o = to_f64(y)
+    assert np.isfinite(o).all()
+    t = tol + (2.0 ** -8 * np.abs(y_ref) if y.dtype == torch.bfloat16 else 0.0)
+    err = np.abs(o - y_ref)
+    k = np.unravel_index(np.argmax(err - t), err.shape)
+    assert (err <= t).all(), f"{what}: {int((err > t).sum())} out of tolerance; worst at {k}: {err[k]:.3e} > {t[k]:.3e}"
+
+
+def _check_tf32_quant(codes, scales, y_ref, tol, what):
+    rows, d = y_ref.shape
+    got_codes = oracle.unpack(codes.cpu().numpy(), 4)
+    got_s = scales.cpu().view(torch.int16).numpy().view(np.uint16)
+    _, ref_s = oracle.quantize(y_ref, 4)
+    s_got, s_ref = oracle.f16_bits_to_f64(got_s), oracle.f16_bits_to_f64(ref_s)
+    # the absmax moves by at most the tolerance at the extreme element; one fp16 rounding on top
+    assert np.all(np.abs(s_got - s_ref) <= tol.max(axis=1) / 7 + 2.0 ** -10 * s_ref + 1e-30), f"{what}: scales"
+    ref_codes, _, pre = oracle.quantize(y_ref, 4, scale_in=got_s, want_prequant=True)
+    diff = got_codes.astype(np.int32) - ref_codes.astype(np.int32)
+    bad = diff != 0
+    if bad.any():
+        assert np.all(np.abs(diff[bad]) == 1), f"{what}: codes differ by more than one"
+        dist = np.abs(pre - np.floor(pre) - 0.5)
+        allowed = tol / np.maximum(s_got, 1e-30)[:, None] + 1e-4
+        assert np.all(dist[bad] <= allowed[bad]), f"{what}: code mismatch away from a rounding boundary"
+    return float(bad.mean())
+
+
+@pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 7, 8, 9, 591, 592, 593, 148 * 8 + 3, 2500])
+def test_tensor_core_composite_5120(rows):
+    p, q1, x, y_ref, tol = _tf32_setup(rows)
+    xd = x.to(DEV)
+    y = p.composite_forward(q1, xd)
+    assert p.device_status() == 0
+    _check_tf32_rows(y, y_ref, tol, "bf16 rows")
+    codes, scales = p.composite_forward_quant(q1, xd, 4)
+    assert p.device_status() == 0
+    frac = _check_tf32_quant(codes, scales, y_ref, tol, "int4")
+    assert frac <= 2e-2
+
+
+@pytest.mark.parametrize("angle_kind,std", [("uniform", 1.0), ("normal", 0.0)])
+def test_tensor_core_composite_5120_angles_and_factors(angle_kind, std):
+    p, q1, x, y_ref, tol = _tf32_setup(333, seed=9, std=std, angle_kind=angle_kind)
+    y = p.composite_forward(q1, x.to(DEV))
+    _check_tf32_rows(y, y_ref, tol, "bf16 rows")
+    codes, scales = p.composite_forward_quant(q1, x.to(DEV), 4)
+    _check_tf32_quant(codes, scales, y_ref, tol, "int4")
+    assert p.device_status() == 0
+
+
+def test_tensor_core_composite_5120_follows_new_angles_and_the_generic_kernels(monkeypatch):
+    p, q1, x, y_ref, tol = _tf32_setup(200, seed=21)
+    xd = x.to(DEV)
+    y1 = p.composite_forward(q1, xd)
+    th = synth.angles(128, "uniform", 77)
+    p.set_angles(th.to(DEV))
+    y2 = p.composite_forward(q1, xd)
+    monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+    y2g = p.composite_forward(q1, xd, out_dtype=torch.float32)
+    monkeypatch.delenv("BFQ_GENERIC_ONLY")
+    assert not torch.equal(y1, y2)
+    Q1 = to_f64(q1)
+    inner = oracle.forward(to_f64(th), to_f64(x).reshape(-1, 128)).reshape(200, 40, 128)
+    tol2 = 2.0 ** -10 * np.einsum("ik,rkj->rij", np.abs(Q1), np.abs(inner)).reshape(200, -1) + 1e-5 * np.abs(to_f64(x)).max()
+    _check_tf32_rows(y2, to_f64(y2g), tol2 + 1e-5 * np.abs(to_f64(x)).max(), "tensor-core path against the generic kernels")
+
+
+def test_tensor_core_composite_5120_padded_rows_and_guards():
+    from parity import Guarded
+    rows = 37
+    p, q1, x, y_ref, tol = _tf32_setup(rows, seed=13)
+    xs = torch.zeros((rows, 5120 + 64), dtype=torch.bfloat16, device=DEV)
+    xs[:, :5120] = x.to(DEV)
+    codes = Guarded((rows, 2560), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    from paper_2509_09679_b200.binding import lib, _check, _stream
+    _check(lib().bfq_composite_forward_quant(p._h, q1.data_ptr(), 40, xs.data_ptr(), 1, rows, xs.stride(0), 4,
+                                             codes.view.data_ptr(), scales.view.data_ptr(), _stream(xs)), "quant")
+    assert p.device_status() == 0
+    assert codes.intact() and scales.intact()
+    _check_tf32_quant(codes.view, scales.view, y_ref, tol, "int4 with a padded leading dimension")
