@@ -175,7 +175,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler captures of a small case)")
-    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward", "int2_8192"],
+    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward", "int2_8192", "composite5120"],
                     help="backward / int2_8192: time only bfq_backward on the learning batch / bfq_forward_quant "
                          "(INT2) on the n = 8192 activations (for profiler captures; prints a short JSON line, "
                          "not the benchmark line)")
@@ -217,6 +217,8 @@ def main():
         return run_backward_only(torch, args, synth, Plan, dev)
     if args.op == "int2_8192":
         return run_int2_8192_only(torch, args, synth, Plan, dev)
+    if args.op == "composite5120":
+        return run_composite_only(torch, args, synth, Plan, dev)
     wl = synth.WORKLOADS[WORKLOAD]
     if args.rows:
         import dataclasses
@@ -310,6 +312,32 @@ def run_int2_8192_only(torch, args, synth, Plan, dev):
     ms = event_time_ms(torch, lambda: plan.forward_quant(x, 2, codes=codes, scales=scales), args.steps)
     print(json.dumps({"op": "int2_8192", "workload": "act8192_int2", "rows": rows, "ms": ms,
                       "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
+
+
+def composite_inputs(torch, synth, Plan, dev, rows=None):
+    """The paper's composite example, d = 5120 = 40 x 128: plan (Q2 angles), Cayley factor Q1, bf16 token rows."""
+    c = synth.COMPOSITE_5120
+    rows = rows or c["n_rows"]
+    plan = Plan(c["n2"], dev)
+    plan.set_angles(synth.angles(c["n2"], "normal", c["seed"], dev))
+    q1 = plan.cayley(synth.cayley_params(c["n1"], c["seed"], device=dev), c["n1"])
+    x = synth.rows(rows, c["n1"] * c["n2"], c["dist"], c["seed"] + 1, outliers=c["outliers"],
+                   outlier_scale=c["outlier_scale"], dtype=torch.bfloat16, device=dev)
+    return plan, q1, x
+
+
+def run_composite_only(torch, args, synth, Plan, dev):
+    """bfq_composite_forward_quant (INT4) alone on (a prefix of) the d = 5120 token rows."""
+    plan, q1, x = composite_inputs(torch, synth, Plan, dev, args.rows)
+    rows = x.shape[0]
+    codes = torch.empty((rows, 2560), dtype=torch.uint8, device=dev)
+    scales = torch.empty((rows,), dtype=torch.float16, device=dev)
+    for _ in range(args.warmup):
+        plan.composite_forward_quant(q1, x, 4, codes=codes, scales=scales)
+    ms = event_time_ms(torch, lambda: plan.composite_forward_quant(q1, x, 4, codes=codes, scales=scales), args.steps)
+    print(json.dumps({"op": "composite5120", "workload": "composite 40x128 int4", "rows": rows, "ms": ms,
+                      "rows_per_s": rows / (ms * 1e-3), "gbs": rows * (2 * 5120 + 2560 + 2) / (ms * 1e-3) / 1e9,
+                      "status": plan.device_status()}))
 
 
 def run_e2e(torch, args, wl, plan, theta, x, codes, scales, barrier, max_over_ranks, world):
@@ -432,6 +460,22 @@ def time_others(torch, synth, Plan, dev):
     W = wl.x(device=dev)
     record("fold_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
            lambda: plan8.fold_weights(W, 2), 5)
+    del W, plan8
+    torch.cuda.empty_cache()
+    # composite 40 x 128 (d = 5120): butterfly-128 on CUDA cores + the dense factor on the tensor cores
+    planc, q1, x = composite_inputs(torch, synth, Plan, dev)
+    rows = x.shape[0]
+    codes = torch.empty((rows, 2560), dtype=torch.uint8, device=dev)
+    scales = torch.empty((rows,), dtype=torch.float16, device=dev)
+    y = torch.empty_like(x)
+    for name, nbytes, fn in (("composite_int4_d5120", 2 * 5120 + 2560 + 2,
+                              lambda: planc.composite_forward_quant(q1, x, 4, codes=codes, scales=scales)),
+                             ("composite_bf16_d5120", 4 * 5120, lambda: planc.composite_forward(q1, x, out=y))):
+        for _ in range(3):
+            fn()
+        ms = event_time_ms(torch, fn, 10)
+        res[name] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": nbytes * rows / (ms * 1e-3) / 1e9, "rows": rows,
+                     "n": 5120}
     return res
 
 

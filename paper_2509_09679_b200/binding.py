@@ -156,21 +156,23 @@ class Plan:
             raise ValueError("q1 must be a contiguous fp32 [n1][n1] tensor")
         return q1.shape[0]
 
-    def composite_forward(self, q1: torch.Tensor, x: torch.Tensor, out_dtype=None) -> torch.Tensor:
+    def composite_forward(self, q1: torch.Tensor, x: torch.Tensor, out_dtype=None, out=None) -> torch.Tensor:
         n1 = self._q1(q1)
         d = n1 * self.n
         rows, ldx = _rows(x, d)
-        y = torch.empty((rows, d), dtype=out_dtype or x.dtype, device=x.device)
+        y = out if out is not None else torch.empty((rows, d), dtype=out_dtype or x.dtype, device=x.device)
         _check(lib().bfq_composite_forward(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(),
                                            _dt(y), d, _stream(x)), "bfq_composite_forward")
         return y
 
-    def composite_forward_quant(self, q1: torch.Tensor, x: torch.Tensor, bits: int):
+    def composite_forward_quant(self, q1: torch.Tensor, x: torch.Tensor, bits: int, codes=None, scales=None):
         n1 = self._q1(q1)
         d = n1 * self.n
         rows, ldx = _rows(x, d)
-        codes = torch.empty((rows, d * bits // 8), dtype=torch.uint8, device=x.device)
-        scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        if codes is None:
+            codes = torch.empty((rows, d * bits // 8), dtype=torch.uint8, device=x.device)
+        if scales is None:
+            scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
         _check(lib().bfq_composite_forward_quant(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, int(bits),
                                                  codes.data_ptr(), scales.data_ptr(), _stream(x)),
                "bfq_composite_forward_quant")

@@ -54,7 +54,9 @@ constexpr int kKSteps = kN1 / 8;           // 5 MMA steps of K = 8
 constexpr int kHalfBytes = kRuns * 128;            // 20480: one 64-element half of every run of a group
 constexpr int kInStageBytes = 2 * kHalfBytes;      // 40960
 constexpr int kInOff = 0;                          // [2 stages][2 halves][160 lines][128 B], 128-byte swizzle
-constexpr int kALbo = 128;                         // A: bytes between the core matrices of consecutive 4-k chunks
+// A: bytes between the core matrices of consecutive 4-k chunks.  144 rather than 128: the 32 lanes of a butterfly warp
+// hold 32 consecutive k and store the same row, so their words sit at 4 (k mod 4) + 144 (k / 4): 32 distinct banks.
+constexpr int kALbo = 144;
 constexpr int kASbo = (kN1 / 4) * kALbo;           // A: bytes between consecutive 8-row groups
 constexpr int kATile = 16 * kASbo;                 // one tile of A: 128 rows x 40 k, TF32
 constexpr int kAOff = kInOff + 2 * kInStageBytes;  // 81920
@@ -67,7 +69,8 @@ constexpr int kSmemBytes = kBarOff + 128 + 1024;   // barriers + alignment slack
 enum : int { kBarInFull = 0, kBarAFull = 2, kBarMmaDone = 3, kBarDEmpty = 5, kNumBars = 7 };
 
 struct Params {
-    float lift[kStages][kN2 / 2][2];  // (nt, sn) of every pair of every stage
+    float nt[kStages][kN2 / 2];  // lifting constants of every pair of every stage: -tan(phi / 2) ...
+    float sn[kStages][kN2 / 2];  // ... and sin(phi)
     uint32_t sign[4];                 // bit j set: position j of a run carries a pending factor -1
     const float* q1;                  // device, [40][40] row-major
     uint8_t* codes;                   // [rows][2560] or null
@@ -95,6 +98,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 __device__ __forceinline__ bool wait_or_fail(uint32_t bar, uint32_t parity, int* status) {
     for (int i = 0; i < (1 << 22); ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(40);
         if ((i & 1023) == 1023 && *reinterpret_cast<volatile int*>(status) != 0) break;
     }
     atomicExch(status, 1);
@@ -140,19 +144,35 @@ __device__ __forceinline__ void load_run(uint32_t line, int u, float (&x)[kN2]) 
     }
 }
 
-// Q2 on the run: stage s couples lo and lo + 2^s; every constant is a kernel parameter at a fixed offset
+// Q2 on the run: stage s couples lo and lo + 2^s; every constant is a kernel parameter at a fixed offset.  Stage 0
+// couples neighbours and runs on scalars; from stage 1 on positions (2 i, 2 i + 1) travel together in one 64-bit
+// register and two pairs rotate per packed FMA, their constants being two consecutive floats of the parameter block.
 __device__ __forceinline__ void butterfly128(const Params& P, float (&x)[kN2]) {
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) {
+    for (int q = 0; q < kN2 / 2; ++q) {
+        const float nt = P.nt[0][q], sn = P.sn[0][q];
+        x[2 * q] = fmaf(nt, x[2 * q + 1], x[2 * q]);
+        x[2 * q + 1] = fmaf(sn, x[2 * q], x[2 * q + 1]);
+        x[2 * q] = fmaf(nt, x[2 * q + 1], x[2 * q]);
+    }
+    u64 X[kN2 / 2];
 #pragma unroll
-        for (int q = 0; q < kN2 / 2; ++q) {
-            const int lo = ((q >> s) << (s + 1)) | (q & ((1 << s) - 1)), hi = lo + (1 << s);
-            const float nt = P.lift[s][q][0], sn = P.lift[s][q][1];
-            x[lo] = fmaf(nt, x[hi], x[lo]);
-            x[hi] = fmaf(sn, x[lo], x[hi]);
-            x[lo] = fmaf(nt, x[hi], x[lo]);
+    for (int i = 0; i < kN2 / 2; ++i) X[i] = pack2(x[2 * i], x[2 * i + 1]);
+#pragma unroll
+    for (int s = 1; s < kStages; ++s) {
+        const u64* nt2 = reinterpret_cast<const u64*>(&P.nt[s][0]);
+        const u64* sn2 = reinterpret_cast<const u64*>(&P.sn[s][0]);
+#pragma unroll
+        for (int q2 = 0; q2 < kN2 / 4; ++q2) {
+            const int q = 2 * q2, lo = ((q >> s) << (s + 1)) | (q & ((1 << s) - 1)), a = lo >> 1, b = a + (1 << (s - 1));
+            const u64 nt = nt2[q2], sn = sn2[q2];
+            X[a] = fma2(nt, X[b], X[a]);
+            X[b] = fma2(sn, X[a], X[b]);
+            X[a] = fma2(nt, X[b], X[a]);
         }
     }
+#pragma unroll
+    for (int i = 0; i < kN2 / 2; ++i) unpack2(X[i], x[2 * i], x[2 * i + 1]);
 }
 
 // A operand, K-major without swizzle: tile t holds rows m = 32 tau + p (position j = 4 p + t); element (m, k) sits at
@@ -255,6 +275,7 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint32_t bars, ui
         const bool valid = token < P.rows;
         uint32_t q[32];
         float inv = 0.f;
+        bool saturated = false;
         if (P.codes != nullptr) {  // row absmax over all 5120 values, then the fp16 scale
             float amax = 0.f;
 #pragma unroll 1
@@ -266,6 +287,8 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint32_t bars, ui
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
             const uint16_t sb = row_scale(amax, 7, &inv);
+            // clamped or subnormal scale (its rounding error is not small), or an infinite / NaN row: keep the clamp
+            saturated = sb == 0x7BFFu || sb < 0x0400u || !(amax < 3.0e38f);
             if (lane == 0 && valid) P.scales[token] = sb;
         }
         float inv_t[4];
@@ -289,12 +312,29 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint32_t bars, ui
             }
             if (P.codes != nullptr) {
                 uint32_t hw[8];  // four 4-bit codes (j = 4 lane .. 4 lane + 3) of each of the eight runs
+                if (!saturated) {
+                    // |y / s| <= 7 (1 + 2^-10) < 7.5 when s is the row's own normal, unsaturated fp16 scale: no clamp needed;
+                    // adding 1.5 * 2^23 + 8 rounds y * inv to the nearest integer r (ties to even, one rounding) and
+                    // leaves r + 8 in [1, 15] in the low mantissa bits; the four biased codes are packed by
+                    // multiply-adds and the bias is turned into two's complement by flipping bit 3 of every nibble
+                    constexpr float kMagic = 12582920.0f;
+                    constexpr uint32_t kUnbias = 0u - 0x4B400000u * 4369u;  // removes the bits of 1.5 * 2^23 from all four terms
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    hw[e] = 0u;
+                    for (int e = 0; e < 8; ++e) {
+                        uint32_t acc = __float_as_uint(fmaf(__uint_as_float(q[e]), inv_t[0], kMagic));
+                        acc += 16u * __float_as_uint(fmaf(__uint_as_float(q[8 + e]), inv_t[1], kMagic));
+                        acc += 256u * __float_as_uint(fmaf(__uint_as_float(q[16 + e]), inv_t[2], kMagic));
+                        acc += 4096u * __float_as_uint(fmaf(__uint_as_float(q[24 + e]), inv_t[3], kMagic));
+                        hw[e] = ((acc + kUnbias) ^ 0x8888u) & 0xFFFFu;
+                    }
+                } else {
 #pragma unroll
-                    for (int t = 0; t < 4; ++t)
-                        hw[e] |= (static_cast<uint32_t>(quant1(__uint_as_float(q[8 * t + e]), inv_t[t], -8, 7)) & 0xFu) << (4 * t);
+                    for (int e = 0; e < 8; ++e) {
+                        hw[e] = 0u;
+#pragma unroll
+                        for (int t = 0; t < 4; ++t)
+                            hw[e] |= (static_cast<uint32_t>(quant1(__uint_as_float(q[8 * t + e]), inv_t[t], -8, 7)) & 0xFu) << (4 * t);
+                    }
                 }
                 // lanes 2 a and 2 a + 1 hold the two halves of one 32-bit word of every run: the even lane
                 // assembles the word of run i, the odd lane that of run i + 1
@@ -384,8 +424,8 @@ static void build_constants(const float* theta, c5k::Params* P) {
             bool flip = false;
             if (psi > pi / 2) psi -= pi, flip = true;
             else if (psi < -pi / 2) psi += pi, flip = true;
-            P->lift[s][q][0] = static_cast<float>(-std::tan(psi / 2));
-            P->lift[s][q][1] = static_cast<float>(std::sin(psi));
+            P->nt[s][q] = static_cast<float>(-std::tan(psi / 2));
+            P->sn[s][q] = static_cast<float>(std::sin(psi));
             if (flip) sign[lo] = -sign[lo], sign[hi] = -sign[hi];
         }
     }
