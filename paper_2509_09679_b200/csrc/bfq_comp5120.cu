@@ -44,9 +44,9 @@ constexpr int kN1 = 40, kN2 = 128, kD = kN1 * kN2, kStages = 7;
 constexpr int kTok = 4;                    // tokens per group
 constexpr int kRuns = kTok * kN1;          // 160 runs per group
 constexpr int kBatches = kRuns / 32;       // 5 batches of 32 runs
-constexpr int kEpiWarps = 4, kBflyWarps = 6;
+constexpr int kEpiWarps = 4, kBflyWarps = 7;
 constexpr int kMmaWarp = kEpiWarps + kBflyWarps;
-constexpr int kThreads = 32 * (kMmaWarp + 1);  // 352
+constexpr int kThreads = 32 * (kMmaWarp + 1);  // 384
 constexpr int kNPad = 48;                  // MMA N: 40 output runs + 8 zero rows of Q1
 constexpr int kKSteps = kN1 / 8;           // 5 MMA steps of K = 8
 
@@ -85,20 +85,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ uint32_t to_tf32(float v) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
-    return r;
-}
+// fp32 -> TF32 (10 mantissa bits), round to nearest with ties away from zero, for finite values: half an ulp is
+// added to the magnitude and the 13 low bits are cleared (what cvt.rna.tf32.f32 gives, without its NaN handling)
+__device__ __forceinline__ uint32_t to_tf32(float v) { return (__float_as_uint(v) + 0x1000u) & 0xFFFFE000u; }
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 // Bounded wait that also gives up early once any thread of the grid has reported a failure.
+template <int SLEEP_NS = 40>
 __device__ __forceinline__ bool wait_or_fail(uint32_t bar, uint32_t parity, int* status) {
     for (int i = 0; i < (1 << 22); ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(40);
+        __nanosleep(SLEEP_NS);
         if ((i & 1023) == 1023 && *reinterpret_cast<volatile int*>(status) != 0) break;
     }
     atomicExch(status, 1);
@@ -228,7 +227,7 @@ __device__ __forceinline__ void mma_role(const Params& P, const CUtensorMap* tma
     if (n_groups > 1) issue_load(tmap, smem, bars, 1, first + stride);
     int committed = -1;
     for (int g = 0; g < n_groups; ++g) {
-        if (!wait_or_fail(bars + 8 * kBarAFull, g & 1, P.status)) break;
+        if (!wait_or_fail<200>(bars + 8 * kBarAFull, g & 1, P.status)) break;
         // every butterfly thread has read stage g & 1 (its loads precede its arrival): refill it
         if (g + 2 < n_groups) issue_load(tmap, smem, bars, g + 2, first + (g + 2) * stride);
         if (g >= 2 && !wait_or_fail(bars + 8 * (kBarDEmpty + (g & 1)), ((g >> 1) - 1) & 1, P.status)) break;
@@ -267,7 +266,7 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint32_t bars, ui
     const uint32_t smask23 = ((sbits & 4u) ? 0x8000u : 0u) | ((sbits & 8u) ? 0x80000000u : 0u);
     for (int g = 0; g < n_groups; ++g) {
         const int buf = g & 1;
-        const bool ok = wait_or_fail(bars + 8 * (kBarMmaDone + buf), (g >> 1) & 1, P.status);
+        const bool ok = wait_or_fail<200>(bars + 8 * (kBarMmaDone + buf), (g >> 1) & 1, P.status);
         if (!__all_sync(0xffffffffu, ok)) break;
         tmem_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * w) << 16) + buf * (4 * kNPad);
