@@ -86,19 +86,26 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // fp32 -> TF32 (10 mantissa bits), round to nearest with ties away from zero, for finite values: half an ulp is
-// added to the magnitude and the 13 low bits are cleared (what cvt.rna.tf32.f32 gives, without its NaN handling)
-__device__ __forceinline__ uint32_t to_tf32(float v) { return (__float_as_uint(v) + 0x1000u) & 0xFFFFE000u; }
+// added to the magnitude; the tensor core reads the upper 19 bits and ignores the 13 low ones
+__device__ __forceinline__ uint32_t to_tf32(float v) { return __float_as_uint(v) + 0x1000u; }
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// Bounded wait that also gives up early once any thread of the grid has reported a failure.
-template <int SLEEP_NS = 40>
+// Bounded wait: the hardware suspends the thread for up to about 2 us per attempt (no issue slots are spent while
+// it sleeps); gives up after 2^20 attempts, or early once any thread of the grid has reported a failure.
 __device__ __forceinline__ bool wait_or_fail(uint32_t bar, uint32_t parity, int* status) {
-    for (int i = 0; i < (1 << 22); ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(SLEEP_NS);
-        if ((i & 1023) == 1023 && *reinterpret_cast<volatile int*>(status) != 0) break;
+    for (int i = 0; i < (1 << 20); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity), "r"(2000u)
+            : "memory");
+        if (ok != 0) return true;
+        if ((i & 63) == 63 && *reinterpret_cast<volatile int*>(status) != 0) break;
     }
     atomicExch(status, 1);
     return false;
@@ -227,7 +234,7 @@ __device__ __forceinline__ void mma_role(const Params& P, const CUtensorMap* tma
     if (n_groups > 1) issue_load(tmap, smem, bars, 1, first + stride);
     int committed = -1;
     for (int g = 0; g < n_groups; ++g) {
-        if (!wait_or_fail<200>(bars + 8 * kBarAFull, g & 1, P.status)) break;
+        if (!wait_or_fail(bars + 8 * kBarAFull, g & 1, P.status)) break;
         // every butterfly thread has read stage g & 1 (its loads precede its arrival): refill it
         if (g + 2 < n_groups) issue_load(tmap, smem, bars, g + 2, first + (g + 2) * stride);
         if (g >= 2 && !wait_or_fail(bars + 8 * (kBarDEmpty + (g & 1)), ((g >> 1) - 1) & 1, P.status)) break;
@@ -266,7 +273,7 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint32_t bars, ui
     const uint32_t smask23 = ((sbits & 4u) ? 0x8000u : 0u) | ((sbits & 8u) ? 0x80000000u : 0u);
     for (int g = 0; g < n_groups; ++g) {
         const int buf = g & 1;
-        const bool ok = wait_or_fail<200>(bars + 8 * (kBarMmaDone + buf), (g >> 1) & 1, P.status);
+        const bool ok = wait_or_fail(bars + 8 * (kBarMmaDone + buf), (g >> 1) & 1, P.status);
         if (!__all_sync(0xffffffffu, ok)) break;
         tmem_fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * w) << 16) + buf * (4 * kNPad);
