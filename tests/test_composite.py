@@ -195,3 +195,35 @@ def test_tensor_core_composite_5120_padded_rows_and_guards():
     assert p.device_status() == 0
     assert codes.intact() and scales.intact()
     _check_tf32_quant(codes.view, scales.view, y_ref, tol, "int4 with a padded leading dimension")
+
+
+def test_full_size_composite_5120_sampled():
+    """The benchmark's configuration (32768 bf16 token rows of d = 5120, INT4), sampled rows against the oracle."""
+    from parity import Guarded
+    c = synth.COMPOSITE_5120
+    n1, n2, rows = c["n1"], c["n2"], c["n_rows"]
+    theta2 = synth.angles(n2, "normal", c["seed"], DEV)
+    params = synth.cayley_params(n1, c["seed"], device=DEV)
+    x = synth.rows(rows, n1 * n2, c["dist"], c["seed"] + 1, outliers=c["outliers"], outlier_scale=c["outlier_scale"],
+                   dtype=torch.bfloat16, device=DEV)
+    p = Plan(n2, DEV)
+    p.set_angles(theta2)
+    q1 = p.cayley(params, n1)
+    codes = Guarded((rows, 2560), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.composite_forward_quant(q1, x, 4, codes=codes.view, scales=scales.view)
+    assert p.device_status() == 0
+    assert codes.intact() and scales.intact()
+    idx = np.unique(np.concatenate([np.arange(8), np.arange(rows - 8, rows),
+                                    np.random.default_rng(0).integers(0, rows, 496)]))
+    ti = torch.from_numpy(idx).to(DEV)
+    Q1 = oracle.cayley(to_f64(params), n1)
+    x64 = to_f64(x[ti])
+    inner = oracle.forward(to_f64(theta2), x64.reshape(-1, n2)).reshape(len(idx), n1, n2)
+    y_ref = np.einsum("ik,rkj->rij", Q1, inner).reshape(len(idx), -1)
+    tol = 2.0 ** -10 * np.einsum("ik,rkj->rij", np.abs(Q1), np.abs(inner)).reshape(len(idx), -1)
+    tol = tol + 1e-5 * np.abs(x64).max(axis=1, keepdims=True)
+    frac = _check_tf32_quant(codes.view[ti], scales.view[ti], y_ref, tol, "composite 5120 int4, full size")
+    assert frac <= 2e-2
+    c2, s2 = p.composite_forward_quant(q1, x, 4)  # bit-identical from run to run
+    assert torch.equal(c2, codes.view) and torch.equal(s2.view(torch.int16), scales.view.view(torch.int16))
