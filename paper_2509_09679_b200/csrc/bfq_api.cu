@@ -169,6 +169,7 @@ static void release_plan(bfq_plan* plan) {
     cudaFree(plan->gsign4096);
     cudaFree(plan->partial);
     cudaFree(plan->status_word);
+    cudaFree(plan->dense128);
     if (plan->theta_host != nullptr) cudaFreeHost(plan->theta_host);
     if (plan->theta_event != nullptr) cudaEventDestroy(plan->theta_event);
     std::free(plan->comp5120);
@@ -218,6 +219,7 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_b4096, bwd4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->dsign4096, bwd4096_dsign_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->gsign4096, bwd4096_gsign_bytes());
+    if (e == cudaSuccess && n == 128) e = cudaMalloc(&plan->dense128, comp5120d_image_bytes());
     if (e == cudaSuccess && n == 128) {  // the composite kernel's constants are computed on the host from the angles
         e = cudaMallocHost(&plan->theta_host, angles * sizeof(float));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->theta_event, cudaEventDisableTiming);
@@ -260,6 +262,7 @@ int bfq_set_angles(bfq_plan* plan, const float* theta, void* stream) {
         k_build_twiddles<<<(count + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(theta, count, plan->tw);
         e = cudaGetLastError();
     }
+    if (e == cudaSuccess && plan->dense128 != nullptr) e = comp5120d_set_angles(plan, static_cast<cudaStream_t>(stream));
     if (e == cudaSuccess && plan->theta_host != nullptr) {
         e = cudaMemcpyAsync(plan->theta_host, theta, sizeof(float) * plan->log_n * (plan->n / 2), cudaMemcpyDeviceToHost,
                             static_cast<cudaStream_t>(stream));
@@ -495,9 +498,17 @@ static int composite_impl(bfq_plan* plan, const float* q1, int n1, const void* x
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
     cudaError_t e;
     if (n1 == 40 && xt == BFQ_BF16 && rows < (int64_t(1) << 31) && (codes == nullptr || bits == 4) &&
-        (y == nullptr || yt == BFQ_BF16) && !env_flag("BFQ_GENERIC_ONLY") && comp5120_available(plan)) {
-        e = comp5120_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
-        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+        (y == nullptr || yt == BFQ_BF16) && !env_flag("BFQ_GENERIC_ONLY")) {
+        // default: both factors on the tensor cores; BFQ_COMPOSITE_FP32_BUTTERFLY=1 keeps Q2 as an fp32 butterfly on
+        // the CUDA cores (only the dense factor on the tensor cores)
+        if (!env_flag("BFQ_COMPOSITE_FP32_BUTTERFLY") && comp5120d_available(plan)) {
+            e = comp5120d_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
+            return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+        }
+        if (comp5120_available(plan)) {
+            e = comp5120_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
+            return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+        }
     }
     e = composite_generic_launch(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, bits, codes, scales,
                                  static_cast<cudaStream_t>(stream));

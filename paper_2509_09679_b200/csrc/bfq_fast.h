@@ -50,4 +50,12 @@ size_t comp5120_param_bytes();
 cudaError_t comp5120_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                             uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 
+
+// composite 40 x 128 on bf16 rows with both factors on the tensor cores (Q2 merged into a dense 128 x 128 block)
+size_t comp5120d_image_bytes();
+bool comp5120d_available(const bfq_plan* plan);
+cudaError_t comp5120d_set_angles(const bfq_plan* plan, cudaStream_t st);
+cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                             uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
+
 }  // namespace bfq

@@ -27,6 +27,8 @@ struct bfq_plan {
     float* theta_host = nullptr;    // pinned host copy of the angles (n = 128 only: the composite kernel's constants
                                     // are kernel parameters computed on the host)
     cudaEvent_t theta_event = nullptr;  // recorded after that copy
+    void* dense128 = nullptr;       // device: Q2 as a dense 128 x 128 block, two bf16 terms, in the MMA operand layout
+                                    // (n = 128 only)
     void* comp5120 = nullptr;       // host: kernel parameters of the 40 x 128 composite kernel
     bool comp5120_valid = false;    // they match the current angles
     float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
