@@ -19,10 +19,10 @@
 // M = 128, N = 48 (40 output runs + 8 zero rows of Q1), K = 8 x 5 steps, A = 40 columns of D1 -> D2 (4 x 48 columns).
 // Both operands of MMA 1 are K-major with the 128-byte swizzle (the layout TMA writes); Q1 is K-major without swizzle.
 //
-// Warps: 0..7 epilogue (warp w reads lanes 32 (w mod 4) .. + 31 of tokens 2 (w / 4), 2 (w / 4) + 1: one position j,
-// forty runs i per thread; the row absmax is combined across the four lane quarters through shared memory; INT4 codes
-// of 8 positions x 8 runs are transposed between 8 lanes by three shuffles so that every lane stores whole 32-bit
-// words); warp 8 lane 0 issues the MMAs; warp 9 lane 0 the TMA loads (three stages).  Every wait is bounded.
+// Warps: 0..15 epilogue (warp w reads lanes 32 (w mod 4) .. + 31 of token w / 4 of the group: one position j, forty
+// runs i per thread; the row absmax is combined across the four lane quarters through shared memory; INT4 codes of
+// 8 positions x 8 runs are transposed between 8 lanes by three shuffles so that every lane stores whole 32-bit
+// words); warp 16 lane 0 issues the MMAs; warp 17 lane 0 the TMA loads (three stages).  Every wait is bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -40,9 +40,9 @@ using namespace ptx;
 constexpr int kN1 = 40, kN2 = 128, kD = kN1 * kN2;
 constexpr int kTok = 4;                 // tokens per group
 constexpr int kRuns = kTok * kN1;       // 160 = N of MMA 1
-constexpr int kEpiWarps = 8;
-constexpr int kMmaWarp = 8, kTmaWarp = 9;
-constexpr int kThreads = 32 * 10;
+constexpr int kEpiWarps = 16;
+constexpr int kMmaWarp = 16, kTmaWarp = 17;
+constexpr int kThreads = 32 * 18;
 constexpr int kNPad = 48, kKSteps2 = kN1 / 8;
 constexpr int kStagesX = 3;
 
@@ -57,13 +57,14 @@ constexpr int kBBlock = kNPad * 8 * 4;              // 1536: one k-step block of
 constexpr int kQ1Off = kQ2Off + kQ2Bytes;
 constexpr int kBarOff = kQ1Off + kKSteps2 * kBBlock;
 constexpr int kAmaxOff = kBarOff + 128;             // float [2 group parities][4 tokens][4 quarters]
-constexpr int kSmemBytes = kAmaxOff + 128 + 1024;
+constexpr int kMiscOff = kAmaxOff + 128;            // tensor-memory base address
+constexpr int kSmemBytes = kMiscOff + 16 + 1024;
 
 // tensor memory columns
 constexpr int kD1Col = 0;                 // two buffers of 160
 constexpr int kD2Col = 2 * kRuns;         // 320: four tokens x 48
 
-enum : int { kBarXFull = 0, kBarXEmpty = 3, kBarMmaDone = 6, kBarD2Empty = 7, kBarAmax = 8, kNumBars = 12 };
+enum : int { kBarXFull = 0, kBarXEmpty = 3, kBarMmaDone = 6, kBarD2Empty = 7, kBarAmax = 8, kNumBars = 16 };
 
 struct Params {
     const uint4* q2img;   // device: the shared-memory image of Q2 (hi, lo) built by k_build_dense128
@@ -205,112 +206,109 @@ __device__ __forceinline__ void mma_role(const Params& P, uint32_t smem, uint32_
 }
 
 // ---- epilogue warps ---------------------------------------------------------------------------------------------------
-// One 8 x 8 block of 4-bit codes held as one word per lane (lane a of 8: position j0 + a, nibble b: run i0 + b) is
+// 8 x 8 blocks of 4-bit codes held as one word per lane (lane a of 8: position j0 + a, nibble b: run i0 + b) are
 // transposed so that lane a holds run i0 + a with nibble p = position j0 + p: three exchanges at lane distance 1, 2, 4
-// swap the off-diagonal nibbles, bytes and half-words.
-__device__ __forceinline__ uint32_t transpose8x8_nibbles(uint32_t w, int a) {
-    uint32_t p = __shfl_xor_sync(0xffffffffu, w, 1);
-    w = (a & 1) ? ((w & 0xF0F0F0F0u) | ((p >> 4) & 0x0F0F0F0Fu)) : ((w & 0x0F0F0F0Fu) | ((p << 4) & 0xF0F0F0F0u));
-    p = __shfl_xor_sync(0xffffffffu, w, 2);
-    w = (a & 2) ? ((w & 0xFF00FF00u) | ((p >> 8) & 0x00FF00FFu)) : ((w & 0x00FF00FFu) | ((p << 8) & 0xFF00FF00u));
-    p = __shfl_xor_sync(0xffffffffu, w, 4);
-    w = (a & 4) ? ((w & 0xFFFF0000u) | (p >> 16)) : ((w & 0x0000FFFFu) | (p << 16));
-    return w;
+// swap the off-diagonal nibbles, bytes and half-words.  Five independent blocks go through each exchange together.
+__device__ __forceinline__ void transpose8x8_nibbles(uint32_t (&w)[5], int a) {
+    uint32_t p[5];
+#pragma unroll
+    for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 1);
+#pragma unroll
+    for (int k = 0; k < 5; ++k)
+        w[k] = (a & 1) ? ((w[k] & 0xF0F0F0F0u) | ((p[k] >> 4) & 0x0F0F0F0Fu)) : ((w[k] & 0x0F0F0F0Fu) | ((p[k] << 4) & 0xF0F0F0F0u));
+#pragma unroll
+    for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 2);
+#pragma unroll
+    for (int k = 0; k < 5; ++k)
+        w[k] = (a & 2) ? ((w[k] & 0xFF00FF00u) | ((p[k] >> 8) & 0x00FF00FFu)) : ((w[k] & 0x00FF00FFu) | ((p[k] << 8) & 0xFF00FF00u));
+#pragma unroll
+    for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 4);
+#pragma unroll
+    for (int k = 0; k < 5; ++k) w[k] = (a & 4) ? ((w[k] & 0xFFFF0000u) | (p[k] >> 16)) : ((w[k] & 0x0000FFFFu) | (p[k] << 16));
 }
 
 __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint32_t bars, uint32_t tmem_base, int n_groups,
                                               int w, int lane) {
-    const int qd = w & 3, set = w >> 2, j = 32 * qd + lane, a = lane & 7;
+    const int qd = w & 3, tau = w >> 2, j = 32 * qd + lane, a = lane & 7;
     float* const amax_slots = reinterpret_cast<float*>(sm + kAmaxOff);
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * qd) << 16) + kD2Col + tau * kNPad;
     for (int g = 0; g < n_groups; ++g) {
         bool ok = wait_or_fail(bars + 8 * kBarMmaDone, g & 1, P.status);
         if (!__all_sync(0xffffffffu, ok)) break;
         tmem_fence_after();
-        // this thread's position j of both tokens of the set: 2 x 40 output runs
-        uint32_t v[2][kN1];
-#pragma unroll
-        for (int tt = 0; tt < 2; ++tt) {
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * qd) << 16) + kD2Col + (2 * set + tt) * kNPad;
-            tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v[tt][0]));
-            tmem_ld8(taddr + 32, reinterpret_cast<uint32_t(&)[8]>(v[tt][32]));
-        }
-#pragma unroll
-        for (int tt = 0; tt < 2; ++tt) {
-            tmem_wait_ld32(reinterpret_cast<uint32_t(&)[32]>(v[tt][0]));
-            tmem_wait_ld8(reinterpret_cast<uint32_t(&)[8]>(v[tt][32]));
-        }
+        // this thread's position j of its token: 40 output runs
+        uint32_t v[kN1];
+        tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v[0]));
+        tmem_ld8(taddr + 32, reinterpret_cast<uint32_t(&)[8]>(v[32]));
+        tmem_wait_ld32(reinterpret_cast<uint32_t(&)[32]>(v[0]));
+        tmem_wait_ld8(reinterpret_cast<uint32_t(&)[8]>(v[32]));
         tmem_fence_before();
         mbar_arrive(bars + 8 * kBarD2Empty);  // D2 is in registers: the next group's second factor may overwrite it
 
-        float inv[2] = {0.f, 0.f};
-        bool saturated[2] = {false, false};
-        if (P.codes != nullptr) {
-            // row absmax: thread -> warp -> the four lane quarters of the set (through shared memory)
+        const int64_t token = int64_t(kTok) * (blockIdx.x + int64_t(g) * gridDim.x) + tau;
+        const bool valid = token < P.rows;
+        if (P.y != nullptr) {
+            // runs i and i + 1: the even lane stores positions (j, j + 1) of run i, the odd lane those of run i + 1
+            const bool odd = lane & 1;
 #pragma unroll
-            for (int tt = 0; tt < 2; ++tt) {
-                float m = 0.f;
-#pragma unroll
-                for (int i = 0; i < kN1; ++i) m = fmaxf(m, fabsf(__uint_as_float(v[tt][i])));
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                if (lane == 0) amax_slots[(g & 1) * 16 + (2 * set + tt) * 4 + qd] = m;
-            }
-            __syncwarp();
-            const uint32_t abar = bars + 8 * (kBarAmax + 2 * (g & 1) + set);
-            if (lane == 0) mbar_arrive(abar);
-            ok = wait_or_fail(abar, (g >> 1) & 1, P.status);
-            if (!__all_sync(0xffffffffu, ok)) break;
-#pragma unroll
-            for (int tt = 0; tt < 2; ++tt) {
-                const float4 q4 = *reinterpret_cast<const float4*>(amax_slots + (g & 1) * 16 + (2 * set + tt) * 4);
-                const float amax = fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w));
-                const uint16_t sb = row_scale(amax, 7, &inv[tt]);
-                saturated[tt] = sb == 0x7BFFu || sb < 0x0400u || !(amax < 3.0e38f);
-                const int64_t token = int64_t(kTok) * (blockIdx.x + int64_t(g) * gridDim.x) + 2 * set + tt;
-                if (qd == 0 && lane == 0 && token < P.rows) P.scales[token] = sb;
+            for (int i = 0; i < kN1; i += 2) {
+                const float mine = __uint_as_float(odd ? v[i + 1] : v[i]);
+                const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(odd ? v[i] : v[i + 1]), 1);
+                const uint32_t word = odd ? pack_bf16x2(other, mine) : pack_bf16x2(mine, other);
+                if (valid) *reinterpret_cast<uint32_t*>(P.y + token * P.ldy + (i + (odd ? 1 : 0)) * kN2 + (j & ~1)) = word;
             }
         }
+        if (P.codes != nullptr) {
+            // row absmax: thread (four partial maxima) -> warp -> the four lane quarters (through shared memory)
+            float m4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int tt = 0; tt < 2; ++tt) {
-            const int64_t token = int64_t(kTok) * (blockIdx.x + int64_t(g) * gridDim.x) + 2 * set + tt;
-            const bool valid = token < P.rows;
-            if (P.y != nullptr) {
-                // runs i and i + 1: the even lane stores positions (j, j + 1) of run i, the odd lane those of run i + 1
-                const bool odd = lane & 1;
+            for (int i = 0; i < kN1; ++i) m4[i & 3] = fmaxf(m4[i & 3], fabsf(__uint_as_float(v[i])));
+            float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
 #pragma unroll
-                for (int i = 0; i < kN1; i += 2) {
-                    const float mine = __uint_as_float(odd ? v[tt][i + 1] : v[tt][i]);
-                    const float other = __shfl_xor_sync(0xffffffffu, __uint_as_float(odd ? v[tt][i] : v[tt][i + 1]), 1);
-                    const uint32_t word = odd ? pack_bf16x2(other, mine) : pack_bf16x2(mine, other);
-                    if (valid)
-                        *reinterpret_cast<uint32_t*>(P.y + token * P.ldy + (i + (odd ? 1 : 0)) * kN2 + (j & ~1)) = word;
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            const uint32_t abar = bars + 8 * (kBarAmax + 4 * (g & 1) + tau);
+            if (lane == 0) {
+                amax_slots[(g & 1) * 16 + tau * 4 + qd] = m;
+                mbar_arrive(abar);
+            }
+            ok = wait_or_fail(abar, (g >> 1) & 1, P.status);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            const float4 q4 = *reinterpret_cast<const float4*>(amax_slots + (g & 1) * 16 + tau * 4);
+            const float amax = fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w));
+            float inv;
+            const uint16_t sb = row_scale(amax, 7, &inv);
+            const bool saturated = sb == 0x7BFFu || sb < 0x0400u || !(amax < 3.0e38f);
+            if (qd == 0 && lane == 0 && valid) P.scales[token] = sb;
+            uint32_t word[5];
+            if (!saturated) {
+                // |y / s| < 7.5 for a normal, unsaturated fp16 scale: y * inv + (1.5 * 2^23 + 8) has r + 8 in [1, 15] in
+                // its low mantissa bits (r = y / s rounded to nearest even); eight of them are summed with weights
+                // 16^b, the exponent bits are removed and bit 3 of every nibble is flipped
+                constexpr float kMagic = 12582920.0f;
+                constexpr uint32_t kUnbias = 0u - 0x4B400000u * 0x11111111u;
+#pragma unroll
+                for (int blk = 0; blk < 5; ++blk) {
+                    uint32_t c[8];
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) c[b] = __float_as_uint(fmaf(__uint_as_float(v[8 * blk + b]), inv, kMagic));
+                    const uint32_t s01 = c[0] + (c[1] << 4), s23 = (c[2] << 8) + (c[3] << 12);
+                    const uint32_t s45 = (c[4] << 16) + (c[5] << 20), s67 = (c[6] << 24) + (c[7] << 28);
+                    word[blk] = (((s01 + s23) + (s45 + s67)) + kUnbias) ^ 0x88888888u;
+                }
+            } else {
+#pragma unroll
+                for (int blk = 0; blk < 5; ++blk) {
+                    word[blk] = 0u;
+#pragma unroll
+                    for (int b = 0; b < 8; ++b)
+                        word[blk] |= (static_cast<uint32_t>(quant1(__uint_as_float(v[8 * blk + b]), inv, -8, 7)) & 0xFu) << (4 * b);
                 }
             }
-            if (P.codes != nullptr) {
+            transpose8x8_nibbles(word, a);
+            if (valid) {
 #pragma unroll
-                for (int blk = 0; blk < kN1 / 8; ++blk) {
-                    uint32_t word;
-                    if (!saturated[tt]) {
-                        // |y / s| < 7.5 for a normal, unsaturated fp16 scale: y * inv + (1.5 * 2^23 + 8) has r + 8 in
-                        // [1, 15] in its low mantissa bits (r = y / s rounded to nearest even); eight of them are summed
-                        // with weights 16^b, the exponent bits are removed and bit 3 of every nibble is flipped
-                        constexpr float kMagic = 12582920.0f;
-                        constexpr uint32_t kUnbias = 0u - 0x4B400000u * 0x11111111u;
-                        uint32_t acc = 0u;
-#pragma unroll
-                        for (int b = 0; b < 8; ++b)
-                            acc += __float_as_uint(fmaf(__uint_as_float(v[tt][8 * blk + b]), inv[tt], kMagic)) << (4 * b);
-                        word = (acc + kUnbias) ^ 0x88888888u;
-                    } else {
-                        word = 0u;
-#pragma unroll
-                        for (int b = 0; b < 8; ++b)
-                            word |= (static_cast<uint32_t>(quant1(__uint_as_float(v[tt][8 * blk + b]), inv[tt], -8, 7)) & 0xFu) << (4 * b);
-                    }
-                    word = transpose8x8_nibbles(word, a);
-                    if (valid)
-                        *reinterpret_cast<uint32_t*>(P.codes + token * (kD / 2) + (8 * blk + a) * (kN2 / 2) + (j >> 3) * 4) = word;
-                }
+                for (int blk = 0; blk < 5; ++blk)
+                    *reinterpret_cast<uint32_t*>(P.codes + token * (kD / 2) + (8 * blk + a) * (kN2 / 2) + (j >> 3) * 4) = word[blk];
             }
         }
     }
@@ -322,7 +320,7 @@ k_comp5120d(const __grid_constant__ Params P, const __grid_constant__ CUtensorMa
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const sm = smem_raw + (smem - smem_u32(smem_raw));
     const uint32_t bars = smem + kBarOff;
-    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(sm + kBarOff + 8 * kNumBars);
+    uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(sm + kMiscOff);
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
     const int n_groups =
         blockIdx.x < total_groups ? static_cast<int>((total_groups - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
@@ -334,7 +332,7 @@ k_comp5120d(const __grid_constant__ Params P, const __grid_constant__ CUtensorMa
         }
         mbar_init(bars + 8 * kBarMmaDone, 1);
         mbar_init(bars + 8 * kBarD2Empty, 32 * kEpiWarps);
-        for (int s = 0; s < 4; ++s) mbar_init(bars + 8 * (kBarAmax + s), 4);
+        for (int s = 0; s < 8; ++s) mbar_init(bars + 8 * (kBarAmax + s), 4);
         mbar_init_fence();
     }
     __syncwarp();
