@@ -209,22 +209,21 @@ __device__ __forceinline__ void mma_role(const Params& P, uint32_t smem, uint32_
 // 8 x 8 blocks of 4-bit codes held as one word per lane (lane a of 8: position j0 + a, nibble b: run i0 + b) are
 // transposed so that lane a holds run i0 + a with nibble p = position j0 + p: three exchanges at lane distance 1, 2, 4
 // swap the off-diagonal nibbles, bytes and half-words.  Five independent blocks go through each exchange together.
-__device__ __forceinline__ void transpose8x8_nibbles(uint32_t (&w)[5], int a) {
-    uint32_t p[5];
+// Per round a lane keeps the nibbles selected by its mask and takes the others from its partner's word rotated left by
+// 4 d or right by 4 d bits (rotl by 32 - 4 d), depending on which side of the exchange it is: keep[] and rot[] are the
+// lane's three masks and rotation counts.
+__device__ __forceinline__ void transpose8x8_nibbles(uint32_t (&w)[5], const uint32_t (&keep)[3], const uint32_t (&rot)[3]) {
 #pragma unroll
-    for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 1);
+    for (int r = 0; r < 3; ++r) {
+        uint32_t p[5];
 #pragma unroll
-    for (int k = 0; k < 5; ++k)
-        w[k] = (a & 1) ? ((w[k] & 0xF0F0F0F0u) | ((p[k] >> 4) & 0x0F0F0F0Fu)) : ((w[k] & 0x0F0F0F0Fu) | ((p[k] << 4) & 0xF0F0F0F0u));
+        for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 1 << r);
 #pragma unroll
-    for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 2);
-#pragma unroll
-    for (int k = 0; k < 5; ++k)
-        w[k] = (a & 2) ? ((w[k] & 0xFF00FF00u) | ((p[k] >> 8) & 0x00FF00FFu)) : ((w[k] & 0x00FF00FFu) | ((p[k] << 8) & 0xFF00FF00u));
-#pragma unroll
-    for (int k = 0; k < 5; ++k) p[k] = __shfl_xor_sync(0xffffffffu, w[k], 4);
-#pragma unroll
-    for (int k = 0; k < 5; ++k) w[k] = (a & 4) ? ((w[k] & 0xFFFF0000u) | (p[k] >> 16)) : ((w[k] & 0x0000FFFFu) | (p[k] << 16));
+        for (int k = 0; k < 5; ++k) {
+            const uint32_t ps = __funnelshift_l(p[k], p[k], rot[r]);
+            w[k] = (w[k] & keep[r]) | (ps & ~keep[r]);
+        }
+    }
 }
 
 __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint32_t bars, uint32_t tmem_base, int n_groups,
@@ -232,6 +231,9 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
     const int qd = w & 3, tau = w >> 2, j = 32 * qd + lane, a = lane & 7;
     float* const amax_slots = reinterpret_cast<float*>(sm + kAmaxOff);
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * qd) << 16) + kD2Col + tau * kNPad;
+    const uint32_t keep[3] = {(a & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu, (a & 2) ? 0xFF00FF00u : 0x00FF00FFu,
+                              (a & 4) ? 0xFFFF0000u : 0x0000FFFFu};
+    const uint32_t rot[3] = {(a & 1) ? 28u : 4u, (a & 2) ? 24u : 8u, 16u};
     for (int g = 0; g < n_groups; ++g) {
         bool ok = wait_or_fail(bars + 8 * kBarMmaDone, g & 1, P.status);
         if (!__all_sync(0xffffffffu, ok)) break;
@@ -291,9 +293,11 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
                     uint32_t c[8];
 #pragma unroll
                     for (int b = 0; b < 8; ++b) c[b] = __float_as_uint(fmaf(__uint_as_float(v[8 * blk + b]), inv, kMagic));
-                    const uint32_t s01 = c[0] + (c[1] << 4), s23 = (c[2] << 8) + (c[3] << 12);
-                    const uint32_t s45 = (c[4] << 16) + (c[5] << 20), s67 = (c[6] << 24) + (c[7] << 28);
-                    word[blk] = (((s01 + s23) + (s45 + s67)) + kUnbias) ^ 0x88888888u;
+                    // shift-and-add pairs, then pairs of pairs (three levels instead of a chain of seven)
+                    const uint32_t s01 = c[1] * 16u + c[0], s23 = c[3] * 16u + c[2];
+                    const uint32_t s45 = c[5] * 16u + c[4], s67 = c[7] * 16u + c[6];
+                    const uint32_t lo = s23 * 256u + s01, hi = s67 * 256u + s45;
+                    word[blk] = ((hi * 65536u + lo) + kUnbias) ^ 0x88888888u;
                 }
             } else {
 #pragma unroll
@@ -304,7 +308,7 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
                         word[blk] |= (static_cast<uint32_t>(quant1(__uint_as_float(v[8 * blk + b]), inv, -8, 7)) & 0xFu) << (4 * b);
                 }
             }
-            transpose8x8_nibbles(word, a);
+            transpose8x8_nibbles(word, keep, rot);
             if (valid) {
 #pragma unroll
                 for (int blk = 0; blk < 5; ++blk)
