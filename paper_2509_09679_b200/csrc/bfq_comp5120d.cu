@@ -64,7 +64,7 @@ constexpr int kSmemBytes = kMiscOff + 16 + 1024;
 constexpr int kD1Col = 0;                 // two buffers of 160
 constexpr int kD2Col = 2 * kRuns;         // 320: four tokens x 48
 
-enum : int { kBarXFull = 0, kBarXEmpty = 3, kBarMmaDone = 6, kBarD2Empty = 7, kBarAmax = 8, kNumBars = 16 };
+enum : int { kBarXFull = 0, kBarXEmpty = 3, kBarMmaDone = 6, kBarD2Empty = 7, kNumBars = 8 };
 
 struct Params {
     const uint4* q2img;   // device: the shared-memory image of Q2 (hi, lo) built by k_build_dense128
@@ -82,18 +82,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// Bounded wait.  Between attempts the warp sleeps SLEEP_NS: a poll costs about ten issue slots, and sixteen epilogue
+// warps polling at full rate took a third of all instructions.
+template <uint32_t SLEEP_NS>
 __device__ __forceinline__ bool wait_or_fail(uint32_t bar, uint32_t parity, int* status) {
-    for (int i = 0; i < (1 << 20); ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity), "r"(2000u)
-            : "memory");
-        if (ok != 0) return true;
-        if ((i & 63) == 63 && *reinterpret_cast<volatile int*>(status) != 0) break;
+    for (int i = 0; i < (1 << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(SLEEP_NS);
+        if ((i & 255) == 255 && *reinterpret_cast<volatile int*>(status) != 0) break;
     }
     atomicExch(status, 1);
     return false;
@@ -150,7 +146,7 @@ __device__ __forceinline__ void tma_role(const Params& P, const CUtensorMap* tma
     for (int g = 0; g < n_groups; ++g) {
         const int stage = g % kStagesX;
         // the stage is free once the MMAs that read it have completed (their commit arrives on x_empty)
-        if (g >= kStagesX && !wait_or_fail(bars + 8 * (kBarXEmpty + stage), ((g / kStagesX) - 1) & 1, P.status)) break;
+        if (g >= kStagesX && !wait_or_fail<500>(bars + 8 * (kBarXEmpty + stage), ((g / kStagesX) - 1) & 1, P.status)) break;
         const uint32_t bar = bars + 8 * (kBarXFull + stage), dst = smem + kXOff + stage * kStageBytes;
         mbar_expect_tx(bar, kStageBytes);
         tma_load_3d(dst, tmap, 0, 0, static_cast<int>(first + g * stride), bar);
@@ -159,13 +155,13 @@ __device__ __forceinline__ void tma_role(const Params& P, const CUtensorMap* tma
     }
     // no copy of this CTA may be in flight when it leaves (returns at once on the normal path)
     for (int g = issued - kStagesX; g < issued; ++g)
-        if (g >= 0) wait_or_fail(bars + 8 * (kBarXFull + g % kStagesX), (g / kStagesX) & 1, P.status);
+        if (g >= 0) wait_or_fail<500>(bars + 8 * (kBarXFull + g % kStagesX), (g / kStagesX) & 1, P.status);
 }
 
 // ---- MMA thread -------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ bool issue_mma1(const Params& P, uint32_t smem, uint32_t bars, uint32_t tmem_base, int g) {
     const int stage = g % kStagesX;
-    if (!wait_or_fail(bars + 8 * (kBarXFull + stage), (g / kStagesX) & 1, P.status)) return false;
+    if (!wait_or_fail<100>(bars + 8 * (kBarXFull + stage), (g / kStagesX) & 1, P.status)) return false;
     tmem_fence_after();
     const uint32_t d1 = tmem_base + kD1Col + (g & 1) * kRuns;
 #pragma unroll
@@ -188,7 +184,7 @@ __device__ __forceinline__ void mma_role(const Params& P, uint32_t smem, uint32_
         // keep the tensor pipe fed: the first factor of the next group goes to the other D1 buffer
         if (g + 1 < n_groups && !issue_mma1(P, smem, bars, tmem_base, g + 1)) break;
         // D2 is single-buffered: the epilogue of the previous group must have read it
-        if (g >= 1 && !wait_or_fail(bars + 8 * kBarD2Empty, (g - 1) & 1, P.status)) break;
+        if (g >= 1 && !wait_or_fail<32>(bars + 8 * kBarD2Empty, (g - 1) & 1, P.status)) break;
         tmem_fence_after();
         const uint32_t d1 = tmem_base + kD1Col + (g & 1) * kRuns;
 #pragma unroll
@@ -202,7 +198,7 @@ __device__ __forceinline__ void mma_role(const Params& P, uint32_t smem, uint32_
         mma_commit(bars + 8 * kBarMmaDone);
         committed = g;
     }
-    if (committed >= 0) wait_or_fail(bars + 8 * kBarMmaDone, committed & 1, P.status);
+    if (committed >= 0) wait_or_fail<500>(bars + 8 * kBarMmaDone, committed & 1, P.status);
 }
 
 // ---- epilogue warps ---------------------------------------------------------------------------------------------------
@@ -234,21 +230,31 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
     const uint32_t keep[3] = {(a & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu, (a & 2) ? 0xFF00FF00u : 0x00FF00FFu,
                               (a & 4) ? 0xFFFF0000u : 0x0000FFFFu};
     const uint32_t rot[3] = {(a & 1) ? 28u : 4u, (a & 2) ? 24u : 8u, 16u};
+    // A warp whose wait gave up stays in the loop without waiting or loading (dead), so that the four warps of a token
+    // always meet at the named barrier of the absmax exchange the same number of times.
+    bool dead = false;
     for (int g = 0; g < n_groups; ++g) {
-        bool ok = wait_or_fail(bars + 8 * kBarMmaDone, g & 1, P.status);
-        if (!__all_sync(0xffffffffu, ok)) break;
+        if (!dead) {
+            const bool ok = wait_or_fail<300>(bars + 8 * kBarMmaDone, g & 1, P.status);
+            dead = !__all_sync(0xffffffffu, ok);
+        }
         tmem_fence_after();
         // this thread's position j of its token: 40 output runs
         uint32_t v[kN1];
-        tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v[0]));
-        tmem_ld8(taddr + 32, reinterpret_cast<uint32_t(&)[8]>(v[32]));
-        tmem_wait_ld32(reinterpret_cast<uint32_t(&)[32]>(v[0]));
-        tmem_wait_ld8(reinterpret_cast<uint32_t(&)[8]>(v[32]));
-        tmem_fence_before();
-        mbar_arrive(bars + 8 * kBarD2Empty);  // D2 is in registers: the next group's second factor may overwrite it
+        if (dead) {
+#pragma unroll
+            for (int i = 0; i < kN1; ++i) v[i] = 0u;
+        } else {
+            tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v[0]));
+            tmem_ld8(taddr + 32, reinterpret_cast<uint32_t(&)[8]>(v[32]));
+            tmem_wait_ld32(reinterpret_cast<uint32_t(&)[32]>(v[0]));
+            tmem_wait_ld8(reinterpret_cast<uint32_t(&)[8]>(v[32]));
+            tmem_fence_before();
+            mbar_arrive(bars + 8 * kBarD2Empty);  // D2 is in registers: the next group's second factor may overwrite it
+        }
 
         const int64_t token = int64_t(kTok) * (blockIdx.x + int64_t(g) * gridDim.x) + tau;
-        const bool valid = token < P.rows;
+        const bool valid = token < P.rows && !dead;
         if (P.y != nullptr) {
             // runs i and i + 1: the even lane stores positions (j, j + 1) of run i, the odd lane those of run i + 1
             const bool odd = lane & 1;
@@ -268,13 +274,9 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
             float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            const uint32_t abar = bars + 8 * (kBarAmax + 4 * (g & 1) + tau);
-            if (lane == 0) {
-                amax_slots[(g & 1) * 16 + tau * 4 + qd] = m;
-                mbar_arrive(abar);
-            }
-            ok = wait_or_fail(abar, (g >> 1) & 1, P.status);
-            if (!__all_sync(0xffffffffu, ok)) break;
+            if (lane == 0) amax_slots[(g & 1) * 16 + tau * 4 + qd] = m;
+            __syncwarp();
+            bar_sync(1 + tau, 128);  // the four warps of this token (slots alternate between groups: one barrier is enough)
             const float4 q4 = *reinterpret_cast<const float4*>(amax_slots + (g & 1) * 16 + tau * 4);
             const float amax = fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w));
             float inv;
@@ -336,7 +338,6 @@ k_comp5120d(const __grid_constant__ Params P, const __grid_constant__ CUtensorMa
         }
         mbar_init(bars + 8 * kBarMmaDone, 1);
         mbar_init(bars + 8 * kBarD2Empty, 32 * kEpiWarps);
-        for (int s = 0; s < 8; ++s) mbar_init(bars + 8 * (kBarAmax + s), 4);
         mbar_init_fence();
     }
     __syncwarp();
