@@ -235,7 +235,7 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
     bool dead = false;
     for (int g = 0; g < n_groups; ++g) {
         if (!dead) {
-            const bool ok = wait_or_fail<300>(bars + 8 * kBarMmaDone, g & 1, P.status);
+            const bool ok = wait_or_fail<40>(bars + 8 * kBarMmaDone, g & 1, P.status);
             dead = !__all_sync(0xffffffffu, ok);
         }
         tmem_fence_after();
