@@ -468,14 +468,22 @@ def time_others(torch, synth, Plan, dev):
     codes = torch.empty((rows, 2560), dtype=torch.uint8, device=dev)
     scales = torch.empty((rows,), dtype=torch.float16, device=dev)
     y = torch.empty_like(x)
-    for name, nbytes, fn in (("composite_int4_d5120", 2 * 5120 + 2560 + 2,
-                              lambda: planc.composite_forward_quant(q1, x, 4, codes=codes, scales=scales)),
-                             ("composite_bf16_d5120", 4 * 5120, lambda: planc.composite_forward(q1, x, out=y))):
-        for _ in range(3):
-            fn()
-        ms = event_time_ms(torch, fn, 10)
-        res[name] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": nbytes * rows / (ms * 1e-3) / 1e9, "rows": rows,
-                     "n": 5120}
+    legs = (("composite_int4_d5120", 2 * 5120 + 2560 + 2,
+             lambda: planc.composite_forward_quant(q1, x, 4, codes=codes, scales=scales)),
+            ("composite_bf16_d5120", 4 * 5120, lambda: planc.composite_forward(q1, x, out=y)))
+    # default: both factors on the tensor cores; *_fp32_butterfly: Q2 as an fp32 butterfly on the CUDA cores
+    for suffix, env in (("", None), ("_fp32_butterfly", "1")):
+        if env is None:
+            os.environ.pop("BFQ_COMPOSITE_FP32_BUTTERFLY", None)
+        else:
+            os.environ["BFQ_COMPOSITE_FP32_BUTTERFLY"] = env
+        for name, nbytes, fn in legs:
+            for _ in range(3):
+                fn()
+            ms = event_time_ms(torch, fn, 10)
+            res[name + suffix] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": nbytes * rows / (ms * 1e-3) / 1e9,
+                                  "rows": rows, "n": 5120}
+    os.environ.pop("BFQ_COMPOSITE_FP32_BUTTERFLY", None)
     return res
 
 
