@@ -238,23 +238,22 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
             const bool ok = wait_or_fail<40>(bars + 8 * kBarMmaDone, g & 1, P.status);
             dead = !__all_sync(0xffffffffu, ok);
         }
+        if (dead) {  // keep the barrier count of the absmax exchange, do nothing else
+            if (P.codes != nullptr) bar_sync(1 + tau, 128);
+            continue;
+        }
         tmem_fence_after();
         // this thread's position j of its token: 40 output runs
         uint32_t v[kN1];
-        if (dead) {
-#pragma unroll
-            for (int i = 0; i < kN1; ++i) v[i] = 0u;
-        } else {
-            tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v[0]));
-            tmem_ld8(taddr + 32, reinterpret_cast<uint32_t(&)[8]>(v[32]));
-            tmem_wait_ld32(reinterpret_cast<uint32_t(&)[32]>(v[0]));
-            tmem_wait_ld8(reinterpret_cast<uint32_t(&)[8]>(v[32]));
-            tmem_fence_before();
-            mbar_arrive(bars + 8 * kBarD2Empty);  // D2 is in registers: the next group's second factor may overwrite it
-        }
+        tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v[0]));
+        tmem_ld8(taddr + 32, reinterpret_cast<uint32_t(&)[8]>(v[32]));
+        tmem_wait_ld32(reinterpret_cast<uint32_t(&)[32]>(v[0]));
+        tmem_wait_ld8(reinterpret_cast<uint32_t(&)[8]>(v[32]));
+        tmem_fence_before();
+        mbar_arrive(bars + 8 * kBarD2Empty);  // D2 is in registers: the next group's second factor may overwrite it
 
         const int64_t token = int64_t(kTok) * (blockIdx.x + int64_t(g) * gridDim.x) + tau;
-        const bool valid = token < P.rows && !dead;
+        const bool valid = token < P.rows;
         if (P.y != nullptr) {
             // runs i and i + 1: the even lane stores positions (j, j + 1) of run i, the odd lane those of run i + 1
             const bool odd = lane & 1;
