@@ -188,30 +188,16 @@ def main():
     from paper_2509_09679_b200 import Plan, lib, synth
 
     lib()  # fail loudly if the CUDA library is missing
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    from paper_2509_09679_b200.replicas import Replicas
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(v: float) -> float:
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    ranks = Replicas(dev)
+    rank, world, dist = ranks.rank, ranks.world, ranks.dist
+    barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     if args.op == "backward":
         return run_backward_only(torch, args, synth, Plan, dev)
@@ -226,7 +212,7 @@ def main():
         wl = dataclasses.replace(wl, n_rows=args.rows)
     # replicas only: every rank runs the whole workload on its own GPU with its own seed
     theta = wl.theta(device=dev, seed=wl.seed)
-    x = wl.x(device=dev, seed=wl.seed + 100 * rank)
+    x = wl.x(device=dev, seed=ranks.seed(wl.seed))
     plan = Plan(wl.n, dev)
     codes = torch.empty((wl.n_rows, wl.n * wl.bits // 8), dtype=torch.uint8, device=dev)
     scales = torch.empty((wl.n_rows,), dtype=torch.float16, device=dev)
@@ -263,7 +249,7 @@ def main():
     status = plan.device_status()
     if status != 0:
         raise SystemExit(f"device status {status}")
-    value = world * wl.n_rows / (ms_step * 1e-3)
+    value = ranks.whole_job_rate(wl.n_rows, ms_step)
 
     # ---- end-to-end through the public API with host buffers --------------------------------------
     e2e = None
