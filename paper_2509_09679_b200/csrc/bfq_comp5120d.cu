@@ -139,18 +139,28 @@ __device__ __forceinline__ void tmem_wait_ld8(uint32_t (&v)[8]) {
 }
 
 // ---- TMA thread: three stages of 4 tokens ---------------------------------------------------------------------------
+__device__ __forceinline__ void issue_load(const CUtensorMap* tmap, uint32_t smem, uint32_t bars, int g) {
+    const int64_t token0 = int64_t(kTok) * (blockIdx.x + int64_t(g) * gridDim.x);
+    const int stage = g % kStagesX;
+    const uint32_t bar = bars + 8 * (kBarXFull + stage), dst = smem + kXOff + stage * kStageBytes;
+    mbar_expect_tx(bar, kStageBytes);
+    tma_load_3d(dst, tmap, 0, 0, static_cast<int>(token0), bar);
+    tma_load_3d(dst + kHalfBytes, tmap, 64, 0, static_cast<int>(token0), bar);
+}
+
+// the first loads (every stage is free) go out before the CTA stages its resident operands
+__device__ __forceinline__ void tma_prologue(const CUtensorMap* tmap, uint32_t smem, uint32_t bars, int n_groups) {
+    for (int g = 0; g < kStagesX && g < n_groups; ++g) issue_load(tmap, smem, bars, g);
+}
+
 __device__ __forceinline__ void tma_role(const Params& P, const CUtensorMap* tmap, uint32_t smem, uint32_t bars,
                                          int n_groups) {
-    const int64_t stride = int64_t(kTok) * gridDim.x, first = int64_t(kTok) * blockIdx.x;
-    int issued = 0;
-    for (int g = 0; g < n_groups; ++g) {
+    int issued = n_groups < kStagesX ? n_groups : kStagesX;
+    for (int g = kStagesX; g < n_groups; ++g) {
         const int stage = g % kStagesX;
         // the stage is free once the MMAs that read it have completed (their commit arrives on x_empty)
-        if (g >= kStagesX && !wait_or_fail<500>(bars + 8 * (kBarXEmpty + stage), ((g / kStagesX) - 1) & 1, P.status)) break;
-        const uint32_t bar = bars + 8 * (kBarXFull + stage), dst = smem + kXOff + stage * kStageBytes;
-        mbar_expect_tx(bar, kStageBytes);
-        tma_load_3d(dst, tmap, 0, 0, static_cast<int>(first + g * stride), bar);
-        tma_load_3d(dst + kHalfBytes, tmap, 64, 0, static_cast<int>(first + g * stride), bar);
+        if (!wait_or_fail<40>(bars + 8 * (kBarXEmpty + stage), ((g / kStagesX) - 1) & 1, P.status)) break;
+        issue_load(tmap, smem, bars, g);
         issued = g + 1;
     }
     // no copy of this CTA may be in flight when it leaves (returns at once on the normal path)
@@ -341,6 +351,8 @@ k_comp5120d(const __grid_constant__ Params P, const __grid_constant__ CUtensorMa
     }
     __syncwarp();
     if (warp == 0) tmem_alloc512(smem_u32(tmem_slot));
+    __syncthreads();  // barriers are initialised: the first loads can go out while the operands are being staged
+    if (warp == kTmaWarp && lane == 0) tma_prologue(&tmap, smem, bars, n_groups);
     // Q2 (two bf16 terms, already in the swizzled operand layout) and Q1 (TF32, K-major without swizzle: row i and
     // contraction index kq = k mod 8 of k-step k / 8 at 256 (i / 8) + 16 (i mod 8) + 128 (kq / 4) + 4 (kq mod 4))
     for (int e = t; e < kQ2Bytes / 16; e += kThreads) reinterpret_cast<uint4*>(sm + kQ2Off)[e] = __ldg(P.q2img + e);
