@@ -261,3 +261,38 @@ def test_full_size_composite_5120_sampled(path, monkeypatch):
     assert frac <= 2e-2
     c2, s2 = p.composite_forward_quant(q1, x, 4)  # bit-identical from run to run
     assert torch.equal(c2, codes.view) and torch.equal(s2.view(torch.int16), scales.view.view(torch.int16))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_tensor_core_composite_5120_degenerate_rows(path, monkeypatch):
+    """Zero rows (scale 0, codes 0), rows so small that the fp16 scale is subnormal, rows so large that it saturates."""
+    _select(monkeypatch, path)
+    rows = 11
+    p, q1, x, _, _ = _tf32_setup(rows, seed=31, path=path)
+    xs = x.clone().float()
+    xs[1] = 0.0
+    xs[2] *= 1e-7
+    xs[3] *= 1e-9
+    xs[5] *= 1e28
+    xs[8] = 0.0
+    xs[8, 4097] = 3.0
+    x = xs.to(torch.bfloat16)
+    x64 = to_f64(x)
+    n1, n2 = 40, 128
+    th2 = to_f64(synth.angles(n2, "normal", 31))
+    Q1 = oracle.cayley(to_f64(synth.cayley_params(n1, 31, 0.1)), n1)
+    inner = oracle.forward(th2, x64.reshape(-1, n2)).reshape(rows, n1, n2)
+    y_ref = np.einsum("ik,rkj->rij", Q1, inner).reshape(rows, -1)
+    tol = 2.0 ** -9 * np.einsum("ik,rkj->rij", np.abs(Q1), np.abs(inner)).reshape(rows, -1)
+    Q2 = oracle.forward(th2, np.eye(n2)).T
+    absin = (np.abs(x64).reshape(-1, n2) @ np.abs(Q2).T).reshape(rows, n1, n2)
+    tol = tol + 2.0 ** -16 * np.einsum("ik,rkj->rij", np.abs(Q1), absin).reshape(rows, -1) + 1e-5 * np.abs(x64).max(axis=1, keepdims=True)
+    codes, scales = p.composite_forward_quant(q1, x.to(DEV), 4)
+    assert p.device_status() == 0
+    s = scales.cpu().view(torch.int16).numpy().view(np.uint16)
+    assert s[1] == 0 and not codes[1].any()          # zero row
+    assert s[5] == 0x7BFF                              # saturated scale: codes clip
+    assert 0 < s[3] < 0x0400 or s[3] == 0              # subnormal (or flushed) scale
+    _check_tf32_quant(codes, scales, y_ref, tol, "degenerate rows")
+    y = p.composite_forward(q1, x.to(DEV))
+    _check_tf32_rows(y, y_ref, tol, "degenerate rows, bf16 out")
