@@ -467,8 +467,9 @@ def time_others(torch, synth, Plan, dev):
             for _ in range(3):
                 fn()
             ms = event_time_ms(torch, fn, 10)
-            res[name + suffix] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": nbytes * rows / (ms * 1e-3) / 1e9,
-                                  "rows": rows, "n": 5120}
+            gbs = nbytes * rows / (ms * 1e-3) / 1e9
+            res[name + suffix] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": gbs,
+                                  "hbm_frac": gbs / measured_peaks()["hbm_gbs"], "rows": rows, "n": 5120}
     os.environ.pop("BFQ_COMPOSITE_FP32_BUTTERFLY", None)
     return res
 
