@@ -315,9 +315,14 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
     cudaError_t e;
-    if (hist != nullptr) {  // statistics: the histogram starts at zero; the generic kernels carry them
+    if (hist != nullptr) {  // statistics: the histogram starts at zero
         e = cudaMemsetAsync(hist, 0, sizeof(unsigned long long) << bits, static_cast<cudaStream_t>(stream));
         if (e != cudaSuccess) return cuda_fail(plan, e);
+        if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+            fwdq4096_available(plan)) {
+            e = fwdq4096_launch_stats(plan, x, rows, ldx, codes, scales, hist, rowstats, static_cast<cudaStream_t>(stream));
+            return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+        }
     } else if (xt == BFQ_BF16 && bits == 4 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq4096_available(plan)) {
         e = fwdq4096_launch(plan, x, rows, ldx, false, codes, scales, nullptr, 0, static_cast<cudaStream_t>(stream));

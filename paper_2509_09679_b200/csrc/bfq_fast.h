@@ -16,6 +16,10 @@ cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaSt
 cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, bool hadamard,
                             uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 
+// the same with the statistics of bfq_forward_quant_stats (hist already zeroed on `st`)
+cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                                  uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st);
+
 // n = 8192, bf16 rows, INT2: two-CTA clusters, one 4096-point half per CTA
 size_t fwdq8192_image_bytes();
 size_t fwdq8192_prep_bytes();

@@ -42,7 +42,8 @@ struct Smem {
     static constexpr uint32_t kExOff = kInOff + G * kInSlots * kRowBytes;  // [G][XB][kExBytes]
     static constexpr uint32_t kBarOff = kExOff + G * XB * kExBytes;       // mbarriers [G][kInSlots]
     static constexpr uint32_t kAmaxOff = kBarOff + 8 * G * kInSlots;      // float [G][2 parities][4 warps]
-    static constexpr uint32_t kTmemOff = kAmaxOff + 32 * G;               // tensor-memory base address
+    static constexpr uint32_t kStatOff = kAmaxOff + 32 * G;               // float [G][2 parities][4 warps][2]: row moments
+    static constexpr uint32_t kTmemOff = kStatOff + 64 * G;               // tensor-memory base address
     static constexpr uint32_t kUsed = kTmemOff + 16;
     static constexpr uint32_t kBytes = kUsed + 1024;  // slack for the 1024-byte alignment of the TMA tiles
 };
@@ -152,10 +153,11 @@ __device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&&
 }
 
 enum : int { kButterfly = 0, kHadamard = 1 };  // TRANSFORM
-enum : int { kOutInt4 = 0, kOutBf16 = 1 };     // OUT
+enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2 };  // OUT
 
 // TRANSFORM: learned butterfly (constants in tensor memory) or the fixed Walsh-Hadamard transform (no constants,
-// no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy).
+// no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy), or
+// codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]).
 template <int G, int CW, int XB, int TRANSFORM, int OUT>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, uint8_t* __restrict__ codes,
@@ -303,7 +305,40 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
         const uint32_t aslot = amax_base + (k & 1) * 16;
         if (lane == 0) sts32(aslot + q * 4, __float_as_uint(amax));
+        const uint32_t mslot = sbase + S::kStatOff + g * 64 + (k & 1) * 32;
+        if constexpr (OUT == kOutInt4Stats) {
+            // sum y^2 and sum y^4 of the row: thread (fixed order), warp (xor tree), then the four warps in order
+            u64 s2v = pack2(0.f, 0.f), s4v = pack2(0.f, 0.f);
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                const u64 sq = mul2(P[m], P[m]);
+                s2v = add2(s2v, sq);
+                s4v = fma2(sq, sq, s4v);
+            }
+            float a2, b2, a4, b4;
+            unpack2(s2v, a2, b2), unpack2(s4v, a4, b4);
+            float s2 = a2 + b2, s4 = a4 + b4;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+                s4 += __shfl_xor_sync(0xFFFFFFFFu, s4, o);
+            }
+            if (lane == 0) sts64(mslot + q * 8, pack2(s2, s4));
+        }
         bar_sync(ex.bar, kGroupThreads);
+        if constexpr (OUT == kOutInt4Stats) {
+            if (t == 0) {
+                float s2 = 0.f, s4 = 0.f;
+#pragma unroll
+                for (int w4 = 0; w4 < 4; ++w4) {
+                    float a, b;
+                    unpack2(lds64(mslot + w4 * 8), a, b);
+                    s2 += a, s4 += b;
+                }
+                float* rs = reinterpret_cast<float*>(yout) + 2 * static_cast<int64_t>(row);
+                rs[0] = s2 * (kPost * kPost), rs[1] = s4 * (kPost * kPost * kPost * kPost);
+            }
+        }
         {
             const uint4 o = lds128(aslot);
             amax = fmaxf(fmaxf(__uint_as_float(o.x), __uint_as_float(o.y)),
@@ -409,6 +444,41 @@ __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restric
     }
 }
 
+// Histogram of the 4-bit codes of packed rows (two per byte): every warp counts whole bytes in its own 256-bin table in
+// shared memory (few lanes of a warp hit the same byte value at once), the CTA folds the byte counts into the 16 code
+// counts (a byte contributes to its low and to its high nibble) and adds them to hist[code + 8] (code = the nibble as a
+// two's complement number).  Counts are exact.
+constexpr int kHistThreads = 256;
+__global__ void __launch_bounds__(kHistThreads) k_hist_int4(const uint4* __restrict__ codes, int64_t chunks,
+                                                            unsigned long long* __restrict__ hist) {
+    __shared__ unsigned int bytes[kHistThreads / 32][256];
+    __shared__ unsigned long long bins[16];
+    const int t = threadIdx.x, warp = t >> 5;
+    for (int e = t; e < (kHistThreads / 32) * 256; e += kHistThreads) (&bytes[0][0])[e] = 0u;
+    if (t < 16) bins[t] = 0ull;
+    __syncthreads();
+    unsigned int* mine = bytes[warp];
+    for (int64_t c = int64_t(blockIdx.x) * kHistThreads + t; c < chunks; c += int64_t(gridDim.x) * kHistThreads) {
+        const uint4 v = __ldg(codes + c);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+#pragma unroll
+            for (int b = 0; b < 4; ++b) atomicAdd(mine + ((w[k] >> (8 * b)) & 0xFFu), 1u);
+        }
+    }
+    __syncthreads();
+    unsigned int n = 0;  // thread t: byte value t
+#pragma unroll
+    for (int wi = 0; wi < kHistThreads / 32; ++wi) n += bytes[wi][t];
+    if (n != 0u) {
+        atomicAdd(&bins[(t & 15) ^ 8], static_cast<unsigned long long>(n));
+        atomicAdd(&bins[(t >> 4) ^ 8], static_cast<unsigned long long>(n));
+    }
+    __syncthreads();
+    if (t < 16 && bins[t] != 0ull) atomicAdd(hist + t, bins[t]);
+}
+
 }  // namespace f4k
 
 // ---- host side ---------------------------------------------------------------------------------------------
@@ -465,6 +535,21 @@ cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, i
     }
     return y == nullptr ? launch_variant<4, 32, 2, kHadamard, kOutInt4>(plan, tmap, rows, codes, scales, y, ldy, st)
                         : launch_variant<4, 32, 2, kHadamard, kOutBf16>(plan, tmap, rows, codes, scales, y, ldy, st);
+}
+
+// bfq_forward_quant_stats on the tuned path: codes + scales + row moments from k_fwdq4096, then the code histogram from
+// the packed codes (hist must have been zeroed on the same stream).
+cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                                  uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st) {
+    CUtensorMap tmap;
+    if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
+    using namespace f4k;
+    cudaError_t e = launch_variant<4, 32, 2, kButterfly, kOutInt4Stats>(plan, tmap, rows, codes, scales, rowstats, 0, st);
+    if (e != cudaSuccess) return e;
+    const int64_t chunks = rows * (kN / 2 / 16);
+    const int64_t want = (chunks + kHistThreads - 1) / kHistThreads, cap = int64_t(plan->sm_count) * 8;
+    k_hist_int4<<<int(want < cap ? want : cap), kHistThreads, 0, st>>>(reinterpret_cast<const uint4*>(codes), chunks, hist);
+    return cudaGetLastError();
 }
 
 }  // namespace bfq

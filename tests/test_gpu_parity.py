@@ -495,6 +495,8 @@ def test_tuned_n4096_hadamard_and_bf16_rows(rows):
 
 # ---- statistics riding on forward + quantize ---------------------------------------------------------------------
 @pytest.mark.parametrize("n,rows,bits,dtype", [(256, 1000, 4, torch.float32), (4096, 333, 4, torch.bfloat16),
+                                               (4096, 1, 4, torch.bfloat16), (4096, 1187, 4, torch.bfloat16),
+                                               (4096, 77, 4, torch.float32),
                                                (8192, 70, 2, torch.bfloat16), (1024, 129, 8, torch.bfloat16)])
 def test_forward_quant_stats(n, rows, bits, dtype):
     theta, x = make(n, rows, dtype, seed=120 + n)
