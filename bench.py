@@ -35,7 +35,7 @@ SLOTS_PER_ROW = 4 * (4096 // 2) * 12 + 4096
 FP32_LANES_PER_SM = 128
 # dram bytes (read + write) per row of the forward+quant kernel, from the committed ncu capture of the
 # current kernel on this workload; set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_ROW = (268.678144e6 + 50.600960e6) / 32768  # profiles/fwdq4096_act4096_int4.md
+NCU_TRAFFIC_BYTES_PER_ROW = (268678912 + 50833408) / 32768  # dram read + write of one k_fwdq4096 launch (profiles/)
 
 
 def measured_peaks():
