@@ -516,3 +516,22 @@ def test_forward_quant_stats(n, rows, bits, dtype):
     np.testing.assert_allclose(to_f64(rowstats), oracle.row_moments(y_ref), rtol=2e-5)
     _, _, hist2, rs2 = p.forward_quant_stats(x.to(DEV), bits)
     assert torch.equal(hist, hist2) and torch.equal(rs2, rowstats)
+
+
+# ---- rows in pinned host memory: chunked copies overlapped with the kernels -------------------------------------------
+@pytest.mark.parametrize("rows,chunks", [(1000, 8), (5, 8), (4096, 3)])
+def test_host_pipeline_matches_the_resident_call(rows, chunks):
+    from paper_2509_09679_b200 import HostForwardQuant
+    theta, x = make(4096, rows, torch.bfloat16, seed=77)
+    p = plan_for(4096, theta)
+    c_ref, s_ref = p.forward_quant(x.to(DEV), 4)
+    x_host = x.pin_memory()
+    c_host = torch.zeros((rows, 2048), dtype=torch.uint8).pin_memory()
+    s_host = torch.zeros((rows,), dtype=torch.float16).pin_memory()
+    pipe = HostForwardQuant(p, rows, 4, chunks=chunks)
+    for _ in range(2):  # second call reuses the buffers and events
+        c_host.zero_()
+        pipe(x_host, c_host, s_host, before=lambda: p.set_angles(theta.to(DEV)))
+        torch.cuda.synchronize()
+        assert torch.equal(c_host, c_ref.cpu()) and torch.equal(s_host.view(torch.int16), s_ref.cpu().view(torch.int16))
+    assert p.device_status() == 0
