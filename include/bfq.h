@@ -176,6 +176,12 @@ int bfq_composite_forward(bfq_plan* plan, const float* q1, int n1, const void* x
                           int64_t ldx, void* y, bfq_dtype yt, int64_t ldy, void* stream);
 int bfq_composite_forward_quant(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,
                                 int64_t ldx, int bits, uint8_t* codes, uint16_t* scales_f16, void* stream);
+/* x = (Q1 (x) Q2)^T y per row, the inverse of bfq_composite_forward (both factors are orthogonal, Sec. 3.3, "Proof of
+ * orthogonality"): X = (Q1^T Y) Q2, i.e. Q1^T across the runs and the inverse butterfly on every run.  Also dL/dx of the
+ * composite for an upstream gradient y.  Same shapes, limits and arithmetic as bfq_composite_forward (for n1 = 40,
+ * n2 = 128, bf16 in and out: both factors on the tensor cores). */
+int bfq_composite_inverse(bfq_plan* plan, const float* q1, int n1, const void* y, bfq_dtype yt, int64_t rows, int64_t ldy,
+                          void* x, bfq_dtype xt, int64_t ldx, void* stream);
 
 /*
  * bfq_backward without any device-memory allocation.  (No counterpart in the paper: this exists for

@@ -218,6 +218,18 @@ def composite_forward(Q1, theta2, x) -> np.ndarray:
     return np.einsum("ik,rkj->rij", Q1, inner).reshape(x.shape)
 
 
+def composite_inverse(Q1, theta2, y) -> np.ndarray:
+    """x = (Q1 kron Q2)^T y per row (= the inverse: both factors are orthogonal, Sec. 3.3): with y as an n1 x n2 matrix Y,
+    X = (Q1^T Y) Q2: Q1^T across the n1 runs, then Q2^T = the inverse butterfly on every run."""
+    Q1 = _f64(Q1)
+    n1 = Q1.shape[0]
+    y = _f64(y)
+    rows = y.reshape(-1, y.shape[-1])
+    n2 = rows.shape[1] // n1
+    mixed = np.einsum("ki,rkj->rij", Q1, rows.reshape(rows.shape[0], n1, n2))
+    return inverse(theta2, mixed.reshape(-1, n2)).reshape(y.shape)
+
+
 def backward(theta, x, g):
     """-> (dx float64 [rows][n], dtheta float64 [L][n/2] summed over rows)."""
     x = _f64(x)

@@ -43,6 +43,7 @@ SIGNATURES = {
     "bfq_cayley": (_i, [_p, _p, _i, _p, _p]),
     "bfq_composite_forward": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
     "bfq_composite_forward_quant": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _i, _p, _p, _p]),
+    "bfq_composite_inverse": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
 }
 
 _lib = None
@@ -164,6 +165,15 @@ class Plan:
         _check(lib().bfq_composite_forward(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(),
                                            _dt(y), d, _stream(x)), "bfq_composite_forward")
         return y
+
+    def composite_inverse(self, q1: torch.Tensor, y: torch.Tensor, out_dtype=None, out=None) -> torch.Tensor:
+        n1 = self._q1(q1)
+        d = n1 * self.n
+        rows, ldy = _rows(y, d)
+        x = out if out is not None else torch.empty((rows, d), dtype=out_dtype or y.dtype, device=y.device)
+        _check(lib().bfq_composite_inverse(self._h, q1.data_ptr(), n1, y.data_ptr(), _dt(y), rows, ldy, x.data_ptr(),
+                                           _dt(x), d, _stream(y)), "bfq_composite_inverse")
+        return x
 
     def composite_forward_quant(self, q1: torch.Tensor, x: torch.Tensor, bits: int, codes=None, scales=None):
         n1 = self._q1(q1)

@@ -481,7 +481,8 @@ int bfq_cayley(bfq_plan* plan, const float* params, int n1, float* q1, void* str
 }
 
 static int composite_impl(bfq_plan* plan, const float* q1, int n1, const void* x, int xt, int64_t rows, int64_t ldx,
-                          void* y, int yt, int64_t ldy, int bits, uint8_t* codes, uint16_t* scales, void* stream) {
+                          void* y, int yt, int64_t ldy, int bits, uint8_t* codes, uint16_t* scales, void* stream,
+                          bool inverse = false) {
     if (plan == nullptr || q1 == nullptr) return BFQ_ERR_NULL;
     if (n1 < 2 || n1 > BFQ_MAX_N1 || plan->n > 1024 || int64_t(n1) * plan->n > BFQ_COMPOSITE_MAX_D)
         return BFQ_ERR_UNSUPPORTED_N;
@@ -506,16 +507,16 @@ static int composite_impl(bfq_plan* plan, const float* q1, int n1, const void* x
         (y == nullptr || yt == BFQ_BF16) && !env_flag("BFQ_GENERIC_ONLY")) {
         // default: both factors on the tensor cores; BFQ_COMPOSITE_FP32_BUTTERFLY=1 keeps Q2 as an fp32 butterfly on
         // the CUDA cores (only the dense factor on the tensor cores)
-        if (!env_flag("BFQ_COMPOSITE_FP32_BUTTERFLY") && comp5120d_available(plan)) {
-            e = comp5120d_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
+        if ((inverse || !env_flag("BFQ_COMPOSITE_FP32_BUTTERFLY")) && comp5120d_available(plan)) {
+            e = comp5120d_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, inverse, static_cast<cudaStream_t>(stream));
             return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
         }
-        if (comp5120_available(plan)) {
+        if (!inverse && comp5120_available(plan)) {
             e = comp5120_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
             return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
         }
     }
-    e = composite_generic_launch(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, bits, codes, scales,
+    e = composite_generic_launch(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, bits, codes, scales, inverse,
                                  static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
@@ -524,6 +525,12 @@ int bfq_composite_forward(bfq_plan* plan, const float* q1, int n1, const void* x
                           int64_t ldx, void* y, bfq_dtype yt, int64_t ldy, void* stream) {
     if (y == nullptr && rows != 0) return BFQ_ERR_NULL;
     return composite_impl(plan, q1, n1, x, xt, rows, ldx, y, yt, ldy, 4, nullptr, nullptr, stream);
+}
+
+int bfq_composite_inverse(bfq_plan* plan, const float* q1, int n1, const void* y, bfq_dtype yt, int64_t rows, int64_t ldy,
+                          void* x, bfq_dtype xt, int64_t ldx, void* stream) {
+    if (x == nullptr && rows != 0) return BFQ_ERR_NULL;
+    return composite_impl(plan, q1, n1, y, yt, rows, ldy, x, xt, ldx, 4, nullptr, nullptr, stream, true);
 }
 
 int bfq_composite_forward_quant(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,

@@ -75,6 +75,7 @@ struct Params {
     int64_t ldy;
     int64_t rows;
     int* status;
+    int transpose_q1;     // 1: apply Q1^T (the inverse transform; q2img then holds Q2^T)
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -358,7 +359,7 @@ k_comp5120d(const __grid_constant__ Params P, const __grid_constant__ CUtensorMa
     for (int e = t; e < kQ2Bytes / 16; e += kThreads) reinterpret_cast<uint4*>(sm + kQ2Off)[e] = __ldg(P.q2img + e);
     for (int e = t; e < kNPad * kN1; e += kThreads) {
         const int i = e / kN1, k = e - i * kN1, kq = k & 7;
-        const float val = i < kN1 ? P.q1[i * kN1 + k] : 0.f;
+        const float val = i < kN1 ? (P.transpose_q1 ? P.q1[k * kN1 + i] : P.q1[i * kN1 + k]) : 0.f;
         *reinterpret_cast<uint32_t*>(sm + kQ1Off + (k >> 3) * kBBlock + 256 * (i >> 3) + 16 * (i & 7) + 128 * (kq >> 2) +
                                      4 * (kq & 3)) = (__float_as_uint(val) + 0x1000u) & 0xFFFFE000u;
     }
@@ -386,6 +387,7 @@ k_comp5120d(const __grid_constant__ Params P, const __grid_constant__ CUtensorMa
 // Dense Q2 from the plan's (cos, sin) table: thread c pushes the unit vector e_c through the 7 stages in float64 and
 // writes column c, split into two bf16 terms, at its place in the swizzled K-major operand image:
 // [term][half = c / 64][row j][16-byte chunk ((c mod 64) / 8) xor (j mod 8)][c mod 8].
+// The second image (offset kQ2Bytes) holds Q2^T in the same layout, for the inverse transform.
 __global__ void __launch_bounds__(kN2) k_build_dense128(const float2* __restrict__ tw, __nv_bfloat16* __restrict__ img) {
     const int c = threadIdx.x;
     double col[kN2];
@@ -406,13 +408,17 @@ __global__ void __launch_bounds__(kN2) k_build_dense128(const float2* __restrict
         const int idx = (c >> 6) * (kQ2Half / 2) + jj * 64 + ((((c & 63) >> 3) ^ (jj & 7)) << 3) + (c & 7);
         img[idx] = hi;
         img[2 * (kQ2Half / 2) + idx] = lo;
+        // transposed: row c, contraction index jj
+        const int idt = (jj >> 6) * (kQ2Half / 2) + c * 64 + ((((jj & 63) >> 3) ^ (c & 7)) << 3) + (jj & 7);
+        img[kQ2Bytes / 2 + idt] = hi;
+        img[kQ2Bytes / 2 + 2 * (kQ2Half / 2) + idt] = lo;
     }
 }
 
 }  // namespace c5d
 
 // ---- host side -----------------------------------------------------------------------------------------------------
-size_t comp5120d_image_bytes() { return c5d::kQ2Bytes; }
+size_t comp5120d_image_bytes() { return 2 * c5d::kQ2Bytes; }  // Q2 and Q2^T
 
 bool comp5120d_available(const bfq_plan* plan) {
     return plan->n == c5d::kN2 && plan->cc_major == 10 && plan->dense128 != nullptr && encode_tiled() != nullptr;
@@ -424,10 +430,11 @@ cudaError_t comp5120d_set_angles(const bfq_plan* plan, cudaStream_t st) {
 }
 
 cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                             uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st) {
+                             uint16_t* scales, void* y_bf16, int64_t ldy, bool inverse, cudaStream_t st) {
     using namespace c5d;
     Params P{};
-    P.q2img = static_cast<const uint4*>(plan->dense128);
+    P.q2img = static_cast<const uint4*>(plan->dense128) + (inverse ? kQ2Bytes / 16 : 0);
+    P.transpose_q1 = inverse ? 1 : 0;
     P.q1 = q1, P.codes = codes, P.scales = scales, P.y = static_cast<__nv_bfloat16*>(y_bf16), P.ldy = ldy;
     P.rows = rows, P.status = plan->status_word;
     // x: [rows][ldx] bf16 seen as {128 positions of a run, 40 runs, rows tokens}; a box is 64 positions of every run of

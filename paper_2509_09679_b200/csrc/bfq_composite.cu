@@ -91,6 +91,7 @@ struct CompositeParams {
     uint16_t* scales;
     int bits;
     int64_t rows;
+    int inverse;  // 1: x = (Q1 kron Q2)^T y: inverse butterfly on every run (stages last to first, G^T), then Q1^T
 };
 
 __global__ void __launch_bounds__(kThreads) k_composite_generic(const CompositeParams p) {
@@ -101,7 +102,10 @@ __global__ void __launch_bounds__(kThreads) k_composite_generic(const CompositeP
     float* q1s = sm + 2 * d;     // [n1p][n1], rows n1..n1p-1 zero
     __shared__ float red[kWarps];
     const int t = threadIdx.x;
-    for (int e = t; e < n1p * n1; e += kThreads) q1s[e] = e < n1 * n1 ? p.q1[e] : 0.f;
+    for (int e = t; e < n1p * n1; e += kThreads) {  // row i of the factor applied: Q1[i][:] or, for the inverse, Q1[:][i]
+        const int i = e / n1, k = e - i * n1;
+        q1s[e] = i < n1 ? (p.inverse ? p.q1[k * n1 + i] : p.q1[e]) : 0.f;
+    }
 
     for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x) {
         __syncthreads();  // previous token's readers of buf / out are done
@@ -111,14 +115,17 @@ __global__ void __launch_bounds__(kThreads) k_composite_generic(const CompositeP
 #pragma unroll
             for (int e = 0; e < 16; ++e) buf[16 * c + e] = v[e];
         }
-        // Q2 on every run: stage s couples lo and lo + 2^s inside the run
-        for (int s = 0; s < p.log_n2; ++s) {
+        // Q2 (or Q2^T) on every run: stage s couples lo and lo + 2^s inside the run
+        for (int ss = 0; ss < p.log_n2; ++ss) {
             __syncthreads();
+            const int s = p.inverse ? p.log_n2 - 1 - ss : ss;
+            const float sgn = p.inverse ? -1.f : 1.f;
             const float2* tws = p.tw + s * h2;
             for (int pr = t; pr < d / 2; pr += kThreads) {
                 const int r = pr / h2, q = pr - r * h2;
                 const int lo = r * n2 + (((q >> s) << (s + 1)) | (q & ((1 << s) - 1))), hi = lo + (1 << s);
-                const float2 cs = __ldg(tws + q);
+                float2 cs = __ldg(tws + q);
+                cs.y *= sgn;
                 const float a = buf[lo], b = buf[hi];
                 buf[lo] = fmaf(cs.x, a, -cs.y * b);
                 buf[hi] = fmaf(cs.y, a, cs.x * b);
@@ -179,11 +186,11 @@ cudaError_t cayley_launch(const float* params, int n1, float* q1, cudaStream_t s
 
 cudaError_t composite_generic_launch(const bfq_plan* plan, const float* q1, int n1, const void* x, int xt, int64_t rows,
                                      int64_t ldx, void* y, int yt, int64_t ldy, int bits, uint8_t* codes,
-                                     uint16_t* scales, cudaStream_t st) {
+                                     uint16_t* scales, bool inverse, cudaStream_t st) {
     comp::CompositeParams p{};
     p.tw = plan->tw, p.q1 = q1, p.n1 = n1, p.n2 = plan->n, p.log_n2 = plan->log_n;
     p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = ldy;
-    p.codes = codes, p.scales = scales, p.bits = bits, p.rows = rows;
+    p.codes = codes, p.scales = scales, p.bits = bits, p.rows = rows, p.inverse = inverse ? 1 : 0;
     const int d = n1 * plan->n, n1p = (n1 + 7) & ~7;
     const size_t smem = sizeof(float) * (size_t(2) * d + size_t(n1p) * n1);
     cudaError_t e = cudaFuncSetAttribute(comp::k_composite_generic, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));

@@ -45,7 +45,7 @@ cudaError_t inv4096_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t 
 cudaError_t cayley_launch(const float* params, int n1, float* q1, cudaStream_t st);
 cudaError_t composite_generic_launch(const bfq_plan* plan, const float* q1, int n1, const void* x, int xt, int64_t rows,
                                      int64_t ldx, void* y, int yt, int64_t ldy, int bits, uint8_t* codes,
-                                     uint16_t* scales, cudaStream_t st);
+                                     uint16_t* scales, bool inverse, cudaStream_t st);
 
 
 // composite 40 x 128 on bf16 rows: butterfly with kernel-parameter constants + tcgen05 TF32 dense factor
@@ -60,6 +60,6 @@ size_t comp5120d_image_bytes();
 bool comp5120d_available(const bfq_plan* plan);
 cudaError_t comp5120d_set_angles(const bfq_plan* plan, cudaStream_t st);
 cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                             uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
+                             uint16_t* scales, void* y_bf16, int64_t ldy, bool inverse, cudaStream_t st);
 
 }  // namespace bfq

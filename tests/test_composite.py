@@ -296,3 +296,42 @@ def test_tensor_core_composite_5120_degenerate_rows(path, monkeypatch):
     _check_tf32_quant(codes, scales, y_ref, tol, "degenerate rows")
     y = p.composite_forward(q1, x.to(DEV))
     _check_tf32_rows(y, y_ref, tol, "degenerate rows, bf16 out")
+
+
+# ---- inverse / transpose of the composite ---------------------------------------------------------------------------
+@pytest.mark.parametrize("n1,n2,rows", [(3, 16, 7), (12, 256, 33), (40, 128, 61), (7, 1024, 20)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_composite_inverse_generic(n1, n2, rows, dtype, monkeypatch):
+    monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+    p, q1, Q1_ref, th2, y = setup(n1, n2, rows, dtype)
+    x_ref = oracle.composite_inverse(Q1_ref, th2, to_f64(y))
+    amax = np.abs(to_f64(y)).max(axis=1)
+    x = p.composite_inverse(q1, y.to(DEV), out_dtype=torch.float32)
+    check_rows_close(x, x_ref, amax, "composite inverse")
+    # forward(inverse(y)) = y
+    back = p.composite_forward(q1, x, out_dtype=torch.float32)
+    check_rows_close(back, to_f64(y), np.sqrt(n1 * n2) * amax, "composite round trip")
+
+
+@pytest.mark.parametrize("rows", [1, 3, 4, 593, 2500])
+def test_tensor_core_composite_inverse_5120(rows):
+    n1, n2 = 40, 128
+    p, q1, y, _, _ = _tf32_setup(rows, seed=41, path="dense")
+    th2 = to_f64(synth.angles(n2, "normal", 41))
+    Q1 = oracle.cayley(to_f64(synth.cayley_params(n1, 41, 0.1)), n1)
+    y64 = to_f64(y)
+    x_ref = oracle.composite_inverse(Q1, th2, y64)
+    # same error model as the forward dense path, with the transposed factors
+    inner = oracle.inverse(th2, y64.reshape(-1, n2)).reshape(rows, n1, n2)
+    Q2 = oracle.forward(th2, np.eye(n2)).T
+    absin = (np.abs(y64).reshape(-1, n2) @ np.abs(Q2)).reshape(rows, n1, n2)
+    tol = 2.0 ** -9 * np.einsum("ki,rkj->rij", np.abs(Q1), np.abs(inner)).reshape(rows, -1) \
+        + 2.0 ** -16 * np.einsum("ki,rkj->rij", np.abs(Q1), absin).reshape(rows, -1) + 1e-5 * np.abs(y64).max(axis=1, keepdims=True)
+    x = p.composite_inverse(q1, y.to(DEV))
+    assert p.device_status() == 0
+    _check_tf32_rows(x, x_ref, tol, "tensor-core composite inverse")
+    # adjoint identity <Q x, z> = <x, Q^T z> on the device results, in float64, within the two paths' tolerances
+    z = p.composite_forward(q1, y.to(DEV))
+    lhs = (to_f64(z) * y64).sum(axis=1)
+    rhs = (y64 * to_f64(x)).sum(axis=1)
+    assert np.all(np.abs(lhs - rhs) <= 2e-2 * (np.abs(y64) ** 2).sum(axis=1))

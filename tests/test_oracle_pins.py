@@ -425,3 +425,8 @@ def test_cayley_and_kronecker_composite():
     np.testing.assert_allclose(K.T @ K, np.eye(n1 * n2), atol=1e-13)
     y = oracle.composite_forward(Q1, rand_theta(128), RNG.standard_normal((2, 5120)))
     assert y.shape == (2, 5120)
+    # the inverse is the transpose of the Kronecker matrix, undoes the forward map and is its adjoint
+    z = RNG.standard_normal((6, n1 * n2))
+    np.testing.assert_allclose(oracle.composite_inverse(Q1s, th2, z), z @ K, atol=1e-13)
+    np.testing.assert_allclose(oracle.composite_inverse(Q1s, th2, oracle.composite_forward(Q1s, th2, x)), x, atol=1e-13)
+    assert abs(np.sum(oracle.composite_forward(Q1s, th2, x) * z) - np.sum(x * oracle.composite_inverse(Q1s, th2, z))) < 1e-12
