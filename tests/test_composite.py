@@ -335,3 +335,38 @@ def test_tensor_core_composite_inverse_5120(rows):
     lhs = (to_f64(z) * y64).sum(axis=1)
     rhs = (y64 * to_f64(x)).sum(axis=1)
     assert np.all(np.abs(lhs - rhs) <= 2e-2 * (np.abs(y64) ** 2).sum(axis=1))
+
+
+# ---- gradients of the composite, composed from the entry points --------------------------------------------------------
+def test_composite_backward_against_float64_and_finite_differences():
+    from paper_2509_09679_b200.composite import cayley_pullback, composite_backward
+    n1, n2, tokens = 6, 64, 37
+    theta2 = synth.angles(n2, "normal", 3)
+    params = synth.cayley_params(n1, 3, 0.3)
+    x = synth.rows(tokens, n1 * n2, "normal", 4)
+    g = synth.rows(tokens, n1 * n2, "normal", 5)
+    p = Plan(n2, DEV)
+    p.set_angles(theta2.to(DEV))
+    q1 = p.cayley(params.to(DEV), n1)
+    dx, dth2, dQ1, dpar = composite_backward(p, q1, params.to(DEV), x.to(DEV), g.to(DEV))
+    # float64 reference from the oracle's pieces: L(theta2, params) = sum(g * composite_forward(x))
+    th64, x64, g64, par64 = to_f64(theta2), to_f64(x), to_f64(g), to_f64(params)
+    Q1 = oracle.cayley(par64, n1)
+    check_rows_close(dx, oracle.composite_inverse(Q1, th64, g64), np.abs(g64).max(axis=1), "composite dx")
+    gp = np.einsum("ki,rkj->rij", Q1, g64.reshape(tokens, n1, n2)).reshape(-1, n2)
+    _, dth_ref = oracle.backward(th64, x64.reshape(-1, n2), gp)
+    from parity import check_dtheta
+    check_dtheta(dth2, dth_ref, "composite dtheta2")
+    xp = oracle.forward(th64, x64.reshape(-1, n2)).reshape(tokens, n1, n2)
+    dQ1_ref = np.einsum("rij,rkj->ik", g64.reshape(tokens, n1, n2), xp)
+    assert np.abs(to_f64(dQ1) - dQ1_ref).max() <= 1e-4 * np.abs(dQ1_ref).max()
+    # the Cayley pull-back against central differences of the oracle (CPU, float64)
+    loss = lambda q: float(np.sum(g64 * oracle.composite_forward(oracle.cayley(q, n1), th64, x64)))
+    fd = np.zeros_like(par64)
+    for k in range(par64.size):
+        e = np.zeros_like(par64)
+        e[k] = 1e-6
+        fd[k] = (loss(par64 + e) - loss(par64 - e)) / 2e-6
+    got = to_f64(cayley_pullback(torch.from_numpy(par64), n1, torch.from_numpy(dQ1_ref)))
+    assert np.abs(got - fd).max() <= 1e-6 * max(1.0, np.abs(fd).max())
+    assert np.abs(to_f64(dpar) - fd).max() <= 2e-4 * np.abs(fd).max()
