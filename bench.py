@@ -416,6 +416,13 @@ def time_others(torch, synth, Plan, dev):
     record("forward_int4_stats_n4096", wl.n_rows, wl.n, wl.L, 4, BYTES_PER_ROW + 8,
            lambda: plan.forward_quant_stats(x, 4), 10)
     record("forward_bf16_n4096", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan.forward(x, out=y), 20)
+    codes2 = torch.empty((wl.n_rows, wl.n // 4), dtype=torch.uint8, device=dev)
+    codes8 = torch.empty((wl.n_rows, wl.n), dtype=torch.uint8, device=dev)
+    record("forward_int2_n4096", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
+           lambda: plan.forward_quant(x, 2, codes=codes2, scales=scales), 20)
+    record("forward_int8_n4096", wl.n_rows, wl.n, wl.L, 4, 3 * wl.n + 2,
+           lambda: plan.forward_quant(x, 8, codes=codes8, scales=scales), 20)
+    del codes2, codes8
     record("hadamard_bf16_n4096", wl.n_rows, wl.n, wl.L, 1, 4 * wl.n, lambda: plan.hadamard(x, out=y), 20)
     del x, y, codes, scales, plan
     # angle-learning step: forward + backward on 128 x 2048 rows of n = 4096

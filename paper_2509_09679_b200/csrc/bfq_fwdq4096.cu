@@ -153,11 +153,12 @@ __device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&&
 }
 
 enum : int { kButterfly = 0, kHadamard = 1 };  // TRANSFORM
-enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2 };  // OUT
+enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutInt8 = 4 };  // OUT
 
 // TRANSFORM: learned butterfly (constants in tensor memory) or the fixed Walsh-Hadamard transform (no constants,
 // no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy), or
-// codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]).
+// codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]), or
+// INT2 / INT8 codes + scales.
 template <int G, int CW, int XB, int TRANSFORM, int OUT>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, uint8_t* __restrict__ codes,
@@ -344,10 +345,53 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             amax = fmaxf(fmaxf(__uint_as_float(o.x), __uint_as_float(o.y)),
                          fmaxf(__uint_as_float(o.z), __uint_as_float(o.w)));
         }
+        constexpr int kQmax = OUT == kOutInt2 ? 1 : (OUT == kOutInt8 ? 127 : 7);
         float inv;
-        const uint16_t s16 = row_scale(amax * kPost, 7, &inv);
+        const uint16_t s16 = row_scale(amax * kPost, kQmax, &inv);
         inv *= kPost;  // the registers still hold the un-normalised values (kPost is a power of two)
         if (t == 0) scales[row] = s16;
+
+        if constexpr (OUT == kOutInt8 || OUT == kOutInt2) {
+            // |v * inv| <= qmax (1 + 2^-10) < qmax + 1/2 for a normal, unsaturated fp16 scale: no clipping; v * inv +
+            // 1.5 * 2^23 then has the code (two's complement) in its low mantissa bits
+            const bool plain8 = (((s16 >> 10) & 31u) != 0u) && (s16 != 0x7BFFu);
+            uint32_t c[16];  // INT8: two bytes; INT2: four bits (two codes) of each packed register
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                uint32_t lo, hi;
+                if (plain8) {
+                    unpack2u(fma2(P[m], pack2(inv, inv), pack2(12582912.0f, 12582912.0f)), lo, hi);
+                } else {
+                    float a, b;
+                    unpack2(P[m], a, b);
+                    lo = static_cast<uint32_t>(quant1(a, inv, -kQmax - 1, kQmax));
+                    hi = static_cast<uint32_t>(quant1(b, inv, -kQmax - 1, kQmax));
+                }
+                c[m] = OUT == kOutInt8 ? ((lo & 0xFFu) | ((hi & 0xFFu) << 8)) : ((lo & 3u) | ((hi & 3u) << 2));
+            }
+            if constexpr (OUT == kOutInt8) {
+                // thread t holds elements 2t + 256m, +1 = bytes 2t + 256m, +1 of the row
+                uint16_t* out16 = reinterpret_cast<uint16_t*>(codes + static_cast<size_t>(row) * kN) + t;
+#pragma unroll
+                for (int m = 0; m < 16; ++m) out16[128 * m] = static_cast<uint16_t>(c[m]);
+            } else {
+                // elements 2t + 256m, +1 are half of byte t/2 + 64m: the low half for even t, the high half for odd t.
+                // The sixteen 4-bit halves travel in two words; the even thread writes bytes m = 0..7, the odd one 8..15.
+                uint32_t w0 = 0u, w1 = 0u;
+#pragma unroll
+                for (int m = 0; m < 8; ++m) w0 |= c[m] << (4 * m), w1 |= c[8 + m] << (4 * m);
+                const bool odd = t & 1;
+                const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, odd ? w0 : w1, 1);
+                const uint32_t mine = odd ? w1 : w0;  // the eight rows m this thread assembles
+                uint8_t* out2 = codes + static_cast<size_t>(row) * (kN / 4) + (t >> 1) + (odd ? 64 * 8 : 0);
+#pragma unroll
+                for (int m = 0; m < 8; ++m) {
+                    const uint32_t a4 = (mine >> (4 * m)) & 0xFu, b4 = (other >> (4 * m)) & 0xFu;
+                    out2[64 * m] = static_cast<uint8_t>(odd ? (b4 | (a4 << 4)) : (a4 | (b4 << 4)));
+                }
+            }
+            continue;
+        }
 
         // codes: thread t holds elements 2t + 256m (+1) = byte t + 128m of the row's packed codes
         const uint32_t e16 = (s16 >> 10) & 31u;
@@ -535,6 +579,16 @@ cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, i
     }
     return y == nullptr ? launch_variant<4, 32, 2, kHadamard, kOutInt4>(plan, tmap, rows, codes, scales, y, ldy, st)
                         : launch_variant<4, 32, 2, kHadamard, kOutBf16>(plan, tmap, rows, codes, scales, y, ldy, st);
+}
+
+// INT2 / INT8 codes (the butterfly only): same kernel, other packing in the epilogue
+cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                                 uint16_t* scales, cudaStream_t st) {
+    CUtensorMap tmap;
+    if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
+    using namespace f4k;
+    return bits == 2 ? launch_variant<4, 32, 2, kButterfly, kOutInt2>(plan, tmap, rows, codes, scales, nullptr, 0, st)
+                     : launch_variant<4, 32, 2, kButterfly, kOutInt8>(plan, tmap, rows, codes, scales, nullptr, 0, st);
 }
 
 // bfq_forward_quant_stats on the tuned path: codes + scales + row moments from k_fwdq4096, then the code histogram from

@@ -535,3 +535,27 @@ def test_host_pipeline_matches_the_resident_call(rows, chunks):
         torch.cuda.synchronize()
         assert torch.equal(c_host, c_ref.cpu()) and torch.equal(s_host.view(torch.int16), s_ref.cpu().view(torch.int16))
     assert p.device_status() == 0
+
+
+@pytest.mark.parametrize("rows", [1, 3, 130, 593, 1001])
+@pytest.mark.parametrize("bits", [2, 8])
+def test_tuned_n4096_int2_and_int8(rows, bits, monkeypatch):
+    theta, x = make(4096, rows, torch.bfloat16, seed=300 + rows)
+    if rows >= 130:  # degenerate rows: zero, tiny (subnormal scale) and huge (saturated scale)
+        xs = x.float()
+        xs[1] = 0.0
+        xs[2] *= 1e-8
+        xs[3] *= 1e30
+        x = xs.to(torch.bfloat16)
+    p = plan_for(4096, theta)
+    y_ref = oracle.forward(to_f64(theta), to_f64(x))
+    codes = Guarded((rows, 4096 * bits // 8), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.forward_quant(x.to(DEV), bits, codes=codes.view, scales=scales.view)
+    assert p.device_status() == 0 and codes.intact() and scales.intact()
+    check_quant(codes.view, scales.view, y_ref, bits, f"tuned n=4096 INT{bits}")
+    monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+    c_g, s_g = p.forward_quant(x.to(DEV), bits)
+    monkeypatch.delenv("BFQ_GENERIC_ONLY")
+    assert (s_g.view(torch.int16).int() - scales.view.view(torch.int16).int()).abs().max().item() <= 1
+    assert (c_g != codes.view).float().mean().item() < 1e-3
