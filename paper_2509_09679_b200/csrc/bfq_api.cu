@@ -333,9 +333,9 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
         e = fwdq4096_launch_bits(plan, x, rows, ldx, bits, codes, scales, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
-    if (hist == nullptr && xt == BFQ_BF16 && bits == 2 && y == nullptr && rows < (int64_t(1) << 31) &&
+    if (hist == nullptr && xt == BFQ_BF16 && y == nullptr && rows < (int64_t(1) << 31) &&
         !env_flag("BFQ_GENERIC_ONLY") && fwdq8192_available(plan)) {
-        e = fwdq8192_launch(plan, x, rows, ldx, codes, scales, static_cast<cudaStream_t>(stream));
+        e = fwdq8192_launch(plan, x, rows, ldx, bits, codes, scales, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     GenericParams p{};

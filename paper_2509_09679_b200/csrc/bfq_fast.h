@@ -23,12 +23,12 @@ cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t ro
 cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                   uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st);
 
-// n = 8192, bf16 rows, INT2: two-CTA clusters, one 4096-point half per CTA
+// n = 8192, bf16 rows, INT2 (INT4 / INT8 through another epilogue): two-CTA clusters, one 4096-point half per CTA
 size_t fwdq8192_image_bytes();
 size_t fwdq8192_prep_bytes();
 bool fwdq8192_available(const bfq_plan* plan);
 cudaError_t fwdq8192_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st);
-cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st);
 
 // n = 4096, bf16 x / g / dx: backward with tensor-memory constants and accumulators

@@ -105,7 +105,8 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
     return (static_cast<uint32_t>(qa) & 3u) | ((static_cast<uint32_t>(qb) & 3u) << 2);
 }
 
-template <int G>
+// BITS = 2 (the tuned workload), 4 or 8: only the epilogue differs.
+template <int G, int BITS>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
            const float* __restrict__ img, uint8_t* __restrict__ codes, uint16_t* __restrict__ scales, int rows,
@@ -275,8 +276,43 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         mbar_wait_cluster_bounded(bar_amax, k & 1, status);
         amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
         float inv;
-        const uint16_t s16 = row_scale(amax, 1, &inv);
+        constexpr int kQmax = (1 << (BITS - 1)) - 1;
+        const uint16_t s16 = row_scale(amax, kQmax, &inv);
         if (rank == 0 && t == 0) scales[row] = s16;
+        if constexpr (BITS != 2) {
+            // A[i] holds elements 2048 rank + 256 i + 2 t (+1) of the row, B[i] the same 4096 further on: with 4 or 8 bits
+            // a register pair is one byte / one 16-bit word of its own.  |v * inv| < qmax + 1/2 for a normal, unsaturated
+            // scale, so v * inv + 1.5 * 2^23 carries the two's complement code in its low mantissa bits.
+            const bool plain = (((s16 >> 10) & 31u) != 0u) && (s16 != 0x7BFFu);
+            const u64 inv2 = pack2(inv, inv);
+            auto code2 = [&](u64 v) -> uint32_t {
+                uint32_t lo, hi;
+                if (plain) {
+                    unpack2u(fma2(v, inv2, pack2(12582912.0f, 12582912.0f)), lo, hi);
+                } else {
+                    float a, b;
+                    unpack2(v, a, b);
+                    lo = static_cast<uint32_t>(static_cast<int>(fminf(fmaxf(rintf(a * inv), float(-kQmax - 1)), float(kQmax))));
+                    hi = static_cast<uint32_t>(static_cast<int>(fminf(fmaxf(rintf(b * inv), float(-kQmax - 1)), float(kQmax))));
+                }
+                constexpr uint32_t kMask = (1u << BITS) - 1u;
+                return (lo & kMask) | ((hi & kMask) << BITS);
+            };
+            const size_t base = static_cast<size_t>(row) * (kN8 * BITS / 8);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t ca = code2(A[i]), cb = code2(B[i]);
+                if constexpr (BITS == 4) {
+                    codes[base + 1024 * rank + 128 * i + t] = static_cast<uint8_t>(ca);
+                    codes[base + 2048 + 1024 * rank + 128 * i + t] = static_cast<uint8_t>(cb);
+                } else {
+                    uint16_t* c16 = reinterpret_cast<uint16_t*>(codes + base);
+                    c16[1024 * rank + 128 * i + t] = static_cast<uint16_t>(ca);
+                    c16[2048 + 1024 * rank + 128 * i + t] = static_cast<uint16_t>(cb);
+                }
+            }
+            continue;
+        }
 
         const uint32_t e16 = (s16 >> 10) & 31u;
         const bool plain = (e16 != 0u) && (s16 != 0x7BFFu);  // normal fp16 scale: |v*inv| <= 1.0005, no clipping
@@ -395,11 +431,12 @@ bool fwdq8192_available(const bfq_plan* plan) {
            encode_tiled() != nullptr;
 }
 
-cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                            uint16_t* scales, cudaStream_t st) {
+template <int BITS>
+static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
+                                        uint16_t* scales, cudaStream_t st) {
     constexpr int G = 4;
     using S = f8k::Smem<G>;
-    auto kern = f8k::k_fwdq8192<G>;
+    auto kern = f8k::k_fwdq8192<G, BITS>;
     static bool attr_set[kMaxDevices] = {false};
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
@@ -427,6 +464,13 @@ cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, i
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192), codes, scales,
                               int(rows), plan->status_word);
+}
+
+cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                            uint16_t* scales, cudaStream_t st) {
+    if (bits == 2) return fwdq8192_launch_bits<2>(plan, x, rows, ldx, codes, scales, st);
+    if (bits == 4) return fwdq8192_launch_bits<4>(plan, x, rows, ldx, codes, scales, st);
+    return fwdq8192_launch_bits<8>(plan, x, rows, ldx, codes, scales, st);
 }
 
 }  // namespace bfq

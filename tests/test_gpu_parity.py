@@ -538,22 +538,22 @@ def test_host_pipeline_matches_the_resident_call(rows, chunks):
 
 
 @pytest.mark.parametrize("rows", [1, 3, 130, 593, 1001])
-@pytest.mark.parametrize("bits", [2, 8])
-def test_tuned_n4096_int2_and_int8(rows, bits, monkeypatch):
-    theta, x = make(4096, rows, torch.bfloat16, seed=300 + rows)
+@pytest.mark.parametrize("n,bits", [(4096, 2), (4096, 8), (8192, 4), (8192, 8)])
+def test_tuned_kernels_other_bit_widths(rows, n, bits, monkeypatch):
+    theta, x = make(n, rows, torch.bfloat16, seed=300 + rows)
     if rows >= 130:  # degenerate rows: zero, tiny (subnormal scale) and huge (saturated scale)
         xs = x.float()
         xs[1] = 0.0
         xs[2] *= 1e-8
         xs[3] *= 1e30
         x = xs.to(torch.bfloat16)
-    p = plan_for(4096, theta)
+    p = plan_for(n, theta)
     y_ref = oracle.forward(to_f64(theta), to_f64(x))
-    codes = Guarded((rows, 4096 * bits // 8), torch.uint8, DEV)
+    codes = Guarded((rows, n * bits // 8), torch.uint8, DEV)
     scales = Guarded((rows,), torch.float16, DEV)
     p.forward_quant(x.to(DEV), bits, codes=codes.view, scales=scales.view)
     assert p.device_status() == 0 and codes.intact() and scales.intact()
-    check_quant(codes.view, scales.view, y_ref, bits, f"tuned n=4096 INT{bits}")
+    check_quant(codes.view, scales.view, y_ref, bits, f"tuned n={n} INT{bits}")
     monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
     c_g, s_g = p.forward_quant(x.to(DEV), bits)
     monkeypatch.delenv("BFQ_GENERIC_ONLY")
