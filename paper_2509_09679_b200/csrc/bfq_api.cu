@@ -291,6 +291,11 @@ int bfq_forward(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64
                                         static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
+    if (xt == BFQ_BF16 && yt == BFQ_BF16 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq8192_available(plan)) {
+        cudaError_t e = fwdq8192_launch_bf16(plan, x, rows, ldx, y, ldy, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     GenericParams p{};
     p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = ldy, p.rows = rows;
     cudaError_t e = launch_generic<kModeForward>(plan, p, static_cast<cudaStream_t>(stream));

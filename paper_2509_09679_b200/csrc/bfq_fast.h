@@ -30,6 +30,8 @@ bool fwdq8192_available(const bfq_plan* plan);
 cudaError_t fwdq8192_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st);
 cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st);
+cudaError_t fwdq8192_launch_bf16(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, void* y, int64_t ldy,
+                                 cudaStream_t st);
 
 // n = 4096, bf16 x / g / dx: backward with tensor-memory constants and accumulators
 size_t bwd4096_image_bytes();

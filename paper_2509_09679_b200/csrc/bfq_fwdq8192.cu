@@ -105,12 +105,14 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
     return (static_cast<uint32_t>(qa) & 3u) | ((static_cast<uint32_t>(qb) & 3u) << 2);
 }
 
-// BITS = 2 (the tuned workload), 4 or 8: only the epilogue differs.
+// BITS = 2 (the tuned workload), 4 or 8: only the epilogue differs.  BITS = 16: the rotated rows themselves in bf16
+// (`codes` then points to them, leading dimension ldy); the absmax hand-shake between the two CTAs is kept, since it is
+// also what tells a CTA that its peer has read the exchange box of the row.
 template <int G, int BITS>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
-           const float* __restrict__ img, uint8_t* __restrict__ codes, uint16_t* __restrict__ scales, int rows,
-           int* __restrict__ status) {
+           const float* __restrict__ img, uint8_t* __restrict__ codes, uint16_t* __restrict__ scales, int64_t ldy,
+           int rows, int* __restrict__ status) {
     using S = Smem<G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -276,10 +278,24 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         mbar_wait_cluster_bounded(bar_amax, k & 1, status);
         amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
         float inv;
-        constexpr int kQmax = (1 << (BITS - 1)) - 1;
+        if constexpr (BITS == 16) {
+            // A[i] holds elements 2048 rank + 256 i + 2 t (+1), B[i] the same 4096 further on: one 32-bit word each
+            uint32_t* yrow = reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(codes) + static_cast<int64_t>(row) * ldy);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float a0, a1, b0, b1;
+                unpack2(A[i], a0, a1);
+                unpack2(B[i], b0, b1);
+                const __nv_bfloat162 va = __floats2bfloat162_rn(a0, a1), vb = __floats2bfloat162_rn(b0, b1);
+                yrow[1024 * rank + 128 * i + t] = *reinterpret_cast<const uint32_t*>(&va);
+                yrow[2048 + 1024 * rank + 128 * i + t] = *reinterpret_cast<const uint32_t*>(&vb);
+            }
+            continue;
+        }
+        constexpr int kQmax = BITS == 16 ? 1 : (1 << (BITS - 1)) - 1;
         const uint16_t s16 = row_scale(amax, kQmax, &inv);
         if (rank == 0 && t == 0) scales[row] = s16;
-        if constexpr (BITS != 2) {
+        if constexpr (BITS != 2 && BITS != 16) {
             // A[i] holds elements 2048 rank + 256 i + 2 t (+1) of the row, B[i] the same 4096 further on: with 4 or 8 bits
             // a register pair is one byte / one 16-bit word of its own.  |v * inv| < qmax + 1/2 for a normal, unsaturated
             // scale, so v * inv + 1.5 * 2^23 carries the two's complement code in its low mantissa bits.
@@ -433,7 +449,7 @@ bool fwdq8192_available(const bfq_plan* plan) {
 
 template <int BITS>
 static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                                        uint16_t* scales, cudaStream_t st) {
+                                        uint16_t* scales, int64_t ldy, cudaStream_t st) {
     constexpr int G = 4;
     using S = f8k::Smem<G>;
     auto kern = f8k::k_fwdq8192<G, BITS>;
@@ -462,15 +478,21 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192), codes, scales,
+    return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192), codes, scales, ldy,
                               int(rows), plan->status_word);
 }
 
 cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st) {
-    if (bits == 2) return fwdq8192_launch_bits<2>(plan, x, rows, ldx, codes, scales, st);
-    if (bits == 4) return fwdq8192_launch_bits<4>(plan, x, rows, ldx, codes, scales, st);
-    return fwdq8192_launch_bits<8>(plan, x, rows, ldx, codes, scales, st);
+    if (bits == 2) return fwdq8192_launch_bits<2>(plan, x, rows, ldx, codes, scales, 0, st);
+    if (bits == 4) return fwdq8192_launch_bits<4>(plan, x, rows, ldx, codes, scales, 0, st);
+    return fwdq8192_launch_bits<8>(plan, x, rows, ldx, codes, scales, 0, st);
+}
+
+// y = Q x in bf16 (the weight-only setting: activations stay 16-bit)
+cudaError_t fwdq8192_launch_bf16(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, void* y, int64_t ldy,
+                                 cudaStream_t st) {
+    return fwdq8192_launch_bits<16>(plan, x, rows, ldx, static_cast<uint8_t*>(y), nullptr, ldy, st);
 }
 
 }  // namespace bfq

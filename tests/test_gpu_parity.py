@@ -559,3 +559,18 @@ def test_tuned_kernels_other_bit_widths(rows, n, bits, monkeypatch):
     monkeypatch.delenv("BFQ_GENERIC_ONLY")
     assert (s_g.view(torch.int16).int() - scales.view.view(torch.int16).int()).abs().max().item() <= 1
     assert (c_g != codes.view).float().mean().item() < 1e-3
+
+
+@pytest.mark.parametrize("rows", [1, 2, 3, 75, 297, 1000])
+def test_tuned_n8192_bf16_rows(rows):
+    """y = Q x in bf16 at n = 8192 (weight-only setting: 16-bit activations) on the cluster kernel, padded leading dimensions."""
+    theta, x = make(8192, rows, torch.bfloat16, seed=500 + rows)
+    p = plan_for(8192, theta)
+    xs = torch.zeros((rows, 8192 + 64), dtype=torch.bfloat16, device=DEV)
+    xs[:, :8192] = x.to(DEV)
+    ybuf = Guarded((rows, 8192 + 128), torch.bfloat16, DEV)
+    y = ybuf.view[:, :8192]
+    p.forward(xs[:, :8192], out=y)
+    assert p.device_status() == 0 and ybuf.intact()
+    assert (ybuf.view[:, 8192:].view(torch.int16) == torch.tensor(0xA5A5, dtype=torch.uint16).view(torch.int16).item()).all()
+    check_rows_close(y, oracle.forward(to_f64(theta), to_f64(x)), absmax_rows(x), "tuned n=8192 bf16 rows")
