@@ -335,7 +335,7 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     }
     if (hist == nullptr && xt == BFQ_BF16 && (bits == 2 || bits == 8) && y == nullptr && rows < (int64_t(1) << 31) &&
         !env_flag("BFQ_GENERIC_ONLY") && fwdq4096_available(plan)) {
-        e = fwdq4096_launch_bits(plan, x, rows, ldx, bits, codes, scales, static_cast<cudaStream_t>(stream));
+        e = fwdq4096_launch_bits(plan, x, rows, ldx, false, bits, codes, scales, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     if (hist == nullptr && xt == BFQ_BF16 && y == nullptr && rows < (int64_t(1) << 31) &&
@@ -409,9 +409,9 @@ int bfq_hadamard_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if (xt == BFQ_BF16 && bits == 4 && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
-        fwdq4096_available(plan)) {
-        e = fwdq4096_launch(plan, x, rows, ldx, true, codes, scales_f16, nullptr, 0, st);
+    if (xt == BFQ_BF16 && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") && fwdq4096_available(plan)) {
+        e = bits == 4 ? fwdq4096_launch(plan, x, rows, ldx, true, codes, scales_f16, nullptr, 0, st)
+                      : fwdq4096_launch_bits(plan, x, rows, ldx, true, bits, codes, scales_f16, st);
     } else {
         GenericParams p{};
         p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = nullptr, p.yt = BFQ_F32, p.ldy = plan->n;

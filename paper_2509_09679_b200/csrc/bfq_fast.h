@@ -17,8 +17,8 @@ cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, i
                             uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 
 // INT2 / INT8 codes from the same kernel (bits = 2 or 8)
-cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
-                                 uint16_t* scales, cudaStream_t st);
+cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, bool hadamard, int bits,
+                                 uint8_t* codes, uint16_t* scales, cudaStream_t st);
 // the same with the statistics of bfq_forward_quant_stats (hist already zeroed on `st`)
 cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                   uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st);

@@ -581,12 +581,16 @@ cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, i
                         : launch_variant<4, 32, 2, kHadamard, kOutBf16>(plan, tmap, rows, codes, scales, y, ldy, st);
 }
 
-// INT2 / INT8 codes (the butterfly only): same kernel, other packing in the epilogue
-cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
-                                 uint16_t* scales, cudaStream_t st) {
+// INT2 / INT8 codes: same kernel, other packing in the epilogue
+cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, bool hadamard, int bits,
+                                 uint8_t* codes, uint16_t* scales, cudaStream_t st) {
     CUtensorMap tmap;
     if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
     using namespace f4k;
+    if (hadamard) {
+        return bits == 2 ? launch_variant<4, 32, 2, kHadamard, kOutInt2>(plan, tmap, rows, codes, scales, nullptr, 0, st)
+                         : launch_variant<4, 32, 2, kHadamard, kOutInt8>(plan, tmap, rows, codes, scales, nullptr, 0, st);
+    }
     return bits == 2 ? launch_variant<4, 32, 2, kButterfly, kOutInt2>(plan, tmap, rows, codes, scales, nullptr, 0, st)
                      : launch_variant<4, 32, 2, kButterfly, kOutInt8>(plan, tmap, rows, codes, scales, nullptr, 0, st);
 }
