@@ -7,7 +7,8 @@
 //     Y = Q1 (X Q2^T):   the butterfly on every run, then the dense factor across the runs.
 //
 // This file holds the Cayley solve and the kernels that work for every (n1 <= 64, n2 <= 1024, n1 n2 <= 16384);
-// the tensor-core kernel for 40 x 128 lives in bfq_comp5120.cu and must agree with these.
+// the tensor-core kernels for 40 x 128 live in bfq_comp5120d.cu (both factors as MMAs) and bfq_comp5120.cu (fp32
+// butterfly + MMA dense factor) and must agree with these.
 #include <cuda_runtime.h>
 
 #include "bfq_fast.h"
