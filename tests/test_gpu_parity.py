@@ -574,3 +574,24 @@ def test_tuned_n8192_bf16_rows(rows):
     assert p.device_status() == 0 and ybuf.intact()
     assert (ybuf.view[:, 8192:].view(torch.int16) == torch.tensor(0xA5A5, dtype=torch.uint16).view(torch.int16).item()).all()
     check_rows_close(y, oracle.forward(to_f64(theta), to_f64(x)), absmax_rows(x), "tuned n=8192 bf16 rows")
+
+
+def test_fold_weights_n4096_int2_on_the_tuned_kernel():
+    """2-bit weights of an n = 4096 layer (the paper's W2 setting at the 7B shape): W Q^T through the tuned kernel's INT2
+    epilogue, and computational invariance of the quantized product against the oracle's own."""
+    n, m = 4096, 300
+    theta = synth.angles(n, "normal", 31)
+    W = synth.rows(m, n, "normal", 32, scale=0.02, dtype=torch.bfloat16)
+    x = synth.rows(24, n, "student_t3", 33, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    th64 = to_f64(theta)
+    codes, scales, _ = p.fold_weights(W.to(DEV), 2)
+    WQt_ref = oracle.forward(th64, to_f64(W))
+    check_quant(codes, scales, WQt_ref, 2, "fold n=4096 INT2")
+    Qx = to_f64(p.forward(x.to(DEV), out_dtype=torch.float32))
+    ref = to_f64(W) @ to_f64(x).T
+    o_codes, o_scales = oracle.quantize(WQt_ref, 2)
+    err_ref = np.linalg.norm(oracle.dequantize(o_codes, o_scales) @ oracle.forward(th64, to_f64(x)).T - ref)
+    deq = oracle.dequantize(oracle.unpack(codes.cpu().numpy(), 2), scales.cpu().view(torch.int16).numpy().view(np.uint16))
+    assert abs(np.linalg.norm(deq @ Qx.T - ref) - err_ref) <= 1e-3 * err_ref
+    assert p.device_status() == 0
