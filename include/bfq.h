@@ -169,7 +169,9 @@ int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int
  * tensor cores: Q2 merged into a dense 128 x 128 block held as two bf16 terms, Q1 in TF32 (10 mantissa bits) applied to
  * the fp32 intermediate read as TF32, fp32 accumulation: |error| <= 2^-9 sum_k |Q1[i][k]| |(Q2 x_k)[j]| there.  With the
  * environment variable BFQ_COMPOSITE_FP32_BUTTERFLY=1 Q2 stays an fp32 butterfly on the CUDA cores and only Q1 uses the
- * tensor cores (TF32, |error| <= 2^-10 of the same sum).  fp32 arithmetic everywhere else.  x and y must not overlap.
+ * tensor cores (TF32, |error| <= 2^-10 of the same sum); in that mode the first call after bfq_set_angles waits on the
+ * host for a copy of the angles (the rotation constants become kernel parameters), so it must not be made during stream
+ * capture.  fp32 arithmetic everywhere else.  x and y must not overlap.
  */
 int bfq_cayley(bfq_plan* plan, const float* params, int n1, float* q1, void* stream);
 int bfq_composite_forward(bfq_plan* plan, const float* q1, int n1, const void* x, bfq_dtype xt, int64_t rows,
