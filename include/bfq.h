@@ -165,7 +165,7 @@ int bfq_fold_weights(bfq_plan* plan, const void* W, bfq_dtype wt, int64_t m, int
  * bfq_composite_forward / _quant: x: [rows][ldx] of xt with ldx >= d; y: [rows][ldy]; codes: [rows][d*bits/8] and one
  * fp16 scale per row over all d elements (the quantizer of bfq_forward_quant).  q1 is read as given: any n1 x n1
  * matrix works, the caller keeps it orthogonal.  Needs 16 <= n2 <= 1024 and d <= BFQ_COMPOSITE_MAX_D, else
- * BFQ_ERR_UNSUPPORTED_N.  For n1 = 40, n2 = 128 and bf16 rows (INT4 codes and / or bf16 rows out) both factors run on the
+ * BFQ_ERR_UNSUPPORTED_N.  For n1 = 40, n2 = 128 and bf16 rows (INT4 / INT8 codes or bf16 rows out) both factors run on the
  * tensor cores: Q2 merged into a dense 128 x 128 block held as two bf16 terms, Q1 in TF32 (10 mantissa bits) applied to
  * the fp32 intermediate read as TF32, fp32 accumulation: |error| <= 2^-9 sum_k |Q1[i][k]| |(Q2 x_k)[j]| there.  With the
  * environment variable BFQ_COMPOSITE_FP32_BUTTERFLY=1 Q2 stays an fp32 butterfly on the CUDA cores and only Q1 uses the

@@ -513,15 +513,16 @@ static int composite_impl(bfq_plan* plan, const float* q1, int n1, const void* x
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
     cudaError_t e;
-    if (n1 == 40 && xt == BFQ_BF16 && rows < (int64_t(1) << 31) && (codes == nullptr || bits == 4) &&
-        (y == nullptr || yt == BFQ_BF16) && !env_flag("BFQ_GENERIC_ONLY")) {
-        // default: both factors on the tensor cores; BFQ_COMPOSITE_FP32_BUTTERFLY=1 keeps Q2 as an fp32 butterfly on
-        // the CUDA cores (only the dense factor on the tensor cores)
-        if ((inverse || !env_flag("BFQ_COMPOSITE_FP32_BUTTERFLY")) && comp5120d_available(plan)) {
-            e = comp5120d_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, inverse, static_cast<cudaStream_t>(stream));
+    if (n1 == 40 && xt == BFQ_BF16 && rows < (int64_t(1) << 31) && (y == nullptr || yt == BFQ_BF16) &&
+        !env_flag("BFQ_GENERIC_ONLY")) {
+        // default: both factors on the tensor cores (INT4 or INT8 codes, or bf16 rows); BFQ_COMPOSITE_FP32_BUTTERFLY=1
+        // keeps Q2 as an fp32 butterfly on the CUDA cores (only the dense factor on the tensor cores; INT4 or bf16 rows)
+        const bool dense_ok = codes == nullptr || bits == 4 || bits == 8, bfly_ok = codes == nullptr || bits == 4;
+        if (dense_ok && (inverse || !bfly_ok || !env_flag("BFQ_COMPOSITE_FP32_BUTTERFLY")) && comp5120d_available(plan)) {
+            e = comp5120d_launch(plan, q1, x, rows, ldx, bits, codes, scales, y, ldy, inverse, static_cast<cudaStream_t>(stream));
             return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
         }
-        if (!inverse && comp5120_available(plan)) {
+        if (!inverse && bfly_ok && comp5120_available(plan)) {
             e = comp5120_launch(plan, q1, x, rows, ldx, codes, scales, y, ldy, static_cast<cudaStream_t>(stream));
             return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
         }

@@ -76,6 +76,7 @@ struct Params {
     int64_t rows;
     int* status;
     int transpose_q1;     // 1: apply Q1^T (the inverse transform; q2img then holds Q2^T)
+    int bits;             // 4 or 8 (codes != null)
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -290,9 +291,37 @@ __device__ __forceinline__ void epilogue_role(const Params& P, uint8_t* sm, uint
             const float4 q4 = *reinterpret_cast<const float4*>(amax_slots + (g & 1) * 16 + tau * 4);
             const float amax = fmaxf(fmaxf(q4.x, q4.y), fmaxf(q4.z, q4.w));
             float inv;
-            const uint16_t sb = row_scale(amax, 7, &inv);
+            const uint16_t sb = row_scale(amax, P.bits == 8 ? 127 : 7, &inv);
             const bool saturated = sb == 0x7BFFu || sb < 0x0400u || !(amax < 3.0e38f);
             if (qd == 0 && lane == 0 && valid) P.scales[token] = sb;
+            if (P.bits == 8) {
+                // one byte per element: |y / s| < 127.5 for a normal scale, y * inv + 1.5 * 2^23 has the two's complement
+                // code in its low byte.  A thread packs four runs into a word; 4 x 4 byte blocks are transposed between
+                // four lanes (two byte-permute exchanges) so that lane a stores run 4 blk + a, positions j0 .. j0 + 3.
+                const int a4 = lane & 3;
+                const uint32_t sel1 = (a4 & 1) ? 0x3715u : 0x6240u, sel2 = (a4 & 2) ? 0x3276u : 0x5410u;
+                uint32_t wb[kN1 / 4];
+#pragma unroll
+                for (int blk = 0; blk < kN1 / 4; ++blk) {
+                    uint32_t c[4];
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const float y = __uint_as_float(v[4 * blk + b]);
+                        c[b] = saturated ? static_cast<uint32_t>(quant1(y, inv, -128, 127)) : __float_as_uint(fmaf(y, inv, 12582912.0f));
+                    }
+                    wb[blk] = __byte_perm(__byte_perm(c[0], c[1], 0x0040u), __byte_perm(c[2], c[3], 0x0040u), 0x5410u);
+                }
+#pragma unroll
+                for (int blk = 0; blk < kN1 / 4; ++blk) wb[blk] = __byte_perm(wb[blk], __shfl_xor_sync(0xffffffffu, wb[blk], 1), sel1);
+#pragma unroll
+                for (int blk = 0; blk < kN1 / 4; ++blk) wb[blk] = __byte_perm(wb[blk], __shfl_xor_sync(0xffffffffu, wb[blk], 2), sel2);
+                if (valid) {
+#pragma unroll
+                    for (int blk = 0; blk < kN1 / 4; ++blk)
+                        *reinterpret_cast<uint32_t*>(P.codes + token * kD + (4 * blk + a4) * kN2 + (j & ~3)) = wb[blk];
+                }
+                continue;
+            }
             uint32_t word[5];
             if (!saturated) {
                 // |y / s| < 7.5 for a normal, unsaturated fp16 scale: y * inv + (1.5 * 2^23 + 8) has r + 8 in [1, 15] in
@@ -429,10 +458,11 @@ cudaError_t comp5120d_set_angles(const bfq_plan* plan, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                             uint16_t* scales, void* y_bf16, int64_t ldy, bool inverse, cudaStream_t st) {
+cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, int bits,
+                             uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, bool inverse, cudaStream_t st) {
     using namespace c5d;
     Params P{};
+    P.bits = bits;
     P.q2img = static_cast<const uint4*>(plan->dense128) + (inverse ? kQ2Bytes / 16 : 0);
     P.transpose_q1 = inverse ? 1 : 0;
     P.q1 = q1, P.codes = codes, P.scales = scales, P.y = static_cast<__nv_bfloat16*>(y_bf16), P.ldy = ldy;

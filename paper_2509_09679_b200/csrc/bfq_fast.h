@@ -64,7 +64,7 @@ cudaError_t comp5120_launch(bfq_plan* plan, const float* q1, const void* x, int6
 size_t comp5120d_image_bytes();
 bool comp5120d_available(const bfq_plan* plan);
 cudaError_t comp5120d_set_angles(const bfq_plan* plan, cudaStream_t st);
-cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                             uint16_t* scales, void* y_bf16, int64_t ldy, bool inverse, cudaStream_t st);
+cudaError_t comp5120d_launch(bfq_plan* plan, const float* q1, const void* x, int64_t rows, int64_t ldx, int bits,
+                             uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, bool inverse, cudaStream_t st);
 
 }  // namespace bfq
