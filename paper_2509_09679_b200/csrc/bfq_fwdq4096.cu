@@ -429,27 +429,23 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
 
 // ---- table preparation -----------------------------------------------------------------------------------
 // Step 1 (one thread per angle): the generic (cos, sin) table entry, the reduced-angle lifting
-// constants and whether the reduction negates the pair.  With r = theta mod 2 pi in [-pi, pi], the pair
-// is negated iff |r| > pi/2, and phi = r -+ pi in that case; tan(phi/2) and sin(phi) are odd in phi,
+// constants and whether the reduction negates the pair.  The pair is negated iff cos(theta) < 0, and
+// phi = theta -+ pi in that case; tan(phi/2) and sin(phi) are odd in phi,
 // so the constants for the mirrored rotation G(-theta) are the negatives of the stored ones.
 __global__ void __launch_bounds__(256) k_prep_angles4096(const float* __restrict__ theta, float2* __restrict__ tw,
                                                           float4* __restrict__ prep, uint8_t* __restrict__ flip) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= 12 * (kN / 2)) return;
-    const double kPi = 3.14159265358979323846;
     const double th = static_cast<double>(theta[k]);
     double sn, c;
     sincos(th, &sn, &c);
     tw[k] = make_float2(static_cast<float>(c), static_cast<float>(sn));
-    double te = remainder(th, 2.0 * kPi);
-    bool f = false;
-    if (te > 0.5 * kPi) {
-        te -= kPi, f = true;
-    } else if (te < -0.5 * kPi) {
-        te += kPi, f = true;
-    }
+    // phi = theta -+ pi when cos(theta) < 0 (|phi| <= pi/2 then): sin(phi) = -sin(theta), cos(phi) = -cos(theta), and
+    // tan(phi/2) = sin(phi) / (1 + cos(phi)) with a denominator >= 1: no second reduction, no tan
+    const bool f = c < 0.0;
+    const double sp = f ? -sn : sn, cp = f ? -c : c;
     flip[k] = f ? 1 : 0;
-    prep[k] = make_float4(static_cast<float>(-tan(0.5 * te)), static_cast<float>(sin(te)), static_cast<float>(c),
+    prep[k] = make_float4(static_cast<float>(-sp / (1.0 + cp)), static_cast<float>(sp), static_cast<float>(c),
                           static_cast<float>(sn));
 }
 

@@ -88,10 +88,13 @@ __device__ __forceinline__ void stage_lift(u64 (&P)[16], const uint32_t (&T)[CW]
 // sign carried by element i when it enters stage s: the product of the negations (flip = 1) of the pairs
 // it belonged to in stages 0..s-1
 __device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int i, int s) {
+    // all (at most twelve) flag loads are issued together: a loop with a run-time trip count would wait for each in turn
     int f = 0;
-    for (int sp = 0; sp < s; ++sp) {
+#pragma unroll
+    for (int sp = 0; sp < 12; ++sp) {
         const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
-        f ^= flip[sp * (kN / 2) + j];
+        const int v = sp < s ? flip[sp * (kN / 2) + j] : 0;
+        f ^= v;
     }
     return f ? -1 : 1;
 }
