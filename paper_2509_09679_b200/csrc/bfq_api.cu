@@ -228,8 +228,9 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
             if (plan->comp5120 == nullptr) e = cudaErrorMemoryAllocation;
         }
     }
-    if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, 4 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, 4 * sizeof(int));
+    if (e == cudaSuccess) plan->form_flag = plan->status_word + 1;
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         release_plan(plan);

@@ -714,7 +714,7 @@ bool bwd4096_available(const bfq_plan* plan) {
 cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st) {
     const int count = 12 * (f4k::kN / 2);
     const float4* prep = reinterpret_cast<const float4*>(plan->prep4096);
-    const uint8_t* flip = reinterpret_cast<const uint8_t*>(prep + count);
+    const uint8_t* flip = reinterpret_cast<const uint8_t*>(reinterpret_cast<const double2*>(prep + count) + count);
     b4k::k_build_image_bwd4096<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img_b4096, plan->dsign4096);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -15,18 +15,22 @@
 //    registers and a warp-level sync only.  The second crosses warps: scalar stores, 64-bit loads,
 //    one named barrier.  The buffer layouts are additive in the index bits (padded, not
 //    XOR-swizzled) so that every access is base + immediate and bank-conflict free.
-//  * Rotations use the three-shear (lifting) form  a += -t*b; b += s*a; a += -t*b  with
-//    t = tan(phi/2), s = sin(phi): three FMAs and two constants per pair.  Angles are reduced to
-//    |phi| <= pi/2 (so |t| <= 1); the sign flips that the reduction introduces are tracked per
-//    element when the tables are built and are absorbed by later stages' angles; the last stage
-//    uses a general 2x2 form whose constants restore the true signs.  All of this is table
-//    preparation: the kernel sees only constants.
+//  * Rotations use the scaled form  lo' = lo + k1*hi, hi' = hi + k2*lo  (two independent FMAs and two constants
+//    per pair): every element carries an implicit factor d, the product of the cosines of the rotations it has
+//    been through, which the table build folds into k1, k2 and into the general 2x2 of the last stage, so the
+//    kernel sees only constants.  The form is singular where a cosine vanishes; when some element's factor leaves
+//    [2^-64, 1] the table build raises a flag and the kernel takes the three-shear (lifting) form instead:
+//    a += -t*b; b += s*a; a += -t*b  with t = tan(phi/2), s = sin(phi), three FMAs per pair, angles reduced to
+//    |phi| <= pi/2 (so |t| <= 1), the sign flips of the reduction tracked per element at table-build time.  Both
+//    images have the same layout.
 //  * The constants (416 words per thread role, 53248 in all) live in tensor memory, one strip per
 //    lane; every group reads the same strips.  They are streamed into registers with tcgen05.ld,
 //    one chunk ahead of use.
 //  * Rows arrive by TMA (128-byte swizzled tiles, two-deep ring per group, mbarrier completion).
 //    The per-row absmax is a warp reduction plus one step across the group's four warps; INT4
 //    codes are produced with the magic-number rounding trick, one byte per packed register.
+#include <type_traits>
+
 #include "bfq_fast.h"
 #include "bfq_generic.cuh"
 #include "bfq_n4096.cuh"
@@ -78,12 +82,18 @@ struct Chunks {
     static constexpr int kAfterPhase2 = 8 * kPerStage - 1;  // last chunk of stage 7
 };
 
-template <int C, int CW>
+enum : int { kFormScaled = 0, kFormShear = 1 };  // FORM: how stages 0..10 rotate (the image must match)
+
+template <int FORM, int C, int CW>
 __device__ __forceinline__ void run_chunk(u64 (&P)[16], const uint32_t (&T)[CW]) {
     using CH = Chunks<CW>;
     constexpr int NU = CW / 4;
     if constexpr (C < CH::kLift) {
-        stage_lift<(C / CH::kPerStage) & 3, (C % CH::kPerStage) * NU, NU, CW>(P, T);
+        if constexpr (FORM == kFormScaled) {
+            stage_scaled<(C / CH::kPerStage) & 3, (C % CH::kPerStage) * NU, NU, CW>(P, T);
+        } else {
+            stage_lift<(C / CH::kPerStage) & 3, (C % CH::kPerStage) * NU, NU, CW>(P, T);
+        }
     } else {
         stage_general<(C - CH::kLift) * (CW / 8), CW / 8, CW>(P, T);
     }
@@ -115,19 +125,19 @@ __device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
 // Chunk C is in Tcur (load already issued); the load of chunk C+1 is issued right after the wait so
 // that exactly one tensor-memory load is in flight while chunk C is being used.  `issue_next` runs
 // once per row, after the second regrouping's barrier (all reads of the input slot are done by then).
-template <int C, int CW, int XB, class F>
+template <int FORM, int C, int CW, int XB, class F>
 __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[CW], uint32_t (&Tnext)[CW], uint32_t tbase,
                                            const ExAddr& ex, F&& issue_next) {
     using CH = Chunks<CW>;
     tmem_wait_ld(Tcur);
     if constexpr (C + 1 < CH::kCount) tmem_ld(tbase + CW * (C + 1), Tnext);
-    run_chunk<C, CW>(P, Tcur);
+    run_chunk<FORM, C, CW>(P, Tcur);
     if constexpr (C == CH::kAfterPhase1) regroup1(P, ex);
     if constexpr (C == CH::kAfterPhase2) {
         regroup2<XB>(P, ex);
         issue_next();
     }
-    if constexpr (C + 1 < CH::kCount) run_chunks<C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, issue_next);
+    if constexpr (C + 1 < CH::kCount) run_chunks<FORM, C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, issue_next);
 }
 
 // Walsh-Hadamard stages 4*PH .. 4*PH+3 of a phase: (a, b) -> (a + b, a - b), no constants; the 1/sqrt(n) is
@@ -161,7 +171,8 @@ enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutIn
 // INT2 / INT8 codes + scales.
 template <int G, int CW, int XB, int TRANSFORM, int OUT>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
-k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, uint8_t* __restrict__ codes,
+k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, const int* __restrict__ form,
+           uint8_t* __restrict__ codes,
            uint16_t* __restrict__ scales, __nv_bfloat16* __restrict__ yout, int64_t ldy, int rows,
            int* __restrict__ status) {
     using S = Smem<G, XB>;
@@ -172,6 +183,12 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = warp & 3, g = warp >> 2;
     const int t = q * 32 + lane;  // role within the group: 0..127
+    // which of the two images (and stage forms) the table build selected for the current angles
+    bool shear = false;
+    if constexpr (kTmem) {
+        shear = __ldg(form) != 0;
+        if (shear) img += 128 * kCols;
+    }
 
     if constexpr (kTmem) {
         if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
@@ -238,6 +255,9 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const uint32_t amax_base = sbase + S::kAmaxOff + g * 32;
     uint8_t* const out_t = codes + t;
 
+    // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
+    auto row_loop = [&](auto form_tag) {
+    constexpr int FORM = decltype(form_tag)::value;
     u64 P[16];
     uint32_t T0[CW], T1[CW];
 
@@ -273,7 +293,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             }
         };
         if constexpr (kTmem) {
-            run_chunks<0, CW, XB>(P, T0, T1, tlane, ex, issue_next);
+            run_chunks<FORM, 0, CW, XB>(P, T0, T1, tlane, ex, issue_next);
         } else {
             run_hadamard<XB>(P, ex, issue_next);
         }
@@ -419,6 +439,12 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             }
         }
     }
+    };
+    if (!shear) {
+        row_loop(std::integral_constant<int, kFormScaled>());
+    } else if constexpr (kTmem) {
+        row_loop(std::integral_constant<int, kFormShear>());
+    }
 
     if constexpr (kTmem) {
         tmem_fence_before();
@@ -428,18 +454,21 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
 }
 
 // ---- table preparation -----------------------------------------------------------------------------------
-// Step 1 (one thread per angle): the generic (cos, sin) table entry, the reduced-angle lifting
-// constants and whether the reduction negates the pair.  The pair is negated iff cos(theta) < 0, and
-// phi = theta -+ pi in that case; tan(phi/2) and sin(phi) are odd in phi,
-// so the constants for the mirrored rotation G(-theta) are the negatives of the stored ones.
+// Step 1 (one thread per angle): the generic (cos, sin) table entry, cos and sin in double for step 2, the
+// reduced-angle lifting constants and whether the reduction negates the pair.  The pair is negated iff
+// cos(theta) < 0, and phi = theta -+ pi in that case; tan(phi/2) and sin(phi) are odd in phi, so the constants for
+// the mirrored rotation G(-theta) are the negatives of the stored ones.
 __global__ void __launch_bounds__(256) k_prep_angles4096(const float* __restrict__ theta, float2* __restrict__ tw,
-                                                          float4* __restrict__ prep, uint8_t* __restrict__ flip) {
+                                                          float4* __restrict__ prep, uint8_t* __restrict__ flip,
+                                                          double2* __restrict__ cs, int* __restrict__ form) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k == 0) *form = kFormScaled;  // step 2 raises it when the scaled form is out of range
     if (k >= 12 * (kN / 2)) return;
     const double th = static_cast<double>(theta[k]);
     double sn, c;
     sincos(th, &sn, &c);
     tw[k] = make_float2(static_cast<float>(c), static_cast<float>(sn));
+    cs[k] = make_double2(c, sn);
     // phi = theta -+ pi when cos(theta) < 0 (|phi| <= pi/2 then): sin(phi) = -sin(theta), cos(phi) = -cos(theta), and
     // tan(phi/2) = sin(phi) / (1 + cos(phi)) with a denominator >= 1: no second reduction, no tan
     const bool f = c < 0.0;
@@ -449,16 +478,33 @@ __global__ void __launch_bounds__(256) k_prep_angles4096(const float* __restrict
                           static_cast<float>(sn));
 }
 
-// Step 2 (one thread per angle): place the constants of pair (s, j) in the tensor-memory image
-// img[role][column], with the role / register / half of the pair's low element in its phase.
-__global__ void __launch_bounds__(256) k_build_image4096(const float4* __restrict__ prep,
-                                                          const uint8_t* __restrict__ flip, float* __restrict__ img) {
+// factor carried by element i when it enters stage s: the product of the cosines of the pairs it belonged to in
+// stages 0..s-1 (its sign is the tracked sign of the three-shear form)
+__device__ __forceinline__ double factor_before(const double2* __restrict__ cs, int i, int s) {
+    double c[11];
+#pragma unroll
+    for (int sp = 0; sp < 11; ++sp) {  // all loads issued together
+        const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
+        c[sp] = sp < s ? cs[sp * (kN / 2) + j].x : 1.0;
+    }
+    double d = 1.0;
+#pragma unroll
+    for (int sp = 0; sp < 11; ++sp) d *= c[sp];
+    return d;
+}
+
+// Step 2 (one thread per angle): place the constants of pair (s, j) in both tensor-memory images
+// img[form][role][column], with the role / register / half of the pair's low element in its phase, and raise *form
+// when an element's factor leaves the range the scaled form is used in.
+__global__ void __launch_bounds__(256) k_build_image4096(const float4* __restrict__ prep, const double2* __restrict__ cs,
+                                                          float* __restrict__ img, int* __restrict__ form) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= 12 * (kN / 2)) return;
     const int s = k / (kN / 2), j = k % (kN / 2);
     const int lo = ((j >> s) << (s + 1)) | (j & ((1 << s) - 1));
     const int hi = lo + (1 << s);
-    const int sa = sign_before(flip, lo, s), sb = sign_before(flip, hi, s);
+    const double da = factor_before(cs, lo, s), db = factor_before(cs, hi, s);
+    const int sa = da < 0.0 ? -1 : 1, sb = db < 0.0 ? -1 : 1;
     const int kk = s & 3;
     int r, m, h;
     if (s < 4) {
@@ -470,17 +516,29 @@ __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restric
     }
     const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
     const float4 p = prep[k];
-    float* strip = img + r * kCols;
+    const double2 own = cs[k];
+    float* scaled = img + kFormScaled * (128 * kCols) + r * kCols;
+    float* shear = img + kFormShear * (128 * kCols) + r * kCols;
     if (s < 11) {
         const float sg = (sa == sb) ? 1.f : -1.f;
-        strip[32 * s + 4 * u + h] = sg * p.x;
-        strip[32 * s + 4 * u + h + 2] = sg * p.y;
+        shear[32 * s + 4 * u + h] = sg * p.x;
+        shear[32 * s + 4 * u + h + 2] = sg * p.y;
+        // k1 = -tan(theta) db/da, k2 = tan(theta) da/db, with one division
+        const double w = own.y / (own.x * da * db);
+        scaled[32 * s + 4 * u + h] = static_cast<float>(-w * db * db);
+        scaled[32 * s + 4 * u + h + 2] = static_cast<float>(w * da * da);
+        const double lim = 5.421010862427522e-20;  // 2^-64
+        if (!(fabs(own.x * da) >= lim && fabs(own.x * db) >= lim)) *form = kFormShear;
     } else {
         const int col = 352 + 8 * u + h;
-        strip[col + 0] = p.z * sa;
-        strip[col + 2] = -p.w * sb;
-        strip[col + 4] = p.w * sa;
-        strip[col + 6] = p.z * sb;
+        shear[col + 0] = p.z * sa;
+        shear[col + 2] = -p.w * sb;
+        shear[col + 4] = p.w * sa;
+        shear[col + 6] = p.z * sb;
+        scaled[col + 0] = static_cast<float>(own.x * da);
+        scaled[col + 2] = static_cast<float>(-own.y * db);
+        scaled[col + 4] = static_cast<float>(own.y * da);
+        scaled[col + 6] = static_cast<float>(own.x * db);
     }
 }
 
@@ -522,18 +580,21 @@ __global__ void __launch_bounds__(kHistThreads) k_hist_int4(const uint4* __restr
 }  // namespace f4k
 
 // ---- host side ---------------------------------------------------------------------------------------------
-size_t fwdq4096_image_bytes() { return size_t(128) * f4k::kCols * sizeof(float); }
-size_t fwdq4096_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1); }
+// two images: scaled form, three-shear form
+size_t fwdq4096_image_bytes() { return size_t(2) * 128 * f4k::kCols * sizeof(float); }
+// per angle: float4 (three-shear constants, cos, sin), double2 (cos, sin), one negation flag
+size_t fwdq4096_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + sizeof(double2) + 1); }
 
 // Builds the generic (cos, sin) table and the tensor-memory image from the angles (two launches).
 cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st) {
     const int count = 12 * (f4k::kN / 2);
     float4* prep = reinterpret_cast<float4*>(plan->prep4096);
-    uint8_t* flip = reinterpret_cast<uint8_t*>(prep + count);
-    f4k::k_prep_angles4096<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, flip);
+    double2* cs = reinterpret_cast<double2*>(prep + count);
+    uint8_t* flip = reinterpret_cast<uint8_t*>(cs + count);
+    f4k::k_prep_angles4096<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, flip, cs, plan->form_flag);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    f4k::k_build_image4096<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img4096);
+    f4k::k_build_image4096<<<(count + 255) / 256, 256, 0, st>>>(prep, cs, plan->img4096, plan->form_flag);
     return cudaGetLastError();
 }
 
@@ -554,7 +615,7 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
     }
     const int64_t want = (rows + G - 1) / G;
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
-    kern<<<grid, G * f4k::kGroupThreads, S::kBytes, st>>>(tmap, plan->img4096, codes, scales,
+    kern<<<grid, G * f4k::kGroupThreads, S::kBytes, st>>>(tmap, plan->img4096, plan->form_flag, codes, scales,
                                                           static_cast<__nv_bfloat16*>(y), ldy, int(rows),
                                                           plan->status_word);
     return cudaGetLastError();

@@ -85,6 +85,23 @@ __device__ __forceinline__ void stage_lift(u64 (&P)[16], const uint32_t (&T)[CW]
     }
 }
 
+// The same stage as two independent FMAs per pair on implicitly scaled values: with true value = d * stored value and
+// per-element factors d fixed by the angles alone (d' = cos(theta) * d for both elements of a pair),
+//     lo' = lo + k1 * hi,   hi' = hi + k2 * lo      (both from the old values)
+// is the rotation.  T holds (k1, k1', k2, k2') for NU consecutive pairs starting at pair U0; the factors are folded into
+// k1, k2 when the tables are built and into the constants of the last stage, which is a general 2x2.
+template <int K, int U0, int NU, int CW>
+__device__ __forceinline__ void stage_scaled(u64 (&P)[16], const uint32_t (&T)[CW]) {
+    static_assert(4 * NU <= CW, "chunk too small");
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int u = U0 + i, m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        const u64 a = P[m_lo], b = P[m_hi];
+        P[m_lo] = fma2(pack2u(T[4 * i], T[4 * i + 1]), b, a);
+        P[m_hi] = fma2(pack2u(T[4 * i + 2], T[4 * i + 3]), a, b);
+    }
+}
+
 // sign carried by element i when it enters stage s: the product of the negations (flip = 1) of the pairs
 // it belonged to in stages 0..s-1
 __device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int i, int s) {

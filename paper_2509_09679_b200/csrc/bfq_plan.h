@@ -34,6 +34,7 @@ struct bfq_plan {
     float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
     int64_t partial_slots = 0;
     int* status_word = nullptr;  // device: non-zero when a bounded wait gave up
+    int* form_flag = nullptr;    // device (status_word + 1): stage form the table build selected for the tuned kernels
     int last_cuda_error = 0;
     int last_backward_partials = 0;
 };
