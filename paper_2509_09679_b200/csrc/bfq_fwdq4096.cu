@@ -122,22 +122,44 @@ __device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
     for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r2 + ex2_rd_local(m));
 }
 
+// The FP32 pipes and the shared-memory pipe are both heavily used; left alone, the row groups drift into step (all
+// rotating, then all regrouping) and the pipes take turns idling.  The groups therefore pass tokens around: a group
+// rotates (one phase of four stages) only while it holds a token and hands it on when it starts a regrouping or its
+// epilogue, so that some groups' rotations overlap the others' memory phases.  A token is a named barrier per group:
+// 128 arrivals from the previous holder + the 128 waiting threads.
+struct Turn {
+    int wait_id, pass_id;  // named barriers: this group's, the next group's in the ring
+    bool on;
+    __device__ __forceinline__ void acquire() const {
+        if (on) bar_sync(wait_id, 2 * kGroupThreads);
+    }
+    __device__ __forceinline__ void pass() const {
+        if (on) bar_arrive(pass_id, 2 * kGroupThreads);
+    }
+};
+
 // Chunk C is in Tcur (load already issued); the load of chunk C+1 is issued right after the wait so
 // that exactly one tensor-memory load is in flight while chunk C is being used.  `issue_next` runs
 // once per row, after the second regrouping's barrier (all reads of the input slot are done by then).
 template <int FORM, int C, int CW, int XB, class F>
 __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[CW], uint32_t (&Tnext)[CW], uint32_t tbase,
-                                           const ExAddr& ex, F&& issue_next) {
+                                           const ExAddr& ex, const Turn& turn, F&& issue_next) {
     using CH = Chunks<CW>;
+    if constexpr (C == 0 || C == CH::kAfterPhase1 + 1 || C == CH::kAfterPhase2 + 1) turn.acquire();
     tmem_wait_ld(Tcur);
     if constexpr (C + 1 < CH::kCount) tmem_ld(tbase + CW * (C + 1), Tnext);
     run_chunk<FORM, C, CW>(P, Tcur);
-    if constexpr (C == CH::kAfterPhase1) regroup1(P, ex);
+    if constexpr (C == CH::kAfterPhase1) {
+        turn.pass();
+        regroup1(P, ex);
+    }
     if constexpr (C == CH::kAfterPhase2) {
+        turn.pass();
         regroup2<XB>(P, ex);
         issue_next();
     }
-    if constexpr (C + 1 < CH::kCount) run_chunks<FORM, C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, issue_next);
+    if constexpr (C + 1 == CH::kCount) turn.pass();
+    if constexpr (C + 1 < CH::kCount) run_chunks<FORM, C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, turn, issue_next);
 }
 
 // Walsh-Hadamard stages 4*PH .. 4*PH+3 of a phase: (a, b) -> (a + b, a - b), no constants; the 1/sqrt(n) is
@@ -169,7 +191,10 @@ enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutIn
 // no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy), or
 // codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]), or
 // INT2 / INT8 codes + scales.
-template <int G, int CW, int XB, int TRANSFORM, int OUT>
+constexpr int kTurnBar0 = 8;  // named barriers 8 .. 8 + G - 1 carry the tokens (1 .. G are the groups' own)
+
+// STEP: group g passes its token to group (g + STEP) % G, so gcd(STEP, G) groups rotate at a time (0: no tokens).
+template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, const int* __restrict__ form,
            uint8_t* __restrict__ codes,
@@ -183,11 +208,26 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = warp & 3, g = warp >> 2;
     const int t = q * 32 + lane;  // role within the group: 0..127
-    // which of the two images (and stage forms) the table build selected for the current angles
+    // Constants of this thread's role, fetched before anything else so that the L2 latency overlaps the set-up: the
+    // image is stored [column quad][role][4], a warp's load is 512 contiguous bytes, and all of a thread's loads
+    // are in flight together.  The G warps of a lane quarter share its 26 blocks of 16 columns.  The scaled-form
+    // image is fetched on the assumption that the table build selected it; the flag is checked below.
+    constexpr int kFillBlocks = (kCols / 16 + G - 1) / G;
+    float4 fill[kTmem ? kFillBlocks : 1][4];
+    auto fetch_image = [&](const float4* __restrict__ base) {
+#pragma unroll
+        for (int j = 0; j < kFillBlocks; ++j) {
+            const int b = g + j * G;
+            if (b < kCols / 16) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) fill[j][i] = __ldg(base + (4 * b + i) * 128 + t);
+            }
+        }
+    };
     bool shear = false;
     if constexpr (kTmem) {
+        fetch_image(reinterpret_cast<const float4*>(img));
         shear = __ldg(form) != 0;
-        if (shear) img += 128 * kCols;
     }
 
     if constexpr (kTmem) {
@@ -207,28 +247,40 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const int first = blockIdx.x * G + g;
     const int stride = gridDim.x * G;
     const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
+    // rows of group 0, the largest count of the CTA: every group takes that many turns with a token
+    const int turns = static_cast<int>(blockIdx.x) * G < rows ? (rows - blockIdx.x * G + stride - 1) / stride : 0;
     const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
     const uint32_t bar_base = sbase + S::kBarOff + 8 * g * kInSlots;
+    static_assert(STEP >= 0 && (STEP == 0 || G % STEP == 0), "the rings must have equal length");
+    constexpr int kRings = STEP == 0 ? 1 : STEP;  // gcd(STEP, G)
+    Turn turn;
+    turn.on = kTmem && STEP > 0;
+    turn.wait_id = kTurnBar0 + g;
+    turn.pass_id = kTurnBar0 + (g + STEP) % G;
+    const bool seeds_ring = (g + STEP) % G < kRings;  // this group's successor starts with the token
 
-    // first rows of this group: issued before the table fill so that HBM latency overlaps it
+    // first rows of this group
     if (t == 0) {
         for (int k = 0; k < kInSlots && k < count; ++k) {
             mbar_expect_tx(bar_base + 8 * k, kRowBytes);
             tma_load_3d(in_base + k * kRowBytes, &tmap, 0, 0, first + k * stride, bar_base + 8 * k);
         }
     }
-    // fill tensor memory: the G warps of a lane quarter share its 26 blocks of 16 columns
+    // fill tensor memory
     if constexpr (kTmem) {
-        const float4* src = reinterpret_cast<const float4*>(img + (q * 32 + lane) * kCols);
-        for (int c = 16 * g; c < kCols; c += 16 * G) {
-            uint32_t v[16];
+        if (shear) fetch_image(reinterpret_cast<const float4*>(img) + (kCols / 4) * 128);  // the other image after all
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 f = __ldg(src + (c >> 2) + i);
-                v[4 * i + 0] = __float_as_uint(f.x), v[4 * i + 1] = __float_as_uint(f.y);
-                v[4 * i + 2] = __float_as_uint(f.z), v[4 * i + 3] = __float_as_uint(f.w);
+        for (int j = 0; j < kFillBlocks; ++j) {
+            const int b = g + j * G;
+            if (b < kCols / 16) {
+                uint32_t v[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[4 * i + 0] = __float_as_uint(fill[j][i].x), v[4 * i + 1] = __float_as_uint(fill[j][i].y);
+                    v[4 * i + 2] = __float_as_uint(fill[j][i].z), v[4 * i + 3] = __float_as_uint(fill[j][i].w);
+                }
+                tmem_st16(tlane + 16 * b, v);
             }
-            tmem_st16(tlane + c, v);
         }
         tmem_wait_st();
         tmem_fence_before();
@@ -261,6 +313,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     u64 P[16];
     uint32_t T0[CW], T1[CW];
 
+    if (seeds_ring) turn.pass();
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
         const int slot = k & 1;
@@ -293,7 +346,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             }
         };
         if constexpr (kTmem) {
-            run_chunks<FORM, 0, CW, XB>(P, T0, T1, tlane, ex, issue_next);
+            run_chunks<FORM, 0, CW, XB>(P, T0, T1, tlane, ex, turn, issue_next);
         } else {
             run_hadamard<XB>(P, ex, issue_next);
         }
@@ -321,11 +374,14 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             m0 = fmaxf(m0, fabsf(a));
             m1 = fmaxf(m1, fabsf(b));
         }
+        // non-negative floats order like their bit patterns: one integer max-reduction over the warp (fmaxf has
+        // already dropped NaNs)
         float amax = fmaxf(m0, m1);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
         const uint32_t aslot = amax_base + (k & 1) * 16;
-        if (lane == 0) sts32(aslot + q * 4, __float_as_uint(amax));
+        {
+            const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax));
+            if (lane == 0) sts32(aslot + q * 4, wmax);
+        }
         const uint32_t mslot = sbase + S::kStatOff + g * 64 + (k & 1) * 32;
         if constexpr (OUT == kOutInt4Stats) {
             // sum y^2 and sum y^4 of the row: thread (fixed order), warp (xor tree), then the four warps in order
@@ -439,6 +495,12 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             }
         }
     }
+    // a group with fewer rows than group 0 keeps the tokens moving
+    for (int k = count; k < turns; ++k) {
+#pragma unroll
+        for (int ph = 0; ph < 3; ++ph) turn.acquire(), turn.pass();
+    }
+    if (g < kRings) turn.acquire();  // each ring's first group takes its token back: no arrival stays pending
     };
     if (!shear) {
         row_loop(std::integral_constant<int, kFormScaled>());
@@ -517,28 +579,30 @@ __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restric
     const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
     const float4 p = prep[k];
     const double2 own = cs[k];
-    float* scaled = img + kFormScaled * (128 * kCols) + r * kCols;
-    float* shear = img + kFormShear * (128 * kCols) + r * kCols;
+    // image layout [column quad][role][4]: column col of role r is word ((col >> 2) * 128 + r) * 4 + (col & 3)
+    float* scaled = img + kFormScaled * (128 * kCols) + 4 * r;
+    float* shear = img + kFormShear * (128 * kCols) + 4 * r;
+    auto at = [](int col) { return (col >> 2) * 512 + (col & 3); };
     if (s < 11) {
         const float sg = (sa == sb) ? 1.f : -1.f;
-        shear[32 * s + 4 * u + h] = sg * p.x;
-        shear[32 * s + 4 * u + h + 2] = sg * p.y;
+        shear[at(32 * s + 4 * u + h)] = sg * p.x;
+        shear[at(32 * s + 4 * u + h + 2)] = sg * p.y;
         // k1 = -tan(theta) db/da, k2 = tan(theta) da/db, with one division
         const double w = own.y / (own.x * da * db);
-        scaled[32 * s + 4 * u + h] = static_cast<float>(-w * db * db);
-        scaled[32 * s + 4 * u + h + 2] = static_cast<float>(w * da * da);
+        scaled[at(32 * s + 4 * u + h)] = static_cast<float>(-w * db * db);
+        scaled[at(32 * s + 4 * u + h + 2)] = static_cast<float>(w * da * da);
         const double lim = 5.421010862427522e-20;  // 2^-64
         if (!(fabs(own.x * da) >= lim && fabs(own.x * db) >= lim)) *form = kFormShear;
     } else {
         const int col = 352 + 8 * u + h;
-        shear[col + 0] = p.z * sa;
-        shear[col + 2] = -p.w * sb;
-        shear[col + 4] = p.w * sa;
-        shear[col + 6] = p.z * sb;
-        scaled[col + 0] = static_cast<float>(own.x * da);
-        scaled[col + 2] = static_cast<float>(-own.y * db);
-        scaled[col + 4] = static_cast<float>(own.y * da);
-        scaled[col + 6] = static_cast<float>(own.x * db);
+        shear[at(col + 0)] = p.z * sa;
+        shear[at(col + 2)] = -p.w * sb;
+        shear[at(col + 4)] = p.w * sa;
+        shear[at(col + 6)] = p.z * sb;
+        scaled[at(col + 0)] = static_cast<float>(own.x * da);
+        scaled[at(col + 2)] = static_cast<float>(-own.y * db);
+        scaled[at(col + 4)] = static_cast<float>(own.y * da);
+        scaled[at(col + 6)] = static_cast<float>(own.x * db);
     }
 }
 
