@@ -208,9 +208,8 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = warp & 3, g = warp >> 2;
     const int t = q * 32 + lane;  // role within the group: 0..127
-    // Constants of this thread's role, fetched before anything else so that the L2 latency overlaps the set-up: the
-    // image is stored [column quad][role][4], a warp's load is 512 contiguous bytes, and all of a thread's loads
-    // are in flight together.  The G warps of a lane quarter share its 26 blocks of 16 columns.  The scaled-form
+    // Constants of this thread's role: the image is stored [column quad][role][4], a warp's load is 512 contiguous
+    // bytes, and all of a thread's loads are in flight together, issued before the set-up barrier.  The G warps of a lane quarter share its 26 blocks of 16 columns.  The scaled-form
     // image is fetched on the assumption that the table build selected it; the flag is checked below.
     constexpr int kFillBlocks = (kCols / 16 + G - 1) / G;
     float4 fill[kTmem ? kFillBlocks : 1][4];
@@ -224,18 +223,20 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             }
         }
     };
-    bool shear = false;
-    if constexpr (kTmem) {
-        fetch_image(reinterpret_cast<const float4*>(img));
-        shear = __ldg(form) != 0;
-    }
-
+    grid_dep_launch();
     if constexpr (kTmem) {
         if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
     }
     if (threadIdx.x < G * kInSlots) {
         mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
         mbar_init_fence();
+    }
+    // everything above overlaps the end of the kernel before this one; global memory is touched from here on
+    grid_dep_wait();
+    bool shear = false;
+    if constexpr (kTmem) {
+        fetch_image(reinterpret_cast<const float4*>(img));
+        shear = __ldg(form) != 0;
     }
     if constexpr (kTmem) tmem_fence_before();
     __syncthreads();
@@ -244,11 +245,13 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     if constexpr (kTmem) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
     const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 
-    const int first = blockIdx.x * G + g;
+    // row r belongs to group (r / gridDim.x) % G of CTA r % gridDim.x: a last, partial round of rows spreads over
+    // the CTAs instead of filling all groups of the first few
+    const int first = g * gridDim.x + blockIdx.x;
     const int stride = gridDim.x * G;
     const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
     // rows of group 0, the largest count of the CTA: every group takes that many turns with a token
-    const int turns = static_cast<int>(blockIdx.x) * G < rows ? (rows - blockIdx.x * G + stride - 1) / stride : 0;
+    const int turns = static_cast<int>(blockIdx.x) < rows ? (rows - blockIdx.x + stride - 1) / stride : 0;
     const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
     const uint32_t bar_base = sbase + S::kBarOff + 8 * g * kInSlots;
     static_assert(STEP >= 0 && (STEP == 0 || G % STEP == 0), "the rings must have equal length");
@@ -524,6 +527,8 @@ __global__ void __launch_bounds__(256) k_prep_angles4096(const float* __restrict
                                                           float4* __restrict__ prep, uint8_t* __restrict__ flip,
                                                           double2* __restrict__ cs, int* __restrict__ form) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
     if (k == 0) *form = kFormScaled;  // step 2 raises it when the scaled form is out of range
     if (k >= 12 * (kN / 2)) return;
     const double th = static_cast<double>(theta[k]);
@@ -561,6 +566,8 @@ __device__ __forceinline__ double factor_before(const double2* __restrict__ cs, 
 __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restrict__ prep, const double2* __restrict__ cs,
                                                           float* __restrict__ img, int* __restrict__ form) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dep_launch();
+    grid_dep_wait();
     if (k >= 12 * (kN / 2)) return;
     const int s = k / (kN / 2), j = k % (kN / 2);
     const int lo = ((j >> s) << (s + 1)) | (j & ((1 << s) - 1));
@@ -655,11 +662,11 @@ cudaError_t fwdq4096_set_angles(const bfq_plan* plan, const float* theta, cudaSt
     float4* prep = reinterpret_cast<float4*>(plan->prep4096);
     double2* cs = reinterpret_cast<double2*>(prep + count);
     uint8_t* flip = reinterpret_cast<uint8_t*>(cs + count);
-    f4k::k_prep_angles4096<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, flip, cs, plan->form_flag);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_overlapped(f4k::k_prep_angles4096, dim3((count + 255) / 256), dim3(256), 0, st, theta, plan->tw,
+                                      prep, flip, cs, plan->form_flag);
     if (e != cudaSuccess) return e;
-    f4k::k_build_image4096<<<(count + 255) / 256, 256, 0, st>>>(prep, cs, plan->img4096, plan->form_flag);
-    return cudaGetLastError();
+    return launch_overlapped(f4k::k_build_image4096, dim3((count + 255) / 256), dim3(256), 0, st, prep, cs, plan->img4096,
+                             plan->form_flag);
 }
 
 bool fwdq4096_available(const bfq_plan* plan) {
@@ -679,10 +686,9 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
     }
     const int64_t want = (rows + G - 1) / G;
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
-    kern<<<grid, G * f4k::kGroupThreads, S::kBytes, st>>>(tmap, plan->img4096, plan->form_flag, codes, scales,
-                                                          static_cast<__nv_bfloat16*>(y), ldy, int(rows),
-                                                          plan->status_word);
-    return cudaGetLastError();
+    return launch_overlapped(kern, dim3(grid), dim3(G * f4k::kGroupThreads), S::kBytes, st, tmap, plan->img4096,
+                             plan->form_flag, codes, scales, static_cast<__nv_bfloat16*>(y), ldy, int(rows),
+                             plan->status_word);
 }
 
 // Four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest among the

@@ -118,6 +118,20 @@ __device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int
 
 }  // namespace f4k
 
+// ---- host side: launch that lets the kernel's set-up overlap the tail of the kernel before it in the stream ----
+// (the kernel calls grid_dep_wait() before it touches global memory)
+template <class... KArgs, class... Args>
+static inline cudaError_t launch_overlapped(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                            Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // ---- host side: cuTensorMapEncodeTiled through the runtime's driver entry point ------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

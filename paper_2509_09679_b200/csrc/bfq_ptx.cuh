@@ -53,6 +53,14 @@ __device__ __forceinline__ u64 mul2(u64 a, u64 b) {
     return d;
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start while the kernel before it in the
+// stream is still running; grid_dep_wait() returns once that kernel has completed and its writes are visible
+// (at once for an ordinary launch).  grid_dep_launch() lets the next kernel of the stream start early under the
+// same rule.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- named barriers (producer / consumer hand-off between warp teams) ---------------------------------
 __device__ __forceinline__ void bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
