@@ -122,43 +122,6 @@ __device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
     for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r2 + ex2_rd_local(m));
 }
 
-// fp16 scale of a row from its absmax, as row_scale() but with straight-line arithmetic: a / QMAX as
-// q0 = a * r, q = fma(fma(-q0, QMAX, a), r, q0) with r = RN(1 / QMAX), which is the correctly rounded quotient for
-// every non-negative finite a when QMAX is 1, 7 or 127 (checked exhaustively), and an approximate reciprocal (one
-// unit in the last place) for the multiplier applied to the values.
-template <int QMAX>
-__device__ __forceinline__ uint16_t row_scale_fast(float amax, float* inv) {
-    static_assert(QMAX == 1 || QMAX == 7 || QMAX == 127, "quotient checked for these divisors only");
-    constexpr float r = 1.0f / QMAX;
-    const float q0 = __fmul_rn(amax, r);
-    const float sf = __fmaf_rn(__fmaf_rn(-q0, static_cast<float>(QMAX), amax), r, q0);
-    const uint16_t bits = sf >= 65520.f ? static_cast<uint16_t>(0x7BFFu) : __half_as_ushort(__float2half_rn(sf));
-    const float sc = __half2float(__ushort_as_half(bits));
-    float rc;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(sc));
-    *inv = sc > 0.f ? rc : 0.f;
-    return bits;
-}
-
-// stores by one thread of a warp or group without a divergent branch around them
-__device__ __forceinline__ void sts32_if(bool p, uint32_t a, uint32_t v) {
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %0, 0;\n\t@q st.shared.u32 [%1], %2;\n\t}" ::"r"(static_cast<uint32_t>(p)),
-                 "r"(a), "r"(v)
-                 : "memory");
-}
-__device__ __forceinline__ void stg16_if(bool p, uint16_t* a, uint16_t v) {
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %0, 0;\n\t@q st.global.u16 [%1], %2;\n\t}" ::"r"(static_cast<uint32_t>(p)),
-                 "l"(a), "h"(v)
-                 : "memory");
-}
-// the two bf16 halves of a word as fp32 bit patterns, on the integer pipe (a shift would go to the FP32 pipe as a
-// multiply)
-__device__ __forceinline__ uint32_t bf16_lo(uint32_t w) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, 0, 0x1044;" : "=r"(r) : "r"(w));
-    return r;
-}
-
 // The FP32 pipes and the shared-memory pipe are both heavily used; left alone, the row groups drift into step (all
 // rotating, then all regrouping) and the pipes take turns idling.  The groups therefore pass tokens around: a group
 // rotates (one phase of four stages) only while it holds a token and hands it on when it starts a regrouping or its

@@ -12,6 +12,11 @@
 // general 2x2 form that also restores the signs the angle reduction tracked, exchange their absmax,
 // and each writes the INT2 codes of the elements it finished.  Every cross-CTA wait is a bounded
 // mbarrier wait; the cluster-wide barriers at entry and exit involve every thread unconditionally.
+// Stages 0-11 rotate in the scaled two-FMA form of the n = 4096 kernel (every element carries the product of the
+// cosines it has been through; stage 12's general 2x2 absorbs the factors), with the three-shear form as the fallback
+// the table build selects when a factor leaves [2^-64, 1].
+#include <type_traits>
+
 #include "bfq_fast.h"
 #include "bfq_generic.cuh"
 #include "bfq_n4096.cuh"
@@ -22,7 +27,8 @@ using namespace ptx;
 using namespace f4k;
 
 constexpr int kN8 = 8192;
-constexpr int kCols8 = 384 + 64;  // 12 three-shear stages of this half + this rank's share of stage 12
+constexpr int kCols8 = 384 + 64;  // 12 stages of this half + this rank's share of stage 12
+enum : int { kFormScaled = 0, kFormShear = 1 };  // how stages 0..11 rotate (the image must match)
 
 template <int G>
 struct Smem {
@@ -63,18 +69,22 @@ __device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
 
 // 12 three-shear stages in chunks of 32 constants; chunk C is in Tcur, chunk C+1 (after the last stage:
 // the first half of this rank's stage-12 constants) is requested right after the wait
-template <int C, class F>
+template <int FORM, int C, class F>
 __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[32], uint32_t (&Tnext)[32], uint32_t tbase,
                                            const ExAddr& ex, F&& issue_next) {
     tmem_wait_ld32(Tcur);
     tmem_ld32(tbase + 32 * (C + 1), Tnext);
-    stage_lift<C & 3, 0, 8, 32>(P, Tcur);
+    if constexpr (FORM == kFormScaled) {
+        stage_scaled<C & 3, 0, 8, 32>(P, Tcur);
+    } else {
+        stage_lift<C & 3, 0, 8, 32>(P, Tcur);
+    }
     if constexpr (C == 3) regroup1(P, ex);
     if constexpr (C == 7) {
         regroup2(P, ex);
         issue_next();
     }
-    if constexpr (C + 1 < 12) run_chunks<C + 1>(P, Tnext, Tcur, tbase, ex, issue_next);
+    if constexpr (C + 1 < 12) run_chunks<FORM, C + 1>(P, Tnext, Tcur, tbase, ex, issue_next);
 }
 
 // stage 12 on four (lower-half, upper-half) register pairs: out_lo = k1*a + k2*b, out_hi = k3*a + k4*b
@@ -111,8 +121,8 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
 template <int G, int BITS>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
-           const float* __restrict__ img, uint8_t* __restrict__ codes, uint16_t* __restrict__ scales, int64_t ldy,
-           int rows, int* __restrict__ status) {
+           const float* __restrict__ img, const int* __restrict__ form, uint8_t* __restrict__ codes,
+           uint16_t* __restrict__ scales, int64_t ldy, int rows, int* __restrict__ status) {
     using S = Smem<G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -152,17 +162,38 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             tma_load_3d(in_base + k * kRowBytes, tmap, 0, 0, first + k * stride, bar_in + 8 * k);
         }
     }
+    // constants of this thread's role: image [form][rank][column quad][role][4], all loads in flight together; the
+    // scaled-form image is fetched on the assumption that the table build selected it
+    constexpr int kFillBlocks = (kCols8 / 16 + G - 1) / G;
+    bool shear;
     {
-        const float4* src = reinterpret_cast<const float4*>(img + (static_cast<size_t>(rank) * 128 + q * 32 + lane) * kCols8);
-        for (int c = 16 * g; c < kCols8; c += 16 * G) {
-            uint32_t v[16];
+        float4 fill[kFillBlocks][4];
+        auto fetch_image = [&](int which) {
+            const float4* base = reinterpret_cast<const float4*>(img) + (static_cast<size_t>(which) * 2 + rank) * (kCols8 / 4) * 128;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float4 f = __ldg(src + (c >> 2) + i);
-                v[4 * i + 0] = __float_as_uint(f.x), v[4 * i + 1] = __float_as_uint(f.y);
-                v[4 * i + 2] = __float_as_uint(f.z), v[4 * i + 3] = __float_as_uint(f.w);
+            for (int j = 0; j < kFillBlocks; ++j) {
+                const int b = g + j * G;
+                if (b < kCols8 / 16) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) fill[j][i] = __ldg(base + (4 * b + i) * 128 + t);
+                }
             }
-            tmem_st16(tlane + c, v);
+        };
+        fetch_image(kFormScaled);
+        shear = __ldg(form) != 0;
+        if (shear) fetch_image(kFormShear);
+#pragma unroll
+        for (int j = 0; j < kFillBlocks; ++j) {
+            const int b = g + j * G;
+            if (b < kCols8 / 16) {
+                uint32_t v[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[4 * i + 0] = __float_as_uint(fill[j][i].x), v[4 * i + 1] = __float_as_uint(fill[j][i].y);
+                    v[4 * i + 2] = __float_as_uint(fill[j][i].z), v[4 * i + 3] = __float_as_uint(fill[j][i].w);
+                }
+                tmem_st16(tlane + 16 * b, v);
+            }
         }
         tmem_wait_st();
     }
@@ -191,6 +222,9 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     // even lane stores the bytes of the lower half of the row, the odd lane those of the upper half.
     uint8_t* const out_t = codes + (t >> 1) + 64 * 8 * rank + ((t & 1) ? 1024 : 0);
 
+    // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
+    auto row_loop = [&](auto form_tag) {
+    constexpr int FORM = decltype(form_tag)::value;
     u64 P[16];
     uint32_t T0[32], T1[32];
 
@@ -212,12 +246,12 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
                 const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    P[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
+                    P[8 * c + 2 * j + 0] = pack2u(bf16_lo(a[j]), bf16_lo(b[j]));
                     P[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
                 }
             }
         }
-        run_chunks<0>(P, T0, T1, tlane, ex, [&]() {
+        run_chunks<FORM, 0>(P, T0, T1, tlane, ex, [&]() {
             if (t == 0 && k + kInSlots < count) {
                 mbar_expect_tx(bar_in + 8 * slot, kRowBytes);
                 tma_load_3d(in_base + slot * kRowBytes, tmap, 0, 0, first + (k + kInSlots) * stride, bar_in + 8 * slot);
@@ -261,11 +295,10 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             m0 = fmaxf(m0, fmaxf(fabsf(a0), fabsf(b0)));
             m1 = fmaxf(m1, fmaxf(fabsf(a1), fabsf(b1)));
         }
+        // non-negative floats order like their bit patterns: one integer max-reduction over the warp
         float amax = fmaxf(m0, m1);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
         const uint32_t aslot = amax_base + (k & 1) * 32;
-        if (lane == 0) sts32(aslot + q * 4, __float_as_uint(amax));
+        sts32_if(lane == 0, aslot + q * 4, __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax)));
         bar_sync(ex.bar, kGroupThreads);
         {
             const uint4 o = lds128(aslot);
@@ -293,8 +326,8 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             continue;
         }
         constexpr int kQmax = BITS == 16 ? 1 : (1 << (BITS - 1)) - 1;
-        const uint16_t s16 = row_scale(amax, kQmax, &inv);
-        if (rank == 0 && t == 0) scales[row] = s16;
+        const uint16_t s16 = row_scale_fast<kQmax>(amax, &inv);
+        stg16_if(rank == 0 && t == 0, scales + row, s16);
         if constexpr (BITS != 2 && BITS != 16) {
             // A[i] holds elements 2048 rank + 256 i + 2 t (+1) of the row, B[i] the same 4096 further on: with 4 or 8 bits
             // a register pair is one byte / one 16-bit word of its own.  |v * inv| < qmax + 1/2 for a normal, unsaturated
@@ -342,6 +375,12 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             out[64 * i] = static_cast<uint8_t>((t & 1) ? (got | (nh << 4)) : (nl | (got << 4)));
         }
     }
+    };
+    if (!shear) {
+        row_loop(std::integral_constant<int, kFormScaled>());
+    } else {
+        row_loop(std::integral_constant<int, kFormShear>());
+    }
 
     tmem_fence_before();
     __syncthreads();
@@ -350,53 +389,58 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
 }
 
 // ---- table preparation -----------------------------------------------------------------------------------
-// Step 1 (one thread per angle): cos/sin table entry, reduced-angle three-shear constants and whether the
-// reduction negates the pair (as for n = 4096: r = theta mod 2 pi, negated iff |r| > pi/2).
+// Step 1 (one thread per angle): cos/sin table entry (fp32 for the generic kernels, double for step 2), the
+// three-shear constants of the angle reduced to |phi| <= pi/2 and whether the reduction negates the pair (iff
+// cos(theta) < 0: phi = theta -+ pi, sin(phi) = -sin(theta), tan(phi/2) = sin(phi) / (1 + cos(phi))).
 __global__ void __launch_bounds__(256) k_prep_angles8192(const float* __restrict__ theta, float2* __restrict__ tw,
-                                                          float4* __restrict__ prep, uint8_t* __restrict__ flip) {
+                                                          float4* __restrict__ prep, double2* __restrict__ cs,
+                                                          int* __restrict__ form) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k == 0) *form = kFormScaled;  // step 2 raises it when the scaled form is out of range
     if (k >= 13 * (kN8 / 2)) return;
-    const double kPi = 3.14159265358979323846;
     const double th = static_cast<double>(theta[k]);
     double sn, c;
     sincos(th, &sn, &c);
     tw[k] = make_float2(static_cast<float>(c), static_cast<float>(sn));
-    double te = remainder(th, 2.0 * kPi);
-    bool f = false;
-    if (te > 0.5 * kPi) {
-        te -= kPi, f = true;
-    } else if (te < -0.5 * kPi) {
-        te += kPi, f = true;
-    }
-    flip[k] = f ? 1 : 0;
-    prep[k] = make_float4(static_cast<float>(-tan(0.5 * te)), static_cast<float>(sin(te)), static_cast<float>(c),
+    cs[k] = make_double2(c, sn);
+    const bool f = c < 0.0;
+    const double sp = f ? -sn : sn, cp = f ? -c : c;
+    prep[k] = make_float4(static_cast<float>(-sp / (1.0 + cp)), static_cast<float>(sp), static_cast<float>(c),
                           static_cast<float>(sn));
 }
 
-// sign carried by element i (0..4095) of half `half` when it enters stage s <= 12: stages 0..11 pair inside
-// the half, and pair j of such a stage belongs to the upper half iff j >= 2048
-__device__ __forceinline__ int sign_before8(const uint8_t* __restrict__ flip, int half, int i, int s) {
-    int f = 0;
-    for (int sp = 0; sp < s; ++sp) {
+// factor carried by element i (0..4095) of half `half` when it enters stage s <= 12: the product of the cosines of
+// the pairs it belonged to in stages 0..s-1 (stages 0..11 pair inside the half; pair j of such a stage belongs to the
+// upper half iff j >= 2048).  Its sign is the tracked sign of the three-shear form.
+__device__ __forceinline__ double factor_before8(const double2* __restrict__ cs, int half, int i, int s) {
+    double c[12];
+#pragma unroll
+    for (int sp = 0; sp < 12; ++sp) {  // all loads issued together
         const int j = ((i >> (sp + 1)) << sp) | (i & ((1 << sp) - 1));
-        f ^= flip[sp * (kN8 / 2) + half * (kN / 2) + j];
+        c[sp] = sp < s ? cs[sp * (kN8 / 2) + half * (kN / 2) + j].x : 1.0;
     }
-    return f ? -1 : 1;
+    double d = 1.0;
+#pragma unroll
+    for (int sp = 0; sp < 12; ++sp) d *= c[sp];
+    return d;
 }
 
-// Step 2 (one thread per angle): constants of pair (s, j) into the image of the CTA rank that uses them,
-// img[rank][role][column]
-__global__ void __launch_bounds__(256) k_build_image8192(const float4* __restrict__ prep,
-                                                          const uint8_t* __restrict__ flip, float* __restrict__ img) {
+// Step 2 (one thread per angle): constants of pair (s, j) into both images of the CTA rank that uses them,
+// img[form][rank][column quad][role][4]; raises *form when an element's factor leaves the scaled form's range.
+__global__ void __launch_bounds__(256) k_build_image8192(const float4* __restrict__ prep, const double2* __restrict__ cs,
+                                                          float* __restrict__ img, int* __restrict__ form) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= 13 * (kN8 / 2)) return;
     const int s = k / (kN8 / 2), j = k % (kN8 / 2);
     const float4 p = prep[k];
+    const double2 own = cs[k];
+    constexpr size_t kImage = size_t(128) * kCols8;  // one (form, rank) image
+    auto at = [](int r, int col) { return (col >> 2) * 512 + 4 * r + (col & 3); };
     if (s < 12) {
         const int half = j >> 11, jj = j & 2047;
         const int lo = ((jj >> s) << (s + 1)) | (jj & ((1 << s) - 1));  // inside the half
         const int hi = lo + (1 << s);
-        const int sa = sign_before8(flip, half, lo, s), sb = sign_before8(flip, half, hi, s);
+        const double da = factor_before8(cs, half, lo, s), db = factor_before8(cs, half, hi, s);
         const int kk = s & 3;
         int r, m, h;
         if (s < 4) {
@@ -407,38 +451,54 @@ __global__ void __launch_bounds__(256) k_build_image8192(const float4* __restric
             r = (lo >> 1) & 127, m = lo >> 8, h = lo & 1;
         }
         const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
-        const float sg = (sa == sb) ? 1.f : -1.f;
-        float* strip = img + (static_cast<size_t>(half) * 128 + r) * kCols8;
-        strip[32 * s + 4 * u + h] = sg * p.x;
-        strip[32 * s + 4 * u + h + 2] = sg * p.y;
+        const float sg = ((da < 0.0) == (db < 0.0)) ? 1.f : -1.f;
+        float* scaled = img + (size_t(kFormScaled) * 2 + half) * kImage;
+        float* shear = img + (size_t(kFormShear) * 2 + half) * kImage;
+        const int col = 32 * s + 4 * u + h;
+        shear[at(r, col)] = sg * p.x;
+        shear[at(r, col + 2)] = sg * p.y;
+        // k1 = -tan(theta) db/da, k2 = tan(theta) da/db, with one division
+        const double w = own.y / (own.x * da * db);
+        scaled[at(r, col)] = static_cast<float>(-w * db * db);
+        scaled[at(r, col + 2)] = static_cast<float>(w * da * da);
+        const double lim = 5.421010862427522e-20;  // 2^-64
+        if (!(fabs(own.x * da) >= lim && fabs(own.x * db) >= lim)) *form = kFormShear;
     } else {
         // stage 12: element j of the lower half with element j of the upper half, in phase-3 ownership;
         // registers 0-7 are finished by rank 0, 8-15 by rank 1
-        const int sa = sign_before8(flip, 0, j, 12), sb = sign_before8(flip, 1, j, 12);
+        const double da = factor_before8(cs, 0, j, 12), db = factor_before8(cs, 1, j, 12);
+        const int sa = da < 0.0 ? -1 : 1, sb = db < 0.0 ? -1 : 1;
         const int r = (j >> 1) & 127, m = j >> 8, h = j & 1;
-        float* strip = img + (static_cast<size_t>(m >> 3) * 128 + r) * kCols8;
+        float* scaled = img + (size_t(kFormScaled) * 2 + (m >> 3)) * kImage;
+        float* shear = img + (size_t(kFormShear) * 2 + (m >> 3)) * kImage;
         const int col = 384 + 8 * (m & 7) + h;
-        strip[col + 0] = p.z * sa;
-        strip[col + 2] = -p.w * sb;
-        strip[col + 4] = p.w * sa;
-        strip[col + 6] = p.z * sb;
+        shear[at(r, col + 0)] = p.z * sa;
+        shear[at(r, col + 2)] = -p.w * sb;
+        shear[at(r, col + 4)] = p.w * sa;
+        shear[at(r, col + 6)] = p.z * sb;
+        scaled[at(r, col + 0)] = static_cast<float>(own.x * da);
+        scaled[at(r, col + 2)] = static_cast<float>(-own.y * db);
+        scaled[at(r, col + 4)] = static_cast<float>(own.y * da);
+        scaled[at(r, col + 6)] = static_cast<float>(own.x * db);
     }
 }
 
 }  // namespace f8k
 
 // ---- host side ---------------------------------------------------------------------------------------------
-size_t fwdq8192_image_bytes() { return size_t(2) * 128 * f8k::kCols8 * sizeof(float); }
-size_t fwdq8192_prep_bytes() { return size_t(13) * (f8k::kN8 / 2) * (sizeof(float4) + 1); }
+// two forms x two CTA ranks
+size_t fwdq8192_image_bytes() { return size_t(4) * 128 * f8k::kCols8 * sizeof(float); }
+// per angle: float4 (three-shear constants, cos, sin) and double2 (cos, sin)
+size_t fwdq8192_prep_bytes() { return size_t(13) * (f8k::kN8 / 2) * (sizeof(float4) + sizeof(double2)); }
 
 cudaError_t fwdq8192_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st) {
     const int count = 13 * (f8k::kN8 / 2);
     float4* prep = reinterpret_cast<float4*>(plan->prep8192);
-    uint8_t* flip = reinterpret_cast<uint8_t*>(prep + count);
-    f8k::k_prep_angles8192<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, flip);
+    double2* cs = reinterpret_cast<double2*>(prep + count);
+    f8k::k_prep_angles8192<<<(count + 255) / 256, 256, 0, st>>>(theta, plan->tw, prep, cs, plan->form_flag);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    f8k::k_build_image8192<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img8192);
+    f8k::k_build_image8192<<<(count + 255) / 256, 256, 0, st>>>(prep, cs, plan->img8192, plan->form_flag);
     return cudaGetLastError();
 }
 
@@ -478,8 +538,8 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192), codes, scales, ldy,
-                              int(rows), plan->status_word);
+    return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192),
+                              static_cast<const int*>(plan->form_flag), codes, scales, ldy, int(rows), plan->status_word);
 }
 
 cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
