@@ -163,6 +163,7 @@ static void release_plan(bfq_plan* plan) {
     cudaFree(plan->img4096);
     cudaFree(plan->prep4096);
     cudaFree(plan->img_b4096);
+    cudaFree(plan->img_i4096);
     cudaFree(plan->img8192);
     cudaFree(plan->prep8192);
     cudaFree(plan->dsign4096);
@@ -217,6 +218,7 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->img8192, fwdq8192_image_bytes());
     if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->prep8192, fwdq8192_prep_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_b4096, bwd4096_image_bytes());
+    if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_i4096, inv4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->dsign4096, bwd4096_dsign_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->gsign4096, bwd4096_gsign_bytes());
     if (e == cudaSuccess && n == 128) e = cudaMalloc(&plan->dense128, comp5120d_image_bytes());

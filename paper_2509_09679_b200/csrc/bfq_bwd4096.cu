@@ -16,6 +16,8 @@
 // d-theta accumulators are owned by thread role (no atomics): stages 0-7 in the tensor-memory columns the
 // constants leave free, stages 8-11 in shared memory.  Each CTA walks its row pairs in a fixed order and
 // writes its sums to its own slot; a second kernel adds the slots in index order: bit-reproducible.
+#include <type_traits>
+
 #include "bfq_fast.h"
 #include "bfq_generic.cuh"
 #include "bfq_n4096.cuh"
@@ -32,6 +34,8 @@ constexpr int kBarRev = 1, kBarFwd = 2, kBarFull = 3, kBarEmpty = 4;  // named b
 constexpr int kConstCols = 384;              // 12 stages x 32 words
 constexpr int kAccCol = 384;                 // accumulators of stages 0..7: 16 columns each
 constexpr uint32_t kPairBytes = 2 * kRowBytes;  // two bf16 rows
+constexpr int kInvCols = 416;  // scaled inverse: stages 11..1 (32 columns each, stage s at 32 (s - 1)), then stage 0 (64)
+enum : int { kFormScaled = 0, kFormShear = 1 };
 
 struct Smem {
     static constexpr uint32_t kXOff = 0;                                   // [kSlots][2][kRowBytes]
@@ -527,6 +531,59 @@ __global__ void __launch_bounds__(256) k_build_gsign4096(const uint8_t* __restri
 }
 
 
+// One thread per angle: the constants of the scaled reverse walk (x = Q^T y, stages 11 down to 0).  Element i enters
+// reverse stage s carrying the factor e = product of the cosines of the pairs it belongs to in stages s+1..11; stage s
+// then is  lo = lo' + j1 hi',  hi = hi' + j2 lo'  with  j1 = tan(theta) e_hi / e_lo,  j2 = -tan(theta) e_lo / e_hi  and
+// both factors are multiplied by cos(theta).  Stage 0 is a general 2x2 that absorbs the factors.  Image layout
+// [column quad][role][4]; stage s >= 1 at columns 32 (s - 1), stage 0 at 352.  *form is raised when a factor leaves
+// [2^-64, 1]: the kernel then walks in the three-shear form.
+__global__ void __launch_bounds__(256) k_build_image_inv4096(const double2* __restrict__ cs, float* __restrict__ img,
+                                                              int* __restrict__ form) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 12 * (kN / 2)) return;
+    const int s = k / (kN / 2), j = k % (kN / 2);
+    const int lo = ((j >> s) << (s + 1)) | (j & ((1 << s) - 1));
+    const int hi = lo + (1 << s);
+    double cl[11], ch[11];
+#pragma unroll
+    for (int sp = 1; sp < 12; ++sp) {  // all loads issued together
+        const int jl = ((lo >> (sp + 1)) << sp) | (lo & ((1 << sp) - 1));
+        const int jh = ((hi >> (sp + 1)) << sp) | (hi & ((1 << sp) - 1));
+        cl[sp - 1] = sp > s ? cs[sp * (kN / 2) + jl].x : 1.0;
+        ch[sp - 1] = sp > s ? cs[sp * (kN / 2) + jh].x : 1.0;
+    }
+    double el = 1.0, eh = 1.0;
+#pragma unroll
+    for (int i = 0; i < 11; ++i) el *= cl[i], eh *= ch[i];
+    const int kk = s & 3;
+    int r, m, h;
+    if (s < 4) {
+        r = ((lo >> 4) & 15) | ((lo >> 9) << 4), m = lo & 15, h = (lo >> 8) & 1;
+    } else if (s < 8) {
+        r = (lo & 15) | ((lo >> 9) << 4), m = (lo >> 4) & 15, h = (lo >> 8) & 1;
+    } else {
+        r = (lo >> 1) & 127, m = lo >> 8, h = lo & 1;
+    }
+    const int u = ((m >> (kk + 1)) << kk) | (m & ((1 << kk) - 1));
+    const double2 own = cs[k];
+    float* strip = img + 4 * r;
+    auto at = [](int col) { return (col >> 2) * 512 + (col & 3); };
+    if (s > 0) {
+        const double w = own.y / (own.x * el * eh);  // tan(theta) / (e_lo e_hi)
+        const int col = 32 * (s - 1) + 4 * u + h;
+        strip[at(col)] = static_cast<float>(w * eh * eh);
+        strip[at(col + 2)] = static_cast<float>(-w * el * el);
+        const double lim = 5.421010862427522e-20;  // 2^-64
+        if (!(fabs(own.x * el) >= lim && fabs(own.x * eh) >= lim)) *form = kFormShear;
+    } else {
+        const int col = 352 + 8 * u + h;
+        strip[at(col + 0)] = static_cast<float>(own.x * el);
+        strip[at(col + 2)] = static_cast<float>(own.y * eh);
+        strip[at(col + 4)] = static_cast<float>(-own.y * el);
+        strip[at(col + 6)] = static_cast<float>(own.x * eh);
+    }
+}
+
 // =================================================================================================================
 // Inverse / transpose for n = 4096 bf16 rows:  x = Q^T y.  The reverse walk of the backward kernel on one array,
 // organised like the forward kernel: four row groups of 128 threads per CTA, 32 constants per tensor-memory chunk.
@@ -541,13 +598,43 @@ struct InvSmem {
     static constexpr uint32_t kBytes = kUsed + 1024;
 };
 
-// stage S (11..0) is in Tcur; stage S-1 is requested right after the wait
-template <int S, class F>
+// general 2x2 on local bit 0 (stage 0 of the reverse walk): out_lo = k1*a + k2*b, out_hi = k3*a + k4*b for the
+// register pairs (2u, 2u + 1), u = U0..U0+NU-1
+template <int U0, int NU>
+__device__ __forceinline__ void stage_general_k0(u64 (&P)[16], const uint32_t (&T)[32]) {
+    static_assert(8 * NU <= 32, "chunk too small");
+#pragma unroll
+    for (int i = 0; i < NU; ++i) {
+        const int m_lo = 2 * (U0 + i), m_hi = m_lo + 1;
+        const u64 K1 = pack2u(T[8 * i], T[8 * i + 1]), K2 = pack2u(T[8 * i + 2], T[8 * i + 3]);
+        const u64 K3 = pack2u(T[8 * i + 4], T[8 * i + 5]), K4 = pack2u(T[8 * i + 6], T[8 * i + 7]);
+        const u64 a = P[m_lo], b = P[m_hi];
+        P[m_lo] = fma2(K2, b, mul2(K1, a));
+        P[m_hi] = fma2(K4, b, mul2(K3, a));
+    }
+}
+
+// stage S (11..0) is in Tcur; the next constants are requested right after the wait.  Three-shear form: stage s at
+// column 32 s, all twelve stages alike.  Scaled form: stages 11..1 are two-FMA stages on values that carry the product of
+// the cosines of the stages above, stage 0 is a general 2x2 (two chunks) that absorbs the factors.
+template <int FORM, int S, class F>
 __device__ __forceinline__ void inv_stages(u64 (&P)[16], uint32_t (&Tcur)[32], uint32_t (&Tnext)[32], uint32_t tlane,
                                            const Addr& a, uint32_t buf2, uint32_t buf1, F&& after_phase3) {
     tmem_wait_ld32(Tcur);
-    if constexpr (S > 0) tmem_ld32(tlane + 32 * (S - 1), Tnext);
-    stage_lift<S & 3, 0, 8, 32>(P, Tcur);
+    if constexpr (FORM == kFormShear) {
+        if constexpr (S > 0) tmem_ld32(tlane + 32 * (S - 1), Tnext);
+        stage_lift<S & 3, 0, 8, 32>(P, Tcur);
+    } else {
+        if constexpr (S > 1) tmem_ld32(tlane + 32 * (S - 2), Tnext);
+        if constexpr (S == 1) tmem_ld32(tlane + 352, Tnext);
+        if constexpr (S > 0) stage_scaled<S & 3, 0, 8, 32>(P, Tcur);
+        if constexpr (S == 0) {
+            tmem_ld32(tlane + 384, Tnext);
+            stage_general_k0<0, 4>(P, Tcur);
+            tmem_wait_ld32(Tnext);
+            stage_general_k0<4, 4>(P, Tnext);
+        }
+    }
     if constexpr (S == 8) {
         bar_sync(a.bar, kThreads);  // every warp is past its scalar reads of the previous row
         rev2_store(P, buf2, a);
@@ -561,13 +648,14 @@ __device__ __forceinline__ void inv_stages(u64 (&P)[16], uint32_t (&Tcur)[32], u
         __syncwarp();
         rev1_load(P, buf1, a);
     }
-    if constexpr (S > 0) inv_stages<S - 1>(P, Tnext, Tcur, tlane, a, buf2, buf1, after_phase3);
+    if constexpr (S > 0) inv_stages<FORM, S - 1>(P, Tnext, Tcur, tlane, a, buf2, buf1, after_phase3);
 }
 
 template <int G, bool OUT_BF16>
 __global__ void __launch_bounds__(G * kThreads, 1)
-k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ img, const uint32_t* __restrict__ gsign,
-          void* __restrict__ xout, int64_t ldx, int rows, int* __restrict__ status) {
+k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ img, const float* __restrict__ img_scaled,
+          const int* __restrict__ form, const uint32_t* __restrict__ gsign, void* __restrict__ xout, int64_t ldx, int rows,
+          int* __restrict__ status) {
     using S = InvSmem<G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -598,7 +686,36 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
             tma_load_3d(in_base + k * kRowBytes, &ymap, 0, 0, first + k * stride, bar_base + 8 * k);
         }
     }
-    {
+    // constants: the scaled-form image ([column quad][role][4], coalesced, all loads in flight) unless the table build
+    // flagged it out of range; then the three-shear image ([role][384])
+    const bool shear = __ldg(form) != 0;
+    if (!shear) {
+        constexpr int kFillBlocks = (kInvCols / 16 + G - 1) / G;
+        float4 fill[kFillBlocks][4];
+        const float4* base = reinterpret_cast<const float4*>(img_scaled);
+#pragma unroll
+        for (int j = 0; j < kFillBlocks; ++j) {
+            const int b = g + j * G;
+            if (b < kInvCols / 16) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) fill[j][i] = __ldg(base + (4 * b + i) * 128 + t);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kFillBlocks; ++j) {
+            const int b = g + j * G;
+            if (b < kInvCols / 16) {
+                uint32_t v[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[4 * i + 0] = __float_as_uint(fill[j][i].x), v[4 * i + 1] = __float_as_uint(fill[j][i].y);
+                    v[4 * i + 2] = __float_as_uint(fill[j][i].z), v[4 * i + 3] = __float_as_uint(fill[j][i].w);
+                }
+                tmem_st16(tlane + 16 * b, v);
+            }
+        }
+        tmem_wait_st();
+    } else {
         const float4* src = reinterpret_cast<const float4*>(img + (q * 32 + lane) * kConstCols);
         for (int c = 16 * g; c < kConstCols; c += 16 * G) {
             uint32_t v[16];
@@ -633,32 +750,40 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
     const uint32_t sgn_a = par_t ? 0x80000000u : 0u, sgn_b = par_t ? 0u : 0x80000000u;
     const uint4* gsv = reinterpret_cast<const uint4*>(gsign);
 
+    // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
+    auto row_loop = [&](auto form_tag) {
+    constexpr int FORM = decltype(form_tag)::value;
+    constexpr bool kSigns = FORM == kFormShear;  // the three-shear walk runs in the sign-tracked parity basis
     u64 P[16];
     uint32_t T0[32], T1[32];
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
         const int slot = k & 1;
-        tmem_ld32(tlane + 32 * 11, T0);
+        tmem_ld32(tlane + (FORM == kFormShear ? 32 * 11 : 32 * 10), T0);
         mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
         const uint32_t tile = in_base + slot * kRowBytes;
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
-            const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
-            const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+            uint32_t s4[4] = {0u, 0u, 0u, 0u};
+            if constexpr (kSigns) {
+                const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
+                s4[0] = sw.x, s4[1] = sw.y, s4[2] = sw.z, s4[3] = sw.w;
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int m = 4 * qq + i;
                 const uint32_t w = lds32(tile + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
-                P[m] = pack2u(w << 16, w & 0xFFFF0000u);
+                P[m] = pack2u(bf16_lo(w), w & 0xFFFF0000u);
             }
         }
-        inv_stages<11>(P, T0, T1, tlane, a, a.ex, a.ex + kExBytes, [&]() {
+        inv_stages<FORM, 11>(P, T0, T1, tlane, a, a.ex, a.ex + kExBytes, [&]() {
             if (t == 0 && k + kInSlots < count) {
                 mbar_expect_tx(bar_base + 8 * slot, kRowBytes);
                 tma_load_3d(in_base + slot * kRowBytes, &ymap, 0, 0, first + (k + kInSlots) * stride, bar_base + 8 * slot);
             }
         });
-        // phase-1 ownership: two runs of 16 consecutive elements; undo the parity sign
+        // phase-1 ownership: two runs of 16 consecutive elements; the three-shear form undoes the parity sign here
+        const uint32_t sa_ = kSigns ? sgn_a : 0u, sb_ = kSigns ? sgn_b : 0u;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int64_t off = static_cast<int64_t>(row) * ldx + 16 * (t & 15) + 512 * (t >> 4) + 256 * h;
@@ -671,8 +796,8 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
                     unpack2u(P[2 * j + 1], lo1, hi1);
                     const float e0 = __uint_as_float(h ? hi0 : lo0), e1 = __uint_as_float(h ? hi1 : lo1);
                     const bool odd_c = ((__builtin_popcount(2 * j) + h) & 1) != 0;
-                    const uint32_t neg_lo = odd_c ? (sgn_b >> 16) : (sgn_a >> 16);
-                    const uint32_t neg_hi = odd_c ? sgn_a : sgn_b;
+                    const uint32_t neg_lo = odd_c ? (sb_ >> 16) : (sa_ >> 16);
+                    const uint32_t neg_hi = odd_c ? sa_ : sb_;
                     w[j] = cvt_bf16x2(e0, e1) ^ (neg_lo | neg_hi);
                 }
                 uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(xout) + off);
@@ -685,13 +810,19 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
                     uint32_t lo, hi;
                     unpack2u(P[m], lo, hi);
                     const bool odd_c = ((__builtin_popcount(m) + h) & 1) != 0;  // parity popcount(m) ^ h ^ popcount(t)
-                    w[m] = (h ? hi : lo) ^ (odd_c ? sgn_b : sgn_a);
+                    w[m] = (h ? hi : lo) ^ (odd_c ? sb_ : sa_);
                 }
                 uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(xout) + off);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) dst[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
             }
         }
+    }
+    };
+    if (!shear) {
+        row_loop(std::integral_constant<int, kFormScaled>());
+    } else {
+        row_loop(std::integral_constant<int, kFormShear>());
     }
     tmem_fence_before();
     __syncthreads();
@@ -702,6 +833,7 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
 
 // ---- host side ---------------------------------------------------------------------------------------------
 size_t bwd4096_image_bytes() { return size_t(128) * b4k::kConstCols * sizeof(float); }
+size_t inv4096_image_bytes() { return size_t(128) * b4k::kInvCols * sizeof(float); }
 size_t bwd4096_dsign_bytes() { return size_t(12) * (f4k::kN / 2); }
 size_t bwd4096_gsign_bytes() { return size_t(16) * b4k::kThreads * sizeof(uint32_t); }
 
@@ -719,6 +851,13 @@ cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     b4k::k_build_gsign4096<<<(16 * b4k::kThreads + 255) / 256, 256, 0, st>>>(flip, plan->gsign4096);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    // the scaled reverse walk of the inverse kernel and its range flag (word 1 of the plan's form flags)
+    e = cudaMemsetAsync(plan->form_flag + 1, 0, sizeof(int), st);
+    if (e != cudaSuccess) return e;
+    b4k::k_build_image_inv4096<<<(count + 255) / 256, 256, 0, st>>>(reinterpret_cast<const double2*>(prep + count),
+                                                                   plan->img_i4096, plan->form_flag + 1);
     return cudaGetLastError();
 }
 
@@ -764,10 +903,12 @@ cudaError_t inv4096_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t 
     const int64_t want = (rows + G - 1) / G;
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
     if (x_bf16) {
-        b4k::k_inv4096<G, true><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->gsign4096, x, ldx,
+        b4k::k_inv4096<G, true><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->img_i4096,
+                                                                            plan->form_flag + 1, plan->gsign4096, x, ldx,
                                                                             int(rows), plan->status_word);
     } else {
-        b4k::k_inv4096<G, false><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->gsign4096, x, ldx,
+        b4k::k_inv4096<G, false><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->img_i4096,
+                                                                             plan->form_flag + 1, plan->gsign4096, x, ldx,
                                                                              int(rows), plan->status_word);
     }
     return cudaGetLastError();

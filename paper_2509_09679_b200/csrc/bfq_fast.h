@@ -35,6 +35,7 @@ cudaError_t fwdq8192_launch_bf16(const bfq_plan* plan, const void* x, int64_t ro
 
 // n = 4096, bf16 x / g / dx: backward with tensor-memory constants and accumulators
 size_t bwd4096_image_bytes();
+size_t inv4096_image_bytes();
 size_t bwd4096_dsign_bytes();
 size_t bwd4096_gsign_bytes();
 bool bwd4096_available(const bfq_plan* plan);

@@ -19,6 +19,7 @@ struct bfq_plan {
     float* img4096 = nullptr;    // [128][416] tensor-memory image of the rotation constants (n = 4096 only)
     void* prep4096 = nullptr;    // staging for the image build: per-angle constants and negation flags (n = 4096 only)
     float* img_b4096 = nullptr;  // [128][384] constants of the backward kernel (n = 4096 only)
+    float* img_i4096 = nullptr;  // [104][128][4] scaled-form constants of the inverse kernel (n = 4096 only)
     int8_t* dsign4096 = nullptr; // [12][2048] sign applied to the accumulated d-theta (n = 4096 only)
     uint32_t* gsign4096 = nullptr;  // [16 * 128] sign words applied to bf16 g rows (n = 4096 only)
     bool bwd_tables_valid = false;  // the three above match the current angles
