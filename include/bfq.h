@@ -216,8 +216,39 @@ int bfq_device_status(bfq_plan* plan);
 /* Last cudaError_t seen by this plan (0 = cudaSuccess).  (No counterpart in the paper.) */
 int bfq_last_cuda_error(const bfq_plan* plan);
 
+/*
+ * Which rotation form the tuned kernels (n = 4096, n = 8192) run with the current angles.  They use the scaled two-FMA
+ * form (paper Sec. "Inference Efficiency": two FMAs per pair) in which every element carries the product of the
+ * cosines it has been through; when such a product leaves [2^-64, 1] (an angle within ~1e-19 .. of an odd multiple of
+ * pi/2 along some path, e.g. angles that are exact multiples of pi/2) the table build selects the three-shear form
+ * instead, which has no such limit.  Returns bit 0 = forward tables use the fallback, bit 1 = inverse tables (built by
+ * the first bfq_inverse / bfq_backward after bfq_set_angles) use the fallback; or a negative bfq_status.  Synchronises
+ * the device.  With the scaled form, inputs must stay below about 2^56 in magnitude (intermediate values are the true
+ * values divided by the factor).  (No counterpart in the paper; informational.)
+ */
+int bfq_stage_form(bfq_plan* plan);
+
+/*
+ * Test hook (no counterpart in the paper): while enabled, the tuned n = 4096 forward kernels of this plan announce 16
+ * bytes more per row load than the load delivers and bound their waits at 4096 polls, so that every wait runs out:
+ * the kernels return normally with meaningless outputs (inside their buffers) and bfq_device_status reports
+ * BFQ_ERR_DEVICE_TIMEOUT once.  Exercises the bounded-wait path without hanging or faulting the GPU.
+ */
+int bfq_test_stuck_wait(bfq_plan* plan, int enable);
+
 /* Static string for a status code. */
 const char* bfq_status_string(int status);
+
+/*
+ * Measures, on the current device, how many SM cycles one warp scheduler needs per FP32 FMA instruction with register
+ * operands only (no memory traffic in the timed loops): out[0] packed fma.rn.f32x2 with three distinct register
+ * operands (the pattern of a rotation with per-pair constants), out[1] packed with two distinct operands, out[2] /
+ * out[3] the same for scalar FMAs.  `cycles_per_instruction` is a HOST array of 4 floats.  Synchronous: allocates and
+ * frees a few hundred bytes of device memory and synchronises the device; meant for benchmarks, which print the
+ * measured issue rate beside the nominal peak of one FMA per lane per cycle (the paper counts FLOPs, appendix table
+ * "FLOP comparison"; it has no counterpart of this call).  Returns BFQ_OK, BFQ_ERR_NULL or BFQ_ERR_CUDA.
+ */
+int bfq_measure_fma_rates(float* cycles_per_instruction);
 
 /* Number of CTAs the backward pass uses (= number of d-theta partial sums); informational. */
 int bfq_backward_partials(const bfq_plan* plan);

@@ -39,6 +39,9 @@ SIGNATURES = {
     "bfq_last_cuda_error": (_i, [_p]),
     "bfq_status_string": (ctypes.c_char_p, [_i]),
     "bfq_backward_partials": (_i, [_p]),
+    "bfq_measure_fma_rates": (_i, [_p]),
+    "bfq_stage_form": (_i, [_p]),
+    "bfq_test_stuck_wait": (_i, [_p, _i]),
     "bfq_backward_noalloc": (_i, [_i, _p, _p, _i, _p, _i, _i64, _i64, _p, _i, _p, _p]),
     "bfq_cayley": (_i, [_p, _p, _i, _p, _p]),
     "bfq_composite_forward": (_i, [_p, _p, _i, _p, _i, _i64, _i64, _p, _i, _i64, _p]),
@@ -84,10 +87,33 @@ def _dt(t: torch.Tensor) -> int:
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 
-def _rows(t: torch.Tensor, n: int):
-    if t.dim() != 2 or t.shape[1] != n or t.stride(1) != 1:
-        raise ValueError(f"expected a [rows][{n}] tensor with unit inner stride, got {tuple(t.shape)}")
+def _rows(t: torch.Tensor, n: int, device=None, rows=None, what: str = "rows"):
+    """Checks a [rows][n] row tensor (unit inner stride; on `device` when given; `rows` rows when given) and returns
+    (rows, leading dimension).  Only this layer knows the buffers' sizes: the C ABI takes bare pointers."""
+    if not isinstance(t, torch.Tensor) or t.dim() != 2 or t.shape[1] != n or t.stride(1) != 1:
+        raise ValueError(f"{what}: expected a [rows][{n}] tensor with unit inner stride, got "
+                         f"{tuple(t.shape) if isinstance(t, torch.Tensor) else type(t)}")
+    if device is not None:
+        _on(t, device, what)
+    if rows is not None and t.shape[0] != rows:
+        raise ValueError(f"{what}: expected {rows} rows, got {t.shape[0]}")
+    if t.shape[0] > 1 and t.stride(0) < n:
+        raise ValueError(f"{what}: rows overlap (row stride {t.stride(0)} < {n})")
     return t.shape[0], (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), n))
+
+
+def _on(t: torch.Tensor, device, what: str):
+    if not t.is_cuda or t.device != device:
+        raise ValueError(f"{what}: tensor is on {t.device}, the plan works on {device}")
+
+
+def _exact(t: torch.Tensor, dtype, shape, device, what: str):
+    """A contiguous tensor of exactly this dtype and shape on `device` (tables, codes, scales, statistics)."""
+    if not isinstance(t, torch.Tensor) or t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        got = (t.dtype, tuple(t.shape)) if isinstance(t, torch.Tensor) else type(t)
+        raise ValueError(f"{what}: expected a contiguous {dtype} tensor of shape {tuple(shape)}, got {got}")
+    _on(t, device, what)
+    return t
 
 
 def _stream(t: torch.Tensor):
@@ -121,24 +147,32 @@ class Plan:
 
     # -- the C ABI, one method per entry point ------------------------------------------------------
     def set_angles(self, theta: torch.Tensor):
-        if theta.dtype != torch.float32 or tuple(theta.shape) != (self.L, self.n // 2) or not theta.is_contiguous():
-            raise ValueError(f"theta must be a contiguous fp32 [{self.L}][{self.n // 2}] tensor")
+        _exact(theta, torch.float32, (self.L, self.n // 2), self.device, "theta")
         _check(lib().bfq_set_angles(self._h, theta.data_ptr(), _stream(theta)), "bfq_set_angles")
 
     def forward(self, x: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
-        rows, ldx = _rows(x, self.n)
+        rows, ldx = _rows(x, self.n, self.device, what="x")
         y = out if out is not None else torch.empty((rows, self.n), dtype=out_dtype or x.dtype, device=x.device)
-        _, ldy = _rows(y, self.n)
+        _, ldy = _rows(y, self.n, self.device, rows, "out")
         _check(lib().bfq_forward(self._h, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(), _dt(y), ldy, _stream(x)),
                "bfq_forward")
         return y
 
-    def forward_quant(self, x: torch.Tensor, bits: int, codes=None, scales=None):
-        rows, ldx = _rows(x, self.n)
+    def _outputs(self, rows: int, width: int, bits: int, codes, scales):
+        """Allocates or checks the codes uint8 [rows][width * bits / 8] and scales fp16 [rows] buffers."""
+        if bits not in (2, 4, 8):
+            raise ValueError("bits must be 2, 4 or 8")
         if codes is None:
-            codes = torch.empty((rows, self.n * bits // 8), dtype=torch.uint8, device=x.device)
+            codes = torch.empty((rows, width * bits // 8), dtype=torch.uint8, device=self.device)
         if scales is None:
-            scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+            scales = torch.empty((rows,), dtype=torch.float16, device=self.device)
+        _exact(codes, torch.uint8, (rows, width * bits // 8), self.device, "codes")
+        _exact(scales, torch.float16, (rows,), self.device, "scales")
+        return codes, scales
+
+    def forward_quant(self, x: torch.Tensor, bits: int, codes=None, scales=None):
+        rows, ldx = _rows(x, self.n, self.device, what="x")
+        codes, scales = self._outputs(rows, self.n, bits, codes, scales)
         _check(lib().bfq_forward_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
                                        scales.data_ptr(), _stream(x)), "bfq_forward_quant")
         return codes, scales
@@ -148,6 +182,7 @@ class Plan:
         """Q1 = (I - A)(I + A)^-1 from the n1 (n1 - 1) / 2 upper-triangle entries of the skew A -> fp32 [n1][n1]."""
         if params.dtype != torch.float32 or params.numel() != n1 * (n1 - 1) // 2 or not params.is_contiguous():
             raise ValueError("params must be a contiguous fp32 tensor of n1 (n1 - 1) / 2 entries")
+        _on(params, self.device, "params")
         q1 = torch.empty((n1, n1), dtype=torch.float32, device=params.device)
         _check(lib().bfq_cayley(self._h, params.data_ptr(), int(n1), q1.data_ptr(), _stream(params)), "bfq_cayley")
         return q1
@@ -155,13 +190,16 @@ class Plan:
     def _q1(self, q1: torch.Tensor) -> int:
         if q1.dtype != torch.float32 or q1.dim() != 2 or q1.shape[0] != q1.shape[1] or not q1.is_contiguous():
             raise ValueError("q1 must be a contiguous fp32 [n1][n1] tensor")
+        _on(q1, self.device, "q1")
         return q1.shape[0]
 
     def composite_forward(self, q1: torch.Tensor, x: torch.Tensor, out_dtype=None, out=None) -> torch.Tensor:
         n1 = self._q1(q1)
         d = n1 * self.n
-        rows, ldx = _rows(x, d)
+        rows, ldx = _rows(x, d, self.device, what="x")
         y = out if out is not None else torch.empty((rows, d), dtype=out_dtype or x.dtype, device=x.device)
+        if _rows(y, d, self.device, rows, "out")[1] != d:
+            raise ValueError("out: rows must be contiguous")
         _check(lib().bfq_composite_forward(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(),
                                            _dt(y), d, _stream(x)), "bfq_composite_forward")
         return y
@@ -169,8 +207,10 @@ class Plan:
     def composite_inverse(self, q1: torch.Tensor, y: torch.Tensor, out_dtype=None, out=None) -> torch.Tensor:
         n1 = self._q1(q1)
         d = n1 * self.n
-        rows, ldy = _rows(y, d)
+        rows, ldy = _rows(y, d, self.device, what="y")
         x = out if out is not None else torch.empty((rows, d), dtype=out_dtype or y.dtype, device=y.device)
+        if _rows(x, d, self.device, rows, "out")[1] != d:
+            raise ValueError("out: rows must be contiguous")
         _check(lib().bfq_composite_inverse(self._h, q1.data_ptr(), n1, y.data_ptr(), _dt(y), rows, ldy, x.data_ptr(),
                                            _dt(x), d, _stream(y)), "bfq_composite_inverse")
         return x
@@ -178,11 +218,8 @@ class Plan:
     def composite_forward_quant(self, q1: torch.Tensor, x: torch.Tensor, bits: int, codes=None, scales=None):
         n1 = self._q1(q1)
         d = n1 * self.n
-        rows, ldx = _rows(x, d)
-        if codes is None:
-            codes = torch.empty((rows, d * bits // 8), dtype=torch.uint8, device=x.device)
-        if scales is None:
-            scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        rows, ldx = _rows(x, d, self.device, what="x")
+        codes, scales = self._outputs(rows, d, bits, codes, scales)
         _check(lib().bfq_composite_forward_quant(self._h, q1.data_ptr(), n1, x.data_ptr(), _dt(x), rows, ldx, int(bits),
                                                  codes.data_ptr(), scales.data_ptr(), _stream(x)),
                "bfq_composite_forward_quant")
@@ -190,9 +227,8 @@ class Plan:
 
     def forward_quant_stats(self, x: torch.Tensor, bits: int):
         """-> (codes, scales, hist int64 [2^bits], rowstats fp32 [rows][2] = (sum y^2, sum y^4))."""
-        rows, ldx = _rows(x, self.n)
-        codes = torch.empty((rows, self.n * bits // 8), dtype=torch.uint8, device=x.device)
-        scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        rows, ldx = _rows(x, self.n, self.device, what="x")
+        codes, scales = self._outputs(rows, self.n, bits, None, None)
         hist = torch.empty((1 << bits,), dtype=torch.int64, device=x.device)
         rowstats = torch.empty((rows, 2), dtype=torch.float32, device=x.device)
         _check(lib().bfq_forward_quant_stats(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
@@ -201,49 +237,48 @@ class Plan:
         return codes, scales, hist, rowstats
 
     def hadamard(self, x: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
-        rows, ldx = _rows(x, self.n)
+        rows, ldx = _rows(x, self.n, self.device, what="x")
         y = out if out is not None else torch.empty((rows, self.n), dtype=out_dtype or x.dtype, device=x.device)
-        _, ldy = _rows(y, self.n)
+        _, ldy = _rows(y, self.n, self.device, rows, "out")
         _check(lib().bfq_hadamard(self._h, x.data_ptr(), _dt(x), rows, ldx, y.data_ptr(), _dt(y), ldy, _stream(x)),
                "bfq_hadamard")
         return y
 
     def hadamard_quant(self, x: torch.Tensor, bits: int, codes=None, scales=None):
-        rows, ldx = _rows(x, self.n)
-        if codes is None:
-            codes = torch.empty((rows, self.n * bits // 8), dtype=torch.uint8, device=x.device)
-        if scales is None:
-            scales = torch.empty((rows,), dtype=torch.float16, device=x.device)
+        rows, ldx = _rows(x, self.n, self.device, what="x")
+        codes, scales = self._outputs(rows, self.n, bits, codes, scales)
         _check(lib().bfq_hadamard_quant(self._h, x.data_ptr(), _dt(x), rows, ldx, int(bits), codes.data_ptr(),
                                         scales.data_ptr(), _stream(x)), "bfq_hadamard_quant")
         return codes, scales
 
     def inverse(self, y: torch.Tensor, out_dtype=None, out: torch.Tensor | None = None) -> torch.Tensor:
-        rows, ldy = _rows(y, self.n)
+        rows, ldy = _rows(y, self.n, self.device, what="y")
         x = out if out is not None else torch.empty((rows, self.n), dtype=out_dtype or y.dtype, device=y.device)
-        _, ldx = _rows(x, self.n)
+        _, ldx = _rows(x, self.n, self.device, rows, "out")
         _check(lib().bfq_inverse(self._h, y.data_ptr(), _dt(y), rows, ldy, x.data_ptr(), _dt(x), ldx, _stream(y)),
                "bfq_inverse")
         return x
 
     def backward(self, x: torch.Tensor, g: torch.Tensor, dx_dtype=None, want_dx: bool = True, dx=None, dtheta=None):
-        rows, ld = _rows(x, self.n)
-        rows_g, ld_g = _rows(g, self.n)
+        rows, ld = _rows(x, self.n, self.device, what="x")
+        rows_g, ld_g = _rows(g, self.n, self.device, what="g")
         if rows_g != rows or ld_g != ld:
             raise ValueError("x and g must have the same shape and row stride")
         if want_dx and dx is None:
             dx = torch.empty_strided((rows, self.n), (ld, 1), dtype=dx_dtype or x.dtype, device=x.device)
+        if want_dx and _rows(dx, self.n, self.device, rows, "dx")[1] != ld:
+            raise ValueError("dx must have the row stride of x")
         if dtheta is None:
             dtheta = torch.empty((self.L, self.n // 2), dtype=torch.float32, device=x.device)
+        _exact(dtheta, torch.float32, (self.L, self.n // 2), self.device, "dtheta")
         _check(lib().bfq_backward(self._h, x.data_ptr(), _dt(x), g.data_ptr(), _dt(g), rows, ld,
                                   dx.data_ptr() if want_dx else None, _dt(dx) if want_dx else BFQ_F32,
                                   dtheta.data_ptr(), _stream(x)), "bfq_backward")
         return (dx if want_dx else None), dtheta
 
     def fold_weights(self, W: torch.Tensor, bits: int, want_rotated: bool = False, rotated_dtype=None):
-        m, ldw = _rows(W, self.n)
-        codes = torch.empty((m, self.n * bits // 8), dtype=torch.uint8, device=W.device)
-        scales = torch.empty((m,), dtype=torch.float16, device=W.device)
+        m, ldw = _rows(W, self.n, self.device, what="W")
+        codes, scales = self._outputs(m, self.n, bits, None, None)
         rot = torch.empty((m, self.n), dtype=rotated_dtype or W.dtype, device=W.device) if want_rotated else None
         _check(lib().bfq_fold_weights(self._h, W.data_ptr(), _dt(W), m, ldw, int(bits), codes.data_ptr(),
                                       scales.data_ptr(), rot.data_ptr() if rot is not None else None,
@@ -252,6 +287,16 @@ class Plan:
 
     def device_status(self) -> int:
         return int(lib().bfq_device_status(self._h))
+
+    def stage_form(self) -> int:
+        """bit 0 / bit 1: the forward / inverse tables of the tuned kernels use the three-shear fallback."""
+        r = int(lib().bfq_stage_form(self._h))
+        if r < 0:
+            raise BfqError(r, "bfq_stage_form")
+        return r
+
+    def test_stuck_wait(self, enable: bool):
+        _check(lib().bfq_test_stuck_wait(self._h, int(bool(enable))), "bfq_test_stuck_wait")
 
     def backward_partials(self) -> int:
         return int(lib().bfq_backward_partials(self._h))
@@ -263,16 +308,33 @@ def backward_noalloc(theta: torch.Tensor, x: torch.Tensor, g: torch.Tensor, dx: 
     library (for hosts that must not call cudaMalloc; row length at most 1024).  Every buffer,
     outputs included, is the caller's; pass dx=None to skip dL/dx.  Runs on x's device, which is
     made current for the call.  Calls share one fixed scratch array per GPU: do not overlap them."""
+    if not isinstance(x, torch.Tensor) or x.dim() != 2 or not x.is_cuda:
+        raise ValueError("x must be a [rows][n] CUDA tensor")
     n = x.shape[1]
-    rows, ld = _rows(x, n)
-    rows_g, ld_g = _rows(g, n)
+    L = n.bit_length() - 1
+    if n < 16 or (1 << L) != n:
+        raise ValueError("n must be a power of two >= 16")
+    rows, ld = _rows(x, n, x.device, what="x")
+    rows_g, ld_g = _rows(g, n, x.device, what="g")
     if rows_g != rows or ld_g != ld:
         raise ValueError("x and g must have the same shape and row stride")
-    if dx is not None and _rows(dx, n) != (rows, ld):
+    if dx is not None and _rows(dx, n, x.device, rows, "dx") != (rows, ld):
         raise ValueError("dx must have the shape and row stride of x")
+    _exact(theta, torch.float32, (L, n // 2), x.device, "theta")
+    _exact(dtheta, torch.float32, (L, n // 2), x.device, "dtheta")
     with torch.cuda.device(x.device):
         _check(lib().bfq_backward_noalloc(n, theta.data_ptr(), x.data_ptr(), _dt(x), g.data_ptr(), _dt(g), rows, ld,
                                           dx.data_ptr() if dx is not None else None,
                                           _dt(dx) if dx is not None else BFQ_F32, dtheta.data_ptr(), _stream(x)),
                "bfq_backward_noalloc")
     return dx, dtheta
+
+
+def measure_fma_rates(device=None):
+    """bfq_measure_fma_rates on `device` (default: the current one): SM cycles per FMA instruction per scheduler for
+    (packed, three register operands), (packed, two), (scalar, three), (scalar, two)."""
+    out = (ctypes.c_float * 4)()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        _check(lib().bfq_measure_fma_rates(ctypes.cast(out, ctypes.c_void_p)), "bfq_measure_fma_rates")
+    return {"packed_3reg": out[0], "packed_2reg": out[1], "scalar_3reg": out[2], "scalar_2reg": out[3]}

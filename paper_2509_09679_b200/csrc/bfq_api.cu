@@ -570,6 +570,24 @@ int bfq_device_status(bfq_plan* plan) {
 
 int bfq_last_cuda_error(const bfq_plan* plan) { return plan == nullptr ? 0 : plan->last_cuda_error; }
 
+int bfq_test_stuck_wait(bfq_plan* plan, int enable) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    plan->test_stuck_wait = enable != 0;
+    return BFQ_OK;
+}
+
+int bfq_stage_form(bfq_plan* plan) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    if (plan->form_flag == nullptr || !plan->angles_set) return BFQ_ERR_WORKSPACE;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaError_t e = cudaDeviceSynchronize();
+    int words[2] = {0, 0};
+    if (e == cudaSuccess) e = cudaMemcpy(words, plan->form_flag, sizeof(words), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(plan, e);
+    return (words[0] != 0 ? 1 : 0) | (words[1] != 0 ? 2 : 0);
+}
+
 int bfq_backward_partials(const bfq_plan* plan) { return plan == nullptr ? 0 : plan->last_backward_partials; }
 
 const char* bfq_status_string(int status) {

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, const int* __restrict__ form,
            uint8_t* __restrict__ codes,
            uint16_t* __restrict__ scales, __nv_bfloat16* __restrict__ yout, int64_t ldy, int rows,
-           int* __restrict__ status) {
+           int* __restrict__ status, uint32_t tx_bytes, int wait_limit) {
     using S = Smem<G, XB>;
     constexpr bool kTmem = TRANSFORM == kButterfly;
     constexpr float kPost = TRANSFORM == kHadamard ? 1.0f / 64.0f : 1.0f;  // 1/sqrt(4096), exact
@@ -265,7 +265,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     // first rows of this group
     if (t == 0) {
         for (int k = 0; k < kInSlots && k < count; ++k) {
-            mbar_expect_tx(bar_base + 8 * k, kRowBytes);
+            mbar_expect_tx(bar_base + 8 * k, tx_bytes);
             tma_load_3d(in_base + k * kRowBytes, &tmap, 0, 0, first + k * stride, bar_base + 8 * k);
         }
     }
@@ -321,7 +321,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         const int row = first + k * stride;
         const int slot = k & 1;
         if constexpr (kTmem) tmem_ld(tlane, T0);
-        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status, wait_limit);
         const uint32_t src = in_base + slot * kRowBytes + in_line;
         {
             // run (h, c) holds elements 8c..8c+7 of half h; element m of half h is half h of P[m]
@@ -343,7 +343,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         }
         auto issue_next = [&]() {
             if (t == 0 && k + kInSlots < count) {
-                mbar_expect_tx(bar_base + 8 * slot, kRowBytes);
+                mbar_expect_tx(bar_base + 8 * slot, tx_bytes);
                 tma_load_3d(in_base + slot * kRowBytes, &tmap, 0, 0, first + (k + kInSlots) * stride,
                             bar_base + 8 * slot);
             }
@@ -686,9 +686,13 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
     }
     const int64_t want = (rows + G - 1) / G;
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
+    // bytes a row's load is expected to deliver and the bound on polls of its barrier; the test hook announces more
+    // bytes than arrive, so that every wait runs out (quickly) and reports through the status word
+    const uint32_t tx_bytes = f4k::kRowBytes + (plan->test_stuck_wait ? 16u : 0u);
+    const int wait_limit = plan->test_stuck_wait ? 4096 : (1 << 22);
     return launch_overlapped(kern, dim3(grid), dim3(G * f4k::kGroupThreads), S::kBytes, st, tmap, plan->img4096,
                              plan->form_flag, codes, scales, static_cast<__nv_bfloat16*>(y), ldy, int(rows),
-                             plan->status_word);
+                             plan->status_word, tx_bytes, wait_limit);
 }
 
 // Four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest among the

@@ -57,3 +57,53 @@ def test_validation_that_precedes_any_cuda_call(lib):
     assert lib.bfq_backward_noalloc(2048, None, None, 0, None, 0, 0, 2048, None, 0, None, None) == -10
     assert lib.bfq_backward_noalloc(100, None, None, 0, None, 0, 0, 100, None, 0, None, None) == -2
     assert lib.bfq_backward_noalloc(256, None, None, 0, None, 0, 0, 256, None, 0, None, None) == -1
+
+
+def _planless(n=256):
+    """A Plan object without a device handle: every check below must raise before the library is reached."""
+    import torch
+
+    p = object.__new__(binding.Plan)
+    p.n, p.L, p.device, p._h = n, n.bit_length() - 1, torch.device("cuda", 0), ctypes.c_void_p()
+    return p
+
+
+def test_binding_rejects_bad_tensors_before_any_launch(monkeypatch):
+    import torch
+
+    def no_library():
+        raise AssertionError("a bad tensor reached the C ABI")
+
+    monkeypatch.setattr(binding, "lib", no_library)
+    p = _planless(256)
+    x = torch.zeros((4, 256))
+    with pytest.raises(ValueError, match="is on cpu"):
+        p.forward_quant(x, 4)                                   # host tensor
+    with pytest.raises(ValueError, match="is on cpu"):
+        p.backward(x, x)
+    with pytest.raises(ValueError):
+        p.forward(torch.zeros((4, 128)))                        # wrong row length
+    with pytest.raises(ValueError):
+        p.forward(torch.zeros((4, 512))[:, ::2])                # inner stride 2
+    with pytest.raises(ValueError):
+        p.set_angles(torch.zeros((8, 64)))                      # theta of a smaller n
+    with pytest.raises(ValueError):
+        p.set_angles(torch.zeros((8, 128), dtype=torch.float64))
+    with pytest.raises(ValueError, match="bits"):
+        p._outputs(4, 256, 3, None, None)
+    # caller-supplied outputs: exact dtype and shape, checked before the device
+    with pytest.raises(ValueError, match="codes"):
+        p._outputs(4, 256, 4, torch.zeros((4, 64), dtype=torch.uint8), torch.zeros((4,), dtype=torch.float16))
+    with pytest.raises(ValueError, match="scales: expected"):
+        binding._exact(torch.zeros((3,), dtype=torch.float16), torch.float16, (4,), p.device, "scales")
+    with pytest.raises(ValueError, match="codes: tensor is on cpu"):
+        p._outputs(4, 256, 4, torch.zeros((4, 128), dtype=torch.uint8), torch.zeros((4,), dtype=torch.float16))
+    with pytest.raises(ValueError, match="codes"):
+        p._outputs(4, 256, 4, torch.zeros((4, 128), dtype=torch.int8), torch.zeros((4,), dtype=torch.float16))
+    # the plan-less entry point sizes theta and dtheta from x
+    with pytest.raises(ValueError):
+        binding.backward_noalloc(torch.zeros((8, 128)), x, x, None, torch.zeros((8, 128)))
+    with pytest.raises(ValueError):
+        binding._rows(torch.zeros((4, 300)).as_strided((4, 256), (100, 1)), 256)   # overlapping rows
+    with pytest.raises(ValueError, match="expected 4 rows"):
+        binding._rows(torch.zeros((5, 256)), 256, None, 4, "out")

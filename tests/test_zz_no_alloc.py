@@ -1,4 +1,4 @@
-"""bfq_backward_noalloc against bfq_backward.
+"""bfq_backward_noalloc against bfq_backward and against the CPU oracle.
 
 The no-allocation entry point serves hosts that cannot let the library call cudaMalloc (all device
 memory owned by a caching allocator, or no tolerance for the device-wide synchronisation an
@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2509_09679_b200 import BfqError, Plan, backward_noalloc, synth
 from parity import check_dtheta, check_rows_close, to_f64
 
@@ -37,6 +38,11 @@ def _check_against_plan(n, rows, dtype, seed):
     check_rows_close(dx, to_f64(dx_ref), np.abs(to_f64(g)).max(axis=1), f"noalloc dx n={n}")
     # d-theta is summed over a different number of CTAs: the d-theta tolerance of the parity tests
     check_dtheta(dth, to_f64(dth_ref), f"noalloc dtheta n={n}")
+    # and against the oracle itself (at these sizes both paths run the same generic kernel: comparing them with each
+    # other alone would compare the kernel with itself)
+    dx_o, dth_o = oracle.backward(to_f64(theta), to_f64(x), to_f64(g))
+    check_rows_close(dx, dx_o, np.abs(to_f64(g)).max(axis=1), f"noalloc dx vs oracle n={n}")
+    check_dtheta(dth, dth_o, f"noalloc dtheta vs oracle n={n}")
     # reproducible from call to call
     dth2 = torch.empty_like(dth)
     backward_noalloc(theta, x, g, None, dth2)
@@ -46,6 +52,13 @@ def _check_against_plan(n, rows, dtype, seed):
 def test_two_calls_in_a_row_match_the_plan_based_backward():
     _check_against_plan(1024, 777, torch.bfloat16, 301)
     _check_against_plan(256, 1500, torch.float32, 302)  # smaller n right after: stale scratch must not matter
+
+
+def test_fewer_partial_sums_after_more():
+    """A long batch fills every partial-sum slot the grid cap allows; the short batch right after uses (and must zero
+    and reduce) only a few of them, whatever the first call left in the others."""
+    _check_against_plan(1024, 6000, torch.bfloat16, 305)
+    _check_against_plan(1024, 9, torch.bfloat16, 306)
 
 
 def test_limits_and_empty_batch():
