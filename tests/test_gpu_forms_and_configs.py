@@ -78,8 +78,8 @@ def test_rotation_forms_n8192(kind):
         codes, scales = p.forward_quant(x.to(DEV), bits)
         check_quant(codes, scales, y_ref, bits, f"{kind} n=8192 INT{bits}")
     check_rows_close(p.forward(x.to(DEV)), y_ref, absmax_rows(x), f"{kind} n=8192 bf16 rows")
-    # thirteen stages: |tan| = 33 everywhere already leaves the range (0.03^12 < 2^-64)
-    assert (p.stage_form() & 1) == (1 if kind in ("steep", "singular") else 0)
+    # twelve scaled stages per half (the thirteenth is a general 2x2): 0.03^12 = 2^-60.7 is still in range
+    assert (p.stage_form() & 1) == (1 if kind == "singular" else 0)
     assert p.device_status() == 0
 
 
