@@ -159,9 +159,9 @@ class Plan:
         return y
 
     def _outputs(self, rows: int, width: int, bits: int, codes, scales):
-        """Allocates or checks the codes uint8 [rows][width * bits / 8] and scales fp16 [rows] buffers."""
-        if bits not in (2, 4, 8):
-            raise ValueError("bits must be 2, 4 or 8")
+        """Allocates or checks the codes uint8 [rows][width * bits / 8] and scales fp16 [rows] buffers (the bit width
+        itself is the C side's to reject, before any launch)."""
+        bits = int(bits)
         if codes is None:
             codes = torch.empty((rows, width * bits // 8), dtype=torch.uint8, device=self.device)
         if scales is None:

@@ -89,8 +89,6 @@ def test_binding_rejects_bad_tensors_before_any_launch(monkeypatch):
         p.set_angles(torch.zeros((8, 64)))                      # theta of a smaller n
     with pytest.raises(ValueError):
         p.set_angles(torch.zeros((8, 128), dtype=torch.float64))
-    with pytest.raises(ValueError, match="bits"):
-        p._outputs(4, 256, 3, None, None)
     # caller-supplied outputs: exact dtype and shape, checked before the device
     with pytest.raises(ValueError, match="codes"):
         p._outputs(4, 256, 4, torch.zeros((4, 64), dtype=torch.uint8), torch.zeros((4,), dtype=torch.float16))
