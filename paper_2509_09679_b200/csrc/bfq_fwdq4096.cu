@@ -122,22 +122,6 @@ __device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
     for (int m = 0; m < 16; ++m) P[m] = lds64(ex.r2 + ex2_rd_local(m));
 }
 
-// The FP32 pipes and the shared-memory pipe are both heavily used; left alone, the row groups drift into step (all
-// rotating, then all regrouping) and the pipes take turns idling.  The groups therefore pass tokens around: a group
-// rotates (one phase of four stages) only while it holds a token and hands it on when it starts a regrouping or its
-// epilogue, so that some groups' rotations overlap the others' memory phases.  A token is a named barrier per group:
-// 128 arrivals from the previous holder + the 128 waiting threads.
-struct Turn {
-    int wait_id, pass_id;  // named barriers: this group's, the next group's in the ring
-    bool on;
-    __device__ __forceinline__ void acquire() const {
-        if (on) bar_sync(wait_id, 2 * kGroupThreads);
-    }
-    __device__ __forceinline__ void pass() const {
-        if (on) bar_arrive(pass_id, 2 * kGroupThreads);
-    }
-};
-
 // Chunk C is in Tcur (load already issued); the load of chunk C+1 is issued right after the wait so
 // that exactly one tensor-memory load is in flight while chunk C is being used.  `issue_next` runs
 // once per row, after the second regrouping's barrier (all reads of the input slot are done by then).
@@ -191,8 +175,6 @@ enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutIn
 // no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy), or
 // codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]), or
 // INT2 / INT8 codes + scales.
-constexpr int kTurnBar0 = 8;  // named barriers 8 .. 8 + G - 1 carry the tokens (1 .. G are the groups' own)
-
 // STEP: group g passes its token to group (g + STEP) % G, so gcd(STEP, G) groups rotate at a time (0: no tokens).
 template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)

@@ -71,7 +71,8 @@ __device__ __forceinline__ void regroup2(u64 (&P)[16], const ExAddr& ex) {
 // the first half of this rank's stage-12 constants) is requested right after the wait
 template <int FORM, int C, class F>
 __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[32], uint32_t (&Tnext)[32], uint32_t tbase,
-                                           const ExAddr& ex, F&& issue_next) {
+                                           const ExAddr& ex, const Turn& turn, F&& issue_next) {
+    if constexpr (C == 0 || C == 4 || C == 8) turn.acquire();
     tmem_wait_ld32(Tcur);
     tmem_ld32(tbase + 32 * (C + 1), Tnext);
     if constexpr (FORM == kFormScaled) {
@@ -79,12 +80,17 @@ __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[32], u
     } else {
         stage_lift<C & 3, 0, 8, 32>(P, Tcur);
     }
-    if constexpr (C == 3) regroup1(P, ex);
+    if constexpr (C == 3) {
+        turn.pass();
+        regroup1(P, ex);
+    }
     if constexpr (C == 7) {
+        turn.pass();
         regroup2(P, ex);
         issue_next();
     }
-    if constexpr (C + 1 < 12) run_chunks<FORM, C + 1>(P, Tnext, Tcur, tbase, ex, issue_next);
+    if constexpr (C == 11) turn.pass();  // before the exchange with the peer CTA: no group waits on it with a token in hand
+    if constexpr (C + 1 < 12) run_chunks<FORM, C + 1>(P, Tnext, Tcur, tbase, ex, turn, issue_next);
 }
 
 // stage 12 on four (lower-half, upper-half) register pairs: out_lo = k1*a + k2*b, out_hi = k3*a + k4*b
@@ -118,7 +124,8 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
 // BITS = 2 (the tuned workload), 4 or 8: only the epilogue differs.  BITS = 16: the rotated rows themselves in bf16
 // (`codes` then points to them, leading dimension ldy); the absmax hand-shake between the two CTAs is kept, since it is
 // also what tells a CTA that its peer has read the exchange box of the row.
-template <int G, int BITS>
+// STEP: token passing between the row groups of a CTA as in the n = 4096 kernel (0: none).
+template <int G, int BITS, int STEP = 2>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
            const float* __restrict__ img, const int* __restrict__ form, uint8_t* __restrict__ codes,
@@ -134,6 +141,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
 
     const uint32_t bar_in = sbase + S::kBarOff + 8 * g * (kInSlots + 2);  // [kInSlots] TMA, then swap, then absmax
     const uint32_t bar_swap = bar_in + 8 * kInSlots, bar_amax = bar_swap + 8;
+    grid_dep_launch();
     if (warp == 0) tmem_alloc512(sbase + S::kTmemOff);
     if (t == 0) {
         for (int k = 0; k < kInSlots; ++k) mbar_init(bar_in + 8 * k, 1);
@@ -145,14 +153,25 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     __syncthreads();
     tmem_fence_after();
     cluster_sync_all();  // the peer's barriers exist before anything arrives on them
+    grid_dep_wait();     // everything above overlaps the end of the kernel before this one
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
     const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 
+    // row r belongs to group (r / n_clusters) % G of cluster r % n_clusters
     const int n_clusters = gridDim.x >> 1;
-    const int first = (blockIdx.x >> 1) * G + g;
+    const int first = g * n_clusters + (blockIdx.x >> 1);
     const int stride = n_clusters * G;
     const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
+    // rows of group 0, the largest count of the CTA: every group takes that many turns with a token
+    const int turns = static_cast<int>(blockIdx.x >> 1) < rows ? (rows - (blockIdx.x >> 1) + stride - 1) / stride : 0;
+    static_assert(STEP >= 0 && (STEP == 0 || G % STEP == 0), "the rings must have equal length");
+    constexpr int kRings = STEP == 0 ? 1 : STEP;
+    Turn turn;
+    turn.on = STEP > 0;
+    turn.wait_id = kTurnBar0 + g;
+    turn.pass_id = kTurnBar0 + (g + STEP) % G;
+    const bool seeds_ring = (g + STEP) % G < kRings;  // this group's successor starts with the token
     const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
     const CUtensorMap* tmap = rank == 0 ? &map_lo : &map_hi;
 
@@ -228,6 +247,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     u64 P[16];
     uint32_t T0[32], T1[32];
 
+    if (seeds_ring) turn.pass();
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
         const int slot = k & 1;
@@ -251,7 +271,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
                 }
             }
         }
-        run_chunks<FORM, 0>(P, T0, T1, tlane, ex, [&]() {
+        run_chunks<FORM, 0>(P, T0, T1, tlane, ex, turn, [&]() {
             if (t == 0 && k + kInSlots < count) {
                 mbar_expect_tx(bar_in + 8 * slot, kRowBytes);
                 tma_load_3d(in_base + slot * kRowBytes, tmap, 0, 0, first + (k + kInSlots) * stride, bar_in + 8 * slot);
@@ -375,6 +395,12 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             out[64 * i] = static_cast<uint8_t>((t & 1) ? (got | (nh << 4)) : (nl | (got << 4)));
         }
     }
+    // a group with fewer rows than group 0 keeps the tokens moving
+    for (int k = count; k < turns; ++k) {
+#pragma unroll
+        for (int ph = 0; ph < 3; ++ph) turn.acquire(), turn.pass();
+    }
+    if (g < kRings) turn.acquire();  // each ring's first group takes its token back: no arrival stays pending
     };
     if (!shear) {
         row_loop(std::integral_constant<int, kFormScaled>());
@@ -531,13 +557,15 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
     cfg.blockDim = dim3(G * f4k::kGroupThreads, 1, 1);
     cfg.dynamicSmemBytes = S::kBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the set-up overlaps the previous kernel's tail
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192),
                               static_cast<const int*>(plan->form_flag), codes, scales, ldy, int(rows), plan->status_word);
 }

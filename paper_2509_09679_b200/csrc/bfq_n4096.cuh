@@ -80,6 +80,24 @@ __device__ __forceinline__ uint32_t bf16_lo(uint32_t w) {
     return r;
 }
 
+constexpr int kTurnBar0 = 8;  // named barriers 8 .. 8 + G - 1 carry the tokens (1 .. G are the groups' own)
+
+// The FP32 pipes and the shared-memory pipe are both heavily used; left alone, the row groups drift into step (all
+// rotating, then all regrouping) and the pipes take turns idling.  The groups therefore pass tokens around: a group
+// rotates (one phase of four stages) only while it holds a token and hands it on when it starts a regrouping or its
+// epilogue, so that some groups' rotations overlap the others' memory phases.  A token is a named barrier per group:
+// 128 arrivals from the previous holder + the 128 waiting threads.
+struct Turn {
+    int wait_id, pass_id;  // named barriers: this group's, the next group's in the ring
+    bool on;
+    __device__ __forceinline__ void acquire() const {
+        if (on) bar_sync(wait_id, 2 * kGroupThreads);
+    }
+    __device__ __forceinline__ void pass() const {
+        if (on) bar_arrive(pass_id, 2 * kGroupThreads);
+    }
+};
+
 // ---- element held by role t, packed register m, half h in each phase -----------------------------------
 //   phase 1: i = m | (t & 15) << 4 | h << 8 | (t >> 4) << 9
 //   phase 2: i = (t & 15) | m << 4 | h << 8 | (t >> 4) << 9
