@@ -1,10 +1,12 @@
 // Tuned backward pass for n = 4096 bf16 rows on sm_100a:  dx = Q^T g  and  d-theta summed over rows.
 //
 // One persistent CTA per SM works on two rows at a time (row pair p of the CTA is rows 2p, 2p+1) with two
-// groups of 128 threads: the forward group recomputes y for pair k+1 while the reverse group walks pair k
-// down; y changes hands through one shared-memory buffer.  Only the reverse group touches the d-theta
-// accumulators.  The thread roles, phases and regrouping layouts are those of the forward kernel
-// (bfq_n4096.cuh).  Per row pair:
+// groups of 128 threads.  The upper group recomputes y for a pair and takes the reverse walk through stages 11, 10
+// and 9 (which need no regrouping: their partners are in the thread's own registers); y and g then change hands through
+// shared memory and the lower group walks stages 8 .. 0 and writes dx, while the upper group is already on the next
+// pair.  The split balances the two groups' arithmetic (12 + 3 against 9 stage-equivalents of rotations, the lower
+// group also carrying both regroupings).  Each group owns the d-theta accumulators of its stages.  The thread roles,
+// phases and regrouping layouts are those of the forward kernel (bfq_n4096.cuh).  Per row pair:
 //   1. y = Q x with the three-shear constants, all 12 stages, in the tracked-sign basis sigma.
 //   2. y and g are moved to the basis sigma * (-1)^popcount(index).  Any two indices that a stage pairs
 //      differ in one bit, so in this basis the high element of every pair of every stage is negated
@@ -14,7 +16,7 @@
 //      form of g^T (dG/dtheta) z; its sign in this basis is fixed per pair and applied when the sums
 //      are written out), then y and g are both un-rotated.  After stage 0, g is dx up to the parity sign.
 // d-theta accumulators are owned by thread role (no atomics): stages 0-7 in the tensor-memory columns the
-// constants leave free, stages 8-11 in shared memory.  Each CTA walks its row pairs in a fixed order and
+// constants leave free, stages 8-11 in shared memory (stage 8 the lower group's, 9-11 the upper group's).  Each CTA walks its row pairs in a fixed order and
 // writes its sums to its own slot; a second kernel adds the slots in index order: bit-reproducible.
 #include <type_traits>
 
@@ -33,6 +35,7 @@ constexpr int kSlots = 2;                    // TMA ring depth (row pairs), x an
 constexpr int kBarRev = 1, kBarFwd = 2, kBarFull = 3, kBarEmpty = 4;  // named barriers
 constexpr int kConstCols = 384;              // 12 stages x 32 words
 constexpr int kAccCol = 384;                 // accumulators of stages 0..7: 16 columns each
+constexpr int kUpperSteps = 8;               // half-stage steps of the reverse walk done by the upper group: stages 11 .. 8
 constexpr uint32_t kPairBytes = 2 * kRowBytes;  // two bf16 rows
 constexpr int kInvCols = 416;  // scaled inverse: stages 11..1 (32 columns each, stage s at 32 (s - 1)), then stage 0 (64)
 enum : int { kFormScaled = 0, kFormShear = 1 };
@@ -40,11 +43,12 @@ enum : int { kFormScaled = 0, kFormShear = 1 };
 struct Smem {
     static constexpr uint32_t kXOff = 0;                                   // [kSlots][2][kRowBytes]
     static constexpr uint32_t kGOff = kXOff + kSlots * kPairBytes;         // [kSlots][2][kRowBytes]
-    static constexpr uint32_t kExFOff = kGOff + kSlots * kPairBytes;       // forward group: [2][kExBytes]
-    static constexpr uint32_t kExROff = kExFOff + 2 * kExBytes;            // reverse group: [4][kExBytes]: y0, y1, g0, g1
-    static constexpr uint32_t kHandOff = kExROff + 4 * kExBytes;           // y hand-off: [2 rows][16][128] packed pairs
-    static constexpr uint32_t kAccOff = kHandOff + 2 * 16 * kThreads * 8;  // [16][128] float4: stages 8..11
-    static constexpr uint32_t kBarOff = kAccOff + 16 * kThreads * 16;      // mbarriers: x ring, g ring
+    static constexpr uint32_t kExFOff = kGOff + kSlots * kPairBytes;       // upper group, forward recompute: [2][kExBytes]
+    // y0, y1, g0, g1 of a row pair in the regrouping layouts: written by the upper group after stage 8 (this is both
+    // the phase-3 -> phase-2 regrouping and the hand-off), re-used by the lower group for the regrouping after stage 4
+    static constexpr uint32_t kExROff = kExFOff + 2 * kExBytes;            // [4][kExBytes]
+    static constexpr uint32_t kAccOff = kExROff + 4 * kExBytes;            // [16][128] float4: stages 8..11
+    static constexpr uint32_t kBarOff = kAccOff + 16 * kThreads * 16;      // mbarriers, one per input slot
     static constexpr uint32_t kTmemOff = kBarOff + 8 * 2 * kSlots;
     static constexpr uint32_t kUsed = kTmemOff + 16;
     static constexpr uint32_t kBytes = kUsed + 1024;
@@ -163,10 +167,11 @@ struct RevStep {
     static constexpr uint32_t kAccSmem = ((s - 8) * 4 + 2 * c) * kThreads * 16;  // stages 8..11: two float4
 };
 
-template <int I, class F>
+// steps I .. END-1 (END = 24: down to stage 0); hook(integral_constant<I>) runs after step I (regroupings, hand-off)
+template <int I, int END, class F>
 __device__ __forceinline__ void rev_steps(u64 (&Y0)[16], u64 (&Y1)[16], u64 (&G0)[16], u64 (&G1)[16],
                                           uint32_t (&Tcur)[16], uint32_t (&Tnext)[16], uint32_t (&Acur)[8],
-                                          uint32_t (&Anext)[8], const Ctx& cx, F&& after_phase3) {
+                                          uint32_t (&Anext)[8], const Ctx& cx, F&& hook) {
     using S = RevStep<I>;
     if constexpr (S::kAccInTmem) {
         tmem_wait_ld16_8(Tcur, Acur);
@@ -176,7 +181,7 @@ __device__ __forceinline__ void rev_steps(u64 (&Y0)[16], u64 (&Y1)[16], u64 (&G0
         Acur[0] = a0.x, Acur[1] = a0.y, Acur[2] = a0.z, Acur[3] = a0.w;
         Acur[4] = a1.x, Acur[5] = a1.y, Acur[6] = a1.z, Acur[7] = a1.w;
     }
-    if constexpr (I + 1 < 24) {
+    if constexpr (I + 1 < END) {
         using N = RevStep<I + 1>;
         tmem_ld16(cx.tlane + N::kTCol, Tnext);
         if constexpr (N::kAccInTmem) tmem_ld8(cx.tlane + N::kAccCol, Anext);
@@ -201,32 +206,8 @@ __device__ __forceinline__ void rev_steps(u64 (&Y0)[16], u64 (&Y1)[16], u64 (&G0
     }
     stage_lift<S::K, S::U0, 4, 16>(G0, Tcur);
     stage_lift<S::K, S::U0, 4, 16>(G1, Tcur);
-    if constexpr (I == 7) {  // phase 3 -> phase 2, across warps
-        bar_sync(cx.a.bar, kThreads);  // every warp is past its half-warp reads for the previous row pair
-        rev2_store(Y0, cx.a.ex + 0 * kExBytes, cx.a);
-        rev2_store(Y1, cx.a.ex + 1 * kExBytes, cx.a);
-        rev2_store(G0, cx.a.ex + 2 * kExBytes, cx.a);
-        rev2_store(G1, cx.a.ex + 3 * kExBytes, cx.a);
-        bar_sync(cx.a.bar, kThreads);
-        after_phase3();  // all reads of the input slot are done: the next row pair may be requested
-        rev2_load(Y0, cx.a.ex + 0 * kExBytes, cx.a);
-        rev2_load(Y1, cx.a.ex + 1 * kExBytes, cx.a);
-        rev2_load(G0, cx.a.ex + 2 * kExBytes, cx.a);
-        rev2_load(G1, cx.a.ex + 3 * kExBytes, cx.a);
-    }
-    if constexpr (I == 15) {  // phase 2 -> phase 1, inside each half-warp, but the buffers were read across warps
-        bar_sync(cx.a.bar, kThreads);
-        rev1_store(Y0, cx.a.ex + 0 * kExBytes, cx.a);
-        rev1_store(Y1, cx.a.ex + 1 * kExBytes, cx.a);
-        rev1_store(G0, cx.a.ex + 2 * kExBytes, cx.a);
-        rev1_store(G1, cx.a.ex + 3 * kExBytes, cx.a);
-        __syncwarp();
-        rev1_load(Y0, cx.a.ex + 0 * kExBytes, cx.a);
-        rev1_load(Y1, cx.a.ex + 1 * kExBytes, cx.a);
-        rev1_load(G0, cx.a.ex + 2 * kExBytes, cx.a);
-        rev1_load(G1, cx.a.ex + 3 * kExBytes, cx.a);
-    }
-    if constexpr (I + 1 < 24) rev_steps<I + 1>(Y0, Y1, G0, G1, Tnext, Tcur, Anext, Acur, cx, after_phase3);
+    hook(std::integral_constant<int, I>());
+    if constexpr (I + 1 < END) rev_steps<I + 1, END>(Y0, Y1, G0, G1, Tnext, Tcur, Anext, Acur, cx, hook);
 }
 
 __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
@@ -270,7 +251,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     cx.acc_smem = sbase + S::kAccOff + t * 16;
     {
         const uint32_t t4 = (t >> 4) & 1, t5 = (t >> 5) & 1, t6 = (t >> 6) & 1;
-        cx.a.ex = sbase + (is_fwd ? S::kExFOff : S::kExROff);
+        cx.a.ex = sbase + (is_fwd ? S::kExFOff : S::kExROff);  // the group's own regrouping buffers
         cx.a.bar = is_fwd ? kBarFwd : kBarRev;
         cx.a.w1 = 4u * (2u * (t & 15) + 32u * (t >> 4));
         cx.a.r1 = 4u * (258u * (t & 15) + 32u * (t >> 4));
@@ -282,20 +263,22 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     const int first = blockIdx.x;
     const int stride = gridDim.x;
     const int count = first < pairs ? (pairs - first + stride - 1) / stride : 0;
-    const uint32_t ring = sbase + (is_fwd ? S::kXOff : S::kGOff);                 // this group's input ring
-    const uint32_t bar_base = sbase + S::kBarOff + (is_fwd ? 0 : 8 * kSlots);     // and its mbarriers
-    const CUtensorMap* tmap = is_fwd ? &xmap : &gmap;
+    // both input rings belong to the upper group: one mbarrier per slot counts the x pair and the g pair
+    const uint32_t xring = sbase + S::kXOff, gring = sbase + S::kGOff;
+    const uint32_t bar_base = sbase + S::kBarOff;
 
     // a row index past the end is legal for the tensor map: the tile is filled with zeros
     auto request = [&](int k) {
         const int slot = k & 1;
         const int r0 = 2 * (first + k * stride);
-        const uint32_t dst = ring + slot * kPairBytes, bar = bar_base + 8 * slot;
-        mbar_expect_tx(bar, kPairBytes);
-        tma_load_3d(dst, tmap, 0, 0, r0, bar);
-        tma_load_3d(dst + kRowBytes, tmap, 0, 0, r0 + 1, bar);
+        const uint32_t bar = bar_base + 8 * slot;
+        mbar_expect_tx(bar, 2 * kPairBytes);
+        tma_load_3d(xring + slot * kPairBytes, &xmap, 0, 0, r0, bar);
+        tma_load_3d(xring + slot * kPairBytes + kRowBytes, &xmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(gring + slot * kPairBytes, &gmap, 0, 0, r0, bar);
+        tma_load_3d(gring + slot * kPairBytes + kRowBytes, &gmap, 0, 0, r0 + 1, bar);
     };
-    if (t == 0) {
+    if (is_fwd && t == 0) {
         for (int k = 0; k < kSlots && k < count; ++k) request(k);
     }
     // constants into tensor memory (each group fills half of the columns), accumulators to zero
@@ -327,24 +310,33 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     // parity of the role: popcount(t) & 1
     const uint32_t par_t = __popc(t) & 1;
     const uint32_t sgn_a = par_t ? 0x80000000u : 0u, sgn_b = par_t ? 0u : 0x80000000u;
-    const uint32_t hand = sbase + S::kHandOff + t * 8;  // + (row * 16 + m) * 1024: conflict free, same role both sides
+    const uint32_t exr = sbase + S::kExROff;  // where a row pair changes hands
 
+    u64 Y0[16], Y1[16], G0[16], G1[16];
+    uint32_t T0[16], T1[16], A0[8], A1[8];
     if (is_fwd) {
-        // =============================== forward group: y = Q x ===============================
+        // ================= upper group: y = Q x, then d-theta and the reverse walk of stages 11, 10, 9 =================
         // x tile, phase-1 ownership (as in the forward kernel)
         const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
         const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
-        u64 X0[16], X1[16];
-        uint32_t T0[16], T1[16];
+        // g tile, phase-3 ownership: the 32-bit word of elements 2t + 256m, 2t + 256m + 1 is word t & 3 of
+        // 16-byte chunk (t & 31) >> 2 of 128-byte line (t >> 5) + 4m; the swizzle moves the chunk to
+        // chunk ^ (line & 7)
+        const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
+        const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
+        const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
+        const uint4* gsv = reinterpret_cast<const uint4*>(gsign);
         for (int k = 0; k < count; ++k) {
             const int slot = k & 1;
+            // every thread of this group is past its reads of the other input slot (each iteration ends in a
+            // barrier with the lower group)
+            if (t == 0 && k >= 1 && k + 1 < count) request(k + 1);
             tmem_ld16(cx.tlane, T0);
             mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
-            const uint32_t tile = ring + slot * kPairBytes;
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-                u64(&X)[16] = r == 0 ? X0 : X1;
-                const uint32_t src = tile + r * kRowBytes + in_line;
+                u64(&X)[16] = r == 0 ? Y0 : Y1;
+                const uint32_t src = xring + slot * kPairBytes + r * kRowBytes + in_line;
                 uint4 w[2][2];
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
@@ -356,71 +348,78 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
                     const uint32_t b[4] = {w[1][c].x, w[1][c].y, w[1][c].z, w[1][c].w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        X[8 * c + 2 * j + 0] = pack2u(a[j] << 16, b[j] << 16);
+                        X[8 * c + 2 * j + 0] = pack2u(bf16_lo(a[j]), bf16_lo(b[j]));
                         X[8 * c + 2 * j + 1] = pack2u(a[j] & 0xFFFF0000u, b[j] & 0xFFFF0000u);
                     }
                 }
             }
-            fwd_chunks<0>(X0, X1, T0, T1, cx);
-            // every thread of the group read its part of the x tile before the barriers inside fwd_chunks
-            if (t == 0 && k + kSlots < count) request(k + kSlots);
-            // y to the parity basis, then hand it over once the reverse group has taken the previous pair
-            bar_sync(kBarEmpty, kCtaThreads);
+            fwd_chunks<0>(Y0, Y1, T0, T1, cx);
+            // y to the parity basis
 #pragma unroll
             for (int m = 0; m < 16; ++m) {
                 const bool odd = (__builtin_popcount(m) & 1) != 0;  // compile-time after unrolling
                 const u64 mask = odd ? pack2u(sgn_b, sgn_a) : pack2u(sgn_a, sgn_b);
-                sts64(hand + (0 * 16 + m) * 1024u, X0[m] ^ mask);
-                sts64(hand + (1 * 16 + m) * 1024u, X1[m] ^ mask);
+                Y0[m] ^= mask;
+                Y1[m] ^= mask;
             }
+            // g into the same basis
+            tmem_ld16(cx.tlane + RevStep<0>::kTCol, T0);
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                u64(&G)[16] = r == 0 ? G0 : G1;
+                const uint32_t src = gring + slot * kPairBytes + r * kRowBytes;
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
+                    const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int m = 4 * qq + i;
+                        const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
+                        G[m] = pack2u(bf16_lo(w), w & 0xFFFF0000u);
+                    }
+                }
+            }
+            rev_steps<0, kUpperSteps>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [](auto) {});
+            // phase 3 -> phase 2 regrouping = the hand-over: once the lower group is past its reads of the buffers for
+            // the previous pair, store in the layout it reads
+            bar_sync(kBarEmpty, kCtaThreads);
+            rev2_store(Y0, exr + 0 * kExBytes, cx.a);
+            rev2_store(Y1, exr + 1 * kExBytes, cx.a);
+            rev2_store(G0, exr + 2 * kExBytes, cx.a);
+            rev2_store(G1, exr + 3 * kExBytes, cx.a);
             __threadfence_block();
             bar_arrive(kBarFull, kCtaThreads);
         }
     } else {
-        // =============================== reverse group: d-theta and dx ===============================
-        // g tile, phase-3 ownership: the 32-bit word of elements 2t + 256m, 2t + 256m + 1 is word t & 3 of
-        // 16-byte chunk (t & 31) >> 2 of 128-byte line (t >> 5) + 4m; the swizzle moves the chunk to
-        // chunk ^ (line & 7)
-        const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
-        const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
-        const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
-        uint32_t gs[16];  // sign words of this role's 16 words of a g row
-        {
-            const uint4* src = reinterpret_cast<const uint4*>(gsign);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint4 v = __ldg(src + q * kThreads + t);
-                gs[4 * q] = v.x, gs[4 * q + 1] = v.y, gs[4 * q + 2] = v.z, gs[4 * q + 3] = v.w;
-            }
-        }
-        u64 Y0[16], Y1[16], G0[16], G1[16];
-        uint32_t T0[16], T1[16], A0[8], A1[8];
-        if (count > 0) bar_arrive(kBarEmpty, kCtaThreads);  // the hand-off buffer starts empty
+        // ================= lower group: stages 8 .. 0, dx =================
+        if (count > 0) bar_arrive(kBarEmpty, kCtaThreads);  // the buffers start empty (the upper group's first wait)
         for (int k = 0; k < count; ++k) {
-            const int slot = k & 1;
             const int r0 = 2 * (first + k * stride);
-            tmem_ld16(cx.tlane + 32 * 11, T0);
-            mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
-            const uint32_t tile = ring + slot * kPairBytes;
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                u64(&G)[16] = r == 0 ? G0 : G1;
-                const uint32_t src = tile + r * kRowBytes;
-#pragma unroll
-                for (int m = 0; m < 16; ++m) {
-                    const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ gs[m];
-                    G[m] = pack2u(w << 16, w & 0xFFFF0000u);
-                }
-            }
+            tmem_ld16(cx.tlane + RevStep<kUpperSteps>::kTCol, T0);
+            tmem_ld8(cx.tlane + RevStep<kUpperSteps>::kAccCol, A0);
             bar_sync(kBarFull, kCtaThreads);
-#pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                Y0[m] = lds64(hand + (0 * 16 + m) * 1024u);
-                Y1[m] = lds64(hand + (1 * 16 + m) * 1024u);
-            }
-            if (k + 1 < count) bar_arrive(kBarEmpty, kCtaThreads);  // each thread re-reads only its own words
-            rev_steps<0>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [&]() {
-                if (t == 0 && k + kSlots < count) request(k + kSlots);
+            rev2_load(Y0, exr + 0 * kExBytes, cx.a);
+            rev2_load(Y1, exr + 1 * kExBytes, cx.a);
+            rev2_load(G0, exr + 2 * kExBytes, cx.a);
+            rev2_load(G1, exr + 3 * kExBytes, cx.a);
+            rev_steps<kUpperSteps, 24>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [&](auto step) {
+                constexpr int I = decltype(step)::value;
+                if constexpr (I == 15) {  // phase 2 -> phase 1, inside each half-warp, but the buffers were read across warps
+                    bar_sync(cx.a.bar, kThreads);
+                    rev1_store(Y0, exr + 0 * kExBytes, cx.a);
+                    rev1_store(Y1, exr + 1 * kExBytes, cx.a);
+                    rev1_store(G0, exr + 2 * kExBytes, cx.a);
+                    rev1_store(G1, exr + 3 * kExBytes, cx.a);
+                    __syncwarp();
+                    rev1_load(Y0, exr + 0 * kExBytes, cx.a);
+                    rev1_load(Y1, exr + 1 * kExBytes, cx.a);
+                    rev1_load(G0, exr + 2 * kExBytes, cx.a);
+                    rev1_load(G1, exr + 3 * kExBytes, cx.a);
+                }
+                if constexpr (I == 17) {  // stage 3 has used every value of that regrouping: the buffers are free
+                    if (k + 1 < count) bar_arrive(kBarEmpty, kCtaThreads);
+                }
             });
 
             // ---- dx = parity sign * g, bf16, phase-1 ownership: two runs of 16 elements per row ----
@@ -457,6 +456,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     }
 
     // ---- this CTA's sums -> its slot of the partial sums, with the sign of the basis undone ----
+    __syncthreads();  // the upper group's sums of stages 9..11 (shared memory) are complete
     if (!is_fwd) {
         float* out = partial + static_cast<int64_t>(blockIdx.x) * (12 * (kN / 2));
         for (int s = 0; s < 12; ++s) {
