@@ -240,6 +240,31 @@ int bfq_test_stuck_wait(bfq_plan* plan, int enable);
 const char* bfq_status_string(int status);
 
 /*
+ * Dense product with on-the-fly dequantization, for the reconstruction loss of the calibration step (paper Sec. 3.4:
+ * || W x - Dequant(Quant(W B^T)) Dequant(Quant(B x)) ||^2) and its gradients:
+ *     C[i][j] = alpha * sum_{k < K} A(i, k) * B(j, k),   i < m, j < n;   C fp32, row-major, leading dimension ldc >= n.
+ * Each operand is described by (data, kind, transposed, ld, scales):
+ *   kind        BFQ_OP_F32 / BFQ_OP_BF16: rows of numbers;  BFQ_OP_CODES2 / 4 / 8: packed two's-complement codes in
+ *               the layout bfq_forward_quant writes, value = code * scale of its stored row (scales: fp16 bits, device);
+ *   transposed  0: stored [m or n][K] (the contraction runs along a stored row);  1: stored [K][m or n];
+ *   ld          leading dimension in elements (codes: in codes) >= the stored row's length; ld * element bits must be
+ *               a multiple of 128 and data 16-byte aligned.
+ * K must be a multiple of 64; m, n are arbitrary.  All pointers are device pointers.  The products run on the tensor
+ * cores in bf16 with fp32 accumulation: codes are exact, fp32 numbers are split into two bf16 terms (relative error
+ * 2^-17 per element), bf16 numbers are exact.  Asynchronous on `stream`; allocates nothing; a bounded device-side
+ * wait that runs out is reported by bfq_device_status.  Returns BFQ_OK, BFQ_ERR_NULL, BFQ_ERR_STRIDE (sizes, leading
+ * dimensions, K not a multiple of 64), BFQ_ERR_ALIGN, BFQ_ERR_DTYPE (kind) or BFQ_ERR_CUDA.
+ */
+#define BFQ_OP_F32 0
+#define BFQ_OP_BF16 1
+#define BFQ_OP_CODES2 2
+#define BFQ_OP_CODES4 4
+#define BFQ_OP_CODES8 8
+int bfq_dequant_gemm(bfq_plan* plan, int64_t m, int64_t n, int64_t k, float alpha, const void* a, int a_kind,
+                     int a_transposed, int64_t lda, const uint16_t* a_scales, const void* b, int b_kind, int b_transposed,
+                     int64_t ldb, const uint16_t* b_scales, float* c, int64_t ldc, void* stream);
+
+/*
  * Measures, on the current device, how many SM cycles one warp scheduler needs per FP32 FMA instruction with register
  * operands only (no memory traffic in the timed loops): out[0] packed fma.rn.f32x2 with three distinct register
  * operands (the pattern of a rotation with per-pair constants), out[1] packed with two distinct operands, out[2] /

@@ -40,6 +40,7 @@ SIGNATURES = {
     "bfq_status_string": (ctypes.c_char_p, [_i]),
     "bfq_backward_partials": (_i, [_p]),
     "bfq_measure_fma_rates": (_i, [_p]),
+    "bfq_dequant_gemm": (_i, [_p, _i64, _i64, _i64, ctypes.c_float, _p, _i, _i, _i64, _p, _p, _i, _i, _i64, _p, _p, _i64, _p]),
     "bfq_stage_form": (_i, [_p]),
     "bfq_test_stuck_wait": (_i, [_p, _i]),
     "bfq_backward_noalloc": (_i, [_i, _p, _p, _i, _p, _i, _i64, _i64, _p, _i, _p, _p]),
@@ -118,6 +119,26 @@ def _exact(t: torch.Tensor, dtype, shape, device, what: str):
 
 def _stream(t: torch.Tensor):
     return ctypes.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+class GemmOperand:
+    """One operand of Plan.dequant_gemm: rows of fp32 / bf16 numbers, or packed codes with the fp16 scales of their
+    stored rows; `transposed` = stored [K][rows] instead of [rows][K]."""
+
+    def __init__(self, data: torch.Tensor, scales: torch.Tensor | None = None, bits: int = 0, transposed: bool = False):
+        if data.dim() != 2 or data.stride(1) != 1:
+            raise ValueError("operand: expected a 2-D tensor with unit inner stride")
+        self.data, self.scales, self.transposed = data, scales, bool(transposed)
+        if scales is None:
+            self.kind, per = _dt(data), 1
+        else:
+            if bits not in (2, 4, 8) or data.dtype != torch.uint8:
+                raise ValueError("operand: codes are uint8 with bits in {2, 4, 8}")
+            self.kind, per = bits, 8 // bits
+            _exact(scales, torch.float16, (data.shape[0],), data.device, "operand scales")
+        stored_rows, width = data.shape[0], data.shape[1] * per
+        self.rows, self.k = (width, stored_rows) if transposed else (stored_rows, width)
+        self.ld = (data.stride(0) if stored_rows > 1 else data.shape[1]) * per
 
 
 class Plan:
@@ -284,6 +305,21 @@ class Plan:
                                       scales.data_ptr(), rot.data_ptr() if rot is not None else None,
                                       _dt(rot) if rot is not None else BFQ_F32, _stream(W)), "bfq_fold_weights")
         return codes, scales, rot
+
+    def dequant_gemm(self, a: GemmOperand, b: GemmOperand, alpha: float = 1.0, out: torch.Tensor | None = None):
+        """C[i][j] = alpha * sum_k A(i, k) B(j, k) on the tensor cores, low-bit operands dequantized on the fly -> fp32."""
+        if a.k != b.k:
+            raise ValueError(f"operands disagree on K: {a.k} and {b.k}")
+        for op, what in ((a, "A"), (b, "B")):
+            _on(op.data, self.device, what)
+        c = out if out is not None else torch.empty((a.rows, b.rows), dtype=torch.float32, device=self.device)
+        _exact(c, torch.float32, (a.rows, b.rows), self.device, "out")
+        _check(lib().bfq_dequant_gemm(self._h, a.rows, b.rows, a.k, float(alpha), a.data.data_ptr(), a.kind,
+                                      int(a.transposed), a.ld, a.scales.data_ptr() if a.scales is not None else None,
+                                      b.data.data_ptr(), b.kind, int(b.transposed), b.ld,
+                                      b.scales.data_ptr() if b.scales is not None else None, c.data_ptr(), b.rows,
+                                      _stream(c)), "bfq_dequant_gemm")
+        return c
 
     def device_status(self) -> int:
         return int(lib().bfq_device_status(self._h))
