@@ -3,8 +3,9 @@ learning-rate schedule from the identity initialisation on the reconstruction lo
 
     L_recon = mean || W x - Dequant(Quant(W B^T)) . Dequant(Quant(B x)) ||^2 .
 
-Everything that touches the butterfly runs in the bfq kernels (forward, forward + quantize, weight folding,
-backward for the angle gradient); the two dense products and the loss are plain torch.matmul calls.  The
+Everything runs in the bfq kernels: forward, forward + quantize, weight folding, backward for the angle gradient, and
+the dense products (bfq_dequant_gemm: tensor cores, the packed codes dequantized on the fly, fp32 operands split into two
+bf16 terms); only element-wise glue (the error, its square, the scaling of the gradient) is torch.  The
 quantizers are not differentiable; as usual their gradient is passed straight through (the paper does not
 say so explicitly: this is the reading taken here).  With act_bits = None activations stay unquantized
 (the paper's W2A16 setting).  Synthetic (W, x) only: the paper's models and calibration set are not here.
@@ -15,7 +16,7 @@ import math
 
 import torch
 
-from .binding import Plan
+from .binding import GemmOperand, Plan
 
 
 def unpack_codes(codes: torch.Tensor, bits: int) -> torch.Tensor:
@@ -50,21 +51,26 @@ class LayerCalibrator:
         self.plan.set_angles(self.theta)
 
     def loss_and_grad(self, x: torch.Tensor):
-        """x: [tokens][n] calibration rows (same dtype as W).  Returns (loss, dL/dtheta)."""
-        p, W = self.plan, self.W
-        ref = x.to(torch.float32) @ W.to(torch.float32).t()                       # W x, the target
-        w_codes, w_scales, Wr = p.fold_weights(W, self.weight_bits, want_rotated=True, rotated_dtype=torch.float32)
-        Wq = dequantize(w_codes, w_scales, self.weight_bits)                     # Dequant(Quant(W B^T))
+        """x: [tokens][n] calibration rows (same dtype as W); tokens and the layer's output width must be multiples
+        of 64 (the K block of the dense products).  Returns (loss, dL/dtheta)."""
+        p, W, wb = self.plan, self.W, self.weight_bits
+        ref = p.dequant_gemm(GemmOperand(x), GemmOperand(W))                      # W x, the target
+        w_codes, w_scales, _ = p.fold_weights(W, wb)                              # Quant(W B^T), codes + scales
+        Wq = GemmOperand(w_codes, w_scales, wb)
         if self.act_bits is None:
-            yq = p.forward(x, out_dtype=torch.float32)                           # B x, kept in 16+ bits
+            y = p.forward(x)                                                      # B x, kept in 16+ bits
+            Yq, YqT = GemmOperand(y), GemmOperand(y, transposed=True)
         else:
-            a_codes, a_scales = p.forward_quant(x, self.act_bits)
-            yq = dequantize(a_codes, a_scales, self.act_bits)                    # Dequant(Quant(B x))
-        err = yq @ Wq.t() - ref
+            a_codes, a_scales = p.forward_quant(x, self.act_bits)                 # Quant(B x)
+            Yq = GemmOperand(a_codes, a_scales, self.act_bits)
+            YqT = GemmOperand(a_codes, a_scales, self.act_bits, transposed=True)
+        err = p.dequant_gemm(Yq, Wq) - ref                                        # [tokens][out]
         loss = (err * err).mean()
-        k = 2.0 / err.numel()
-        g_y = (k * err) @ Wq                  # dL/d(B x), straight through the activation quantizer
-        g_w = (k * err).t() @ yq              # dL/d(W B^T), straight through the weight quantizer
+        e = err * (2.0 / err.numel())
+        # dL/d(B x) = e Wq and dL/d(W B^T) = e^T yq, straight through the two quantizers: the contraction runs across
+        # the stored rows of the codes (their scales vary along it) and of e
+        g_y = p.dequant_gemm(GemmOperand(e), GemmOperand(w_codes, w_scales, wb, transposed=True))
+        g_w = p.dequant_gemm(GemmOperand(e, transposed=True), YqT)
         # row i of W B^T is B w_i: both gradients flow through the same transform, one on the activation rows
         # and one on the weight rows
         _, dth_x = p.backward(x, g_y.to(x.dtype), want_dx=False)
