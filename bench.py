@@ -551,6 +551,44 @@ def time_others(torch, synth, Plan, dev):
             res[name + suffix] = {"rows_per_s": rows / (ms * 1e-3), "ms": ms, "gbs": gbs,
                                   "hbm_frac": gbs / measured_peaks()["hbm_gbs"], "rows": rows, "n": 5120}
     os.environ.pop("BFQ_COMPOSITE_FP32_BUTTERFLY", None)
+    del planc, q1, x, codes, scales, y
+    torch.cuda.empty_cache()
+    # layer-calibration step (reconstruction loss + angle gradient) on a 4096 x 4096 layer, 2048 tokens, 4-bit weights and
+    # activations, and its dense products alone (bfq_dequant_gemm; TFLOP/s counts 2 m n k once, whatever the number of
+    # bf16 terms an operand is split into)
+    from paper_2509_09679_b200 import GemmOperand
+    from paper_2509_09679_b200.calibrate import LayerCalibrator
+
+    n, out, tokens = 4096, 4096, 2048
+    W = synth.rows(out, n, "normal", 7001, scale=0.02, dtype=torch.bfloat16).to(dev)
+    X = synth.rows(tokens, n, "student_t3", 7002, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16).to(dev)
+    cal = LayerCalibrator(W, 4, 4, theta=synth.angles(n, "normal", 7003, dev) * 0.1)
+    for _ in range(2):
+        cal.loss_and_grad(X)
+    ms = event_time_ms(torch, lambda: cal.loss_and_grad(X), 5)
+    res["calibration_step_n4096_w4a4"] = {"ms": ms, "tokens": tokens, "out": out, "n": n, "tokens_per_s": tokens / (ms * 1e-3)}
+    p = cal.plan
+    wc, ws, _ = p.fold_weights(W, 4)
+    ac, asc = p.forward_quant(X, 4)
+    e = torch.randn((tokens, out), device=dev)
+    peak = None
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak = float(json.load(f)["bf16_tflops"])
+    except (OSError, KeyError, ValueError):
+        pass
+    gemms = (("dequant_gemm_codes_x_codes", lambda: p.dequant_gemm(GemmOperand(ac, asc, 4), GemmOperand(wc, ws, 4)), tokens, out, n),
+             ("dequant_gemm_f32_x_codesT", lambda: p.dequant_gemm(GemmOperand(e), GemmOperand(wc, ws, 4, transposed=True)), tokens, n, out),
+             ("dequant_gemm_f32T_x_codesT", lambda: p.dequant_gemm(GemmOperand(e, transposed=True), GemmOperand(ac, asc, 4, transposed=True)), out, n, tokens))
+    for name, fn, m_, n_, k_ in gemms:
+        for _ in range(2):
+            fn()
+        ms = event_time_ms(torch, fn, 10)
+        tf = 2.0 * m_ * n_ * k_ / (ms * 1e-3) / 1e12
+        res[name] = {"ms": ms, "m": m_, "n": n_, "k": k_, "tflops": tf,
+                     "tensor_frac": None if peak is None else tf / peak}
+    if p.device_status() != 0:
+        raise SystemExit("device status after the calibration legs")
     return res
 
 

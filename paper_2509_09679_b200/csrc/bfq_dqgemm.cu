@@ -5,15 +5,15 @@
 // [K][rows].  This covers the three products of the reconstruction loss (paper Sec. 3.4):
 //     Dequant(Quant(B x)) . Dequant(Quant(W B^T))^T,   err . Dequant(Quant(W B^T)),   err^T . Dequant(Quant(B x)).
 //
-// One CTA per 128 x 128 tile of C.  Four producer warps build the operand tiles of a 64-wide K block in shared memory
-// in the K-major, 128-byte-swizzled layout the tensor core reads (thread = tile row), as 1 or 2 bf16 terms each:
+// One CTA per 128 x 128 tile of C.  Eight producer warps build the operand tiles of a 64-wide K block in shared memory
+// in the K-major, 128-byte-swizzled layout the tensor core reads (thread = tile row of A or of B), as 1 or 2 bf16 terms:
 //   * codes contracted along their stored row: the integer codes are exact in bf16 (one term); the row scale multiplies
 //     the finished row / column of C;
 //   * codes contracted across stored rows (transposed): code x scale has at most 14 significant bits: hi + lo, exact;
 //   * fp32 numbers: hi + lo = 16 significant bits (relative error 2^-17 per element); bf16 numbers: one term, exact.
 // One thread issues tcgen05.mma (kind::f16, M = N = 128, fp32 accumulators in tensor memory) for every pair of terms
 // and commits to the stage's "empty" mbarrier; two stages.  The producer warps then read the accumulators back
-// (tcgen05.ld, a lane quarter each), apply alpha and the row / column scales and store fp32 rows of C.  Every wait is
+// (tcgen05.ld, a lane quarter and half of the columns each), apply alpha and the row / column scales and store fp32 rows of C.  Every wait is
 // bounded and reports through the plan's status word.
 #include "../../include/bfq.h"
 
@@ -32,7 +32,7 @@ using namespace ptx;
 constexpr int kTile = 128;       // rows of A and of B per CTA
 constexpr int kKB = 64;          // K block: one 128-byte swizzle atom of bf16
 constexpr int kStages = 2;
-constexpr int kProducers = 128;  // threads 0..127 build tiles and run the epilogue; thread 128 issues the MMAs
+constexpr int kProducers = 256;  // threads 0..127 build A's tile rows, 128..255 B's; all run the epilogue; thread 256 issues the MMAs
 constexpr uint32_t kTileBytes = kTile * kKB * 2;  // one bf16 term of one operand: 16 KB
 constexpr int kWaitLimit = 1 << 24;
 
@@ -238,28 +238,25 @@ __global__ void __launch_bounds__(kProducers + 32, 1) k_dequant_gemm(const Param
     bool ok = true;
 
     if (tid < kProducers) {
-        // ---- producers: thread = tile row of A and of B ----
-        const int ra = m0 + tid, rb = n0 + tid;
+        // ---- producers: thread = one tile row of A (threads 0..127) or of B (128..255) ----
+        const bool for_a = tid < kTile;
+        const int r = tid & (kTile - 1);
+        const Operand& op = for_a ? p.a : p.b;
+        const int row = (for_a ? m0 : n0) + r;
+        const int terms = for_a ? ta : tb;
         float v[kKB];
         for (int kb = 0; kb < kblocks && ok; ++kb) {
             const int s = kb & 1;
             if (kb >= kStages) ok = wait_bounded(bar_empty + 8 * s, ((kb >> 1) - 1) & 1, p.status);
             if (!ok) break;
-            const uint32_t at = sbase + s * stage_bytes, bt = at + ta * kTileBytes;
-            if (ra < p.a.rows) {
-                load_row(p.a, ra, kb * kKB, v);
+            const uint32_t tile = sbase + s * stage_bytes + (for_a ? 0u : ta * kTileBytes);
+            if (row < op.rows) {
+                load_row(op, row, kb * kKB, v);
             } else {
 #pragma unroll
                 for (int k = 0; k < kKB; ++k) v[k] = 0.f;
             }
-            store_row(at, tid, ta, v);
-            if (rb < p.b.rows) {
-                load_row(p.b, rb, kb * kKB, v);
-            } else {
-#pragma unroll
-                for (int k = 0; k < kKB; ++k) v[k] = 0.f;
-            }
-            store_row(bt, tid, tb, v);
+            store_row(tile, r, terms, v);
             fence_proxy_async();  // the tiles were written through the generic proxy, the tensor core reads them through the async one
             mbar_arrive(bar_full + 8 * s);
         }
@@ -268,13 +265,16 @@ __global__ void __launch_bounds__(kProducers + 32, 1) k_dequant_gemm(const Param
         ok = __all_sync(0xFFFFFFFFu, ok);  // the tensor-memory loads below are warp-wide
         tmem_fence_after();
         if (ok) {
+            // warp w reads lanes 32 (w & 3) .. +31 (rows of the tile) and columns 64 (w >> 2) .. +63
+            const int ra = m0 + 32 * (warp & 3) + (tid & 31);
             const bool row_ok = ra < p.a.rows;
             float rs = p.alpha;
             if (row_ok && is_codes(p.a.kind) && !p.a.transposed) rs *= __half2float(__ushort_as_half(__ldg(p.a.scales + ra)));
             const bool col_scaled = is_codes(p.b.kind) && !p.b.transposed;
             float* crow = p.c + int64_t(row_ok ? ra : 0) * p.ldc + n0;
-            const uint32_t tlane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-            for (int c0 = 0; c0 < kTile; c0 += 32) {
+            const uint32_t tlane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+            const int cbase = 64 * (warp >> 2);
+            for (int c0 = cbase; c0 < cbase + 64; c0 += 32) {
                 uint32_t acc[32];
                 tmem_ld32(tlane + c0, acc);
                 tmem_wait_ld32(acc);
