@@ -38,7 +38,7 @@ EXECUTED_SLOTS_PER_ROW = 2 * (4096 // 2) * 11 + 4 * (4096 // 2) + 4096
 FP32_LANES_PER_SM = 128
 # dram bytes (read + write) per row of the forward+quant kernel, from the committed ncu capture of the
 # current kernel on this workload; set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_ROW = (268697856 + 51188480) / 32768  # dram read + write of one k_fwdq4096 launch (profiles/)
+NCU_TRAFFIC_BYTES_PER_ROW = (268688896 + 51520256) / 32768  # dram read + write of one k_fwdq4096 launch (profiles/)
 
 
 def measured_peaks():
@@ -207,7 +207,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler captures of a small case)")
-    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward", "int2_8192", "composite5120", "fma_peak"],
+    ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward", "inverse", "int2_8192", "composite5120", "dequant_gemm", "fma_peak"],
                     help="backward / int2_8192: time only bfq_backward on the learning batch / bfq_forward_quant "
                          "(INT2) on the n = 8192 activations (for profiler captures; prints a short JSON line, "
                          "not the benchmark line)")
@@ -236,6 +236,10 @@ def main():
         return
     if args.op == "backward":
         return run_backward_only(torch, args, synth, Plan, dev)
+    if args.op == "inverse":
+        return run_inverse_only(torch, args, synth, Plan, dev)
+    if args.op == "dequant_gemm":
+        return run_gemm_only(torch, args, synth, Plan, dev)
     if args.op == "int2_8192":
         return run_int2_8192_only(torch, args, synth, Plan, dev)
     if args.op == "composite5120":
@@ -349,6 +353,42 @@ def run_backward_only(torch, args, synth, Plan, dev):
     ms = event_time_ms(torch, lambda: plan.backward(x, g, dx=dx, dtheta=dth), args.steps)
     print(json.dumps({"op": "backward", "workload": "learn4096", "rows": rows, "ms": ms,
                       "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
+
+
+def run_inverse_only(torch, args, synth, Plan, dev):
+    """bfq_inverse alone on (a prefix of) the learning batch's gradient rows."""
+    wl = synth.WORKLOADS["learn4096"]
+    rows = args.rows or wl.n_rows
+    plan = Plan(wl.n, dev)
+    plan.set_angles(wl.theta(device=dev))
+    g = wl.g(device=dev, n_rows=rows)
+    out = torch.empty_like(g)
+    for _ in range(args.warmup):
+        plan.inverse(g, out=out)
+    ms = event_time_ms(torch, lambda: plan.inverse(g, out=out), args.steps)
+    print(json.dumps({"op": "inverse", "workload": "learn4096", "rows": rows, "ms": ms,
+                      "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
+
+
+def run_gemm_only(torch, args, synth, Plan, dev):
+    """bfq_dequant_gemm alone: 4-bit activation codes x 4-bit weight codes, the forward product of the calibration step
+    (tokens = --rows or 2048, a 4096 x 4096 layer)."""
+    from paper_2509_09679_b200 import GemmOperand
+
+    n, out, tokens = 4096, 4096, args.rows or 2048
+    plan = Plan(n, dev)
+    plan.set_angles(synth.angles(n, "normal", 7003, dev))
+    W = synth.rows(out, n, "normal", 7001, scale=0.02, dtype=torch.bfloat16).to(dev)
+    X = synth.rows(tokens, n, "student_t3", 7002, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16).to(dev)
+    wc, ws, _ = plan.fold_weights(W, 4)
+    ac, asc = plan.forward_quant(X, 4)
+    c = torch.empty((tokens, out), dtype=torch.float32, device=dev)
+    fn = lambda: plan.dequant_gemm(GemmOperand(ac, asc, 4), GemmOperand(wc, ws, 4), out=c)
+    for _ in range(args.warmup):
+        fn()
+    ms = event_time_ms(torch, fn, args.steps)
+    print(json.dumps({"op": "dequant_gemm", "m": tokens, "n": out, "k": n, "ms": ms,
+                      "tflops": 2.0 * tokens * out * n / (ms * 1e-3) / 1e12, "status": plan.device_status()}))
 
 
 def run_int2_8192_only(torch, args, synth, Plan, dev):
