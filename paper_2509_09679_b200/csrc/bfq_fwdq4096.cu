@@ -48,7 +48,9 @@ struct Smem {
     static constexpr uint32_t kAmaxOff = kBarOff + 8 * G * kInSlots;      // float [G][2 parities][4 warps]
     static constexpr uint32_t kStatOff = kAmaxOff + 32 * G;               // float [G][2 parities][4 warps][2]: row moments
     static constexpr uint32_t kTmemOff = kStatOff + 64 * G;               // tensor-memory base address
-    static constexpr uint32_t kUsed = kTmemOff + 16;
+    static constexpr uint32_t kBinsOff = kTmemOff + 16;                   // u64 [16]: the CTA's code counts (statistics)
+    static constexpr uint32_t kHistOff = kBinsOff + 128;                  // u32 [G][256]: counts of packed code bytes
+    static constexpr uint32_t kUsed = kHistOff + 1024 * G;
     static constexpr uint32_t kBytes = kUsed + 1024;  // slack for the 1024-byte alignment of the TMA tiles
 };
 
@@ -173,17 +175,18 @@ enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutIn
 
 // TRANSFORM: learned butterfly (constants in tensor memory) or the fixed Walsh-Hadamard transform (no constants,
 // no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy), or
-// codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]), or
-// INT2 / INT8 codes + scales.
+// codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]) + the
+// tensor-wide counts of the 16 code values added to `hist`, or INT2 / INT8 codes + scales.
 // STEP: group g passes its token to group (g + STEP) % G, so gcd(STEP, G) groups rotate at a time (0: no tokens).
 template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, const int* __restrict__ form,
            uint8_t* __restrict__ codes,
            uint16_t* __restrict__ scales, __nv_bfloat16* __restrict__ yout, int64_t ldy, int rows,
-           int* __restrict__ status, uint32_t tx_bytes, int wait_limit) {
+           int* __restrict__ status, uint32_t tx_bytes, int wait_limit, unsigned long long* __restrict__ hist) {
     using S = Smem<G, XB>;
     constexpr bool kTmem = TRANSFORM == kButterfly;
+    constexpr bool kCount = OUT == kOutInt4Stats;
     constexpr float kPost = TRANSFORM == kHadamard ? 1.0f / 64.0f : 1.0f;  // 1/sqrt(4096), exact
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -212,6 +215,9 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     if (threadIdx.x < G * kInSlots) {
         mbar_init(sbase + S::kBarOff + 8 * threadIdx.x, 1);
         mbar_init_fence();
+    }
+    if constexpr (kCount) {
+        for (uint32_t e = threadIdx.x; e < (128u + 1024u * G) / 4u; e += G * kGroupThreads) sts32(sbase + S::kBinsOff + 4u * e, 0u);
     }
     // everything above overlaps the end of the kernel before this one; global memory is touched from here on
     grid_dep_wait();
@@ -291,6 +297,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
     const uint32_t amax_base = sbase + S::kAmaxOff + g * 32;
     uint8_t* const out_t = codes + t;
+    const uint32_t hist_g = sbase + S::kHistOff + 1024u * g;  // this group's counts of packed code bytes
 
     // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
     auto row_loop = [&](auto form_tag) {
@@ -467,7 +474,9 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             for (int m = 0; m < 16; ++m) {
                 uint32_t lo, hi;
                 unpack2u(fma2(P[m], inv2, magic2), lo, hi);
-                out[128 * m] = static_cast<uint8_t>((hi * 16u + lo) ^ 0x88u);  // offset-binary -> two's complement
+                const uint32_t byte = (hi * 16u + lo) ^ 0x88u;  // offset-binary -> two's complement
+                out[128 * m] = static_cast<uint8_t>(byte);
+                if constexpr (kCount) red_shared_inc(hist_g + 4u * (byte & 0xFFu));
             }
         } else {
 #pragma unroll
@@ -476,7 +485,9 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                 unpack2(P[m], a, b);
                 const int qa = static_cast<int>(fminf(fmaxf(rintf(a * inv), -8.f), 7.f));
                 const int qb = static_cast<int>(fminf(fmaxf(rintf(b * inv), -8.f), 7.f));
-                out[128 * m] = static_cast<uint8_t>((qa & 0xF) | ((qb & 0xF) << 4));
+                const uint32_t byte = static_cast<uint32_t>((qa & 0xF) | ((qb & 0xF) << 4));
+                out[128 * m] = static_cast<uint8_t>(byte);
+                if constexpr (kCount) red_shared_inc(hist_g + 4u * byte);
             }
         }
     }
@@ -493,6 +504,25 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         row_loop(std::integral_constant<int, kFormShear>());
     }
 
+    if constexpr (kCount) {
+        // byte counts of the G groups -> the CTA's 16 code counts (a byte holds two codes) -> the caller's histogram,
+        // indexed by code + 8.  Integer additions: the result does not depend on their order.
+        __syncthreads();
+        if (threadIdx.x < 256) {
+            uint32_t n = 0;
+#pragma unroll
+            for (int gg = 0; gg < G; ++gg) n += lds32(sbase + S::kHistOff + 1024u * gg + 4u * threadIdx.x);
+            if (n != 0u) {
+                red_shared_add64(sbase + S::kBinsOff + 8u * ((threadIdx.x & 15u) ^ 8u), n);
+                red_shared_add64(sbase + S::kBinsOff + 8u * ((threadIdx.x >> 4) ^ 8u), n);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < 16) {
+            const unsigned long long c = lds64(sbase + S::kBinsOff + 8u * threadIdx.x);
+            if (c != 0ull) atomicAdd(hist + threadIdx.x, c);
+        }
+    }
     if constexpr (kTmem) {
         tmem_fence_before();
         __syncthreads();
@@ -595,41 +625,6 @@ __global__ void __launch_bounds__(256) k_build_image4096(const float4* __restric
     }
 }
 
-// Histogram of the 4-bit codes of packed rows (two per byte): every warp counts whole bytes in its own 256-bin table in
-// shared memory (few lanes of a warp hit the same byte value at once), the CTA folds the byte counts into the 16 code
-// counts (a byte contributes to its low and to its high nibble) and adds them to hist[code + 8] (code = the nibble as a
-// two's complement number).  Counts are exact.
-constexpr int kHistThreads = 256;
-__global__ void __launch_bounds__(kHistThreads) k_hist_int4(const uint4* __restrict__ codes, int64_t chunks,
-                                                            unsigned long long* __restrict__ hist) {
-    __shared__ unsigned int bytes[kHistThreads / 32][256];
-    __shared__ unsigned long long bins[16];
-    const int t = threadIdx.x, warp = t >> 5;
-    for (int e = t; e < (kHistThreads / 32) * 256; e += kHistThreads) (&bytes[0][0])[e] = 0u;
-    if (t < 16) bins[t] = 0ull;
-    __syncthreads();
-    unsigned int* mine = bytes[warp];
-    for (int64_t c = int64_t(blockIdx.x) * kHistThreads + t; c < chunks; c += int64_t(gridDim.x) * kHistThreads) {
-        const uint4 v = __ldg(codes + c);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-#pragma unroll
-            for (int b = 0; b < 4; ++b) atomicAdd(mine + ((w[k] >> (8 * b)) & 0xFFu), 1u);
-        }
-    }
-    __syncthreads();
-    unsigned int n = 0;  // thread t: byte value t
-#pragma unroll
-    for (int wi = 0; wi < kHistThreads / 32; ++wi) n += bytes[wi][t];
-    if (n != 0u) {
-        atomicAdd(&bins[(t & 15) ^ 8], static_cast<unsigned long long>(n));
-        atomicAdd(&bins[(t >> 4) ^ 8], static_cast<unsigned long long>(n));
-    }
-    __syncthreads();
-    if (t < 16 && bins[t] != 0ull) atomicAdd(hist + t, bins[t]);
-}
-
 }  // namespace f4k
 
 // ---- host side ---------------------------------------------------------------------------------------------
@@ -657,7 +652,8 @@ bool fwdq4096_available(const bfq_plan* plan) {
 
 template <int G, int CW, int XB, int TRANSFORM, int OUT>
 static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap, int64_t rows, uint8_t* codes,
-                                  uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
+                                  uint16_t* scales, void* y, int64_t ldy, cudaStream_t st,
+                                  unsigned long long* hist = nullptr) {
     using S = f4k::Smem<G, XB>;
     static bool attr_set[kMaxDevices] = {false};
     auto kern = f4k::k_fwdq4096<G, CW, XB, TRANSFORM, OUT>;
@@ -674,7 +670,7 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
     const int wait_limit = plan->test_stuck_wait ? 4096 : (1 << 22);
     return launch_overlapped(kern, dim3(grid), dim3(G * f4k::kGroupThreads), S::kBytes, st, tmap, plan->img4096,
                              plan->form_flag, codes, scales, static_cast<__nv_bfloat16*>(y), ldy, int(rows),
-                             plan->status_word, tx_bytes, wait_limit);
+                             plan->status_word, tx_bytes, wait_limit, hist);
 }
 
 // Four row groups per CTA, 32-word constant chunks, one buffer per regrouping (measured fastest among the
@@ -708,19 +704,14 @@ cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t ro
                      : launch_variant<4, 32, 2, kButterfly, kOutInt8>(plan, tmap, rows, codes, scales, nullptr, 0, st);
 }
 
-// bfq_forward_quant_stats on the tuned path: codes + scales + row moments from k_fwdq4096, then the code histogram from
-// the packed codes (hist must have been zeroed on the same stream).
+// bfq_forward_quant_stats on the tuned path: codes + scales + row moments + code counts from one launch of k_fwdq4096
+// (hist must have been zeroed on the same stream).
 cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                   uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st) {
     CUtensorMap tmap;
     if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
     using namespace f4k;
-    cudaError_t e = launch_variant<4, 32, 2, kButterfly, kOutInt4Stats>(plan, tmap, rows, codes, scales, rowstats, 0, st);
-    if (e != cudaSuccess) return e;
-    const int64_t chunks = rows * (kN / 2 / 16);
-    const int64_t want = (chunks + kHistThreads - 1) / kHistThreads, cap = int64_t(plan->sm_count) * 8;
-    k_hist_int4<<<int(want < cap ? want : cap), kHistThreads, 0, st>>>(reinterpret_cast<const uint4*>(codes), chunks, hist);
-    return cudaGetLastError();
+    return launch_variant<4, 32, 2, kButterfly, kOutInt4Stats>(plan, tmap, rows, codes, scales, rowstats, 0, st, hist);
 }
 
 }  // namespace bfq

@@ -42,6 +42,13 @@ __device__ __forceinline__ void sts32(uint32_t a, uint32_t v) {
 __device__ __forceinline__ void sts64(uint32_t a, u64 v) {
     asm volatile("st.shared.b64 [%0], %1;" ::"r"(a), "l"(v) : "memory");
 }
+// counters in shared memory: add without reading the result back
+__device__ __forceinline__ void red_shared_inc(uint32_t a) {
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(a) : "memory");
+}
+__device__ __forceinline__ void red_shared_add64(uint32_t a, u64 v) {
+    asm volatile("red.shared.add.u64 [%0], %1;" ::"r"(a), "l"(v) : "memory");
+}
 
 // fp16 scale of a row from its absmax, like row_scale() of the generic kernels but with straight-line arithmetic: a / QMAX as
 // q0 = a * r, q = fma(fma(-q0, QMAX, a), r, q0) with r = RN(1 / QMAX), which is the correctly rounded quotient for
