@@ -232,7 +232,15 @@ def main():
     barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     if args.op == "fma_peak":
-        print(json.dumps({"op": "fma_peak", **fma_rates(torch, dev)}))
+        from paper_2509_09679_b200 import measure_mma_rates
+
+        m = measure_mma_rates(dev)
+        # one merged phase of four butterfly stages at n = 4096 = 256 distinct 16 x 16 blocks; 128 token rows per MMA;
+        # two bf16 terms for the block and two for the data = 4 MMAs (M = 128, N = 16, K = 16) per block
+        merged = {"cycles_per_mma_m128_k16": m,
+                  "merged_phase_cycles_per_row_per_sm": 256 * 4 * m["n16"] / 128,
+                  "note": "three such phases per row; the FP32 kernel takes about 1100 cycles per row per SM in all"}
+        print(json.dumps({"op": "fma_peak", **fma_rates(torch, dev), "tensor_core_small_n": merged}))
         return
     if args.op == "backward":
         return run_backward_only(torch, args, synth, Plan, dev)

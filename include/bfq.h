@@ -275,6 +275,16 @@ int bfq_dequant_gemm(bfq_plan* plan, int64_t m, int64_t n, int64_t k, float alph
  */
 int bfq_measure_fma_rates(float* cycles_per_instruction);
 
+/*
+ * Measures, on the current device, the SM cycles one tcgen05.mma (bf16 x bf16 -> fp32, M = 128, K = 16, operands in
+ * shared memory, issued back to back by one thread) takes for N = 16, 64, 128 and 256: `cycles_per_mma` is a HOST
+ * array of 4 floats in that order.  It prices running merged butterfly stages as small dense blocks on the tensor
+ * cores (one 2^k x 2^k block per MMA; the paper's Sec. 3.2.1 structure has a different block for every group of
+ * columns) against the FP32 path; no counterpart in the paper.  Synchronous, allocates and frees a few bytes of device
+ * memory.  Returns BFQ_OK, BFQ_ERR_NULL, BFQ_ERR_CUDA or BFQ_ERR_DEVICE_TIMEOUT (a bounded wait ran out).
+ */
+int bfq_measure_mma_rates(float* cycles_per_mma);
+
 /* Number of CTAs the backward pass uses (= number of d-theta partial sums); informational. */
 int bfq_backward_partials(const bfq_plan* plan);
 

@@ -40,6 +40,7 @@ SIGNATURES = {
     "bfq_status_string": (ctypes.c_char_p, [_i]),
     "bfq_backward_partials": (_i, [_p]),
     "bfq_measure_fma_rates": (_i, [_p]),
+    "bfq_measure_mma_rates": (_i, [_p]),
     "bfq_dequant_gemm": (_i, [_p, _i64, _i64, _i64, ctypes.c_float, _p, _i, _i, _i64, _p, _p, _i, _i, _i64, _p, _p, _i64, _p]),
     "bfq_stage_form": (_i, [_p]),
     "bfq_test_stuck_wait": (_i, [_p, _i]),
@@ -374,3 +375,13 @@ def measure_fma_rates(device=None):
     with torch.cuda.device(dev):
         _check(lib().bfq_measure_fma_rates(ctypes.cast(out, ctypes.c_void_p)), "bfq_measure_fma_rates")
     return {"packed_3reg": out[0], "packed_2reg": out[1], "scalar_3reg": out[2], "scalar_2reg": out[3]}
+
+
+def measure_mma_rates(device=None):
+    """bfq_measure_mma_rates on `device` (default: the current one): SM cycles per tcgen05.mma (bf16, M = 128, K = 16)
+    for N = 16, 64, 128, 256."""
+    out = (ctypes.c_float * 4)()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        _check(lib().bfq_measure_mma_rates(ctypes.cast(out, ctypes.c_void_p)), "bfq_measure_mma_rates")
+    return {"n16": out[0], "n64": out[1], "n128": out[2], "n256": out[3]}

@@ -5,16 +5,26 @@
 // [K][rows].  This covers the three products of the reconstruction loss (paper Sec. 3.4):
 //     Dequant(Quant(B x)) . Dequant(Quant(W B^T))^T,   err . Dequant(Quant(W B^T)),   err^T . Dequant(Quant(B x)).
 //
-// One CTA per 128 x 128 tile of C.  Eight producer warps build the operand tiles of a 64-wide K block in shared memory
-// in the K-major, 128-byte-swizzled layout the tensor core reads (thread = tile row of A or of B), as 1 or 2 bf16 terms:
+// One CTA per 128 x 128 tile of C, K blocks of 64.  An operand tile in shared memory is 128 rows of 128 bytes (64 bf16)
+// with the 128-byte swizzle, and every row is 64 elements that are CONTIGUOUS IN THE STORED OPERAND:
+//   * stored [rows][K]: shared-memory row r = tile row r, 64 consecutive k (the K-major layout of the tensor core);
+//   * stored [K][rows]: shared-memory row 64 h + k = stored row k0 + k, tile rows 64 h .. 64 h + 63 (the MN-major
+//     layout: blocks of 64 tile rows 8192 bytes apart, groups of 8 k 1024 bytes apart).
+// So one producer thread (eight producer warps: threads 0..127 for A, 128..255 for B) always turns 64 contiguous stored
+// elements into one 128-byte row, with 16-byte loads and stores, whatever the orientation; the instruction descriptor
+// tells the tensor core which layout each operand has.  Terms per operand:
 //   * codes contracted along their stored row: the integer codes are exact in bf16 (one term); the row scale multiplies
 //     the finished row / column of C;
-//   * codes contracted across stored rows (transposed): code x scale has at most 14 significant bits: hi + lo, exact;
+//   * codes contracted across stored rows: the scale varies along k, so code x scale (at most 15 significant bits) is
+//     stored as hi + lo, exactly;
 //   * fp32 numbers: hi + lo = 16 significant bits (relative error 2^-17 per element); bf16 numbers: one term, exact.
-// One thread issues tcgen05.mma (kind::f16, M = N = 128, fp32 accumulators in tensor memory) for every pair of terms
-// and commits to the stage's "empty" mbarrier; two stages.  The producer warps then read the accumulators back
-// (tcgen05.ld, a lane quarter and half of the columns each), apply alpha and the row / column scales and store fp32 rows of C.  Every wait is
-// bounded and reports through the plan's status word.
+// Codes become bf16 without integer-to-float conversions: a field u = code + 2^(b-1) OR-ed into the mantissa of 128.0
+// is the bf16 number 128 + u, two fields per 32-bit word at a time, and one packed subtraction removes the offset.
+// The global loads of the next K block are issued before the current one is converted.  One thread issues
+// tcgen05.mma (kind::f16, M = N = 128, fp32 accumulators in tensor memory) for every pair of terms and commits to
+// the stage's "empty" mbarrier; the ring has as many stages as fit 192 KB.  The producer warps then read the
+// accumulators back (tcgen05.ld, a lane quarter and half of the columns each), apply alpha and the row / column
+// scales and store fp32 rows of C.  Every wait is bounded and reports through the plan's status word.
 #include "../../include/bfq.h"
 
 #include <cuda_bf16.h>

@@ -3,6 +3,10 @@
 // butterfly with per-pair constants does, and when it reads two.  No global traffic inside the timed loops; each warp
 // times itself with the SM clock.  The numbers put the roofline's nominal "128 lanes per SM per cycle" beside what the
 // register file actually delivers to this instruction pattern.
+//
+// Second measurement: SM cycles per tcgen05.mma (bf16 x bf16 -> fp32, M = 128, K = 16) as a function of N, operands in
+// shared memory, one thread issuing back to back.  It prices the alternative of running merged butterfly stages as
+// small dense blocks on the tensor cores (a 16 x 16 block per MMA) against the FP32 path.
 #include "../../include/bfq.h"
 
 #include <cuda_runtime.h>
@@ -80,6 +84,74 @@ __global__ void __launch_bounds__(kThreads, 1) k_rate(const float* __restrict__ 
     if ((threadIdx.x & 31) == 0) atomicMax(cycles + PATTERN, static_cast<unsigned long long>(t1 - t0));
 }
 
+// ---- tensor-core issue rate for small N -----------------------------------------------------------------------
+constexpr int kMmaShapes = 4;
+constexpr int kMmaIters = 256;  // x 4 K steps of 16
+__constant__ int c_mma_n[kMmaShapes] = {16, 64, 128, 256};
+
+__device__ __forceinline__ uint64_t desc_k_major_sw128(uint32_t addr) {
+    // K-major tile, 128-byte swizzle: 8-row groups 1024 bytes apart
+    return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(1) << 16) |
+           (static_cast<uint64_t>(1024 >> 4) << 32) | (static_cast<uint64_t>(1) << 46) | (static_cast<uint64_t>(2) << 61);
+}
+
+// One CTA per SM; zero operands (the cycle count does not depend on the values); every wait is bounded.
+__global__ void __launch_bounds__(128, 1) k_mma_rate(unsigned long long* __restrict__ cycles, int* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_tile = sbase, b_tile = sbase + 16384u, bar = sbase + 49152u, slot = bar + 8u;
+    for (uint32_t e = threadIdx.x; e < 49152u / 16u; e += blockDim.x)
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(sbase + 16u * e), "r"(0u) : "memory");
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        mbar_init_fence();
+    }
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(slot) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tmem_fence_before();
+    __syncthreads();
+    tmem_fence_after();
+    uint32_t tmem = 0;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem) : "r"(slot));
+    if (threadIdx.x == 0) {
+        uint32_t parity = 0;
+        for (int sh = 0; sh < kMmaShapes; ++sh) {
+            const uint32_t n = static_cast<uint32_t>(c_mma_n[sh]);
+            // fp32 accumulator, bf16 operands, both K-major, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+            const long long t0 = sm_clock();
+            for (int it = 0; it < kMmaIters; ++it) {
+#pragma unroll
+                for (uint32_t ks = 0; ks < 4; ++ks) {
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t"
+                        "setp.ne.b32 p, %4, 0;\n\t"
+                        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                        ::"r"(tmem), "l"(desc_k_major_sw128(a_tile + 32u * ks)), "l"(desc_k_major_sw128(b_tile + 32u * ks)),
+                        "r"(idesc), "r"(static_cast<uint32_t>(it | ks))
+                        : "memory");
+                }
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+            bool done = false;
+            for (int i = 0; i < (1 << 24) && !done; ++i) done = mbar_try_wait(bar, parity);
+            const long long t1 = sm_clock();
+            if (!done) {
+                atomicExch(status, 1);
+                break;
+            }
+            parity ^= 1u;
+            atomicMax(cycles + sh, static_cast<unsigned long long>(t1 - t0));
+        }
+    }
+    tmem_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+}
+
 }  // namespace rates
 }  // namespace bfq
 
@@ -120,5 +192,34 @@ extern "C" int bfq_measure_fma_rates(float* cycles_per_instruction) {
         const double per_warp = (p < 2 ? 64.0 : 128.0) * kIters;
         cycles_per_instruction[p] = static_cast<float>(static_cast<double>(host_cyc[p]) / (per_warp * warps_per_scheduler));
     }
+    return BFQ_OK;
+}
+
+extern "C" int bfq_measure_mma_rates(float* cycles_per_mma) {
+    using namespace bfq::rates;
+    if (cycles_per_mma == nullptr) return BFQ_ERR_NULL;
+    unsigned long long* cyc = nullptr;
+    cudaError_t e = cudaMalloc(&cyc, (kMmaShapes + 1) * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(cyc, 0, (kMmaShapes + 1) * sizeof(unsigned long long));
+    int sms = 1, dev = 0;
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    constexpr int kSmem = 49152 + 16 + 1024;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_mma_rate, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    unsigned long long host[kMmaShapes + 1] = {0, 0, 0, 0, 0};
+    if (e == cudaSuccess) {
+        int* status = reinterpret_cast<int*>(cyc + kMmaShapes);
+        for (int rep = 0; rep < 2; ++rep) {  // the second round counts
+            if (rep == 1) cudaMemset(cyc, 0, kMmaShapes * sizeof(unsigned long long));
+            k_mma_rate<<<sms, 128, kSmem>>>(cyc, status);
+        }
+        e = cudaDeviceSynchronize();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(host, cyc, sizeof(host), cudaMemcpyDeviceToHost);
+    cudaFree(cyc);
+    if (e != cudaSuccess) return BFQ_ERR_CUDA;
+    if (host[kMmaShapes] != 0) return BFQ_ERR_DEVICE_TIMEOUT;
+    for (int s = 0; s < kMmaShapes; ++s)
+        cycles_per_mma[s] = static_cast<float>(static_cast<double>(host[s]) / (4.0 * kMmaIters));
     return BFQ_OK;
 }
