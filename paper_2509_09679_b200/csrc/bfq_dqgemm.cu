@@ -41,9 +41,10 @@ using namespace ptx;
 
 constexpr int kTile = 128;       // rows of A and of B per CTA
 constexpr int kKB = 64;          // K block: one 128-byte swizzle atom of bf16
-constexpr int kStages = 2;
-constexpr int kProducers = 256;  // threads 0..127 build A's tile rows, 128..255 B's; all run the epilogue; thread 256 issues the MMAs
+constexpr int kMaxStages = 6;
+constexpr int kProducers = 256;  // threads 0..127 build A's tile, 128..255 B's; all run the epilogue; thread 256 issues the MMAs
 constexpr uint32_t kTileBytes = kTile * kKB * 2;  // one bf16 term of one operand: 16 KB
+constexpr uint32_t kRingBytes = 12 * kTileBytes;  // 192 KB of operand tiles
 constexpr int kWaitLimit = 1 << 24;
 
 struct Operand {
@@ -60,6 +61,10 @@ __host__ __device__ __forceinline__ int terms_of(int kind, int transposed) {
     if (kind == BFQ_OP_BF16) return 1;
     if (kind == BFQ_OP_F32) return 2;
     return transposed ? 2 : 1;
+}
+__host__ __device__ __forceinline__ int stages_of(int terms_a, int terms_b) {
+    const int fit = 12 / (terms_a + terms_b);
+    return fit < kMaxStages ? fit : kMaxStages;
 }
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -80,136 +85,97 @@ __device__ __forceinline__ void tmem_alloc128(uint32_t smem_dst) {
 __device__ __forceinline__ void tmem_dealloc128(uint32_t taddr) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 128;" ::"r"(taddr) : "memory");
 }
-// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart; the start address advances by 32 bytes
-// per 16-element K step inside the atom
-__device__ __forceinline__ uint64_t desc_sw128(uint32_t addr) {
-    return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(1) << 16) |
+// Shared-memory descriptor of a 128-byte-swizzled tile.  K-major operand: rows of 128 bytes, 8-row groups 1024 bytes
+// apart (stride field), the leading field unused; one K step of 16 elements is 32 bytes further along the row.
+// MN-major operand: rows of 128 bytes hold 64 tile rows for one k, groups of 8 k are 1024 bytes apart (stride field),
+// blocks of 64 tile rows 8192 bytes apart (leading field); one K step of 16 is two groups = 2048 bytes further.
+__device__ __forceinline__ uint64_t desc_sw128(uint32_t addr, uint32_t leading_bytes) {
+    return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(leading_bytes >> 4) << 16) |
            (static_cast<uint64_t>(1024 >> 4) << 32) | (static_cast<uint64_t>(1) << 46) | (static_cast<uint64_t>(2) << 61);
 }
-// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(kTile >> 3) << 17) | (uint32_t(kTile >> 4) << 24);
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+// bf16 x bf16 -> fp32, M = 128, N = 128; bit 15 / 16: A / B is MN-major
+__device__ __forceinline__ uint32_t make_idesc(int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn_major) << 15) |
+           (static_cast<uint32_t>(b_mn_major) << 16) | (uint32_t(kTile >> 3) << 17) | (uint32_t(kTile >> 4) << 24);
+}
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// ---- one tile row: 64 consecutive k of operand row `row` (already checked < op.rows), as fp32 ----------------
-__device__ __forceinline__ float code_value(uint32_t byte, int shift, int bits) {
-    const int q = static_cast<int>((byte >> shift) & ((1u << bits) - 1u));
-    return static_cast<float>(q >= (1 << (bits - 1)) ? q - (1 << bits) : q);
+// ---- one shared-memory row: 64 elements that are contiguous in the stored operand -------------------------------
+__device__ __forceinline__ void sts128(uint32_t at, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(at), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {  // lo in bits 0..15
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
 }
 
-// codes along the stored row: element k in bits [BITS (k mod 8/BITS), +BITS) of byte k BITS / 8, 16-byte loads; the
-// row's scale is applied to the finished row of C
-template <int BITS>
-__device__ __forceinline__ void codes_along(const Operand& op, int row, int k0, float (&v)[kKB]) {
-    const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(op.data) + (int64_t(row) * op.ld + k0) * BITS / 8);
-    constexpr int kPerWord = 32 / BITS;
-#pragma unroll
-    for (int i = 0; i < kKB * BITS / 128; ++i) {
-        const uint4 w4 = __ldg(p + i);
-        const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int e = 0; e < kPerWord; ++e) {
-                // sign-extend the field: shift it to the top of the word, then arithmetic shift back
-                const int q = static_cast<int>(ws[j] << (32 - BITS * (e + 1))) >> (32 - BITS);
-                v[(4 * i + j) * kPerWord + e] = static_cast<float>(q);
-            }
-    }
-}
-// codes across stored rows: stored row k0 + k holds this tile row's code in its column `row`; the stored row's scale
-// varies along k and is applied here (code x fp16 scale is exact in fp32)
-template <int BITS>
-__device__ __forceinline__ void codes_across(const Operand& op, int row, int k0, float (&v)[kKB]) {
-    const int64_t pitch = op.ld * BITS / 8;
-    const uint8_t* p = static_cast<const uint8_t*>(op.data) + int64_t(k0) * pitch + (int64_t(row) * BITS >> 3);
-    const int shift = (row * BITS) & 7;
-#pragma unroll
-    for (int k = 0; k < kKB; ++k) {
-        const float s = __half2float(__ushort_as_half(__ldg(op.scales + k0 + k)));
-        v[k] = s * code_value(__ldg(p + int64_t(k) * pitch), shift, BITS);
-    }
+// Where chunk j (16 bytes = 8 bf16) of shared-memory row `srow` of a tile goes
+__device__ __forceinline__ uint32_t chunk_addr(uint32_t tile, int srow, int j) {
+    return tile + static_cast<uint32_t>(srow) * 128u + static_cast<uint32_t>((j ^ (srow & 7)) << 4);
 }
 
-__device__ __forceinline__ void load_row(const Operand& op, int row, int k0, float (&v)[kKB]) {
-    if (!op.transposed) {
-        if (op.kind == BFQ_OP_F32) {
-            const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(op.data) + int64_t(row) * op.ld + k0);
-#pragma unroll
-            for (int i = 0; i < kKB / 4; ++i) {
-                const float4 f = __ldg(p + i);
-                v[4 * i] = f.x, v[4 * i + 1] = f.y, v[4 * i + 2] = f.z, v[4 * i + 3] = f.w;
-            }
-        } else if (op.kind == BFQ_OP_BF16) {
-            const uint4* p = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(op.data) + int64_t(row) * op.ld + k0);
-#pragma unroll
-            for (int i = 0; i < kKB / 8; ++i) {
-                const uint4 w = __ldg(p + i);
-                const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    v[8 * i + 2 * j] = __uint_as_float(ws[j] << 16);
-                    v[8 * i + 2 * j + 1] = __uint_as_float(ws[j] & 0xFFFF0000u);
-                }
-            }
-        } else if (op.kind == BFQ_OP_CODES2) {
-            codes_along<2>(op, row, k0, v);
-        } else if (op.kind == BFQ_OP_CODES4) {
-            codes_along<4>(op, row, k0, v);
-        } else {
-            codes_along<8>(op, row, k0, v);
-        }
-    } else {
-        if (op.kind == BFQ_OP_F32) {
-            const float* p = static_cast<const float*>(op.data) + int64_t(k0) * op.ld + row;
-#pragma unroll
-            for (int k = 0; k < kKB; ++k) v[k] = __ldg(p + int64_t(k) * op.ld);
-        } else if (op.kind == BFQ_OP_BF16) {
-            const uint16_t* p = static_cast<const uint16_t*>(op.data) + int64_t(k0) * op.ld + row;
-#pragma unroll
-            for (int k = 0; k < kKB; ++k) v[k] = __uint_as_float(static_cast<uint32_t>(__ldg(p + int64_t(k) * op.ld)) << 16);
-        } else if (op.kind == BFQ_OP_CODES2) {
-            codes_across<2>(op, row, k0, v);
-        } else if (op.kind == BFQ_OP_CODES4) {
-            codes_across<4>(op, row, k0, v);
-        } else {
-            codes_across<8>(op, row, k0, v);
-        }
-    }
+// two fp32 values -> their bf16 words (hi term, remainder term)
+__device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t& lo) {
+    hi = pack_bf16(a, b);
+    lo = pack_bf16(a - __uint_as_float(hi << 16), b - __uint_as_float(hi & 0xFFFF0000u));
 }
 
-// 64 fp32 values of tile row r -> `terms` bf16 tiles (hi, then the rounding remainder) in the swizzled layout:
-// 16-byte chunk j of row r sits at chunk j ^ (r & 7) of its 128-byte line; 8-row groups are 1024 bytes apart
-__device__ __forceinline__ void store_row(uint32_t tile, int r, int terms, const float (&v)[kKB]) {
-    const uint32_t line = tile + (r >> 3) * 1024u + (r & 7) * 128u;
+// Raw 16-byte words of a row's 64 elements: fp32 16, bf16 8, 8-bit codes 4, 4-bit codes 2, 2-bit codes 1
+template <int KIND>
+struct RawWords {
+    static constexpr int kCount = KIND == BFQ_OP_F32 ? 16 : (KIND == BFQ_OP_BF16 ? 8 : (KIND * 64) / 128);
+};
+
+// 8 codes of 4 bits (one word, element e in bits 4e..4e+3, two's complement) -> 4 words of bf16 pairs in element order
+__device__ __forceinline__ void codes4_to_bf16(uint32_t w, uint32_t (&o)[4]) {
+    const uint32_t x = w ^ 0x88888888u;  // u = code + 8
+    // (128 + u_e, 128 + u_{e+4}) as a bf16 pair: the field sits in the low mantissa bits of 128.0 = 0x4300
+    const uint32_t t0 = (x & 0x000F000Fu) | 0x43004300u, t1 = ((x >> 4) & 0x000F000Fu) | 0x43004300u;
+    const uint32_t t2 = ((x >> 8) & 0x000F000Fu) | 0x43004300u, t3 = ((x >> 12) & 0x000F000Fu) | 0x43004300u;
+    const uint32_t off = 0x43084308u;  // 136.0 twice
+    const uint32_t c0 = sub_bf16x2(t0, off), c1 = sub_bf16x2(t1, off), c2 = sub_bf16x2(t2, off), c3 = sub_bf16x2(t3, off);
+    o[0] = prmt(c0, c1, 0x5410u), o[1] = prmt(c2, c3, 0x5410u);  // elements (0,1), (2,3)
+    o[2] = prmt(c0, c1, 0x7632u), o[3] = prmt(c2, c3, 0x7632u);  // elements (4,5), (6,7)
+}
+// 16 codes of 2 bits (one word) -> 8 words of bf16 pairs in element order
+__device__ __forceinline__ void codes2_to_bf16(uint32_t w, uint32_t (&o)[8]) {
+    const uint32_t x = w ^ 0xAAAAAAAAu;  // u = code + 2
+    uint32_t c[8];                       // c[j] = (code_j, code_{j+8})
 #pragma unroll
-    for (int j = 0; j < kKB / 8; ++j) {
-        uint32_t hi[4], lo[4];
+    for (int j = 0; j < 8; ++j) c[j] = sub_bf16x2(((x >> (2 * j)) & 0x00030003u) | 0x43004300u, 0x43024302u);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float a = v[8 * j + 2 * e], b = v[8 * j + 2 * e + 1];
-            const __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
-            hi[e] = static_cast<uint32_t>(__bfloat16_as_ushort(ah)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bh)) << 16);
-            if (terms == 2) {  // the rounding remainder, for operands that are not exact in one bf16 term
-                const __nv_bfloat16 al = __float2bfloat16_rn(a - __bfloat162float(ah)), bl = __float2bfloat16_rn(b - __bfloat162float(bh));
-                lo[e] = static_cast<uint32_t>(__bfloat16_as_ushort(al)) | (static_cast<uint32_t>(__bfloat16_as_ushort(bl)) << 16);
-            }
-        }
-        const uint32_t at = line + ((j ^ (r & 7)) << 4);
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(at), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-        if (terms == 2)
-            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(at + kTileBytes), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3])
-                         : "memory");
+    for (int j = 0; j < 4; ++j) {
+        o[j] = prmt(c[2 * j], c[2 * j + 1], 0x5410u);      // elements (2j, 2j+1)
+        o[4 + j] = prmt(c[2 * j], c[2 * j + 1], 0x7632u);  // elements (8+2j, 9+2j)
     }
+}
+// 4 codes of 8 bits (one word) -> 2 words of bf16 pairs: byte u = code + 128 in the low mantissa bits of 2^23
+__device__ __forceinline__ void codes8_to_bf16(uint32_t w, uint32_t (&o)[2]) {
+    const uint32_t x = w ^ 0x80808080u;
+    const float m = 8388736.0f;  // 2^23 + 128
+    const float f0 = __uint_as_float(prmt(x, 0x4B000000u, 0x7440u)) - m, f1 = __uint_as_float(prmt(x, 0x4B000000u, 0x7441u)) - m;
+    const float f2 = __uint_as_float(prmt(x, 0x4B000000u, 0x7442u)) - m, f3 = __uint_as_float(prmt(x, 0x4B000000u, 0x7443u)) - m;
+    o[0] = pack_bf16(f0, f1), o[1] = pack_bf16(f2, f3);
 }
 
 struct Params {
@@ -221,20 +187,192 @@ struct Params {
     int* status;
 };
 
+// zeroes the elements >= valid of chunk j (elements 8j .. 8j+7, two per word)
+__device__ __forceinline__ void mask_chunk(uint32_t (&o)[4], int j, int valid) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const int e = 8 * j + 2 * w;
+        o[w] = e >= valid ? 0u : (e + 1 >= valid ? (o[w] & 0xFFFFu) : o[w]);
+    }
+}
+
+// One chunk (8 elements as 4 words of exact bf16 pairs) to the tile: as it is, or times the row's scale in two terms
+template <bool SCALED, bool PARTIAL>
+__device__ __forceinline__ void store_bf16_chunk(uint32_t tile, int srow, int j, uint32_t (&o)[4], float s, int valid) {
+    if constexpr (PARTIAL) mask_chunk(o, j, valid);
+    const uint32_t at = chunk_addr(tile, srow, j);
+    if constexpr (!SCALED) {
+        sts128(at, o[0], o[1], o[2], o[3]);
+    } else {
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) split2(__uint_as_float(o[w] << 16) * s, __uint_as_float(o[w] & 0xFFFF0000u) * s, hi[w], lo[w]);
+        sts128(at, hi[0], hi[1], hi[2], hi[3]);
+        sts128(at + kTileBytes, lo[0], lo[1], lo[2], lo[3]);
+    }
+}
+
+// The 64 elements of one shared-memory row from their raw 16-byte words.  SCALED (codes contracted across their stored
+// rows): times `s`, two terms.
+template <int KIND, bool SCALED, bool PARTIAL>
+__device__ __forceinline__ void convert_store(const uint4 (&raw)[RawWords<KIND>::kCount], uint32_t tile, int srow, float s,
+                                              int valid) {
+    if constexpr (KIND == BFQ_OP_F32) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint4 u = raw[2 * j], v = raw[2 * j + 1];
+            uint32_t hi[4], lo[4];
+            split2(__uint_as_float(u.x), __uint_as_float(u.y), hi[0], lo[0]);
+            split2(__uint_as_float(u.z), __uint_as_float(u.w), hi[1], lo[1]);
+            split2(__uint_as_float(v.x), __uint_as_float(v.y), hi[2], lo[2]);
+            split2(__uint_as_float(v.z), __uint_as_float(v.w), hi[3], lo[3]);
+            if constexpr (PARTIAL) mask_chunk(hi, j, valid), mask_chunk(lo, j, valid);
+            const uint32_t at = chunk_addr(tile, srow, j);
+            sts128(at, hi[0], hi[1], hi[2], hi[3]);
+            sts128(at + kTileBytes, lo[0], lo[1], lo[2], lo[3]);
+        }
+    } else if constexpr (KIND == BFQ_OP_BF16) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t o[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+            store_bf16_chunk<false, PARTIAL>(tile, srow, j, o, 1.f, valid);
+        }
+    } else if constexpr (KIND == BFQ_OP_CODES4) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t ws[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                uint32_t o[4];
+                codes4_to_bf16(ws[w], o);
+                store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 4 * i + w, o, s, valid);
+            }
+        }
+    } else if constexpr (KIND == BFQ_OP_CODES2) {
+        const uint32_t ws[4] = {raw[0].x, raw[0].y, raw[0].z, raw[0].w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            uint32_t o8[8];
+            codes2_to_bf16(ws[w], o8);
+            uint32_t oa[4] = {o8[0], o8[1], o8[2], o8[3]}, ob[4] = {o8[4], o8[5], o8[6], o8[7]};
+            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * w, oa, s, valid);
+            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * w + 1, ob, s, valid);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t ws[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t o2a[2], o2b[2];
+                codes8_to_bf16(ws[2 * h], o2a);
+                codes8_to_bf16(ws[2 * h + 1], o2b);
+                uint32_t o[4] = {o2a[0], o2a[1], o2b[0], o2b[1]};
+                store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * i + h, o, s, valid);
+            }
+        }
+    }
+}
+
+struct Ring {
+    uint32_t sbase, stage_bytes, bar_full, bar_empty;
+    int stages;
+};
+
+// Producer loop of one thread: shared-memory row `srow` of every K block of its operand.  ACROSS: the operand is stored
+// [K][rows]; the thread's row is stored row k0 + (r >> 1), tile rows 64 (r & 1) .. + 63.
+template <int KIND, bool ACROSS>
+__device__ __forceinline__ bool produce(const Operand& op, int r, int tile_row0, uint32_t tile_off, const Ring& ring, int kblocks,
+                                        int* status) {
+    constexpr int NW = RawWords<KIND>::kCount;
+    constexpr int kEbits = KIND == BFQ_OP_F32 ? 32 : (KIND == BFQ_OP_BF16 ? 16 : KIND);
+    constexpr int kPerWord = 128 / kEbits;  // elements per 16-byte word
+    constexpr bool kScaled = ACROSS && KIND >= BFQ_OP_CODES2;
+    int srow, valid;
+    const uint8_t* src;
+    int64_t step;  // bytes from one K block to the next
+    int krow = 0;
+    if constexpr (!ACROSS) {
+        const int row = tile_row0 + r;
+        srow = r;
+        valid = row < op.rows ? kKB : 0;
+        src = static_cast<const uint8_t*>(op.data) + (int64_t(row < op.rows ? row : 0) * op.ld) * kEbits / 8;
+        step = kKB * kEbits / 8;
+    } else {
+        const int half = r & 1, first = tile_row0 + 64 * half;
+        krow = r >> 1;
+        srow = 64 * half + krow;
+        const int left = op.rows - first;
+        valid = left < 0 ? 0 : (left > kKB ? kKB : left);
+        src = static_cast<const uint8_t*>(op.data) + (int64_t(krow) * op.ld + (valid > 0 ? first : 0)) * kEbits / 8;
+        step = int64_t(kKB) * op.ld * kEbits / 8;
+    }
+    auto load = [&](uint4 (&raw)[NW], int kb) {
+        const uint4* p = reinterpret_cast<const uint4*>(src + int64_t(kb) * step);
+#pragma unroll
+        for (int i = 0; i < NW; ++i) raw[i] = i * kPerWord < valid ? __ldg(p + i) : make_uint4(0u, 0u, 0u, 0u);
+    };
+    auto scale_at = [&](int kb) -> float {
+        if constexpr (kScaled) return __half2float(__ushort_as_half(__ldg(op.scales + kb * kKB + krow)));
+        return 1.f;
+    };
+    uint4 cur[NW], nxt[NW];
+    load(cur, 0);
+    float s_cur = scale_at(0), s_nxt = 1.f;
+    int s = 0;
+    uint32_t round = 0;  // how many times the ring has wrapped
+    for (int kb = 0; kb < kblocks; ++kb) {
+        if (kb + 1 < kblocks) {
+            load(nxt, kb + 1);
+            s_nxt = scale_at(kb + 1);
+        }
+        if (round > 0 && !wait_bounded(ring.bar_empty + 8 * s, (round - 1) & 1, status)) return false;
+        const uint32_t tile = ring.sbase + s * ring.stage_bytes + tile_off;
+        if (valid == kKB) {
+            convert_store<KIND, kScaled, false>(cur, tile, srow, s_cur, valid);
+        } else {
+            convert_store<KIND, kScaled, true>(cur, tile, srow, s_cur, valid);
+        }
+        fence_proxy_async();  // written through the generic proxy, read by the tensor core through the async one
+        mbar_arrive(ring.bar_full + 8 * s);
+#pragma unroll
+        for (int i = 0; i < NW; ++i) cur[i] = nxt[i];
+        s_cur = s_nxt;
+        if (++s == ring.stages) s = 0, ++round;
+    }
+    return true;
+}
+
+template <bool ACROSS>
+__device__ __forceinline__ bool produce_kind(const Operand& op, int r, int tile_row0, uint32_t tile_off, const Ring& ring,
+                                             int kblocks, int* status) {
+    switch (op.kind) {
+        case BFQ_OP_F32: return produce<BFQ_OP_F32, ACROSS>(op, r, tile_row0, tile_off, ring, kblocks, status);
+        case BFQ_OP_BF16: return produce<BFQ_OP_BF16, ACROSS>(op, r, tile_row0, tile_off, ring, kblocks, status);
+        case BFQ_OP_CODES2: return produce<BFQ_OP_CODES2, ACROSS>(op, r, tile_row0, tile_off, ring, kblocks, status);
+        case BFQ_OP_CODES4: return produce<BFQ_OP_CODES4, ACROSS>(op, r, tile_row0, tile_off, ring, kblocks, status);
+        default: return produce<BFQ_OP_CODES8, ACROSS>(op, r, tile_row0, tile_off, ring, kblocks, status);
+    }
+}
+
 __global__ void __launch_bounds__(kProducers + 32, 1) k_dequant_gemm(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int tid = threadIdx.x, warp = tid >> 5;
     const int ta = terms_of(p.a.kind, p.a.transposed), tb = terms_of(p.b.kind, p.b.transposed);
-    const uint32_t stage_bytes = static_cast<uint32_t>(ta + tb) * kTileBytes;
-    const uint32_t bars = sbase + kStages * 4 * kTileBytes;  // full[2], empty[2], done, then the tensor-memory address
-    const uint32_t bar_full = bars, bar_empty = bars + 8 * kStages, bar_done = bars + 16 * kStages, tmem_slot = bar_done + 8;
+    Ring ring;
+    ring.sbase = sbase;
+    ring.stage_bytes = static_cast<uint32_t>(ta + tb) * kTileBytes;
+    ring.stages = stages_of(ta, tb);
+    const uint32_t bars = sbase + kRingBytes;  // full[6], empty[6], done, then the tensor-memory address
+    ring.bar_full = bars, ring.bar_empty = bars + 8 * kMaxStages;
+    const uint32_t bar_done = bars + 16 * kMaxStages, tmem_slot = bar_done + 8;
 
     if (warp == 0) tmem_alloc128(tmem_slot);
     if (tid == kProducers) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_full + 8 * s, kProducers);
-            mbar_init(bar_empty + 8 * s, 1);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(ring.bar_full + 8 * s, kProducers);
+            mbar_init(ring.bar_empty + 8 * s, 1);
         }
         mbar_init(bar_done, 1);
         mbar_init_fence();
@@ -250,28 +388,13 @@ __global__ void __launch_bounds__(kProducers + 32, 1) k_dequant_gemm(const Param
     bool ok = true;
 
     if (tid < kProducers) {
-        // ---- producers: thread = one tile row of A (threads 0..127) or of B (128..255) ----
+        // ---- producers: threads 0..127 build A's tiles, 128..255 B's ----
         const bool for_a = tid < kTile;
         const int r = tid & (kTile - 1);
         const Operand& op = for_a ? p.a : p.b;
-        const int row = (for_a ? m0 : n0) + r;
-        const int terms = for_a ? ta : tb;
-        float v[kKB];
-        for (int kb = 0; kb < kblocks && ok; ++kb) {
-            const int s = kb & 1;
-            if (kb >= kStages) ok = wait_bounded(bar_empty + 8 * s, ((kb >> 1) - 1) & 1, p.status);
-            if (!ok) break;
-            const uint32_t tile = sbase + s * stage_bytes + (for_a ? 0u : ta * kTileBytes);
-            if (row < op.rows) {
-                load_row(op, row, kb * kKB, v);
-            } else {
-#pragma unroll
-                for (int k = 0; k < kKB; ++k) v[k] = 0.f;
-            }
-            store_row(tile, r, terms, v);
-            fence_proxy_async();  // the tiles were written through the generic proxy, the tensor core reads them through the async one
-            mbar_arrive(bar_full + 8 * s);
-        }
+        const uint32_t tile_off = for_a ? 0u : static_cast<uint32_t>(ta) * kTileBytes;
+        ok = op.transposed ? produce_kind<true>(op, r, for_a ? m0 : n0, tile_off, ring, kblocks, p.status)
+                           : produce_kind<false>(op, r, for_a ? m0 : n0, tile_off, ring, kblocks, p.status);
         // ---- epilogue: accumulators -> alpha * row scale * column scale -> C ----
         if (ok) ok = wait_bounded(bar_done, 0, p.status);
         ok = __all_sync(0xFFFFFFFFu, ok);  // the tensor-memory loads below are warp-wide
@@ -284,38 +407,52 @@ __global__ void __launch_bounds__(kProducers + 32, 1) k_dequant_gemm(const Param
             if (row_ok && is_codes(p.a.kind) && !p.a.transposed) rs *= __half2float(__ushort_as_half(__ldg(p.a.scales + ra)));
             const bool col_scaled = is_codes(p.b.kind) && !p.b.transposed;
             float* crow = p.c + int64_t(row_ok ? ra : 0) * p.ldc + n0;
+            const bool vec = (p.ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(p.c) & 15u) == 0;
             const uint32_t tlane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
             const int cbase = 64 * (warp >> 2);
             for (int c0 = cbase; c0 < cbase + 64; c0 += 32) {
                 uint32_t acc[32];
                 tmem_ld32(tlane + c0, acc);
                 tmem_wait_ld32(acc);
+                float out[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const int col = n0 + c0 + j;
-                    if (row_ok && col < p.b.rows) {
-                        float cs = 1.f;
-                        if (col_scaled) cs = __half2float(__ushort_as_half(__ldg(p.b.scales + col)));
-                        crow[c0 + j] = __uint_as_float(acc[j]) * rs * cs;
-                    }
+                    float cs = rs;
+                    if (col_scaled && n0 + c0 + j < p.b.rows) cs *= __half2float(__ushort_as_half(__ldg(p.b.scales + n0 + c0 + j)));
+                    out[j] = __uint_as_float(acc[j]) * cs;
+                }
+                if (!row_ok) continue;
+                if (vec && n0 + c0 + 32 <= p.b.rows) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(crow + c0 + j) = make_float4(out[j], out[j + 1], out[j + 2], out[j + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (n0 + c0 + j < p.b.rows) crow[c0 + j] = out[j];
                 }
             }
         }
     } else if (tid == kProducers) {
         // ---- one thread issues the MMAs: every pair of terms, four K steps of 16 per block ----
-        for (int kb = 0; kb < kblocks && ok; ++kb) {
-            const int s = kb & 1;
-            ok = wait_bounded(bar_full + 8 * s, (kb >> 1) & 1, p.status);
+        const uint32_t idesc = make_idesc(p.a.transposed, p.b.transposed);
+        const uint32_t a_step = p.a.transposed ? 2048u : 32u, b_step = p.b.transposed ? 2048u : 32u;
+        const uint32_t a_lead = p.a.transposed ? 8192u : 16u, b_lead = p.b.transposed ? 8192u : 16u;
+        int s = 0;
+        uint32_t round = 0;
+        for (int kb = 0; kb < kblocks; ++kb) {
+            ok = wait_bounded(ring.bar_full + 8 * s, round & 1, p.status);
             if (!ok) break;
             tmem_fence_after();
-            const uint32_t at = sbase + s * stage_bytes, bt = at + ta * kTileBytes;
+            const uint32_t at = sbase + s * ring.stage_bytes, bt = at + ta * kTileBytes;
             for (int ia = 0; ia < ta; ++ia)
                 for (int ib = 0; ib < tb; ++ib)
 #pragma unroll
                     for (int ks = 0; ks < kKB / 16; ++ks)
-                        mma_bf16(tmem_base, desc_sw128(at + ia * kTileBytes + ks * 32), desc_sw128(bt + ib * kTileBytes + ks * 32),
-                                 (kb | ia | ib | ks) != 0 ? 1u : 0u);
-            mma_commit(bar_empty + 8 * s);  // arrives when the MMAs issued so far have read their operands and finished
+                        mma_bf16(tmem_base, desc_sw128(at + ia * kTileBytes + ks * a_step, a_lead),
+                                 desc_sw128(bt + ib * kTileBytes + ks * b_step, b_lead), idesc, (kb | ia | ib | ks) != 0 ? 1u : 0u);
+            mma_commit(ring.bar_empty + 8 * s);  // arrives when the MMAs issued so far have read their operands and finished
+            if (++s == ring.stages) s = 0, ++round;
         }
         if (ok) mma_commit(bar_done);
     }
@@ -358,7 +495,7 @@ extern "C" int bfq_dequant_gemm(bfq_plan* plan, int64_t m, int64_t n, int64_t k,
     if (k == 0) {
         e = cudaMemset2DAsync(c, size_t(ldc) * 4, 0, size_t(n) * 4, size_t(m), static_cast<cudaStream_t>(stream));
     } else {
-        constexpr size_t smem = size_t(kStages) * 4 * kTileBytes + 8 * (2 * kStages + 1) + 16 + 1024;
+        constexpr size_t smem = size_t(kRingBytes) + 8 * (2 * kMaxStages + 1) + 16 + 1024;
         static bool attr_set[bfq::kMaxDevices] = {false};
         if (!attr_set[plan->device]) {
             e = cudaFuncSetAttribute(k_dequant_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
