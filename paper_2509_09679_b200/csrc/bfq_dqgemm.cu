@@ -316,28 +316,40 @@ __device__ __forceinline__ bool produce(const Operand& op, int r, int tile_row0,
         if constexpr (kScaled) return __half2float(__ushort_as_half(__ldg(op.scales + kb * kKB + krow)));
         return 1.f;
     };
-    uint4 cur[NW], nxt[NW];
-    load(cur, 0);
-    float s_cur = scale_at(0), s_nxt = 1.f;
+    // the raw words of the next kDepth K blocks are in flight while the current one is converted
+    constexpr int kDepth = NW >= 16 ? 1 : (NW >= 8 ? 2 : 4);
+    uint4 buf[kDepth + 1][NW];
+    float sc[kDepth + 1];
+#pragma unroll
+    for (int d = 0; d <= kDepth; ++d) {
+        sc[d] = 1.f;
+        if (d < kDepth && d < kblocks) {
+            load(buf[d], d);
+            sc[d] = scale_at(d);
+        }
+    }
     int s = 0;
     uint32_t round = 0;  // how many times the ring has wrapped
     for (int kb = 0; kb < kblocks; ++kb) {
-        if (kb + 1 < kblocks) {
-            load(nxt, kb + 1);
-            s_nxt = scale_at(kb + 1);
+        if (kb + kDepth < kblocks) {
+            load(buf[kDepth], kb + kDepth);
+            sc[kDepth] = scale_at(kb + kDepth);
         }
         if (round > 0 && !wait_bounded(ring.bar_empty + 8 * s, (round - 1) & 1, status)) return false;
         const uint32_t tile = ring.sbase + s * ring.stage_bytes + tile_off;
         if (valid == kKB) {
-            convert_store<KIND, kScaled, false>(cur, tile, srow, s_cur, valid);
+            convert_store<KIND, kScaled, false>(buf[0], tile, srow, sc[0], valid);
         } else {
-            convert_store<KIND, kScaled, true>(cur, tile, srow, s_cur, valid);
+            convert_store<KIND, kScaled, true>(buf[0], tile, srow, sc[0], valid);
         }
         fence_proxy_async();  // written through the generic proxy, read by the tensor core through the async one
         mbar_arrive(ring.bar_full + 8 * s);
 #pragma unroll
-        for (int i = 0; i < NW; ++i) cur[i] = nxt[i];
-        s_cur = s_nxt;
+        for (int d = 0; d < kDepth; ++d) {
+#pragma unroll
+            for (int i = 0; i < NW; ++i) buf[d][i] = buf[d + 1][i];
+            sc[d] = sc[d + 1];
+        }
         if (++s == ring.stages) s = 0, ++round;
     }
     return true;
