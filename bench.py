@@ -569,7 +569,14 @@ def time_others(torch, synth, Plan, dev):
            lambda: plan8.forward_quant(x, 2, codes=codes, scales=scales), 5)
     y8 = torch.empty_like(x)
     record("forward_bf16_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan8.forward(x, out=y8), 5)
-    del x, y8
+    # backward at n = 8192 (generic kernel): a quarter of the rows
+    rows8 = wl.n_rows // 4
+    g8 = torch.randn((rows8, wl.n), device=dev, dtype=torch.float32).to(x.dtype)
+    dx8 = torch.empty_like(g8)
+    dth8 = torch.empty((wl.L, wl.n // 2), dtype=torch.float32, device=dev)
+    record("backward_n8192", rows8, wl.n, wl.L, 14, 3 * 2 * wl.n,
+           lambda: plan8.backward(x[:rows8], g8, dx=dx8, dtheta=dth8), 3)
+    del x, y8, g8, dx8
     wl = synth.WORKLOADS["fold8192_int2"]
     W = wl.x(device=dev)
     record("fold_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,

@@ -105,7 +105,8 @@ static cudaError_t launch_generic(const bfq_plan* plan, const GenericParams& p, 
 template <int LOG_N, int R>
 static cudaError_t launch_backward_t(bfq_plan* plan, BackwardParams p, float* dtheta, cudaStream_t st) {
     using G = Geo<LOG_N>;
-    constexpr size_t smem = sizeof(float) * size_t(G::kGroups) * R * G::kN;
+    // row buffers + the d-theta sums of every row group
+    constexpr size_t smem = sizeof(float) * size_t(G::kGroups) * (size_t(R) * G::kN + BwdAcc<LOG_N>::kFloats);
     static int blocks_per_sm[kMaxDevices] = {0};
     auto kern = k_backward_generic<LOG_N, R>;
     int& occ = blocks_per_sm[plan->device];

@@ -415,12 +415,20 @@ __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_generic(const GenericP
 }
 
 // ---- backward ------------------------------------------------------------------------------------
-// One thread owns the same pairs (stage, j) for every row its CTA processes, so its d-theta
-// partial sums need no atomics.  Rows are assigned to CTAs statically (tile = blockIdx.x + k *
+// One thread owns the same pairs (stage, j) for every row its row group processes, so its d-theta sums need no
+// atomics: they are kept in shared memory (one array [L][n/2] per row group; at n = 8192, where that would not fit
+// beside the row buffer, the last stage's eight sums per thread stay in registers) for all rows of the CTA and written
+// to the CTA's partial-sum slot once, at the end.  Rows are assigned to CTAs statically (tile = blockIdx.x + k *
 // gridDim.x), which fixes the summation order.
+template <int LOG_N>
+struct BwdAcc {
+    static constexpr int kSmemStages = LOG_N > 12 ? 12 : LOG_N;  // stages whose sums live in shared memory
+    static constexpr int kFloats = kSmemStages * Geo<LOG_N>::kHalf;
+};
+
 template <int LOG_N, int P, int R>
 __device__ __forceinline__ void backward_phase(float (&v)[R][16], float (&w)[R][16], const float2* __restrict__ tw,
-                                               int t, float* __restrict__ part) {
+                                               int t, float* __restrict__ sacc, float (&racc)[8]) {
     using PH = Phase<LOG_N, P>;
 #pragma unroll
     for (int kk = 0; kk < PH::kNs; ++kk) {
@@ -440,7 +448,11 @@ __device__ __forceinline__ void backward_phase(float (&v)[R][16], float (&w)[R][
                 // stage-output form of g^T (dG/dtheta) z:  g_hi * z'_lo - g_lo * z'_hi
                 d += w[r][e_hi] * v[r][e_lo] - w[r][e_lo] * v[r][e_hi];
             }
-            part[b * Geo<LOG_N>::kHalf + j] += d;
+            if (b < BwdAcc<LOG_N>::kSmemStages) {
+                sacc[b * Geo<LOG_N>::kHalf + j] += d;
+            } else {
+                racc[q] += d;
+            }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const float a = v[r][e_lo], bb = v[r][e_hi];
@@ -456,17 +468,19 @@ __device__ __forceinline__ void backward_phase(float (&v)[R][16], float (&w)[R][
 
 template <int LOG_N, int P, int R>
 __device__ __forceinline__ void backward_from(float (&v)[R][16], float (&w)[R][16], const float2* tw, float* rowbuf,
-                                              int t, float* part) {
-    backward_phase<LOG_N, P, R>(v, w, tw, t, part);
+                                              int t, float* sacc, float (&racc)[8]) {
+    backward_phase<LOG_N, P, R>(v, w, tw, t, sacc, racc);
     if constexpr (P > 0) {
         exchange<LOG_N, P, P - 1, R>(v, rowbuf, t);
         exchange<LOG_N, P, P - 1, R>(w, rowbuf, t);
-        backward_from<LOG_N, P - 1, R>(v, w, tw, rowbuf, t, part);
+        backward_from<LOG_N, P - 1, R>(v, w, tw, rowbuf, t, sacc, racc);
     }
 }
 
-template <int LOG_N, int P>
-__device__ __forceinline__ void zero_partials(int t, float* part) {
+// the pairs thread t owns in phase P (and the phases after it): zero the shared-memory sums (ZERO) or copy the sums to
+// the partial-sum slot in global memory
+template <int LOG_N, int P, bool ZERO>
+__device__ __forceinline__ void visit_partials(int t, float* __restrict__ sacc, const float (&racc)[8], float* __restrict__ part) {
     using PH = Phase<LOG_N, P>;
 #pragma unroll
     for (int k = 0; k < PH::kNs; ++k) {
@@ -477,21 +491,30 @@ __device__ __forceinline__ void zero_partials(int t, float* part) {
             const int e_lo = ((q >> lb) << (lb + 1)) | (q & ((1 << lb) - 1));
             const int i = PH::idx(t, e_lo);
             const int j = ((i >> (b + 1)) << b) | (i & ((1 << b) - 1));
-            part[b * Geo<LOG_N>::kHalf + j] = 0.f;
+            const int at = b * Geo<LOG_N>::kHalf + j;
+            if (b < BwdAcc<LOG_N>::kSmemStages) {
+                if (ZERO) sacc[at] = 0.f; else part[at] = sacc[at];
+            } else if (!ZERO) {
+                part[at] = racc[q];
+            }
         }
     }
-    if constexpr (P + 1 < Geo<LOG_N>::kPhases) zero_partials<LOG_N, P + 1>(t, part);
+    if constexpr (P + 1 < Geo<LOG_N>::kPhases) visit_partials<LOG_N, P + 1, ZERO>(t, sacc, racc, part);
 }
 
 template <int LOG_N, int R>
-__global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_backward_generic(const BackwardParams p) {
+__global__ void __launch_bounds__(Geo<LOG_N>::kThreads, 1) k_backward_generic(const BackwardParams p) {
     using G = Geo<LOG_N>;
     extern __shared__ __align__(16) float smem[];
     const int group = threadIdx.x / G::kTPR;
     const int t = threadIdx.x % G::kTPR;
     float* rowbuf = smem + group * R * G::kN;
+    float* sacc = smem + G::kGroups * R * G::kN + group * BwdAcc<LOG_N>::kFloats;
     float* part = p.partial + (static_cast<int64_t>(blockIdx.x) * G::kGroups + group) * (LOG_N * G::kHalf);
-    zero_partials<LOG_N, 0>(t, part);
+    float racc[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) racc[q] = 0.f;
+    visit_partials<LOG_N, 0, true>(t, sacc, racc, part);  // each slot is only ever touched by its owner: no barrier
 
     constexpr int kRowsPerTile = G::kGroups * R;
     const int64_t tiles = (p.rows + kRowsPerTile - 1) / kRowsPerTile;
@@ -505,13 +528,14 @@ __global__ void __launch_bounds__(Geo<LOG_N>::kThreads) k_backward_generic(const
         }
         forward_from<LOG_N, 0, R>(v, p.tw, rowbuf, t);  // v = y = Q x, last-phase ownership
         if constexpr (G::kPhases > 1) exchange<LOG_N, 0, G::kPhases - 1, R>(w, rowbuf, t);
-        backward_from<LOG_N, G::kPhases - 1, R>(v, w, p.tw, rowbuf, t, part);
+        backward_from<LOG_N, G::kPhases - 1, R>(v, w, p.tw, rowbuf, t, sacc, racc);
         if (p.dx != nullptr) {
 #pragma unroll
             for (int r = 0; r < R; ++r)
                 if (row0 + r < p.rows) store16(p.dx, p.dxt, (row0 + r) * p.ld + t * 16, w[r]);
         }
     }
+    visit_partials<LOG_N, 0, false>(t, sacc, racc, part);
 }
 
 // dtheta[k] = sum over partial slots in slot order (fixed order => reproducible bits)

@@ -57,7 +57,7 @@ static cudaError_t launch(int device, const PerDevice& d, BackwardParams p, cons
                           cudaStream_t st) {
     using G = Geo<LOG_N>;
     constexpr int R = 1;
-    constexpr size_t smem = sizeof(float) * size_t(G::kGroups) * R * G::kN;
+    constexpr size_t smem = sizeof(float) * size_t(G::kGroups) * (size_t(R) * G::kN + BwdAcc<LOG_N>::kFloats);
     constexpr int count = LOG_N * G::kHalf;
     auto kern = k_backward_generic<LOG_N, R>;
     static bool attr_set[kMaxDevices] = {false};
