@@ -187,19 +187,20 @@ struct Params {
     int* status;
 };
 
-// zeroes the elements >= valid of chunk j (elements 8j .. 8j+7, two per word)
-__device__ __forceinline__ void mask_chunk(uint32_t (&o)[4], int j, int valid) {
+// zeroes the elements >= valid of the c-th chunk of a piece (its elements 8c .. 8c+7, two per word)
+__device__ __forceinline__ void mask_chunk(uint32_t (&o)[4], int c, int valid) {
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-        const int e = 8 * j + 2 * w;
+        const int e = 8 * c + 2 * w;
         o[w] = e >= valid ? 0u : (e + 1 >= valid ? (o[w] & 0xFFFFu) : o[w]);
     }
 }
 
-// One chunk (8 elements as 4 words of exact bf16 pairs) to the tile: as it is, or times the row's scale in two terms
+// One chunk (8 elements as 4 words of exact bf16 pairs) to chunk j of row `srow`: as it is, or times the scale in two
+// terms.  c = which chunk of its piece this is (for the masking of a partial piece).
 template <bool SCALED, bool PARTIAL>
-__device__ __forceinline__ void store_bf16_chunk(uint32_t tile, int srow, int j, uint32_t (&o)[4], float s, int valid) {
-    if constexpr (PARTIAL) mask_chunk(o, j, valid);
+__device__ __forceinline__ void store_bf16_chunk(uint32_t tile, int srow, int j, int c, uint32_t (&o)[4], float s, int valid) {
+    if constexpr (PARTIAL) mask_chunk(o, c, valid);
     const uint32_t at = chunk_addr(tile, srow, j);
     if constexpr (!SCALED) {
         sts128(at, o[0], o[1], o[2], o[3]);
@@ -212,64 +213,56 @@ __device__ __forceinline__ void store_bf16_chunk(uint32_t tile, int srow, int j,
     }
 }
 
-// The 64 elements of one shared-memory row from their raw 16-byte words.  SCALED (codes contracted across their stored
-// rows): times `s`, two terms.
+// One raw 16-byte word = piece p of shared-memory row `srow` (the row's 64 elements are 128 / kPerWord pieces).
+// SCALED (codes contracted across their stored rows): times `s`, two terms.  PARTIAL: only the first `valid` elements
+// of the piece exist; the others are stored as zero.
 template <int KIND, bool SCALED, bool PARTIAL>
-__device__ __forceinline__ void convert_store(const uint4 (&raw)[RawWords<KIND>::kCount], uint32_t tile, int srow, float s,
-                                              int valid) {
+__device__ __forceinline__ void convert_word(const uint4 raw, uint32_t tile, int srow, int p, float s, int valid) {
     if constexpr (KIND == BFQ_OP_F32) {
+        // 4 numbers = half of chunk p / 2
+        uint32_t hi[2], lo[2];
+        split2(__uint_as_float(raw.x), __uint_as_float(raw.y), hi[0], lo[0]);
+        split2(__uint_as_float(raw.z), __uint_as_float(raw.w), hi[1], lo[1]);
+        if constexpr (PARTIAL) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint4 u = raw[2 * j], v = raw[2 * j + 1];
-            uint32_t hi[4], lo[4];
-            split2(__uint_as_float(u.x), __uint_as_float(u.y), hi[0], lo[0]);
-            split2(__uint_as_float(u.z), __uint_as_float(u.w), hi[1], lo[1]);
-            split2(__uint_as_float(v.x), __uint_as_float(v.y), hi[2], lo[2]);
-            split2(__uint_as_float(v.z), __uint_as_float(v.w), hi[3], lo[3]);
-            if constexpr (PARTIAL) mask_chunk(hi, j, valid), mask_chunk(lo, j, valid);
-            const uint32_t at = chunk_addr(tile, srow, j);
-            sts128(at, hi[0], hi[1], hi[2], hi[3]);
-            sts128(at + kTileBytes, lo[0], lo[1], lo[2], lo[3]);
-        }
-    } else if constexpr (KIND == BFQ_OP_BF16) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint32_t o[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
-            store_bf16_chunk<false, PARTIAL>(tile, srow, j, o, 1.f, valid);
-        }
-    } else if constexpr (KIND == BFQ_OP_CODES4) {
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const uint32_t ws[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                uint32_t o[4];
-                codes4_to_bf16(ws[w], o);
-                store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 4 * i + w, o, s, valid);
+            for (int w = 0; w < 2; ++w) {
+                const uint32_t m = 2 * w >= valid ? 0u : (2 * w + 1 >= valid ? 0xFFFFu : 0xFFFFFFFFu);
+                hi[w] &= m, lo[w] &= m;
             }
         }
+        const uint32_t at = chunk_addr(tile, srow, p >> 1) + 8u * (p & 1);
+        asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(at), "r"(hi[0]), "r"(hi[1]) : "memory");
+        asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(at + kTileBytes), "r"(lo[0]), "r"(lo[1]) : "memory");
+    } else if constexpr (KIND == BFQ_OP_BF16) {
+        uint32_t o[4] = {raw.x, raw.y, raw.z, raw.w};
+        store_bf16_chunk<false, PARTIAL>(tile, srow, p, 0, o, 1.f, valid);
+    } else if constexpr (KIND == BFQ_OP_CODES4) {
+        const uint32_t ws[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            uint32_t o[4];
+            codes4_to_bf16(ws[w], o);
+            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 4 * p + w, w, o, s, valid);
+        }
     } else if constexpr (KIND == BFQ_OP_CODES2) {
-        const uint32_t ws[4] = {raw[0].x, raw[0].y, raw[0].z, raw[0].w};
+        const uint32_t ws[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
             uint32_t o8[8];
             codes2_to_bf16(ws[w], o8);
             uint32_t oa[4] = {o8[0], o8[1], o8[2], o8[3]}, ob[4] = {o8[4], o8[5], o8[6], o8[7]};
-            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * w, oa, s, valid);
-            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * w + 1, ob, s, valid);
+            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 8 * p + 2 * w, 2 * w, oa, s, valid);
+            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 8 * p + 2 * w + 1, 2 * w + 1, ob, s, valid);
         }
     } else {
+        const uint32_t ws[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t ws[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t o2a[2], o2b[2];
-                codes8_to_bf16(ws[2 * h], o2a);
-                codes8_to_bf16(ws[2 * h + 1], o2b);
-                uint32_t o[4] = {o2a[0], o2a[1], o2b[0], o2b[1]};
-                store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * i + h, o, s, valid);
-            }
+        for (int h = 0; h < 2; ++h) {
+            uint32_t o2a[2], o2b[2];
+            codes8_to_bf16(ws[2 * h], o2a);
+            codes8_to_bf16(ws[2 * h + 1], o2b);
+            uint32_t o[4] = {o2a[0], o2a[1], o2b[0], o2b[1]};
+            store_bf16_chunk<SCALED, PARTIAL>(tile, srow, 2 * p + h, h, o, s, valid);
         }
     }
 }
@@ -279,76 +272,88 @@ struct Ring {
     int stages;
 };
 
-// Producer loop of one thread: shared-memory row `srow` of every K block of its operand.  ACROSS: the operand is stored
-// [K][rows]; the thread's row is stored row k0 + (r >> 1), tile rows 64 (r & 1) .. + 63.
+// Producer loop of one thread of the 128 that build one operand's tiles.  A K block of the operand is 128 shared-memory
+// rows of kLpr 16-byte pieces; piece id = i * 128 + r (i = 0 .. kLpr - 1) is piece id % kLpr of row id / kLpr, so the
+// lanes of a warp read consecutive pieces of the same stored row: global loads are coalesced as far as the stored row
+// allows.  ACROSS: the operand is stored [K][rows]; shared-memory row 64 h + k is stored row k0 + k, tile rows
+// 64 h .. 64 h + 63.
 template <int KIND, bool ACROSS>
 __device__ __forceinline__ bool produce(const Operand& op, int r, int tile_row0, uint32_t tile_off, const Ring& ring, int kblocks,
                                         int* status) {
-    constexpr int NW = RawWords<KIND>::kCount;
+    constexpr int kLpr = RawWords<KIND>::kCount;  // pieces per row = pieces per thread
     constexpr int kEbits = KIND == BFQ_OP_F32 ? 32 : (KIND == BFQ_OP_BF16 ? 16 : KIND);
-    constexpr int kPerWord = 128 / kEbits;  // elements per 16-byte word
+    constexpr int kPerWord = 128 / kEbits;  // elements per piece
     constexpr bool kScaled = ACROSS && KIND >= BFQ_OP_CODES2;
-    int srow, valid;
-    const uint8_t* src;
-    int64_t step;  // bytes from one K block to the next
-    int krow = 0;
-    if constexpr (!ACROSS) {
-        const int row = tile_row0 + r;
-        srow = r;
-        valid = row < op.rows ? kKB : 0;
-        src = static_cast<const uint8_t*>(op.data) + (int64_t(row < op.rows ? row : 0) * op.ld) * kEbits / 8;
-        step = kKB * kEbits / 8;
-    } else {
-        const int half = r & 1, first = tile_row0 + 64 * half;
-        krow = r >> 1;
-        srow = 64 * half + krow;
-        const int left = op.rows - first;
-        valid = left < 0 ? 0 : (left > kKB ? kKB : left);
-        src = static_cast<const uint8_t*>(op.data) + (int64_t(krow) * op.ld + (valid > 0 ? first : 0)) * kEbits / 8;
-        step = int64_t(kKB) * op.ld * kEbits / 8;
-    }
-    auto load = [&](uint4 (&raw)[NW], int kb) {
-        const uint4* p = reinterpret_cast<const uint4*>(src + int64_t(kb) * step);
-#pragma unroll
-        for (int i = 0; i < NW; ++i) raw[i] = i * kPerWord < valid ? __ldg(p + i) : make_uint4(0u, 0u, 0u, 0u);
+    constexpr int kRowStep = kTile / kLpr;  // rows between a thread's consecutive pieces
+    const int p = r % kLpr, row_first = r / kLpr;
+    const uint8_t* const base = static_cast<const uint8_t*>(op.data);
+    const int64_t pitch = op.ld * kEbits / 8;  // bytes of a stored row
+    // per piece: how many of its elements exist (0: nothing is loaded) and where K block 0 of it starts
+    auto srow_of = [&](int i) { return row_first + i * kRowStep; };
+    auto valid_of = [&](int i) -> int {
+        if constexpr (!ACROSS) {
+            return tile_row0 + srow_of(i) < op.rows ? kPerWord : 0;
+        } else {
+            const int left = op.rows - (tile_row0 + 64 * (srow_of(i) >> 6) + p * kPerWord);
+            return left < 0 ? 0 : (left > kPerWord ? kPerWord : left);
+        }
     };
-    auto scale_at = [&](int kb) -> float {
-        if constexpr (kScaled) return __half2float(__ushort_as_half(__ldg(op.scales + kb * kKB + krow)));
-        return 1.f;
+    auto src_of = [&](int i, int kb) -> const uint4* {
+        if constexpr (!ACROSS) {
+            return reinterpret_cast<const uint4*>(base + int64_t(tile_row0 + srow_of(i)) * pitch + int64_t(kb) * (kKB * kEbits / 8) + 16 * p);
+        } else {
+            const int sr = srow_of(i);
+            return reinterpret_cast<const uint4*>(base + (int64_t(kb) * kKB + (sr & 63)) * pitch +
+                                                  int64_t(tile_row0 + 64 * (sr >> 6)) * kEbits / 8 + 16 * p);
+        }
+    };
+    auto load = [&](uint4 (&raw)[kLpr], float (&sc)[kLpr], int kb) {
+#pragma unroll
+        for (int i = 0; i < kLpr; ++i) {
+            raw[i] = valid_of(i) > 0 ? __ldg(src_of(i, kb)) : make_uint4(0u, 0u, 0u, 0u);
+            if constexpr (kScaled) sc[i] = __half2float(__ushort_as_half(__ldg(op.scales + kb * kKB + (srow_of(i) & 63))));
+        }
     };
     // the raw words of the next kDepth K blocks are in flight while the current one is converted
-    constexpr int kDepth = NW >= 16 ? 1 : (NW >= 8 ? 2 : 4);
-    uint4 buf[kDepth + 1][NW];
-    float sc[kDepth + 1];
-#pragma unroll
-    for (int d = 0; d <= kDepth; ++d) {
-        sc[d] = 1.f;
-        if (d < kDepth && d < kblocks) {
-            load(buf[d], d);
-            sc[d] = scale_at(d);
+    constexpr int kDepth = kLpr >= 16 ? 1 : (kLpr >= 8 ? 2 : 4);
+    uint4 buf[kDepth + 1][kLpr];
+    float sc[kDepth + 1][kScaled ? kLpr : 1];
+    auto load_slot = [&](int d, int kb) {
+        if constexpr (kScaled) {
+            load(buf[d], sc[d], kb);
+        } else {
+            float none[kLpr];
+            load(buf[d], none, kb);
         }
-    }
+    };
+#pragma unroll
+    for (int d = 0; d < kDepth; ++d)
+        if (d < kblocks) load_slot(d, d);
     int s = 0;
     uint32_t round = 0;  // how many times the ring has wrapped
     for (int kb = 0; kb < kblocks; ++kb) {
-        if (kb + kDepth < kblocks) {
-            load(buf[kDepth], kb + kDepth);
-            sc[kDepth] = scale_at(kb + kDepth);
-        }
+        if (kb + kDepth < kblocks) load_slot(kDepth, kb + kDepth);
         if (round > 0 && !wait_bounded(ring.bar_empty + 8 * s, (round - 1) & 1, status)) return false;
         const uint32_t tile = ring.sbase + s * ring.stage_bytes + tile_off;
-        if (valid == kKB) {
-            convert_store<KIND, kScaled, false>(buf[0], tile, srow, sc[0], valid);
-        } else {
-            convert_store<KIND, kScaled, true>(buf[0], tile, srow, sc[0], valid);
+#pragma unroll
+        for (int i = 0; i < kLpr; ++i) {
+            const int v = valid_of(i);
+            const float si = kScaled ? sc[0][kScaled ? i : 0] : 1.f;
+            if (v == kPerWord) {
+                convert_word<KIND, kScaled, false>(buf[0][i], tile, srow_of(i), p, si, v);
+            } else {
+                convert_word<KIND, kScaled, true>(buf[0][i], tile, srow_of(i), p, si, v);
+            }
         }
         fence_proxy_async();  // written through the generic proxy, read by the tensor core through the async one
         mbar_arrive(ring.bar_full + 8 * s);
 #pragma unroll
         for (int d = 0; d < kDepth; ++d) {
 #pragma unroll
-            for (int i = 0; i < NW; ++i) buf[d][i] = buf[d + 1][i];
-            sc[d] = sc[d + 1];
+            for (int i = 0; i < kLpr; ++i) {
+                buf[d][i] = buf[d + 1][i];
+                if constexpr (kScaled) sc[d][i] = sc[d + 1][i];
+            }
         }
         if (++s == ring.stages) s = 0, ++round;
     }
