@@ -581,6 +581,8 @@ def time_others(torch, synth, Plan, dev):
     W = wl.x(device=dev)
     record("fold_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
            lambda: plan8.fold_weights(W, 2), 5)
+    record("fold_int2_with_rows_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n + wl.n // 4 + 2,
+           lambda: plan8.fold_weights(W, 2, want_rotated=True), 5)
     del W, plan8
     torch.cuda.empty_cache()
     # composite 40 x 128 (d = 5120): both factors on the tensor cores (default), or butterfly-128 on the CUDA cores

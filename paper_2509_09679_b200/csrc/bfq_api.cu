@@ -337,6 +337,18 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
         e = fwdq4096_launch(plan, x, rows, ldx, false, codes, scales, nullptr, 0, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
+    // weight folding that keeps W Q^T in bf16: codes and rows from one pass of the tuned kernels
+    if (hist == nullptr && xt == BFQ_BF16 && y != nullptr && yt == BFQ_BF16 && rows < (int64_t(1) << 31) &&
+        !env_flag("BFQ_GENERIC_ONLY")) {
+        if (fwdq4096_available(plan)) {
+            e = fwdq4096_launch_codes_rows(plan, x, rows, ldx, bits, codes, scales, y, plan->n, static_cast<cudaStream_t>(stream));
+            return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+        }
+        if (fwdq8192_available(plan)) {
+            e = fwdq8192_launch_codes_rows(plan, x, rows, ldx, bits, codes, scales, y, plan->n, static_cast<cudaStream_t>(stream));
+            return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+        }
+    }
     if (hist == nullptr && xt == BFQ_BF16 && (bits == 2 || bits == 8) && y == nullptr && rows < (int64_t(1) << 31) &&
         !env_flag("BFQ_GENERIC_ONLY") && fwdq4096_available(plan)) {
         e = fwdq4096_launch_bits(plan, x, rows, ldx, false, bits, codes, scales, static_cast<cudaStream_t>(stream));

@@ -19,6 +19,9 @@ cudaError_t fwdq4096_launch(const bfq_plan* plan, const void* x, int64_t rows, i
 // INT2 / INT8 codes from the same kernel (bits = 2 or 8)
 cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, bool hadamard, int bits,
                                  uint8_t* codes, uint16_t* scales, cudaStream_t st);
+// codes + scales (bits = 2, 4, 8) and the rotated rows in bf16 from one pass
+cudaError_t fwdq4096_launch_codes_rows(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits,
+                                       uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 // the same with the statistics of bfq_forward_quant_stats (hist already zeroed on `st`)
 cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                   uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st);
@@ -30,6 +33,8 @@ bool fwdq8192_available(const bfq_plan* plan);
 cudaError_t fwdq8192_set_angles(const bfq_plan* plan, const float* theta, cudaStream_t st);
 cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
                             uint16_t* scales, cudaStream_t st);
+cudaError_t fwdq8192_launch_codes_rows(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits,
+                                       uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 cudaError_t fwdq8192_launch_bf16(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, void* y, int64_t ldy,
                                  cudaStream_t st);
 

@@ -178,7 +178,8 @@ enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutIn
 // codes + scales + the second and fourth moment of every rotated row (`yout` then points to float [rows][2]) + the
 // tensor-wide counts of the 16 code values added to `hist`, or INT2 / INT8 codes + scales.
 // STEP: group g passes its token to group (g + STEP) % G, so gcd(STEP, G) groups rotate at a time (0: no tokens).
-template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2>
+// ROWS (code outputs only): the rotated rows are written as well, in bf16, to `yout` (weight folding that keeps W Q^T).
+template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2, bool ROWS = false>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, const int* __restrict__ form,
            uint8_t* __restrict__ codes,
@@ -343,7 +344,8 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             run_hadamard<XB>(P, ex, issue_next);
         }
 
-        if constexpr (OUT == kOutBf16) {
+        static_assert(!ROWS || OUT == kOutInt4 || OUT == kOutInt2 || OUT == kOutInt8, "rows beside codes only");
+        if constexpr (OUT == kOutBf16 || ROWS) {
             // thread t holds elements 2t + 256m, +1: one 32-bit word of the bf16 row per packed register
             uint32_t* out = reinterpret_cast<uint32_t*>(yout + static_cast<int64_t>(row) * ldy) + t;
 #pragma unroll
@@ -353,6 +355,8 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                 const __nv_bfloat162 v = __floats2bfloat162_rn(a * kPost, b * kPost);
                 out[128 * m] = *reinterpret_cast<const uint32_t*>(&v);
             }
+        }
+        if constexpr (OUT == kOutBf16) {
             bar_sync(ex.bar, kGroupThreads);  // every warp is past its reads of the second regrouping buffer
             continue;
         }
@@ -650,13 +654,13 @@ bool fwdq4096_available(const bfq_plan* plan) {
     return plan->n == f4k::kN && plan->cc_major == 10 && plan->img4096 != nullptr && encode_tiled() != nullptr;
 }
 
-template <int G, int CW, int XB, int TRANSFORM, int OUT>
+template <int G, int CW, int XB, int TRANSFORM, int OUT, bool ROWS = false>
 static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap, int64_t rows, uint8_t* codes,
                                   uint16_t* scales, void* y, int64_t ldy, cudaStream_t st,
                                   unsigned long long* hist = nullptr) {
     using S = f4k::Smem<G, XB>;
     static bool attr_set[kMaxDevices] = {false};
-    auto kern = f4k::k_fwdq4096<G, CW, XB, TRANSFORM, OUT>;
+    auto kern = f4k::k_fwdq4096<G, CW, XB, TRANSFORM, OUT, 2, ROWS>;
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
         if (e != cudaSuccess) return e;
@@ -702,6 +706,17 @@ cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t ro
     }
     return bits == 2 ? launch_variant<4, 32, 2, kButterfly, kOutInt2>(plan, tmap, rows, codes, scales, nullptr, 0, st)
                      : launch_variant<4, 32, 2, kButterfly, kOutInt8>(plan, tmap, rows, codes, scales, nullptr, 0, st);
+}
+
+// weight folding that keeps the rotated rows: codes + scales and W Q^T in bf16 (leading dimension ldy) from one pass
+cudaError_t fwdq4096_launch_codes_rows(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits,
+                                       uint8_t* codes, uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
+    CUtensorMap tmap;
+    if (!encode_row_map(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
+    using namespace f4k;
+    if (bits == 4) return launch_variant<4, 32, 2, kButterfly, kOutInt4, true>(plan, tmap, rows, codes, scales, y, ldy, st);
+    if (bits == 2) return launch_variant<4, 32, 2, kButterfly, kOutInt2, true>(plan, tmap, rows, codes, scales, y, ldy, st);
+    return launch_variant<4, 32, 2, kButterfly, kOutInt8, true>(plan, tmap, rows, codes, scales, y, ldy, st);
 }
 
 // bfq_forward_quant_stats on the tuned path: codes + scales + row moments + code counts from one launch of k_fwdq4096

@@ -125,11 +125,13 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
 // (`codes` then points to them, leading dimension ldy); the absmax hand-shake between the two CTAs is kept, since it is
 // also what tells a CTA that its peer has read the exchange box of the row.
 // STEP: token passing between the row groups of a CTA as in the n = 4096 kernel (0: none).
-template <int G, int BITS, int STEP = 2>
+// ROWS (BITS = 2, 4, 8): the rotated rows are written as well, in bf16, to `yrows` (leading dimension ldy).
+template <int G, int BITS, int STEP = 2, bool ROWS = false>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
            const float* __restrict__ img, const int* __restrict__ form, uint8_t* __restrict__ codes,
-           uint16_t* __restrict__ scales, int64_t ldy, int rows, int* __restrict__ status) {
+           uint16_t* __restrict__ scales, int64_t ldy, int rows, int* __restrict__ status,
+           __nv_bfloat16* __restrict__ yrows) {
     using S = Smem<G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -331,9 +333,11 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         mbar_wait_cluster_bounded(bar_amax, k & 1, status);
         amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
         float inv;
-        if constexpr (BITS == 16) {
+        static_assert(!(ROWS && BITS == 16), "BITS = 16 writes the rows already");
+        if constexpr (BITS == 16 || ROWS) {
             // A[i] holds elements 2048 rank + 256 i + 2 t (+1), B[i] the same 4096 further on: one 32-bit word each
-            uint32_t* yrow = reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(codes) + static_cast<int64_t>(row) * ldy);
+            uint32_t* yrow = reinterpret_cast<uint32_t*>((BITS == 16 ? reinterpret_cast<__nv_bfloat16*>(codes) : yrows) +
+                                                         static_cast<int64_t>(row) * ldy);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 float a0, a1, b0, b1;
@@ -343,8 +347,8 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
                 yrow[1024 * rank + 128 * i + t] = *reinterpret_cast<const uint32_t*>(&va);
                 yrow[2048 + 1024 * rank + 128 * i + t] = *reinterpret_cast<const uint32_t*>(&vb);
             }
-            continue;
         }
+        if constexpr (BITS == 16) continue;
         constexpr int kQmax = BITS == 16 ? 1 : (1 << (BITS - 1)) - 1;
         const uint16_t s16 = row_scale_fast<kQmax>(amax, &inv);
         stg16_if(rank == 0 && t == 0, scales + row, s16);
@@ -533,12 +537,12 @@ bool fwdq8192_available(const bfq_plan* plan) {
            encode_tiled() != nullptr;
 }
 
-template <int BITS>
+template <int BITS, bool ROWS = false>
 static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                                        uint16_t* scales, int64_t ldy, cudaStream_t st) {
+                                        uint16_t* scales, int64_t ldy, cudaStream_t st, void* yrows = nullptr) {
     constexpr int G = 4;
     using S = f8k::Smem<G>;
-    auto kern = f8k::k_fwdq8192<G, BITS>;
+    auto kern = f8k::k_fwdq8192<G, BITS, 2, ROWS>;
     static bool attr_set[kMaxDevices] = {false};
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
@@ -567,7 +571,8 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192),
-                              static_cast<const int*>(plan->form_flag), codes, scales, ldy, int(rows), plan->status_word);
+                              static_cast<const int*>(plan->form_flag), codes, scales, ldy, int(rows), plan->status_word,
+                              static_cast<__nv_bfloat16*>(yrows));
 }
 
 cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
@@ -575,6 +580,14 @@ cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, i
     if (bits == 2) return fwdq8192_launch_bits<2>(plan, x, rows, ldx, codes, scales, 0, st);
     if (bits == 4) return fwdq8192_launch_bits<4>(plan, x, rows, ldx, codes, scales, 0, st);
     return fwdq8192_launch_bits<8>(plan, x, rows, ldx, codes, scales, 0, st);
+}
+
+// codes + scales and the rotated rows in bf16 from one pass (weight folding that keeps W Q^T)
+cudaError_t fwdq8192_launch_codes_rows(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits,
+                                       uint8_t* codes, uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
+    if (bits == 2) return fwdq8192_launch_bits<2, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
+    if (bits == 4) return fwdq8192_launch_bits<4, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
+    return fwdq8192_launch_bits<8, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
 }
 
 // y = Q x in bf16 (the weight-only setting: activations stay 16-bit)

@@ -595,3 +595,20 @@ def test_fold_weights_n4096_int2_on_the_tuned_kernel():
     deq = oracle.dequantize(oracle.unpack(codes.cpu().numpy(), 2), scales.cpu().view(torch.int16).numpy().view(np.uint16))
     assert abs(np.linalg.norm(deq @ Qx.T - ref) - err_ref) <= 1e-3 * err_ref
     assert p.device_status() == 0
+
+
+@pytest.mark.parametrize("n,bits,m", [(4096, 2, 293), (4096, 4, 37), (4096, 8, 5), (8192, 2, 151), (8192, 4, 9)])
+def test_fold_weights_with_rotated_rows_on_the_tuned_kernels(n, bits, m):
+    """bfq_fold_weights that also keeps W Q^T in bf16: codes, scales and rotated rows come from one pass of the tuned
+    kernels and must agree with the oracle like the two outputs do separately; the generic kernel gives the same codes."""
+    theta = synth.angles(n, "normal", 41)
+    W = synth.rows(m, n, "normal", 42, scale=0.02, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    ref = oracle.forward(to_f64(theta), to_f64(W))
+    codes, scales, rot = p.fold_weights(W.to(DEV), bits, want_rotated=True)
+    assert rot.dtype == torch.bfloat16
+    check_quant(codes, scales, ref, bits, f"fold + rows n={n} INT{bits}: codes")
+    check_rows_close(rot, ref, absmax_rows(W), f"fold + rows n={n} INT{bits}: rows")
+    codes2, scales2, _ = p.fold_weights(W.to(DEV), bits)
+    assert torch.equal(codes, codes2) and torch.equal(scales.view(torch.int16), scales2.view(torch.int16))
+    assert p.device_status() == 0
