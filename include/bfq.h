@@ -200,7 +200,7 @@ int bfq_composite_inverse(bfq_plan* plan, const float* q1, int n1, const void* y
  *   - n <= BFQ_NOALLOC_MAX_N (power of two >= BFQ_MIN_N), else BFQ_ERR_TOO_LARGE; rows is unlimited;
  *   - all calls share the one array: calls that may overlap on a GPU (different streams, different
  *     threads) race with each other -- serialise them; contents left by an earlier call are harmless
- *     (each call rewrites the table and zeroes the partial sums it reads);
+ *     (each call rewrites the table and overwrites the partial sums it reads);
  *   - the first call on each device resolves the array's address (cudaGetSymbolAddress) and sets a
  *     kernel attribute; make that first call before any stream capture begins.
  * It calls no cudaMalloc, cudaFree or other allocating routine.  d-theta is bit-reproducible from call

@@ -11,8 +11,8 @@
 //
 // Consequences of the shared array: the row length is limited to BFQ_NOALLOC_MAX_N; all calls (from
 // any stream or thread) use the same bytes, so two calls that overlap on one GPU race; the array
-// keeps the previous call's contents, and each call rewrites the table and zeroes exactly the
-// partial sums it is going to read before it uses them.
+// keeps the previous call's contents, and each call rewrites the table and overwrites exactly the
+// partial sums it is going to read (every CTA stores its finished sums into its own slots).
 #include "../../include/bfq.h"
 
 #include <cuda_runtime.h>
@@ -81,7 +81,7 @@ static cudaError_t launch(int device, const PerDevice& d, BackwardParams p, cons
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     p.tw = tw;
-    p.partial = partial;  // every CTA zeroes its own slots before accumulating into them
+    p.partial = partial;  // every CTA overwrites its own slots with its finished sums
     kern<<<grid, G::kThreads, smem, st>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
