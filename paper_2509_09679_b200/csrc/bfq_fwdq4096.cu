@@ -423,44 +423,82 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         inv *= kPost;  // the registers still hold the un-normalised values (kPost is a power of two)
         stg16_if(t == 0, scales + row, s16);
 
-        if constexpr (OUT == kOutInt8 || OUT == kOutInt2) {
+        if constexpr (OUT == kOutInt8) {
             // |v * inv| <= qmax (1 + 2^-10) < qmax + 1/2 for a normal, unsaturated fp16 scale: no clipping; v * inv +
             // 1.5 * 2^23 then has the code (two's complement) in its low mantissa bits
             const bool plain8 = (((s16 >> 10) & 31u) != 0u) && (s16 != 0x7BFFu);
-            uint32_t c[16];  // INT8: two bytes; INT2: four bits (two codes) of each packed register
+            // thread t holds elements 2t + 256m, +1 = bytes 2t + 256m, +1 of the row
+            uint16_t* out16 = reinterpret_cast<uint16_t*>(codes + static_cast<size_t>(row) * kN) + t;
+            if (plain8) {
+                // u = code + 128 in the low byte of v * inv + (1.5 * 2^23 + 128), whose other low bits are zero:
+                // hi * 256 + lo has u_hi, u_lo in its two low bytes; the XOR turns offset binary into two's complement
+                const u64 inv2 = pack2(inv, inv), magic2 = pack2(12583040.0f, 12583040.0f);
 #pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                uint32_t lo, hi;
-                if (plain8) {
-                    unpack2u(fma2(P[m], pack2(inv, inv), pack2(12582912.0f, 12582912.0f)), lo, hi);
-                } else {
+                for (int m = 0; m < 16; ++m) {
+                    uint32_t lo, hi;
+                    unpack2u(fma2(P[m], inv2, magic2), lo, hi);
+                    out16[128 * m] = static_cast<uint16_t>((hi * 256u + lo) ^ 0x8080u);
+                }
+            } else {
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
                     float a, b;
                     unpack2(P[m], a, b);
-                    lo = static_cast<uint32_t>(quant1(a, inv, -kQmax - 1, kQmax));
-                    hi = static_cast<uint32_t>(quant1(b, inv, -kQmax - 1, kQmax));
+                    const uint32_t lo = static_cast<uint32_t>(quant1(a, inv, -kQmax - 1, kQmax));
+                    const uint32_t hi = static_cast<uint32_t>(quant1(b, inv, -kQmax - 1, kQmax));
+                    out16[128 * m] = static_cast<uint16_t>((lo & 0xFFu) | ((hi & 0xFFu) << 8));
                 }
-                c[m] = OUT == kOutInt8 ? ((lo & 0xFFu) | ((hi & 0xFFu) << 8)) : ((lo & 3u) | ((hi & 3u) << 2));
             }
-            if constexpr (OUT == kOutInt8) {
-                // thread t holds elements 2t + 256m, +1 = bytes 2t + 256m, +1 of the row
-                uint16_t* out16 = reinterpret_cast<uint16_t*>(codes + static_cast<size_t>(row) * kN) + t;
+            continue;
+        }
+        if constexpr (OUT == kOutInt2) {
+            // elements 2t + 256m, +1 are half of byte t/2 + 64m: the low half for even t, the high half for odd t.
+            // The sixteen 4-bit halves (two codes each) travel in two words, registers 0..7 and 8..15.
+            const bool plain2 = (((s16 >> 10) & 31u) != 0u) && (s16 != 0x7BFFu);
+            uint32_t w0 = 0u, w1 = 0u;
+            if (plain2) {
+                // |v * inv| <= 1.0005: v * inv + (1.5 * 2^23 + 2) has u = code + 2 in {1, 2, 3} in its low bits above
+                // the constant pattern C = 0x4B400000, so hi * 4 + lo = 5 C + (4 u_hi + u_lo); a Horner chain over the
+                // registers gives the nibbles times 16^m plus a constant, one subtraction removes it and one XOR turns
+                // every u into the two's complement code
+                const u64 inv2 = pack2(inv, inv), magic2 = pack2(12582914.0f, 12582914.0f);
 #pragma unroll
-                for (int m = 0; m < 16; ++m) out16[128 * m] = static_cast<uint16_t>(c[m]);
-            } else {
-                // elements 2t + 256m, +1 are half of byte t/2 + 64m: the low half for even t, the high half for odd t.
-                // The sixteen 4-bit halves travel in two words; the even thread writes bytes m = 0..7, the odd one 8..15.
-                uint32_t w0 = 0u, w1 = 0u;
-#pragma unroll
-                for (int m = 0; m < 8; ++m) w0 |= c[m] << (4 * m), w1 |= c[8 + m] << (4 * m);
-                const bool odd = t & 1;
-                const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, odd ? w0 : w1, 1);
-                const uint32_t mine = odd ? w1 : w0;  // the eight rows m this thread assembles
-                uint8_t* out2 = codes + static_cast<size_t>(row) * (kN / 4) + (t >> 1) + (odd ? 64 * 8 : 0);
-#pragma unroll
-                for (int m = 0; m < 8; ++m) {
-                    const uint32_t a4 = (mine >> (4 * m)) & 0xFu, b4 = (other >> (4 * m)) & 0xFu;
-                    out2[64 * m] = static_cast<uint8_t>(odd ? (b4 | (a4 << 4)) : (a4 | (b4 << 4)));
+                for (int m = 7; m >= 0; --m) {
+                    uint32_t lo, hi;
+                    unpack2u(fma2(P[m], inv2, magic2), lo, hi);
+                    w0 = w0 * 16u + (hi * 4u + lo);
+                    unpack2u(fma2(P[8 + m], inv2, magic2), lo, hi);
+                    w1 = w1 * 16u + (hi * 4u + lo);
                 }
+                constexpr uint32_t kBias = static_cast<uint32_t>((5ull * 0x4B400000ull * 0x11111111ull) & 0xFFFFFFFFull);
+                w0 = (w0 - kBias) ^ 0xAAAAAAAAu;
+                w1 = (w1 - kBias) ^ 0xAAAAAAAAu;
+            } else {
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    float a, b;
+                    unpack2(P[m], a, b);
+                    const uint32_t c = (static_cast<uint32_t>(quant1(a, inv, -2, 1)) & 3u) |
+                                       ((static_cast<uint32_t>(quant1(b, inv, -2, 1)) & 3u) << 2);
+                    if (m < 8) w0 |= c << (4 * m); else w1 |= c << (4 * (m - 8));
+                }
+            }
+            // the even thread writes bytes m = 0..7 (its nibbles + the odd thread's), the odd one 8..15 (the even
+            // thread's nibbles + its own): one exchange of a word, then nibble m of the two words side by side in byte m
+            const bool odd = t & 1;
+            const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, odd ? w0 : w1, 1);
+            const uint32_t low = odd ? other : w0, high = odd ? w1 : other;
+            auto spread4 = [](uint32_t x) {  // nibbles 0..3 of x into the low halves of bytes 0..3
+                x &= 0xFFFFu;
+                x = (x | (x << 8)) & 0x00FF00FFu;
+                return (x | (x << 4)) & 0x0F0F0F0Fu;
+            };
+            uint8_t* out2 = codes + static_cast<size_t>(row) * (kN / 4) + (t >> 1) + (odd ? 64 * 8 : 0);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t bytes = spread4(low >> (16 * h)) | (spread4(high >> (16 * h)) << 4);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) out2[64 * (4 * h + j)] = static_cast<uint8_t>(bytes >> (8 * j));
             }
             continue;
         }

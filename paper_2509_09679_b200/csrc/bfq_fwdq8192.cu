@@ -361,7 +361,12 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             auto code2 = [&](u64 v) -> uint32_t {
                 uint32_t lo, hi;
                 if (plain) {
-                    unpack2u(fma2(v, inv2, pack2(12582912.0f, 12582912.0f)), lo, hi);
+                    // u = code + 2^(BITS-1) in the low BITS bits of v * inv + (1.5 * 2^23 + 2^(BITS-1)), the bits above
+                    // them up to bit 22 zero: (hi << BITS) + lo has both fields in place; the XOR turns offset binary
+                    // into two's complement
+                    constexpr float kMagic = 12582912.0f + float(1 << (BITS - 1));
+                    unpack2u(fma2(v, inv2, pack2(kMagic, kMagic)), lo, hi);
+                    return ((hi << BITS) + lo) ^ ((1u << (BITS - 1)) | (1u << (2 * BITS - 1)));
                 } else {
                     float a, b;
                     unpack2(v, a, b);
@@ -391,12 +396,46 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         const bool plain = (e16 != 0u) && (s16 != 0x7BFFu);  // normal fp16 scale: |v*inv| <= 1.0005, no clipping
         const u64 inv2 = pack2(inv, inv);
         uint8_t* out = out_t + static_cast<size_t>(row) * (kN8 / 4);
+        // the eight nibbles (two codes each) of the lower-half registers in one word, those of the upper half in another
+        uint32_t wa = 0u, wb = 0u;
+        if (plain) {
+            // v * inv + (1.5 * 2^23 + 2) has u = code + 2 in {1, 2, 3} in its low bits above the constant pattern
+            // C = 0x4B400000, so hi * 4 + lo = 5 C + (4 u_hi + u_lo) and a Horner chain over the registers yields the sum
+            // of the nibbles times 16^i plus a constant; one subtraction removes it, one XOR turns u into the code
+            const u64 magic2 = pack2(12582914.0f, 12582914.0f);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t nl = nibble_int2(A[i], inv2, inv, plain), nh = nibble_int2(B[i], inv2, inv, plain);
-            const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, (t & 1) ? nl : nh, 1);
-            // even lane: its lower-half nibble + the odd lane's; odd lane: the even lane's upper-half nibble + its own
-            out[64 * i] = static_cast<uint8_t>((t & 1) ? (got | (nh << 4)) : (nl | (got << 4)));
+            for (int i = 7; i >= 0; --i) {
+                uint32_t lo, hi;
+                unpack2u(fma2(A[i], inv2, magic2), lo, hi);
+                wa = wa * 16u + (hi * 4u + lo);
+                unpack2u(fma2(B[i], inv2, magic2), lo, hi);
+                wb = wb * 16u + (hi * 4u + lo);
+            }
+            constexpr uint32_t kBias = static_cast<uint32_t>((5ull * 0x4B400000ull * 0x11111111ull) & 0xFFFFFFFFull);
+            wa = (wa - kBias) ^ 0xAAAAAAAAu;
+            wb = (wb - kBias) ^ 0xAAAAAAAAu;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                wa |= nibble_int2(A[i], inv2, inv, false) << (4 * i);
+                wb |= nibble_int2(B[i], inv2, inv, false) << (4 * i);
+            }
+        }
+        // even lane: bytes of the lower half = its nibbles + the odd lane's; odd lane: bytes of the upper half = the even
+        // lane's nibbles + its own.  One exchange of a word, then nibble i of the two words side by side in byte i.
+        const bool odd = t & 1;
+        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, odd ? wa : wb, 1);
+        const uint32_t low = odd ? got : wa, high = odd ? wb : got;
+        auto spread4 = [](uint32_t x) {  // nibbles 0..3 of x into the low halves of bytes 0..3
+            x &= 0xFFFFu;
+            x = (x | (x << 8)) & 0x00FF00FFu;
+            return (x | (x << 4)) & 0x0F0F0F0Fu;
+        };
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t bytes = spread4(low >> (16 * h)) | (spread4(high >> (16 * h)) << 4);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) out[64 * (4 * h + j)] = static_cast<uint8_t>(bytes >> (8 * j));
         }
     }
     // a group with fewer rows than group 0 keeps the tokens moving
