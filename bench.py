@@ -537,6 +537,10 @@ def time_others(torch, synth, Plan, dev):
     record("forward_bf16_n4096", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan.forward(x, out=y), 20)
     codes2 = torch.empty((wl.n_rows, wl.n // 4), dtype=torch.uint8, device=dev)
     codes8 = torch.empty((wl.n_rows, wl.n), dtype=torch.uint8, device=dev)
+    x32 = x.float()
+    record("forward_int4_fp32_rows_n4096", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n + wl.n // 2 + 2,
+           lambda: plan.forward_quant(x32, 4, codes=codes, scales=scales), 20)
+    del x32
     record("forward_int2_n4096", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
            lambda: plan.forward_quant(x, 2, codes=codes2, scales=scales), 20)
     record("forward_int8_n4096", wl.n_rows, wl.n, wl.L, 4, 3 * wl.n + 2,

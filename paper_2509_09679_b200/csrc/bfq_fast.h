@@ -22,6 +22,9 @@ cudaError_t fwdq4096_launch_bits(const bfq_plan* plan, const void* x, int64_t ro
 // codes + scales (bits = 2, 4, 8) and the rotated rows in bf16 from one pass
 cudaError_t fwdq4096_launch_codes_rows(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits,
                                        uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
+// fp32 rows in: codes + scales (bits = 2, 4, 8) or, with bits = 0, the rotated rows in fp32
+cudaError_t fwdq4096_launch_f32(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                                uint16_t* scales, void* y_f32, int64_t ldy, cudaStream_t st);
 // the same with the statistics of bfq_forward_quant_stats (hist already zeroed on `st`)
 cudaError_t fwdq4096_launch_stats(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                   uint16_t* scales, unsigned long long* hist, float* rowstats, cudaStream_t st);

@@ -171,7 +171,7 @@ __device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&&
 }
 
 enum : int { kButterfly = 0, kHadamard = 1 };  // TRANSFORM
-enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutInt8 = 4 };  // OUT
+enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutInt8 = 4, kOutF32 = 5 };  // OUT
 
 // TRANSFORM: learned butterfly (constants in tensor memory) or the fixed Walsh-Hadamard transform (no constants,
 // no tensor memory).  OUT: INT4 codes + fp16 scales, or the rotated rows in bf16 (`yout`, leading dimension ldy), or
@@ -179,7 +179,9 @@ enum : int { kOutInt4 = 0, kOutBf16 = 1, kOutInt4Stats = 2, kOutInt2 = 3, kOutIn
 // tensor-wide counts of the 16 code values added to `hist`, or INT2 / INT8 codes + scales.
 // STEP: group g passes its token to group (g + STEP) % G, so gcd(STEP, G) groups rotate at a time (0: no tokens).
 // ROWS (code outputs only): the rotated rows are written as well, in bf16, to `yout` (weight folding that keeps W Q^T).
-template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2, bool ROWS = false>
+// IN_F32: the rows are fp32 (16 KB each): one input slot per group instead of two, re-armed as soon as the group has
+// read it (after the second regrouping's barrier), so the load still has most of a row's time to arrive.
+template <int G, int CW, int XB, int TRANSFORM, int OUT, int STEP = 2, bool ROWS = false, bool IN_F32 = false>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ img, const int* __restrict__ form,
            uint8_t* __restrict__ codes,
@@ -252,10 +254,13 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     const bool seeds_ring = (g + STEP) % G < kRings;  // this group's successor starts with the token
 
     // first rows of this group
+    constexpr int kSlotsUsed = IN_F32 ? 1 : kInSlots;                // fp32 rows: one slot of 2 * kRowBytes per group
+    constexpr uint32_t kSlotBytes = IN_F32 ? 2 * kRowBytes : kRowBytes;
+    static_assert(kInSlots == 2, "an fp32 row takes the group's two bf16 slots");
     if (t == 0) {
-        for (int k = 0; k < kInSlots && k < count; ++k) {
+        for (int k = 0; k < kSlotsUsed && k < count; ++k) {
             mbar_expect_tx(bar_base + 8 * k, tx_bytes);
-            tma_load_3d(in_base + k * kRowBytes, &tmap, 0, 0, first + k * stride, bar_base + 8 * k);
+            tma_load_3d(in_base + k * kSlotBytes, &tmap, 0, 0, first + k * stride, bar_base + 8 * k);
         }
     }
     // fill tensor memory
@@ -294,8 +299,10 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     // input tile: thread t owns two runs of 32 bytes, at byte 32 (t & 15) + 1024 (t >> 4) + 512 h of the
     // row, i.e. 16-byte chunks 2 (t & 3) + c of 128-byte line ((t >> 2) & 3) + 8 (t >> 4) + 4 h; the TMA
     // swizzle stores chunk j of line l at position j ^ (l & 7)
-    const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
-    const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+    // (fp32 rows: runs of 64 bytes at byte 64 (t & 15) + 2048 (t >> 4) + 1024 h: chunks 4 (t & 1) + c of line
+    // ((t & 15) >> 1) + 16 (t >> 4) + 8 h)
+    const uint32_t in_line = IN_F32 ? ((t & 15) >> 1) * 128u + (t >> 4) * 2048u : ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+    const uint32_t in_x = IN_F32 ? ((((t & 1) << 2) ^ ((t >> 1) & 7)) << 4) : ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
     const uint32_t amax_base = sbase + S::kAmaxOff + g * 32;
     uint8_t* const out_t = codes + t;
     const uint32_t hist_g = sbase + S::kHistOff + 1024u * g;  // this group's counts of packed code bytes
@@ -309,11 +316,25 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     if (seeds_ring) turn.pass();
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
-        const int slot = k & 1;
+        const int slot = IN_F32 ? 0 : (k & 1);
         if constexpr (kTmem) tmem_ld(tlane, T0);
-        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status, wait_limit);
-        const uint32_t src = in_base + slot * kRowBytes + in_line;
-        {
+        mbar_wait_bounded(bar_base + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status, wait_limit);
+        const uint32_t src = in_base + slot * kSlotBytes + in_line;
+        if constexpr (IN_F32) {
+            // run h holds elements 4c .. 4c+3 in 16-byte chunk c; element m of half h is half h of P[m]
+            uint4 w[2][4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) w[h][c] = lds128(src + 1024u * h + (in_x ^ (c << 4)));
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                P[4 * c + 0] = pack2u(w[0][c].x, w[1][c].x);
+                P[4 * c + 1] = pack2u(w[0][c].y, w[1][c].y);
+                P[4 * c + 2] = pack2u(w[0][c].z, w[1][c].z);
+                P[4 * c + 3] = pack2u(w[0][c].w, w[1][c].w);
+            }
+        } else {
             // run (h, c) holds elements 8c..8c+7 of half h; element m of half h is half h of P[m]
             uint4 w[2][2];
 #pragma unroll
@@ -332,9 +353,9 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             }
         }
         auto issue_next = [&]() {
-            if (t == 0 && k + kInSlots < count) {
+            if (t == 0 && k + kSlotsUsed < count) {
                 mbar_expect_tx(bar_base + 8 * slot, tx_bytes);
-                tma_load_3d(in_base + slot * kRowBytes, &tmap, 0, 0, first + (k + kInSlots) * stride,
+                tma_load_3d(in_base + slot * kSlotBytes, &tmap, 0, 0, first + (k + kSlotsUsed) * stride,
                             bar_base + 8 * slot);
             }
         };
@@ -356,7 +377,17 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                 out[128 * m] = *reinterpret_cast<const uint32_t*>(&v);
             }
         }
-        if constexpr (OUT == kOutBf16) {
+        if constexpr (OUT == kOutF32) {
+            // thread t holds elements 2t + 256m, +1: one 64-bit word of the fp32 row per packed register
+            u64* out = reinterpret_cast<u64*>(reinterpret_cast<float*>(yout) + static_cast<int64_t>(row) * ldy) + t;
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                float a, b;
+                unpack2(P[m], a, b);
+                out[128 * m] = pack2(a * kPost, b * kPost);
+            }
+        }
+        if constexpr (OUT == kOutBf16 || OUT == kOutF32) {
             bar_sync(ex.bar, kGroupThreads);  // every warp is past its reads of the second regrouping buffer
             continue;
         }
@@ -692,13 +723,13 @@ bool fwdq4096_available(const bfq_plan* plan) {
     return plan->n == f4k::kN && plan->cc_major == 10 && plan->img4096 != nullptr && encode_tiled() != nullptr;
 }
 
-template <int G, int CW, int XB, int TRANSFORM, int OUT, bool ROWS = false>
+template <int G, int CW, int XB, int TRANSFORM, int OUT, bool ROWS = false, bool IN_F32 = false>
 static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap, int64_t rows, uint8_t* codes,
                                   uint16_t* scales, void* y, int64_t ldy, cudaStream_t st,
                                   unsigned long long* hist = nullptr) {
     using S = f4k::Smem<G, XB>;
     static bool attr_set[kMaxDevices] = {false};
-    auto kern = f4k::k_fwdq4096<G, CW, XB, TRANSFORM, OUT, 2, ROWS>;
+    auto kern = f4k::k_fwdq4096<G, CW, XB, TRANSFORM, OUT, 2, ROWS, IN_F32>;
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
         if (e != cudaSuccess) return e;
@@ -708,7 +739,7 @@ static cudaError_t launch_variant(const bfq_plan* plan, const CUtensorMap& tmap,
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
     // bytes a row's load is expected to deliver and the bound on polls of its barrier; the test hook announces more
     // bytes than arrive, so that every wait runs out (quickly) and reports through the status word
-    const uint32_t tx_bytes = f4k::kRowBytes + (plan->test_stuck_wait ? 16u : 0u);
+    const uint32_t tx_bytes = (IN_F32 ? 2 : 1) * f4k::kRowBytes + (plan->test_stuck_wait ? 16u : 0u);
     const int wait_limit = plan->test_stuck_wait ? 4096 : (1 << 22);
     return launch_overlapped(kern, dim3(grid), dim3(G * f4k::kGroupThreads), S::kBytes, st, tmap, plan->img4096,
                              plan->form_flag, codes, scales, static_cast<__nv_bfloat16*>(y), ldy, int(rows),
@@ -755,6 +786,18 @@ cudaError_t fwdq4096_launch_codes_rows(const bfq_plan* plan, const void* x, int6
     if (bits == 4) return launch_variant<4, 32, 2, kButterfly, kOutInt4, true>(plan, tmap, rows, codes, scales, y, ldy, st);
     if (bits == 2) return launch_variant<4, 32, 2, kButterfly, kOutInt2, true>(plan, tmap, rows, codes, scales, y, ldy, st);
     return launch_variant<4, 32, 2, kButterfly, kOutInt8, true>(plan, tmap, rows, codes, scales, y, ldy, st);
+}
+
+// fp32 rows in: codes + scales (bits = 2, 4, 8), or the rotated rows in fp32 (bits = 0, y with leading dimension ldy)
+cudaError_t fwdq4096_launch_f32(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                                uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
+    CUtensorMap tmap;
+    if (!encode_row_map_f32(&tmap, x, rows, ldx)) return cudaErrorInvalidValue;
+    using namespace f4k;
+    if (bits == 0) return launch_variant<4, 32, 2, kButterfly, kOutF32, false, true>(plan, tmap, rows, codes, scales, y, ldy, st);
+    if (bits == 4) return launch_variant<4, 32, 2, kButterfly, kOutInt4, false, true>(plan, tmap, rows, codes, scales, nullptr, 0, st);
+    if (bits == 2) return launch_variant<4, 32, 2, kButterfly, kOutInt2, false, true>(plan, tmap, rows, codes, scales, nullptr, 0, st);
+    return launch_variant<4, 32, 2, kButterfly, kOutInt8, false, true>(plan, tmap, rows, codes, scales, nullptr, 0, st);
 }
 
 // bfq_forward_quant_stats on the tuned path: codes + scales + row moments + code counts from one launch of k_fwdq4096

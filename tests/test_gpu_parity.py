@@ -612,3 +612,42 @@ def test_fold_weights_with_rotated_rows_on_the_tuned_kernels(n, bits, m):
     codes2, scales2, _ = p.fold_weights(W.to(DEV), bits)
     assert torch.equal(codes, codes2) and torch.equal(scales.view(torch.int16), scales2.view(torch.int16))
     assert p.device_status() == 0
+
+
+@pytest.mark.parametrize("rows", [1, 3, 130, 593, 1001])
+@pytest.mark.parametrize("bits", [0, 2, 4, 8])
+def test_tuned_n4096_fp32_rows(rows, bits, monkeypatch):
+    """fp32 rows at n = 4096 take the tuned kernel (fp32 tensor map, one input slot per row group): rotated rows in fp32
+    (bits = 0) and codes of every width against the oracle, degenerate rows included, a padded leading dimension, and
+    agreement with the generic kernels."""
+    n = 4096
+    theta, x = make(n, rows, torch.float32, seed=500 + rows + bits)
+    if rows >= 130:  # zero, tiny (subnormal scale) and huge (saturated scale) rows
+        x[1] = 0.0
+        x[2] *= 1e-8
+        x[3] *= 1e30
+    p = plan_for(n, theta)
+    xpad = torch.zeros((rows, n + 8), dtype=torch.float32, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    xv = xpad[:, :n]
+    y_ref = oracle.forward(to_f64(theta), to_f64(x))
+    if bits == 0:
+        amax = np.abs(to_f64(x)).max(axis=1)
+        keep = (amax < 1e20) & (amax > 0)  # the absolute tolerance means nothing for the 1e30 row
+        out = Guarded((rows, n), torch.float32, DEV)
+        p.forward(xv, out=out.view)
+        assert out.intact() and p.device_status() == 0
+        if rows >= 130:
+            assert not out.view[1].any()  # the zero row stays zero
+        check_rows_close(out.view[torch.from_numpy(keep).to(DEV)], y_ref[keep], absmax_rows(x)[keep], "tuned fp32 rows")
+        return
+    codes = Guarded((rows, n * bits // 8), torch.uint8, DEV)
+    scales = Guarded((rows,), torch.float16, DEV)
+    p.forward_quant(xv, bits, codes=codes.view, scales=scales.view)
+    assert p.device_status() == 0 and codes.intact() and scales.intact()
+    check_quant(codes.view, scales.view, y_ref, bits, f"tuned fp32 n={n} INT{bits}")
+    monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+    c_g, s_g = p.forward_quant(xv, bits)
+    monkeypatch.delenv("BFQ_GENERIC_ONLY")
+    assert (s_g.view(torch.int16).int() - scales.view.view(torch.int16).int()).abs().max().item() <= 1
+    assert (c_g != codes.view).float().mean().item() < 1e-3
