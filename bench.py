@@ -571,6 +571,10 @@ def time_others(torch, synth, Plan, dev):
     scales = torch.empty((wl.n_rows,), dtype=torch.float16, device=dev)
     record("forward_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
            lambda: plan8.forward_quant(x, 2, codes=codes, scales=scales), 5)
+    x32 = x.float()
+    record("forward_int2_fp32_rows_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n + wl.n // 4 + 2,
+           lambda: plan8.forward_quant(x32, 2, codes=codes, scales=scales), 5)
+    del x32
     y8 = torch.empty_like(x)
     record("forward_bf16_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan8.forward(x, out=y8), 5)
     # backward at n = 8192 (generic kernel): a quarter of the rows

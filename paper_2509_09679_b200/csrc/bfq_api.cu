@@ -300,6 +300,11 @@ int bfq_forward(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64
         cudaError_t e = fwdq4096_launch_f32(plan, x, rows, ldx, 0, nullptr, nullptr, y, ldy, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
+    if (xt == BFQ_F32 && yt == BFQ_F32 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq8192_available(plan)) {
+        cudaError_t e = fwdq8192_launch_f32(plan, x, rows, ldx, 0, nullptr, nullptr, y, ldy, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     if (xt == BFQ_BF16 && yt == BFQ_BF16 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq8192_available(plan)) {
         cudaError_t e = fwdq8192_launch_bf16(plan, x, rows, ldx, y, ldy, static_cast<cudaStream_t>(stream));
@@ -346,6 +351,11 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
     if (hist == nullptr && xt == BFQ_F32 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq4096_available(plan)) {
         e = fwdq4096_launch_f32(plan, x, rows, ldx, bits, codes, scales, nullptr, 0, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
+    if (hist == nullptr && xt == BFQ_F32 && y == nullptr && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+        fwdq8192_available(plan)) {
+        e = fwdq8192_launch_f32(plan, x, rows, ldx, bits, codes, scales, nullptr, 0, static_cast<cudaStream_t>(stream));
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     // weight folding that keeps W Q^T in bf16: codes and rows from one pass of the tuned kernels

@@ -126,7 +126,9 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
 // also what tells a CTA that its peer has read the exchange box of the row.
 // STEP: token passing between the row groups of a CTA as in the n = 4096 kernel (0: none).
 // ROWS (BITS = 2, 4, 8): the rotated rows are written as well, in bf16, to `yrows` (leading dimension ldy).
-template <int G, int BITS, int STEP = 2, bool ROWS = false>
+// IN_F32: fp32 rows (a half row is 16 KB): one input slot per group instead of two, re-armed after the second
+// regrouping's barrier.  BITS = 32 (with IN_F32): the rotated rows in fp32 (`codes` then points to them).
+template <int G, int BITS, int STEP = 2, bool ROWS = false, bool IN_F32 = false>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
            const float* __restrict__ img, const int* __restrict__ form, uint8_t* __restrict__ codes,
@@ -177,10 +179,13 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
     const CUtensorMap* tmap = rank == 0 ? &map_lo : &map_hi;
 
+    constexpr int kSlotsUsed = IN_F32 ? 1 : kInSlots;
+    constexpr uint32_t kSlotBytes = IN_F32 ? 2 * kRowBytes : kRowBytes;
+    static_assert(kInSlots == 2, "an fp32 half row takes the group's two bf16 slots");
     if (t == 0) {
-        for (int k = 0; k < kInSlots && k < count; ++k) {
-            mbar_expect_tx(bar_in + 8 * k, kRowBytes);
-            tma_load_3d(in_base + k * kRowBytes, tmap, 0, 0, first + k * stride, bar_in + 8 * k);
+        for (int k = 0; k < kSlotsUsed && k < count; ++k) {
+            mbar_expect_tx(bar_in + 8 * k, kSlotBytes);
+            tma_load_3d(in_base + k * kSlotBytes, tmap, 0, 0, first + k * stride, bar_in + 8 * k);
         }
     }
     // constants of this thread's role: image [form][rank][column quad][role][4], all loads in flight together; the
@@ -232,8 +237,10 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         ex.r2 = eb2 + 4u * (2u * (t & 15) + 32u * (t >> 4));
         ex.bar = 1 + g;
     }
-    const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
-    const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+    // (fp32 rows: runs of 64 bytes at byte 64 (t & 15) + 2048 (t >> 4) + 1024 h: chunks 4 (t & 1) + c of line
+    // ((t & 15) >> 1) + 16 (t >> 4) + 8 h)
+    const uint32_t in_line = IN_F32 ? ((t & 15) >> 1) * 128u + (t >> 4) * 2048u : ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+    const uint32_t in_x = IN_F32 ? ((((t & 1) << 2) ^ ((t >> 1) & 7)) << 4) : ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
     const uint32_t my_box = sbase + S::kPeerOff + (g * 8 * kGroupThreads + t) * 8;  // + i * 1024: register i from the peer
     const uint32_t peer_box = map_to_cta(my_box, peer);
     const uint32_t amax_base = sbase + S::kAmaxOff + g * 64;                         // [2][8] floats
@@ -252,11 +259,25 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     if (seeds_ring) turn.pass();
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
-        const int slot = k & 1;
+        const int slot = IN_F32 ? 0 : (k & 1);
         tmem_ld32(tlane, T0);
-        mbar_wait_bounded(bar_in + 8 * slot, (k >> 1) & 1, status);
-        const uint32_t src = in_base + slot * kRowBytes + in_line;
-        {
+        mbar_wait_bounded(bar_in + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status);
+        const uint32_t src = in_base + slot * kSlotBytes + in_line;
+        if constexpr (IN_F32) {
+            // run h holds elements 4c .. 4c+3 in 16-byte chunk c; element m of half h is half h of P[m]
+            uint4 w[2][4];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) w[h][c] = lds128(src + 1024u * h + (in_x ^ (c << 4)));
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                P[4 * c + 0] = pack2u(w[0][c].x, w[1][c].x);
+                P[4 * c + 1] = pack2u(w[0][c].y, w[1][c].y);
+                P[4 * c + 2] = pack2u(w[0][c].z, w[1][c].z);
+                P[4 * c + 3] = pack2u(w[0][c].w, w[1][c].w);
+            }
+        } else {
             uint4 w[2][2];
 #pragma unroll
             for (int h = 0; h < 2; ++h)
@@ -274,9 +295,9 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             }
         }
         run_chunks<FORM, 0>(P, T0, T1, tlane, ex, turn, [&]() {
-            if (t == 0 && k + kInSlots < count) {
-                mbar_expect_tx(bar_in + 8 * slot, kRowBytes);
-                tma_load_3d(in_base + slot * kRowBytes, tmap, 0, 0, first + (k + kInSlots) * stride, bar_in + 8 * slot);
+            if (t == 0 && k + kSlotsUsed < count) {
+                mbar_expect_tx(bar_in + 8 * slot, kSlotBytes);
+                tma_load_3d(in_base + slot * kSlotBytes, tmap, 0, 0, first + (k + kSlotsUsed) * stride, bar_in + 8 * slot);
             }
         });  // the first 32 of this rank's stage-12 constants are now requested in T0
 
@@ -348,11 +369,20 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
                 yrow[2048 + 1024 * rank + 128 * i + t] = *reinterpret_cast<const uint32_t*>(&vb);
             }
         }
-        if constexpr (BITS == 16) continue;
-        constexpr int kQmax = BITS == 16 ? 1 : (1 << (BITS - 1)) - 1;
+        if constexpr (BITS == 32) {
+            // one 64-bit word of the fp32 row per packed register
+            u64* yrow = reinterpret_cast<u64*>(reinterpret_cast<float*>(codes) + static_cast<int64_t>(row) * ldy);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                yrow[1024 * rank + 128 * i + t] = A[i];
+                yrow[2048 + 1024 * rank + 128 * i + t] = B[i];
+            }
+        }
+        if constexpr (BITS == 16 || BITS == 32) continue;
+        constexpr int kQmax = BITS >= 16 ? 1 : (1 << (BITS - 1)) - 1;
         const uint16_t s16 = row_scale_fast<kQmax>(amax, &inv);
         stg16_if(rank == 0 && t == 0, scales + row, s16);
-        if constexpr (BITS != 2 && BITS != 16) {
+        if constexpr (BITS != 2 && BITS < 16) {
             // A[i] holds elements 2048 rank + 256 i + 2 t (+1) of the row, B[i] the same 4096 further on: with 4 or 8 bits
             // a register pair is one byte / one 16-bit word of its own.  |v * inv| < qmax + 1/2 for a normal, unsaturated
             // scale, so v * inv + 1.5 * 2^23 carries the two's complement code in its low mantissa bits.
@@ -576,12 +606,12 @@ bool fwdq8192_available(const bfq_plan* plan) {
            encode_tiled() != nullptr;
 }
 
-template <int BITS, bool ROWS = false>
+template <int BITS, bool ROWS = false, bool IN_F32 = false>
 static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                         uint16_t* scales, int64_t ldy, cudaStream_t st, void* yrows = nullptr) {
     constexpr int G = 4;
     using S = f8k::Smem<G>;
-    auto kern = f8k::k_fwdq8192<G, BITS, 2, ROWS>;
+    auto kern = f8k::k_fwdq8192<G, BITS, 2, ROWS, IN_F32>;
     static bool attr_set[kMaxDevices] = {false};
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
@@ -589,9 +619,15 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
         attr_set[plan->device] = true;
     }
     CUtensorMap map_lo, map_hi;
-    const uint16_t* xb = static_cast<const uint16_t*>(x);
-    if (!encode_row_map(&map_lo, xb, rows, ldx) || !encode_row_map(&map_hi, xb + f4k::kN, rows, ldx))
-        return cudaErrorInvalidValue;
+    if constexpr (IN_F32) {
+        const float* xf = static_cast<const float*>(x);
+        if (!encode_row_map_f32(&map_lo, xf, rows, ldx) || !encode_row_map_f32(&map_hi, xf + f4k::kN, rows, ldx))
+            return cudaErrorInvalidValue;
+    } else {
+        const uint16_t* xb = static_cast<const uint16_t*>(x);
+        if (!encode_row_map(&map_lo, xb, rows, ldx) || !encode_row_map(&map_hi, xb + f4k::kN, rows, ldx))
+            return cudaErrorInvalidValue;
+    }
     const int64_t want = (rows + G - 1) / G;
     const int max_clusters = plan->sm_count / 2;
     const int clusters = int(want < max_clusters ? want : max_clusters);
@@ -627,6 +663,15 @@ cudaError_t fwdq8192_launch_codes_rows(const bfq_plan* plan, const void* x, int6
     if (bits == 2) return fwdq8192_launch_bits<2, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
     if (bits == 4) return fwdq8192_launch_bits<4, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
     return fwdq8192_launch_bits<8, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
+}
+
+// fp32 rows in: codes + scales (bits = 2, 4, 8), or the rotated rows in fp32 (bits = 0, y with leading dimension ldy)
+cudaError_t fwdq8192_launch_f32(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                                uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
+    if (bits == 0) return fwdq8192_launch_bits<32, false, true>(plan, x, rows, ldx, static_cast<uint8_t*>(y), nullptr, ldy, st);
+    if (bits == 2) return fwdq8192_launch_bits<2, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
+    if (bits == 4) return fwdq8192_launch_bits<4, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
+    return fwdq8192_launch_bits<8, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
 }
 
 // y = Q x in bf16 (the weight-only setting: activations stay 16-bit)

@@ -616,11 +616,11 @@ def test_fold_weights_with_rotated_rows_on_the_tuned_kernels(n, bits, m):
 
 @pytest.mark.parametrize("rows", [1, 3, 130, 593, 1001])
 @pytest.mark.parametrize("bits", [0, 2, 4, 8])
-def test_tuned_n4096_fp32_rows(rows, bits, monkeypatch):
-    """fp32 rows at n = 4096 take the tuned kernel (fp32 tensor map, one input slot per row group): rotated rows in fp32
-    (bits = 0) and codes of every width against the oracle, degenerate rows included, a padded leading dimension, and
-    agreement with the generic kernels."""
-    n = 4096
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_tuned_fp32_rows(n, rows, bits, monkeypatch):
+    """fp32 rows at n = 4096 / 8192 take the tuned kernels (fp32 tensor map, one input slot per row group): rotated rows
+    in fp32 (bits = 0) and codes of every width against the oracle, degenerate rows included, a padded leading dimension,
+    and agreement with the generic kernels."""
     theta, x = make(n, rows, torch.float32, seed=500 + rows + bits)
     if rows >= 130:  # zero, tiny (subnormal scale) and huge (saturated scale) rows
         x[1] = 0.0
