@@ -468,6 +468,17 @@ int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64
     if (rows == 0) return BFQ_OK;
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    if (yt == BFQ_F32 && xt == BFQ_F32 && rows < (int64_t(1) << 31) && x != y && !env_flag("BFQ_GENERIC_ONLY") &&
+        bwd4096_available(plan)) {  // fp32 rows in and out on the tuned kernel
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        cudaError_t e = cudaSuccess;
+        if (!plan->bwd_tables_valid) {
+            e = bwd4096_build_tables(plan, st);
+            plan->bwd_tables_valid = (e == cudaSuccess);
+        }
+        if (e == cudaSuccess) e = inv4096_launch_f32(plan, y, rows, ldy, x, ldx, st);
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     if (yt == BFQ_BF16 && rows < (int64_t(1) << 31) && x != y && !env_flag("BFQ_GENERIC_ONLY") && bwd4096_available(plan)) {
         cudaStream_t st = static_cast<cudaStream_t>(stream);
         cudaError_t e = cudaSuccess;

@@ -651,7 +651,8 @@ __device__ __forceinline__ void inv_stages(u64 (&P)[16], uint32_t (&Tcur)[32], u
     if constexpr (S > 0) inv_stages<FORM, S - 1>(P, Tnext, Tcur, tlane, a, buf2, buf1, after_phase3);
 }
 
-template <int G, bool OUT_BF16>
+// IN_F32: the rows come in fp32 (16 KB each): one input slot per group instead of two, re-armed after phase 3.
+template <int G, bool OUT_BF16, bool IN_F32 = false>
 __global__ void __launch_bounds__(G * kThreads, 1)
 k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ img, const float* __restrict__ img_scaled,
           const int* __restrict__ form, const uint32_t* __restrict__ gsign, void* __restrict__ xout, int64_t ldx, int rows,
@@ -680,10 +681,13 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
     const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
     const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
     const uint32_t bar_base = sbase + S::kBarOff + 8 * g * kInSlots;
+    constexpr int kSlotsUsed = IN_F32 ? 1 : kInSlots;
+    constexpr uint32_t kSlotBytes = IN_F32 ? 2 * kRowBytes : kRowBytes;
+    static_assert(kInSlots == 2, "an fp32 row takes the group's two bf16 slots");
     if (t == 0) {
-        for (int k = 0; k < kInSlots && k < count; ++k) {
-            mbar_expect_tx(bar_base + 8 * k, kRowBytes);
-            tma_load_3d(in_base + k * kRowBytes, &ymap, 0, 0, first + k * stride, bar_base + 8 * k);
+        for (int k = 0; k < kSlotsUsed && k < count; ++k) {
+            mbar_expect_tx(bar_base + 8 * k, kSlotBytes);
+            tma_load_3d(in_base + k * kSlotBytes, &ymap, 0, 0, first + k * stride, bar_base + 8 * k);
         }
     }
     // constants: the scaled-form image ([column quad][role][4], coalesced, all loads in flight) unless the table build
@@ -746,6 +750,7 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
     const uint32_t g_x = (((t & 31) >> 2) ^ (t >> 5));
     const uint32_t g_a0 = (t >> 5) * 128u + (g_x << 4) + (t & 3) * 4u;
     const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
+    const uint32_t f_a = (t >> 4) * 128u + ((((t & 15) >> 1) ^ (t >> 4)) << 4) + (t & 1) * 8u;  // fp32 rows
     const uint32_t par_t = __popc(t) & 1;
     const uint32_t sgn_a = par_t ? 0x80000000u : 0u, sgn_b = par_t ? 0u : 0x80000000u;
     const uint4* gsv = reinterpret_cast<const uint4*>(gsign);
@@ -758,12 +763,29 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
     uint32_t T0[32], T1[32];
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
-        const int slot = k & 1;
+        const int slot = IN_F32 ? 0 : (k & 1);
         tmem_ld32(tlane + (FORM == kFormShear ? 32 * 11 : 32 * 10), T0);
-        mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
-        const uint32_t tile = in_base + slot * kRowBytes;
+        mbar_wait_bounded(bar_base + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status);
+        const uint32_t tile = in_base + slot * kSlotBytes;
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
+            if constexpr (IN_F32) {
+                // elements 2t + 256m, +1 are the 8-byte word t & 1 of 16-byte chunk (t & 15) >> 1 of 128-byte line
+                // (t >> 4) + 8m; the swizzle moves the chunk to chunk ^ (line & 7)
+                uint32_t s4[4] = {0u, 0u, 0u, 0u};
+                if constexpr (kSigns) {
+                    const uint4 sw = __ldg(gsv + qq * kThreads + t);
+                    s4[0] = sw.x, s4[1] = sw.y, s4[2] = sw.z, s4[3] = sw.w;
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int m = 4 * qq + i;
+                    uint32_t lo, hi;
+                    unpack2u(lds64(tile + f_a + 1024u * m), lo, hi);
+                    P[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
+                }
+                continue;
+            }
             uint32_t s4[4] = {0u, 0u, 0u, 0u};
             if constexpr (kSigns) {
                 const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
@@ -777,9 +799,9 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
             }
         }
         inv_stages<FORM, 11>(P, T0, T1, tlane, a, a.ex, a.ex + kExBytes, [&]() {
-            if (t == 0 && k + kInSlots < count) {
-                mbar_expect_tx(bar_base + 8 * slot, kRowBytes);
-                tma_load_3d(in_base + slot * kRowBytes, &ymap, 0, 0, first + (k + kInSlots) * stride, bar_base + 8 * slot);
+            if (t == 0 && k + kSlotsUsed < count) {
+                mbar_expect_tx(bar_base + 8 * slot, kSlotBytes);
+                tma_load_3d(in_base + slot * kSlotBytes, &ymap, 0, 0, first + (k + kSlotsUsed) * stride, bar_base + 8 * slot);
             }
         });
         // phase-1 ownership: two runs of 16 consecutive elements; the three-shear form undoes the parity sign here
@@ -882,6 +904,27 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
     const int count = 12 * (f4k::kN / 2);
     k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid, count, dtheta);
     plan->last_backward_partials = grid;
+    return cudaGetLastError();
+}
+
+// fp32 rows in, fp32 rows out
+cudaError_t inv4096_launch_f32(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, int64_t ldx,
+                               cudaStream_t st) {
+    constexpr int G = 4;
+    using S = b4k::InvSmem<G>;
+    auto kern = b4k::k_inv4096<G, false, true>;
+    static bool attr_set[kMaxDevices] = {false};
+    if (!attr_set[plan->device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[plan->device] = true;
+    }
+    CUtensorMap ymap;
+    if (!encode_row_map_f32(&ymap, y, rows, ldy)) return cudaErrorInvalidValue;
+    const int64_t want = (rows + G - 1) / G;
+    const int grid = int(want < plan->sm_count ? want : plan->sm_count);
+    kern<<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->img_i4096, plan->form_flag + 1,
+                                                    plan->gsign4096, x, ldx, int(rows), plan->status_word);
     return cudaGetLastError();
 }
 

@@ -54,6 +54,8 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
                            float* dtheta, cudaStream_t st);
 
 // n = 4096, bf16 y -> bf16 / fp32 x: inverse (uses the backward tables)
+cudaError_t inv4096_launch_f32(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, int64_t ldx,
+                               cudaStream_t st);
 cudaError_t inv4096_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, bool x_bf16, int64_t ldx,
                            cudaStream_t st);
 

@@ -640,6 +640,12 @@ def test_tuned_fp32_rows(n, rows, bits, monkeypatch):
         if rows >= 130:
             assert not out.view[1].any()  # the zero row stays zero
         check_rows_close(out.view[torch.from_numpy(keep).to(DEV)], y_ref[keep], absmax_rows(x)[keep], "tuned fp32 rows")
+        if n == 4096:  # the tuned inverse reads fp32 rows the same way
+            inv = Guarded((rows, n), torch.float32, DEV)
+            p.inverse(xv, out=inv.view)
+            assert inv.intact() and p.device_status() == 0
+            xi_ref = oracle.inverse(to_f64(theta), to_f64(x))
+            check_rows_close(inv.view[torch.from_numpy(keep).to(DEV)], xi_ref[keep], absmax_rows(x)[keep], "tuned fp32 inverse")
         return
     codes = Guarded((rows, n * bits // 8), torch.uint8, DEV)
     scales = Guarded((rows,), torch.float16, DEV)
