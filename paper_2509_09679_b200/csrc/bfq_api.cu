@@ -512,14 +512,14 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
         cudaError_t e = cudaMemsetAsync(dtheta, 0, sizeof(float) * size_t(plan->log_n) * (plan->n / 2), st);
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
-    if (xt == BFQ_BF16 && gt == BFQ_BF16 && (dx == nullptr || dxt == BFQ_BF16) && rows < (int64_t(1) << 31) - 1 &&
-        !env_flag("BFQ_GENERIC_ONLY") && bwd4096_available(plan)) {
+    if (xt == gt && (dx == nullptr || dxt == xt) && rows < (int64_t(1) << 31) - 1 && !env_flag("BFQ_GENERIC_ONLY") &&
+        bwd4096_available(plan)) {  // all rows bf16, or all fp32
         cudaError_t e = cudaSuccess;
         if (!plan->bwd_tables_valid) {  // built on first use after bfq_set_angles, on the caller's stream
             e = bwd4096_build_tables(plan, st);
             plan->bwd_tables_valid = (e == cudaSuccess);
         }
-        if (e == cudaSuccess) e = bwd4096_launch(plan, x, g, rows, ld, dx, dtheta, st);
+        if (e == cudaSuccess) e = bwd4096_launch(plan, x, g, rows, ld, dx, dtheta, xt == BFQ_F32, st);
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     BackwardParams p{};

@@ -223,10 +223,14 @@ __device__ __forceinline__ int elem_of(int P, int t, int m, int h) {
     return h | (t << 1) | (m << 8);
 }
 
+// IN_F32: x, g and dx are fp32.  A row pair of x and of g then fills the whole input ring (one slot of 64 KB instead of
+// two of 32 KB): the next pair is requested as soon as the upper group has read g, behind a barrier of that group.
+template <bool IN_F32>
 __global__ void __launch_bounds__(kCtaThreads, 1)
 k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap gmap,
           const float* __restrict__ img, const uint32_t* __restrict__ gsign, const int8_t* __restrict__ dsign,
-          __nv_bfloat16* __restrict__ dx, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status) {
+          void* __restrict__ dx_out, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status) {
+    __nv_bfloat16* const dx = static_cast<__nv_bfloat16*>(dx_out);
     using S = Smem;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -268,18 +272,21 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     const uint32_t bar_base = sbase + S::kBarOff;
 
     // a row index past the end is legal for the tensor map: the tile is filled with zeros
+    constexpr int kSlotsUsed = IN_F32 ? 1 : kSlots;
+    constexpr uint32_t kInRow = IN_F32 ? 2 * kRowBytes : kRowBytes;  // bytes of one input row
+    static_assert(kSlots == 2, "an fp32 row pair takes both bf16 slots of a ring");
     auto request = [&](int k) {
-        const int slot = k & 1;
+        const int slot = IN_F32 ? 0 : (k & 1);
         const int r0 = 2 * (first + k * stride);
         const uint32_t bar = bar_base + 8 * slot;
-        mbar_expect_tx(bar, 2 * kPairBytes);
+        mbar_expect_tx(bar, 4 * kInRow);
         tma_load_3d(xring + slot * kPairBytes, &xmap, 0, 0, r0, bar);
-        tma_load_3d(xring + slot * kPairBytes + kRowBytes, &xmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(xring + slot * kPairBytes + kInRow, &xmap, 0, 0, r0 + 1, bar);
         tma_load_3d(gring + slot * kPairBytes, &gmap, 0, 0, r0, bar);
-        tma_load_3d(gring + slot * kPairBytes + kRowBytes, &gmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(gring + slot * kPairBytes + kInRow, &gmap, 0, 0, r0 + 1, bar);
     };
     if (is_fwd && t == 0) {
-        for (int k = 0; k < kSlots && k < count; ++k) request(k);
+        for (int k = 0; k < kSlotsUsed && k < count; ++k) request(k);
     }
     // constants into tensor memory (each group fills half of the columns), accumulators to zero
     {
@@ -317,8 +324,12 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     if (is_fwd) {
         // ================= upper group: y = Q x, then d-theta and the reverse walk of stages 11, 10, 9 =================
         // x tile, phase-1 ownership (as in the forward kernel)
-        const uint32_t in_line = ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
-        const uint32_t in_x = ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+        // (fp32: runs of 64 bytes at byte 64 (t & 15) + 2048 (t >> 4) + 1024 h: chunks 4 (t & 1) + c of line
+        // ((t & 15) >> 1) + 16 (t >> 4) + 8 h)
+        const uint32_t in_line = IN_F32 ? ((t & 15) >> 1) * 128u + (t >> 4) * 2048u : ((t >> 2) & 3) * 128u + (t >> 4) * 1024u;
+        const uint32_t in_x = IN_F32 ? ((((t & 1) << 2) ^ ((t >> 1) & 7)) << 4) : ((((t & 3) << 1) ^ ((t >> 2) & 3)) << 4);
+        // fp32 g: elements 2t + 256m, +1 are the 8-byte word t & 1 of chunk (t & 15) >> 1 of line (t >> 4) + 8m
+        const uint32_t f_a = (t >> 4) * 128u + ((((t & 15) >> 1) ^ (t >> 4)) << 4) + (t & 1) * 8u;
         // g tile, phase-3 ownership: the 32-bit word of elements 2t + 256m, 2t + 256m + 1 is word t & 3 of
         // 16-byte chunk (t & 31) >> 2 of 128-byte line (t >> 5) + 4m; the swizzle moves the chunk to
         // chunk ^ (line & 7)
@@ -327,16 +338,31 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
         const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
         const uint4* gsv = reinterpret_cast<const uint4*>(gsign);
         for (int k = 0; k < count; ++k) {
-            const int slot = k & 1;
+            const int slot = IN_F32 ? 0 : (k & 1);
             // every thread of this group is past its reads of the other input slot (each iteration ends in a
             // barrier with the lower group)
-            if (t == 0 && k >= 1 && k + 1 < count) request(k + 1);
+            if (!IN_F32 && t == 0 && k >= 1 && k + 1 < count) request(k + 1);
             tmem_ld16(cx.tlane, T0);
-            mbar_wait_bounded(bar_base + 8 * slot, (k >> 1) & 1, status);
+            mbar_wait_bounded(bar_base + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status);
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 u64(&X)[16] = r == 0 ? Y0 : Y1;
-                const uint32_t src = xring + slot * kPairBytes + r * kRowBytes + in_line;
+                const uint32_t src = xring + slot * kPairBytes + r * kInRow + in_line;
+                if constexpr (IN_F32) {
+                    uint4 w[2][4];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) w[h][c] = lds128(src + 1024u * h + (in_x ^ (c << 4)));
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        X[4 * c + 0] = pack2u(w[0][c].x, w[1][c].x);
+                        X[4 * c + 1] = pack2u(w[0][c].y, w[1][c].y);
+                        X[4 * c + 2] = pack2u(w[0][c].z, w[1][c].z);
+                        X[4 * c + 3] = pack2u(w[0][c].w, w[1][c].w);
+                    }
+                    continue;
+                }
                 uint4 w[2][2];
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
@@ -367,7 +393,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 u64(&G)[16] = r == 0 ? G0 : G1;
-                const uint32_t src = gring + slot * kPairBytes + r * kRowBytes;
+                const uint32_t src = gring + slot * kPairBytes + r * kInRow;
 #pragma unroll
                 for (int qq = 0; qq < 4; ++qq) {
                     const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
@@ -375,10 +401,20 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = 4 * qq + i;
-                        const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
-                        G[m] = pack2u(bf16_lo(w), w & 0xFFFF0000u);
+                        if constexpr (IN_F32) {
+                            uint32_t lo, hi;
+                            unpack2u(lds64(src + f_a + 1024u * m), lo, hi);
+                            G[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
+                        } else {
+                            const uint32_t w = lds32(src + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
+                            G[m] = pack2u(bf16_lo(w), w & 0xFFFF0000u);
+                        }
                     }
                 }
+            }
+            if constexpr (IN_F32) {  // the one slot has been read by every thread of the group: next pair
+                bar_sync(cx.a.bar, kThreads);
+                if (t == 0 && k + 1 < count) request(k + 1);
             }
             rev_steps<0, kUpperSteps>(Y0, Y1, G0, G1, T0, T1, A0, A1, cx, [](auto) {});
             // phase 3 -> phase 2 regrouping = the hand-over: once the lower group is past its reads of the buffers for
@@ -428,6 +464,25 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
                 for (int r = 0; r < 2; ++r) {
                     if (r0 + r < rows) {
                         const u64(&G)[16] = r == 0 ? G0 : G1;
+                        if constexpr (IN_F32) {
+                            float* row = static_cast<float*>(dx_out) + static_cast<int64_t>(r0 + r) * ld + 16 * (t & 15) + 512 * (t >> 4);
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                uint32_t w[16];
+#pragma unroll
+                                for (int m = 0; m < 16; ++m) {
+                                    uint32_t lo, hi;
+                                    unpack2u(G[m], lo, hi);
+                                    // element m of half h: parity popcount(m) ^ h ^ popcount(t)
+                                    const bool odd_c = ((__builtin_popcount(m) + h) & 1) != 0;
+                                    w[m] = (h ? hi : lo) ^ (odd_c ? sgn_b : sgn_a);
+                                }
+                                uint4* dst = reinterpret_cast<uint4*>(row + 256 * h);
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) dst[c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                            }
+                            continue;
+                        }
                         __nv_bfloat16* row = dx + static_cast<int64_t>(r0 + r) * ld + 16 * (t & 15) + 512 * (t >> 4);
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
@@ -883,22 +938,33 @@ cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// f32: x, g and dx are fp32 rows (else bf16)
 cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
-                           float* dtheta, cudaStream_t st) {
+                           float* dtheta, bool f32, cudaStream_t st) {
     static bool attr_set[kMaxDevices] = {false};
     if (!attr_set[plan->device]) {
-        cudaError_t e = cudaFuncSetAttribute(b4k::k_bwd4096, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(b4k::k_bwd4096<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              int(b4k::Smem::kBytes));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(b4k::k_bwd4096<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(b4k::Smem::kBytes));
         if (e != cudaSuccess) return e;
         attr_set[plan->device] = true;
     }
     CUtensorMap xmap, gmap;
-    if (!encode_row_map(&xmap, x, rows, ld) || !encode_row_map(&gmap, g, rows, ld)) return cudaErrorInvalidValue;
+    const bool maps = f32 ? (encode_row_map_f32(&xmap, x, rows, ld) && encode_row_map_f32(&gmap, g, rows, ld))
+                          : (encode_row_map(&xmap, x, rows, ld) && encode_row_map(&gmap, g, rows, ld));
+    if (!maps) return cudaErrorInvalidValue;
     const int64_t pairs = (rows + 1) / 2;
     const int grid = int(pairs < plan->sm_count ? pairs : plan->sm_count);
-    b4k::k_bwd4096<<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
-                                                                   plan->dsign4096, static_cast<__nv_bfloat16*>(dx), ld,
-                                                                   plan->partial, int(rows), plan->status_word);
+    if (f32) {
+        b4k::k_bwd4096<true><<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
+                                                                              plan->dsign4096, dx, ld, plan->partial,
+                                                                              int(rows), plan->status_word);
+    } else {
+        b4k::k_bwd4096<false><<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
+                                                                               plan->dsign4096, dx, ld, plan->partial,
+                                                                               int(rows), plan->status_word);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int count = 12 * (f4k::kN / 2);

@@ -51,7 +51,7 @@ size_t bwd4096_gsign_bytes();
 bool bwd4096_available(const bfq_plan* plan);
 cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st);
 cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
-                           float* dtheta, cudaStream_t st);
+                           float* dtheta, bool f32, cudaStream_t st);
 
 // n = 4096, bf16 y -> bf16 / fp32 x: inverse (uses the backward tables)
 cudaError_t inv4096_launch_f32(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, int64_t ldx,
