@@ -560,6 +560,14 @@ def time_others(torch, synth, Plan, dev):
     record("backward_n4096", wl.n_rows, wl.n, wl.L, 14, 3 * 2 * wl.n,
            lambda: plan.backward(x, g, dx=dx, dtheta=dth), 3)
     record("inverse_n4096", wl.n_rows, wl.n, wl.L, 4, 2 * 2 * wl.n, lambda: plan.inverse(g, out=dx), 3)
+    # the same two on fp32 rows (a quarter of the batch)
+    q = wl.n_rows // 4
+    x32, g32 = x[:q].float(), g[:q].float()
+    dx32 = torch.empty_like(x32)
+    record("backward_fp32_rows_n4096", q, wl.n, wl.L, 14, 3 * 4 * wl.n,
+           lambda: plan.backward(x32, g32, dx=dx32, dtheta=dth), 3)
+    record("inverse_fp32_rows_n4096", q, wl.n, wl.L, 4, 2 * 4 * wl.n, lambda: plan.inverse(g32, out=dx32), 3)
+    del x32, g32, dx32
     del x, g, dx
     torch.cuda.empty_cache()
     # n = 8192 INT2
