@@ -30,6 +30,7 @@
 #ifndef BFQ_H_
 #define BFQ_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -263,6 +264,27 @@ const char* bfq_status_string(int status);
 int bfq_dequant_gemm(bfq_plan* plan, int64_t m, int64_t n, int64_t k, float alpha, const void* a, int a_kind,
                      int a_transposed, int64_t lda, const uint16_t* a_scales, const void* b, int b_kind, int b_transposed,
                      int64_t ldb, const uint16_t* b_scales, float* c, int64_t ldc, void* stream);
+
+/*
+ * bfq_forward_quant for rows that live in HOST memory (paper Sec. 3.4 quantizer on y = Q x, as bfq_forward_quant): the
+ * same result, with the host -> device copy of the rows, the kernels and the device -> host copy of codes and scales
+ * overlapped chunk by chunk on two streams the plan owns.
+ *   x_host          HOST pointer, [rows][ldx] of type xt; pinned (page-locked) memory for the copies to be asynchronous
+ *   codes_host      HOST pointer, [rows][n*bits/8] packed codes; scales_host_f16: HOST pointer, [rows] fp16 bits
+ *   workspace       DEVICE pointer, 16-byte aligned, owned by the caller, workspace_bytes long: holds two chunks of rows
+ *                   with their codes and scales; bfq_forward_quant_host_workspace(plan, xt, bits, chunk_rows) gives the
+ *                   size for a wanted chunk (rows are processed in chunks of a multiple of 8 rows that fit twice)
+ * Enqueued on `stream` and the plan's two copy streams; when the work enqueued on `stream` by this call is done, the
+ * host buffers hold the results.  The host buffers must stay valid until then.  Allocates nothing.  The paper has no
+ * counterpart of this call (it is the end-to-end form of the online activation path).
+ * Returns BFQ_OK, BFQ_ERR_NULL, BFQ_ERR_DTYPE, BFQ_ERR_BITS, BFQ_ERR_STRIDE, BFQ_ERR_ALIGN, BFQ_ERR_WORKSPACE (no angles
+ * set, or a workspace too small for 8 rows twice) or BFQ_ERR_CUDA.
+ */
+int bfq_forward_quant_host(bfq_plan* plan, const void* x_host, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
+                           uint8_t* codes_host, uint16_t* scales_host_f16, void* workspace, size_t workspace_bytes,
+                           void* stream);
+/* Bytes of device workspace that let bfq_forward_quant_host work in chunks of chunk_rows rows (0 on bad arguments). */
+size_t bfq_forward_quant_host_workspace(const bfq_plan* plan, bfq_dtype xt, int bits, int64_t chunk_rows);
 
 /*
  * Measures, on the current device, how many SM cycles one warp scheduler needs per FP32 FMA instruction with register

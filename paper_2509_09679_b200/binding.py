@@ -39,6 +39,8 @@ SIGNATURES = {
     "bfq_last_cuda_error": (_i, [_p]),
     "bfq_status_string": (ctypes.c_char_p, [_i]),
     "bfq_backward_partials": (_i, [_p]),
+    "bfq_forward_quant_host": (_i, [_p, _p, _i, _i64, _i64, _i, _p, _p, _p, ctypes.c_size_t, _p]),
+    "bfq_forward_quant_host_workspace": (ctypes.c_size_t, [_p, _i, _i, _i64]),
     "bfq_measure_fma_rates": (_i, [_p]),
     "bfq_measure_mma_rates": (_i, [_p]),
     "bfq_dequant_gemm": (_i, [_p, _i64, _i64, _i64, ctypes.c_float, _p, _i, _i, _i64, _p, _p, _i, _i, _i64, _p, _p, _i64, _p]),
@@ -297,6 +299,34 @@ class Plan:
                                   dx.data_ptr() if want_dx else None, _dt(dx) if want_dx else BFQ_F32,
                                   dtheta.data_ptr(), _stream(x)), "bfq_backward")
         return (dx if want_dx else None), dtheta
+
+    def forward_quant_host_workspace(self, dtype, bits: int, chunk_rows: int) -> int:
+        """Bytes of device workspace for forward_quant_host in chunks of chunk_rows rows."""
+        xt = BFQ_F32 if dtype == torch.float32 else BFQ_BF16
+        return int(lib().bfq_forward_quant_host_workspace(self._h, xt, int(bits), int(chunk_rows)))
+
+    def forward_quant_host(self, x_host: torch.Tensor, bits: int, codes_host: torch.Tensor, scales_host: torch.Tensor,
+                           workspace: torch.Tensor):
+        """bfq_forward_quant_host: rows, codes and scales in (pinned) host memory, a uint8 device workspace; enqueued on
+        the current stream of the plan's device."""
+        if x_host.is_cuda or codes_host.is_cuda or scales_host.is_cuda:
+            raise ValueError("x_host, codes_host and scales_host must be host tensors")
+        if x_host.dim() != 2 or x_host.shape[1] != self.n or x_host.stride(1) != 1:
+            raise ValueError(f"x_host must be [rows][{self.n}] with unit inner stride")
+        if x_host.dtype not in (torch.float32, torch.bfloat16):
+            raise ValueError("x_host must be float32 or bfloat16")
+        rows = x_host.shape[0]
+        for t, dtype, shape, what in ((codes_host, torch.uint8, (rows, self.n * int(bits) // 8), "codes_host"),
+                                      (scales_host, torch.float16, (rows,), "scales_host")):
+            if t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+                raise ValueError(f"{what}: expected a contiguous {dtype} host tensor of shape {shape}")
+        if not workspace.is_cuda or workspace.device != self.device or workspace.dtype != torch.uint8 or not workspace.is_contiguous():
+            raise ValueError("workspace must be a contiguous uint8 tensor on the plan's device")
+        with torch.cuda.device(self.device):
+            stream = torch.cuda.current_stream(self.device).cuda_stream
+            _check(lib().bfq_forward_quant_host(self._h, x_host.data_ptr(), _dt(x_host), rows, x_host.stride(0), int(bits),
+                                                codes_host.data_ptr(), scales_host.data_ptr(), workspace.data_ptr(),
+                                                workspace.numel(), stream), "bfq_forward_quant_host")
 
     def fold_weights(self, W: torch.Tensor, bits: int, want_rotated: bool = False, rotated_dtype=None):
         m, ldw = _rows(W, self.n, self.device, what="W")

@@ -171,6 +171,10 @@ static void release_plan(bfq_plan* plan) {
     cudaFree(plan->gsign4096);
     cudaFree(plan->partial);
     cudaFree(plan->status_word);
+    if (plan->host_in != nullptr) cudaStreamDestroy(plan->host_in);
+    if (plan->host_out != nullptr) cudaStreamDestroy(plan->host_out);
+    for (int i = 0; i < 8; ++i)
+        if (plan->host_ev[i] != nullptr) cudaEventDestroy(plan->host_ev[i]);
     cudaFree(plan->dense128);
     if (plan->theta_host != nullptr) cudaFreeHost(plan->theta_host);
     if (plan->theta_event != nullptr) cudaEventDestroy(plan->theta_event);
@@ -231,6 +235,9 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
             if (plan->comp5120 == nullptr) e = cudaErrorMemoryAllocation;
         }
     }
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&plan->host_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&plan->host_out, cudaStreamNonBlocking);
+    for (int i = 0; i < 8 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&plan->host_ev[i], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMalloc(&plan->status_word, 4 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(plan->status_word, 0, 4 * sizeof(int));
     if (e == cudaSuccess) plan->form_flag = plan->status_word + 1;
@@ -390,6 +397,82 @@ static int forward_quant_impl(bfq_plan* plan, const void* x, int xt, int64_t row
 int bfq_forward_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
                       uint8_t* codes, uint16_t* scales_f16, void* stream) {
     return forward_quant_impl(plan, x, xt, rows, ldx, bits, codes, scales_f16, nullptr, BFQ_F32, stream);
+}
+
+// ---- rows in host memory ----------------------------------------------------------------------------------
+static size_t host_row_bytes(int n, int xt, int bits) {
+    return size_t(n) * (xt == BFQ_F32 ? 4 : 2) + size_t(n) * bits / 8 + 2;
+}
+
+size_t bfq_forward_quant_host_workspace(const bfq_plan* plan, bfq_dtype xt, int bits, int64_t chunk_rows) {
+    if (plan == nullptr || chunk_rows <= 0 || (bits != 2 && bits != 4 && bits != 8)) return 0;
+    const int64_t r = (chunk_rows + 7) / 8 * 8;
+    return size_t(2) * size_t(r) * host_row_bytes(plan->n, xt, bits);
+}
+
+int bfq_forward_quant_host(bfq_plan* plan, const void* x_host, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,
+                           uint8_t* codes_host, uint16_t* scales_host_f16, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+    if (plan == nullptr) return BFQ_ERR_NULL;
+    if (xt != BFQ_F32 && xt != BFQ_BF16) return BFQ_ERR_DTYPE;
+    if (bits != 2 && bits != 4 && bits != 8) return BFQ_ERR_BITS;
+    if (rows < 0 || ldx < plan->n) return BFQ_ERR_STRIDE;
+    if (rows == 0) return BFQ_OK;
+    if (x_host == nullptr || codes_host == nullptr || scales_host_f16 == nullptr || workspace == nullptr) return BFQ_ERR_NULL;
+    if (!aligned16(workspace)) return BFQ_ERR_ALIGN;
+    if (!plan->angles_set) return BFQ_ERR_WORKSPACE;
+    const int n = plan->n;
+    const size_t esz = xt == BFQ_F32 ? 4 : 2, code_row = size_t(n) * bits / 8;
+    // two buffers of `chunk` rows each: rows, then codes, then scales (chunk is a multiple of 8: 16-byte aligned parts)
+    int64_t chunk = int64_t(workspace_bytes / (2 * host_row_bytes(n, xt, bits))) / 8 * 8;
+    if (chunk < 8) return BFQ_ERR_WORKSPACE;
+    if (chunk > rows) chunk = (rows + 7) / 8 * 8;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
+    cudaStream_t main = static_cast<cudaStream_t>(stream), s_in = plan->host_in, s_out = plan->host_out;
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    const size_t buf_bytes = size_t(chunk) * host_row_bytes(n, xt, bits);
+    auto xbuf = [&](int b) { return base + b * buf_bytes; };
+    auto cbuf = [&](int b) { return base + b * buf_bytes + size_t(chunk) * n * esz; };
+    auto sbuf = [&](int b) { return reinterpret_cast<uint16_t*>(base + b * buf_bytes + size_t(chunk) * (n * esz + code_row)); };
+    cudaEvent_t* loaded = plan->host_ev;        // [2] the rows of buffer b have arrived
+    cudaEvent_t* consumed = plan->host_ev + 2;  // [2] the kernels have read the rows of buffer b
+    cudaEvent_t* computed = plan->host_ev + 4;  // [2] codes and scales of buffer b are written
+    cudaEvent_t* drained = plan->host_ev + 6;   // [2] codes and scales of buffer b are back on the host
+    cudaError_t e = cudaEventRecord(loaded[0], main);  // the side streams start after the caller's earlier work
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_in, loaded[0], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, loaded[0], 0);
+    int rc = BFQ_OK;
+    const int64_t nchunks = (rows + chunk - 1) / chunk;
+    for (int64_t c = 0; c < nchunks && e == cudaSuccess && rc == BFQ_OK; ++c) {
+        const int b = int(c & 1);
+        const int64_t r0 = c * chunk, r = (rows - r0 < chunk) ? rows - r0 : chunk;
+        if (c >= 2) e = cudaStreamWaitEvent(s_in, consumed[b], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(xbuf(b), size_t(n) * esz, static_cast<const uint8_t*>(x_host) + size_t(r0) * ldx * esz,
+                                  size_t(ldx) * esz, size_t(n) * esz, size_t(r), cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(loaded[b], s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(main, loaded[b], 0);
+        if (e == cudaSuccess && c >= 2) e = cudaStreamWaitEvent(main, drained[b], 0);
+        if (e != cudaSuccess) break;
+        rc = forward_quant_impl(plan, xbuf(b), xt, r, n, bits, cbuf(b), sbuf(b), nullptr, BFQ_F32, main);
+        if (rc != BFQ_OK) break;
+        e = cudaEventRecord(consumed[b], main);
+        if (e == cudaSuccess) e = cudaEventRecord(computed[b], main);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, computed[b], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(codes_host + size_t(r0) * code_row, cbuf(b), size_t(r) * code_row, cudaMemcpyDeviceToHost, s_out);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(scales_host_f16 + r0, sbuf(b), size_t(r) * 2, cudaMemcpyDeviceToHost, s_out);
+        if (e == cudaSuccess) e = cudaEventRecord(drained[b], s_out);
+    }
+    // the caller's stream is done when both side streams are
+    if (e == cudaSuccess) e = cudaEventRecord(loaded[0], s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(main, loaded[0], 0);
+    if (e == cudaSuccess) e = cudaEventRecord(loaded[1], s_out);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(main, loaded[1], 0);
+    if (rc != BFQ_OK) return rc;
+    return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
 }
 
 int bfq_forward_quant_stats(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int64_t ldx, int bits,

@@ -36,6 +36,9 @@ struct bfq_plan {
     int64_t partial_slots = 0;
     int* status_word = nullptr;  // device: non-zero when a bounded wait gave up
     int* form_flag = nullptr;    // device (status_word + 1): stage form the table build selected for the tuned kernels
+    // bfq_forward_quant_host: copy-in and copy-out streams and the events that order them with the caller's stream
+    cudaStream_t host_in = nullptr, host_out = nullptr;
+    cudaEvent_t host_ev[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     bool test_stuck_wait = false;  // bfq_test_stuck_wait: the n = 4096 forward kernel announces bytes that never arrive
     int last_cuda_error = 0;
     int last_backward_partials = 0;

@@ -53,6 +53,8 @@ def test_validation_that_precedes_any_cuda_call(lib):
     assert lib.bfq_last_cuda_error(None) == 0
     assert lib.bfq_backward_partials(None) == 0
     assert lib.bfq_forward_quant(None, None, 0, 0, 0, 4, None, None, None) == -1
+    assert lib.bfq_forward_quant_host(None, None, 0, 0, 0, 4, None, None, None, 0, None) == -1
+    assert lib.bfq_forward_quant_host_workspace(None, 0, 4, 128) == 0
     # the no-allocation backward checks its sizes before it touches the device
     assert lib.bfq_backward_noalloc(2048, None, None, 0, None, 0, 0, 2048, None, 0, None, None) == -10
     assert lib.bfq_backward_noalloc(100, None, None, 0, None, 0, 0, 100, None, 0, None, None) == -2

@@ -538,6 +538,27 @@ def test_host_pipeline_matches_the_resident_call(rows, chunks):
     assert p.device_status() == 0
 
 
+@pytest.mark.parametrize("n,rows,bits,dtype", [(256, 77, 8, torch.float32), (4096, 300, 2, torch.float32),
+                                               (8192, 41, 2, torch.bfloat16)])
+def test_host_entry_point_other_shapes(n, rows, bits, dtype):
+    """bfq_forward_quant_host through the binding: fp32 rows, a padded leading dimension on the host, chunks that do not
+    divide the row count, generic and tuned kernels; results equal the device-resident call bit for bit."""
+    theta, x = make(n, rows, dtype, seed=91)
+    p = plan_for(n, theta)
+    c_ref, s_ref = p.forward_quant(x.to(DEV), bits)
+    x_host = torch.zeros((rows, n + 16), dtype=dtype).pin_memory()
+    x_host[:, :n] = x
+    c_host = torch.zeros((rows, n * bits // 8), dtype=torch.uint8).pin_memory()
+    s_host = torch.zeros((rows,), dtype=torch.float16).pin_memory()
+    ws = torch.empty((p.forward_quant_host_workspace(dtype, bits, 24),), dtype=torch.uint8, device=DEV)
+    p.forward_quant_host(x_host[:, :n], bits, c_host, s_host, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(c_host, c_ref.cpu()) and torch.equal(s_host.view(torch.int16), s_ref.cpu().view(torch.int16))
+    with pytest.raises(BfqError):  # a workspace too small for two chunks of eight rows
+        p.forward_quant_host(x_host[:, :n], bits, c_host, s_host, ws[:64])
+    assert p.device_status() == 0
+
+
 @pytest.mark.parametrize("rows", [1, 3, 130, 593, 1001])
 @pytest.mark.parametrize("n,bits", [(4096, 2), (4096, 8), (8192, 4), (8192, 8)])
 def test_tuned_kernels_other_bit_widths(rows, n, bits, monkeypatch):
