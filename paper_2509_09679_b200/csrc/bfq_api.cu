@@ -167,6 +167,12 @@ static void release_plan(bfq_plan* plan) {
     cudaFree(plan->img_i4096);
     cudaFree(plan->img8192);
     cudaFree(plan->prep8192);
+    for (int h = 0; h < 2; ++h) {
+        cudaFree(plan->img_b8192[h]);
+        cudaFree(plan->dsign8192[h]);
+        cudaFree(plan->gsign8192[h]);
+    }
+    cudaFree(plan->prep_half8192);
     cudaFree(plan->dsign4096);
     cudaFree(plan->gsign4096);
     cudaFree(plan->partial);
@@ -222,6 +228,12 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->prep4096, fwdq4096_prep_bytes());
     if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->img8192, fwdq8192_image_bytes());
     if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->prep8192, fwdq8192_prep_bytes());
+    for (int h = 0; h < 2 && n == 8192; ++h) {
+        if (e == cudaSuccess) e = cudaMalloc(&plan->img_b8192[h], bwd4096_image_bytes());
+        if (e == cudaSuccess) e = cudaMalloc(&plan->dsign8192[h], bwd4096_dsign_bytes());
+        if (e == cudaSuccess) e = cudaMalloc(&plan->gsign8192[h], bwd4096_gsign_bytes());
+    }
+    if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->prep_half8192, bwd8192_prep_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_b4096, bwd4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img_i4096, inv4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->dsign4096, bwd4096_dsign_bytes());
@@ -603,6 +615,19 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
             plan->bwd_tables_valid = (e == cudaSuccess);
         }
         if (e == cudaSuccess) e = bwd4096_launch(plan, x, g, rows, ld, dx, dtheta, xt == BFQ_F32, st);
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
+    if (xt == BFQ_BF16 && gt == BFQ_BF16 && (dx == nullptr || dxt == BFQ_BF16) && rows < (int64_t(1) << 31) - 1 &&
+        !env_flag("BFQ_GENERIC_ONLY") && bwd8192_available(plan) && fwdq8192_available(plan)) {
+        // n = 8192: stage 12's sums from the forward cluster kernel, stages 0 .. 11 and dx from two launches of the
+        // n = 4096 backward kernel (one per half of the elements)
+        cudaError_t e = cudaSuccess;
+        if (!plan->bwd_tables_valid) {
+            e = bwd8192_build_tables(plan, st);
+            plan->bwd_tables_valid = (e == cudaSuccess);
+        }
+        if (e == cudaSuccess) e = fwdq8192_launch_dtheta12(plan, x, g, rows, ld, dtheta + 12 * (plan->n / 2), st);
+        if (e == cudaSuccess) e = bwd8192_launch_halves(plan, x, g, rows, ld, dx, dtheta, st);
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     BackwardParams p{};

@@ -225,12 +225,19 @@ __device__ __forceinline__ int elem_of(int P, int t, int m, int h) {
 
 // IN_F32: x, g and dx are fp32.  A row pair of x and of g then fills the whole input ring (one slot of 64 KB instead of
 // two of 32 KB): the next pair is requested as soon as the upper group has read g, behind a barrier of that group.
-template <bool IN_F32>
+// WIDE (bf16 rows): the launch handles half `half` of n = 8192 rows, i.e. stages 0 .. 11 of that half, whose tables it
+// is given.  x rows are the half's 4096 elements (the tensor map starts there); g rows are whole 8192-element rows (16 KB),
+// and the gradient that enters the half is the transposed stage-12 rotation of the two halves of g, formed as g is read:
+// g'_own = c g_own +- s g_other with (cos, sin) of stage 12 from `tw12`.  dx is written at column 4096 * half.  One input
+// slot, as for fp32 rows.
+template <bool IN_F32, bool WIDE = false>
 __global__ void __launch_bounds__(kCtaThreads, 1)
 k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap gmap,
           const float* __restrict__ img, const uint32_t* __restrict__ gsign, const int8_t* __restrict__ dsign,
-          void* __restrict__ dx_out, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status) {
-    __nv_bfloat16* const dx = static_cast<__nv_bfloat16*>(dx_out);
+          void* __restrict__ dx_out, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status,
+          const float2* __restrict__ tw12, int half) {
+    static_assert(!(IN_F32 && WIDE), "the wide mode takes bf16 rows");
+    __nv_bfloat16* const dx = static_cast<__nv_bfloat16*>(dx_out) + (WIDE ? 4096 * half : 0);
     using S = Smem;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -272,18 +279,20 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     const uint32_t bar_base = sbase + S::kBarOff;
 
     // a row index past the end is legal for the tensor map: the tile is filled with zeros
-    constexpr int kSlotsUsed = IN_F32 ? 1 : kSlots;
-    constexpr uint32_t kInRow = IN_F32 ? 2 * kRowBytes : kRowBytes;  // bytes of one input row
-    static_assert(kSlots == 2, "an fp32 row pair takes both bf16 slots of a ring");
+    constexpr bool kOneSlot = IN_F32 || WIDE;
+    constexpr int kSlotsUsed = kOneSlot ? 1 : kSlots;
+    constexpr uint32_t kInRow = IN_F32 ? 2 * kRowBytes : kRowBytes;                // bytes of one x row
+    constexpr uint32_t kGRow = (IN_F32 || WIDE) ? 2 * kRowBytes : kRowBytes;       // bytes of one g row
+    static_assert(kSlots == 2, "an fp32 / wide row pair takes both bf16 slots of a ring");
     auto request = [&](int k) {
-        const int slot = IN_F32 ? 0 : (k & 1);
+        const int slot = kOneSlot ? 0 : (k & 1);
         const int r0 = 2 * (first + k * stride);
         const uint32_t bar = bar_base + 8 * slot;
-        mbar_expect_tx(bar, 4 * kInRow);
+        mbar_expect_tx(bar, 2 * kInRow + 2 * kGRow);
         tma_load_3d(xring + slot * kPairBytes, &xmap, 0, 0, r0, bar);
         tma_load_3d(xring + slot * kPairBytes + kInRow, &xmap, 0, 0, r0 + 1, bar);
         tma_load_3d(gring + slot * kPairBytes, &gmap, 0, 0, r0, bar);
-        tma_load_3d(gring + slot * kPairBytes + kInRow, &gmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(gring + slot * kPairBytes + kGRow, &gmap, 0, 0, r0 + 1, bar);
     };
     if (is_fwd && t == 0) {
         for (int k = 0; k < kSlotsUsed && k < count; ++k) request(k);
@@ -338,12 +347,12 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
         const uint32_t g_a1 = (t >> 5) * 128u + ((g_x ^ 4u) << 4) + (t & 3) * 4u;
         const uint4* gsv = reinterpret_cast<const uint4*>(gsign);
         for (int k = 0; k < count; ++k) {
-            const int slot = IN_F32 ? 0 : (k & 1);
+            const int slot = kOneSlot ? 0 : (k & 1);
             // every thread of this group is past its reads of the other input slot (each iteration ends in a
             // barrier with the lower group)
-            if (!IN_F32 && t == 0 && k >= 1 && k + 1 < count) request(k + 1);
+            if (!kOneSlot && t == 0 && k >= 1 && k + 1 < count) request(k + 1);
             tmem_ld16(cx.tlane, T0);
-            mbar_wait_bounded(bar_base + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status);
+            mbar_wait_bounded(bar_base + 8 * slot, (kOneSlot ? k : (k >> 1)) & 1, status);
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 u64(&X)[16] = r == 0 ? Y0 : Y1;
@@ -393,7 +402,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 u64(&G)[16] = r == 0 ? G0 : G1;
-                const uint32_t src = gring + slot * kPairBytes + r * kInRow;
+                const uint32_t src = gring + slot * kPairBytes + r * kGRow;
 #pragma unroll
                 for (int qq = 0; qq < 4; ++qq) {
                     const uint4 sw = __ldg(gsv + qq * kThreads + t);  // 2 KB in all: stays in L1
@@ -401,7 +410,18 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = 4 * qq + i;
-                        if constexpr (IN_F32) {
+                        if constexpr (WIDE) {
+                            // elements 2t + 256m, +1 of both halves of the row (the upper half is 8192 bytes further on, the
+                            // same line modulo 8) and (cos, sin) of the two stage-12 pairs they form
+                            const uint32_t at = src + ((m & 1) ? g_a1 : g_a0) + 512u * m;
+                            const uint32_t wo = lds32(at + 8192u * half), wx = lds32(at + 8192u * (half ^ 1));
+                            const float4 cs = __ldg(reinterpret_cast<const float4*>(tw12 + 2 * t + 256 * m));
+                            const float sg = half ? -1.f : 1.f;
+                            const u64 own = pack2u(bf16_lo(wo), wo & 0xFFFF0000u), oth = pack2u(bf16_lo(wx), wx & 0xFFFF0000u);
+                            uint32_t lo, hi;
+                            unpack2u(fma2(pack2(sg * cs.y, sg * cs.w), oth, mul2(pack2(cs.x, cs.z), own)), lo, hi);
+                            G[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
+                        } else if constexpr (IN_F32) {
                             uint32_t lo, hi;
                             unpack2u(lds64(src + f_a + 1024u * m), lo, hi);
                             G[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
@@ -412,7 +432,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
                     }
                 }
             }
-            if constexpr (IN_F32) {  // the one slot has been read by every thread of the group: next pair
+            if constexpr (kOneSlot) {  // the one slot has been read by every thread of the group: next pair
                 bar_sync(cx.a.bar, kThreads);
                 if (t == 0 && k + 1 < count) request(k + 1);
             }
@@ -909,6 +929,101 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
 }  // namespace b4k
 
 // ---- host side ---------------------------------------------------------------------------------------------
+namespace b4k {
+// One thread per angle of stages 0 .. 11 of half `half` of an n = 8192 transform: the staging entries the table builds
+// above read (three-shear constants, cos, sin; negation flag), from the (cos, sin) in double that bfq_set_angles left.
+__global__ void __launch_bounds__(256) k_prep_half8192(const double2* __restrict__ cs8192, int half, float4* __restrict__ prep,
+                                                        uint8_t* __restrict__ flip) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= 12 * (kN / 2)) return;
+    const int s = k / (kN / 2), j = k % (kN / 2);
+    const double2 v = cs8192[s * kN + (kN / 2) * half + j];
+    const double c = v.x, sn = v.y;
+    const bool f = c < 0.0;
+    const double sp = f ? -sn : sn, cp = f ? -c : c;
+    flip[k] = f ? 1 : 0;
+    prep[k] = make_float4(static_cast<float>(-sp / (1.0 + cp)), static_cast<float>(sp), static_cast<float>(c),
+                          static_cast<float>(sn));
+}
+
+// out[s * out_stride + out_offset + j] = sum over slots of partial[slot][s * width + j], slots in index order
+__global__ void k_reduce_partials_strided(const float* __restrict__ partial, int slots, int stages, int width, int out_stride,
+                                          int out_offset, float* __restrict__ out) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= stages * width) return;
+    float acc = 0.f;
+    for (int s = 0; s < slots; ++s) acc += partial[static_cast<int64_t>(s) * stages * width + k];
+    out[(k / width) * out_stride + out_offset + (k % width)] = acc;
+}
+}  // namespace b4k
+
+size_t bwd8192_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1); }
+
+bool bwd8192_available(const bfq_plan* plan) {
+    return plan->n == 2 * f4k::kN && plan->cc_major == 10 && plan->img_b8192[0] != nullptr && plan->img_b8192[1] != nullptr &&
+           plan->prep_half8192 != nullptr && plan->prep8192 != nullptr && plan->partial_slots >= plan->sm_count &&
+           encode_tiled() != nullptr;
+}
+
+// the two halves' tables from the staging area bfq_set_angles filled (cos, sin in double after the 13 x 4096 float4 entries)
+cudaError_t bwd8192_build_tables(const bfq_plan* plan, cudaStream_t st) {
+    const int count = 12 * (f4k::kN / 2), count8 = 13 * f4k::kN;
+    const double2* cs = reinterpret_cast<const double2*>(reinterpret_cast<const float4*>(plan->prep8192) + count8);
+    float4* prep = reinterpret_cast<float4*>(plan->prep_half8192);
+    uint8_t* flip = reinterpret_cast<uint8_t*>(prep + count);
+    for (int h = 0; h < 2; ++h) {
+        b4k::k_prep_half8192<<<(count + 255) / 256, 256, 0, st>>>(cs, h, prep, flip);
+        b4k::k_build_image_bwd4096<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img_b8192[h], plan->dsign8192[h]);
+        b4k::k_build_gsign4096<<<(16 * b4k::kThreads + 255) / 256, 256, 0, st>>>(flip, plan->gsign8192[h]);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// Stages 0 .. 11 of an n = 8192 backward (bf16 rows): one launch per half of the rows' elements; dx complete, d-theta rows
+// 0 .. 11.  Row 12 of d-theta is the caller's business.
+cudaError_t bwd8192_launch_halves(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
+                                  float* dtheta, cudaStream_t st) {
+    static bool attr_set[kMaxDevices] = {false};
+    auto kern = b4k::k_bwd4096<false, true>;
+    if (!attr_set[plan->device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(b4k::Smem::kBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[plan->device] = true;
+    }
+    const int64_t pairs = (rows + 1) / 2;
+    const int grid = int(pairs < plan->sm_count ? pairs : plan->sm_count);
+    const int n8 = 2 * f4k::kN;
+    for (int h = 0; h < 2; ++h) {
+        CUtensorMap xmap, gmap;
+        // x: the half's 4096 elements of every row; g: whole rows of 8192 bf16 = 128 lines of 128 bytes
+        if (!encode_row_map(&xmap, static_cast<const uint16_t*>(x) + f4k::kN * h, rows, ld)) return cudaErrorInvalidValue;
+        {
+            const cuuint64_t dims[3] = {64, 128, static_cast<cuuint64_t>(rows)};
+            const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ld) * 2};
+            const cuuint32_t box[3] = {64, 128, 1};
+            const cuuint32_t estr[3] = {1, 1, 1};
+            if (encode_tiled()(&gmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(g), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return cudaErrorInvalidValue;
+        }
+        kern<<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b8192[h], plan->gsign8192[h],
+                                                              plan->dsign8192[h], dx, ld, plan->partial, int(rows),
+                                                              plan->status_word, plan->tw + 12 * f4k::kN, h);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        const int count = 12 * (f4k::kN / 2);
+        b4k::k_reduce_partials_strided<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid, 12, f4k::kN / 2, n8 / 2,
+                                                                          (f4k::kN / 2) * h, dtheta);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    plan->last_backward_partials = grid;
+    return cudaSuccess;
+}
+
 size_t bwd4096_image_bytes() { return size_t(128) * b4k::kConstCols * sizeof(float); }
 size_t inv4096_image_bytes() { return size_t(128) * b4k::kInvCols * sizeof(float); }
 size_t bwd4096_dsign_bytes() { return size_t(12) * (f4k::kN / 2); }
@@ -959,11 +1074,11 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
     if (f32) {
         b4k::k_bwd4096<true><<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
                                                                               plan->dsign4096, dx, ld, plan->partial,
-                                                                              int(rows), plan->status_word);
+                                                                              int(rows), plan->status_word, nullptr, 0);
     } else {
         b4k::k_bwd4096<false><<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
                                                                                plan->dsign4096, dx, ld, plan->partial,
-                                                                               int(rows), plan->status_word);
+                                                                               int(rows), plan->status_word, nullptr, 0);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -23,6 +23,11 @@ struct bfq_plan {
     int8_t* dsign4096 = nullptr; // [12][2048] sign applied to the accumulated d-theta (n = 4096 only)
     uint32_t* gsign4096 = nullptr;  // [16 * 128] sign words applied to bf16 g rows (n = 4096 only)
     bool bwd_tables_valid = false;  // the three above match the current angles
+    // n = 8192: backward tables of the two 4096-element halves (stages 0 .. 11), built on first use like the above
+    float* img_b8192[2] = {nullptr, nullptr};
+    int8_t* dsign8192[2] = {nullptr, nullptr};
+    uint32_t* gsign8192[2] = {nullptr, nullptr};
+    void* prep_half8192 = nullptr;  // staging of one half: three-shear constants and negation flags
     float* img8192 = nullptr;    // [2][128][448] constants of the n = 8192 forward kernel, one image per CTA rank
     void* prep8192 = nullptr;    // staging for that image build
     float* theta_host = nullptr;    // pinned host copy of the angles (n = 128 only: the composite kernel's constants

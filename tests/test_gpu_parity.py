@@ -323,6 +323,11 @@ def test_tuned_backward_n4096_ragged_row_counts(rows, angle_kind, dtype):
     # d-theta only, and again: same bits
     _, dth2 = p.backward(xpad[:, :n], gpad[:, :n], want_dx=False)
     assert torch.equal(dth2, dth.view)
+    monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+    dx_gen, dth_gen = p.backward(xpad[:, :n], gpad[:, :n], dx_dtype=torch.float32)
+    monkeypatch.delenv("BFQ_GENERIC_ONLY")
+    check_rows_close(dxbuf.view[:, :n], to_f64(dx_gen), absmax_rows(g), "n=8192 tuned vs generic dx")
+    check_dtheta(dth.view, to_f64(dth_gen), "n=8192 tuned vs generic dtheta")
 
 
 def test_tuned_backward_follows_new_angles_and_agrees_with_the_generic_kernels(monkeypatch):
@@ -679,3 +684,41 @@ def test_tuned_fp32_rows(n, rows, bits, monkeypatch):
     monkeypatch.delenv("BFQ_GENERIC_ONLY")
     assert (s_g.view(torch.int16).int() - scales.view.view(torch.int16).int()).abs().max().item() <= 1
     assert (c_g != codes.view).float().mean().item() < 1e-3
+
+
+@pytest.mark.parametrize("rows", [1, 2, 3, 75, 297, 1001])
+@pytest.mark.parametrize("angle_kind", ["normal", "uniform"])
+def test_tuned_backward_n8192_ragged_row_counts(rows, angle_kind, monkeypatch):
+    """n = 8192 bf16 rows: stage 12's sums come from the forward cluster kernel, stages 0 .. 11 and dx from two launches of
+    the n = 4096 backward kernel (one per half of the elements): everything against the oracle, a padded leading
+    dimension, the same bits when run again, and agreement with the generic kernel."""
+    n = 8192
+    theta = synth.angles(n, angle_kind, 80 + rows)
+    if angle_kind == "uniform":
+        theta[:, ::7] = math.pi / 2
+        theta[:, 1::7] = -math.pi
+        theta[:, 4::7] = 100.0
+    x = synth.rows(rows, n, "laplace", 81 + rows, outliers=16, outlier_scale=100.0, dtype=torch.bfloat16)
+    g = synth.rows(rows, n, "normal", 82 + rows, dtype=torch.bfloat16)
+    p = plan_for(n, theta)
+    ld = n + 8
+    xpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    gpad = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    xpad[:, :n] = x.to(DEV)
+    gpad[:, :n] = g.to(DEV)
+    dxbuf = Guarded((rows, ld), torch.bfloat16, DEV)
+    dth = Guarded((p.L, n // 2), torch.float32, DEV)
+    p.backward(xpad[:, :n], gpad[:, :n], dx=dxbuf.view[:, :n], dtheta=dth.view)
+    assert p.device_status() == 0
+    dx_ref, dth_ref = oracle.backward(to_f64(theta), to_f64(x), to_f64(g))
+    check_rows_close(dxbuf.view[:, :n], dx_ref, absmax_rows(g), f"n=8192 dx rows={rows}")
+    check_dtheta(dth.view, dth_ref, f"n=8192 dtheta rows={rows}")
+    assert dxbuf.intact() and dth.intact()
+    assert (dxbuf.view[:, n:].contiguous().view(torch.int16) == torch.tensor(0xA5A5, dtype=torch.uint16).view(torch.int16)).all()
+    _, dth2 = p.backward(xpad[:, :n], gpad[:, :n], want_dx=False)
+    assert torch.equal(dth2, dth.view)
+    monkeypatch.setenv("BFQ_GENERIC_ONLY", "1")
+    dx_gen, dth_gen = p.backward(xpad[:, :n], gpad[:, :n], dx_dtype=torch.float32)
+    monkeypatch.delenv("BFQ_GENERIC_ONLY")
+    check_rows_close(dxbuf.view[:, :n], to_f64(dx_gen), absmax_rows(g), "n=8192 tuned vs generic dx")
+    check_dtheta(dth.view, to_f64(dth_gen), "n=8192 tuned vs generic dtheta")
