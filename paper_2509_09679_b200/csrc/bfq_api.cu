@@ -223,7 +223,10 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     const size_t angles = size_t(plan->log_n) * (n / 2);
     plan->partial_slots = backward_slots(plan->log_n, plan->sm_count);
     e = cudaMalloc(&plan->tw, angles * sizeof(float2));
-    if (e == cudaSuccess) e = cudaMalloc(&plan->partial, size_t(plan->partial_slots) * angles * sizeof(float));
+    plan->partial_floats = size_t(plan->partial_slots) * angles;
+    if (n == 8192 && plan->partial_floats < bwd8192_partial_floats(plan->sm_count))
+        plan->partial_floats = bwd8192_partial_floats(plan->sm_count);
+    if (e == cudaSuccess) e = cudaMalloc(&plan->partial, plan->partial_floats * sizeof(float));
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->img4096, fwdq4096_image_bytes());
     if (e == cudaSuccess && n == 4096) e = cudaMalloc(&plan->prep4096, fwdq4096_prep_bytes());
     if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->img8192, fwdq8192_image_bytes());
@@ -618,15 +621,13 @@ int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
     if (xt == BFQ_BF16 && gt == BFQ_BF16 && (dx == nullptr || dxt == BFQ_BF16) && rows < (int64_t(1) << 31) - 1 &&
-        !env_flag("BFQ_GENERIC_ONLY") && bwd8192_available(plan) && fwdq8192_available(plan)) {
-        // n = 8192: stage 12's sums from the forward cluster kernel, stages 0 .. 11 and dx from two launches of the
-        // n = 4096 backward kernel (one per half of the elements)
+        !env_flag("BFQ_GENERIC_ONLY") && bwd8192_available(plan)) {
+        // n = 8192: the n = 4096 backward kernel on both halves of the elements, the last stage folded into its read of g
         cudaError_t e = cudaSuccess;
         if (!plan->bwd_tables_valid) {
             e = bwd8192_build_tables(plan, st);
             plan->bwd_tables_valid = (e == cudaSuccess);
         }
-        if (e == cudaSuccess) e = fwdq8192_launch_dtheta12(plan, x, g, rows, ld, dtheta + 12 * (plan->n / 2), st);
         if (e == cudaSuccess) e = bwd8192_launch_halves(plan, x, g, rows, ld, dx, dtheta, st);
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }

@@ -52,8 +52,13 @@ struct Smem {
     static constexpr uint32_t kTmemOff = kBarOff + 8 * 2 * kSlots;
     static constexpr uint32_t kUsed = kTmemOff + 16;
     static constexpr uint32_t kBytes = kUsed + 1024;
+    // wide mode only: the upper group's sums of the stage that joins the halves, [16][128] packed pairs
+    static constexpr uint32_t kAcc12Off = (kUsed + 15u) & ~15u;
+    static constexpr uint32_t kBytesWide = kAcc12Off + 16 * kThreads * 8 + 1024;
 };
-static_assert(Smem::kBytes <= 232448, "shared memory budget of one CTA");
+static_assert(Smem::kBytesWide <= 232448, "shared memory budget of one CTA");
+constexpr int kSlotFloats = 12 * (kN / 2);            // one CTA's sums of stages 0 .. 11
+constexpr int kSlotFloatsWide = kSlotFloats + kN;     // ... followed by its share of stage 12's (wide mode)
 
 __device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -229,15 +234,35 @@ __device__ __forceinline__ int elem_of(int P, int t, int m, int h) {
 // is given.  x rows are the half's 4096 elements (the tensor map starts there); g rows are whole 8192-element rows (16 KB),
 // and the gradient that enters the half is the transposed stage-12 rotation of the two halves of g, formed as g is read:
 // g'_own = c g_own +- s g_other with (cos, sin) of stage 12 from `tw12`.  dx is written at column 4096 * half.  One input
-// slot, as for fp32 rows.
+// slot, as for fp32 rows.  Stage 12's sums g_hi y_lo - g_lo y_hi are the same expression in g' and the halves' outputs
+// z before that stage (a rotation keeps the cross product of two vectors), so each launch adds its share while both are
+// in registers: half 0 has z_lo and forms g'_hi, half 1 has z_hi and forms g'_lo; the upper group keeps these sums in
+// shared memory and the CTA's slot of `partial` is kSlotFloatsWide long (sign of the share included).
+// what the CTAs of the upper half use in the wide mode instead of xmap, img, gsign, dsign
+struct alignas(64) WideHalf {
+    CUtensorMap xmap;
+    const float* img;
+    const uint32_t* gsign;
+    const int8_t* dsign;
+};
+
 template <bool IN_F32, bool WIDE = false>
 __global__ void __launch_bounds__(kCtaThreads, 1)
 k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap gmap,
-          const float* __restrict__ img, const uint32_t* __restrict__ gsign, const int8_t* __restrict__ dsign,
+          const float* __restrict__ img_lo, const uint32_t* __restrict__ gsign_lo, const int8_t* __restrict__ dsign_lo,
           void* __restrict__ dx_out, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status,
-          const float2* __restrict__ tw12, int half) {
+          const float2* __restrict__ tw12, const __grid_constant__ WideHalf upper) {
     static_assert(!(IN_F32 && WIDE), "the wide mode takes bf16 rows");
-    __nv_bfloat16* const dx = static_cast<__nv_bfloat16*>(dx_out) + (WIDE ? 4096 * half : 0);
+    // wide mode: the first half of the grid works on the lower halves of the rows, the second on the upper halves (the
+    // hardware hands out CTAs in index order, so the second set fills the SMs as the first set's CTAs finish)
+    const int ctas = WIDE ? int(gridDim.x >> 1) : int(gridDim.x);
+    const int half = WIDE ? int(blockIdx.x >= unsigned(ctas)) : 0;
+    const CUtensorMap* const xm = (WIDE && half) ? &upper.xmap : &xmap;
+    const float* const img = (WIDE && half) ? upper.img : img_lo;
+    const uint32_t* const gsign = (WIDE && half) ? upper.gsign : gsign_lo;
+    const int8_t* const dsign = (WIDE && half) ? upper.dsign : dsign_lo;
+    // (only dereferenced when dx_out is not null)
+    __nv_bfloat16* const dx = static_cast<__nv_bfloat16*>(dx_out) + (WIDE && dx_out != nullptr ? 4096 * half : 0);
     using S = Smem;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -271,8 +296,8 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     }
 
     const int pairs = (rows + 1) / 2;
-    const int first = blockIdx.x;
-    const int stride = gridDim.x;
+    const int first = int(blockIdx.x) - half * ctas;
+    const int stride = ctas;
     const int count = first < pairs ? (pairs - first + stride - 1) / stride : 0;
     // both input rings belong to the upper group: one mbarrier per slot counts the x pair and the g pair
     const uint32_t xring = sbase + S::kXOff, gring = sbase + S::kGOff;
@@ -289,8 +314,8 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
         const int r0 = 2 * (first + k * stride);
         const uint32_t bar = bar_base + 8 * slot;
         mbar_expect_tx(bar, 2 * kInRow + 2 * kGRow);
-        tma_load_3d(xring + slot * kPairBytes, &xmap, 0, 0, r0, bar);
-        tma_load_3d(xring + slot * kPairBytes + kInRow, &xmap, 0, 0, r0 + 1, bar);
+        tma_load_3d(xring + slot * kPairBytes, xm, 0, 0, r0, bar);
+        tma_load_3d(xring + slot * kPairBytes + kInRow, xm, 0, 0, r0 + 1, bar);
         tma_load_3d(gring + slot * kPairBytes, &gmap, 0, 0, r0, bar);
         tma_load_3d(gring + slot * kPairBytes + kGRow, &gmap, 0, 0, r0 + 1, bar);
     };
@@ -316,6 +341,8 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
             for (int i = 0; i < 16; ++i) z[i] = 0u;
             for (int c = kAccCol; c < 512; c += 16) tmem_st16(cx.tlane + c, z);
             for (int q = 0; q < 16; ++q) sts128(cx.acc_smem + q * kThreads * 16, make_uint4(0u, 0u, 0u, 0u));
+        } else if constexpr (WIDE) {
+            for (int m = 0; m < 16; ++m) sts64(sbase + S::kAcc12Off + (m * kThreads + t) * 8, 0ull);
         }
         tmem_wait_st();
     }
@@ -399,8 +426,41 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
             }
             // g into the same basis
             tmem_ld16(cx.tlane + RevStep<0>::kTCol, T0);
+            if constexpr (WIDE) {
+                // elements 2t + 256m, +1 of both halves of the row (the upper half is 8192 bytes further on, the same
+                // line modulo 8) and (cos, sin) of the two stage-12 pairs they form; y carries the signs of the walk's basis
+                // here, the sign of each sum is put right when the sums are written out
+                const float sg = half ? -1.f : 1.f;
+                const uint32_t acc12 = sbase + S::kAcc12Off + t * 8;
+                const uint32_t src = gring;
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
+                for (int qq = 0; qq < 4; ++qq) {
+                    const uint4 sw = __ldg(gsv + qq * kThreads + t);
+                    const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int m = 4 * qq + i;
+                        const float4 cs = __ldg(reinterpret_cast<const float4*>(tw12 + 2 * t + 256 * m));
+                        const u64 c2 = pack2(cs.x, cs.z), s2 = pack2(sg * cs.y, sg * cs.w), ns2 = pack2(-sg * cs.y, -sg * cs.w);
+                        u64 acc = lds64(acc12 + m * kThreads * 8);
+#pragma unroll
+                        for (int r = 0; r < 2; ++r) {
+                            u64(&G)[16] = r == 0 ? G0 : G1;
+                            const u64(&Y)[16] = r == 0 ? Y0 : Y1;
+                            const uint32_t at = src + r * kGRow + ((m & 1) ? g_a1 : g_a0) + 512u * m;
+                            const uint32_t wo = lds32(at + 8192u * half), wx = lds32(at + 8192u * (half ^ 1));
+                            const u64 own = pack2u(bf16_lo(wo), wo & 0xFFFF0000u), oth = pack2u(bf16_lo(wx), wx & 0xFFFF0000u);
+                            acc = fma2(fma2(ns2, own, mul2(c2, oth)), Y[m], acc);
+                            uint32_t lo, hi;
+                            unpack2u(fma2(s2, oth, mul2(c2, own)), lo, hi);
+                            G[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
+                        }
+                        sts64(acc12 + m * kThreads * 8, acc);
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < (WIDE ? 0 : 2); ++r) {
                 u64(&G)[16] = r == 0 ? G0 : G1;
                 const uint32_t src = gring + slot * kPairBytes + r * kGRow;
 #pragma unroll
@@ -410,18 +470,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = 4 * qq + i;
-                        if constexpr (WIDE) {
-                            // elements 2t + 256m, +1 of both halves of the row (the upper half is 8192 bytes further on, the
-                            // same line modulo 8) and (cos, sin) of the two stage-12 pairs they form
-                            const uint32_t at = src + ((m & 1) ? g_a1 : g_a0) + 512u * m;
-                            const uint32_t wo = lds32(at + 8192u * half), wx = lds32(at + 8192u * (half ^ 1));
-                            const float4 cs = __ldg(reinterpret_cast<const float4*>(tw12 + 2 * t + 256 * m));
-                            const float sg = half ? -1.f : 1.f;
-                            const u64 own = pack2u(bf16_lo(wo), wo & 0xFFFF0000u), oth = pack2u(bf16_lo(wx), wx & 0xFFFF0000u);
-                            uint32_t lo, hi;
-                            unpack2u(fma2(pack2(sg * cs.y, sg * cs.w), oth, mul2(pack2(cs.x, cs.z), own)), lo, hi);
-                            G[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
-                        } else if constexpr (IN_F32) {
+                        if constexpr (IN_F32) {
                             uint32_t lo, hi;
                             unpack2u(lds64(src + f_a + 1024u * m), lo, hi);
                             G[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
@@ -479,7 +528,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
             });
 
             // ---- dx = parity sign * g, bf16, phase-1 ownership: two runs of 16 elements per row ----
-            if (dx != nullptr) {
+            if (dx_out != nullptr) {
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
                     if (r0 + r < rows) {
@@ -532,8 +581,23 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
 
     // ---- this CTA's sums -> its slot of the partial sums, with the sign of the basis undone ----
     __syncthreads();  // the upper group's sums of stages 9..11 (shared memory) are complete
+    float* const slot_out = partial + static_cast<int64_t>(blockIdx.x) * (WIDE ? kSlotFloatsWide : kSlotFloats);
+    if constexpr (WIDE) {
+        if (is_fwd) {
+            // this half's share of stage 12: pairs 2t + 256m, +1; y carried the signs of the basis g enters (the sign
+            // words), half 1's share is subtracted
+            const float sg = half ? -1.f : 1.f;
+            for (int m = 0; m < 16; ++m) {
+                float a0, a1;
+                unpack2(lds64(sbase + S::kAcc12Off + (m * kThreads + t) * 8), a0, a1);
+                const uint32_t sw = __ldg(gsign + (m >> 2) * 4 * kThreads + 4 * t + (m & 3));
+                *reinterpret_cast<float2*>(slot_out + kSlotFloats + 2 * t + 256 * m) =
+                    make_float2((sw & 0x8000u) ? -sg * a0 : sg * a0, (sw & 0x80000000u) ? -sg * a1 : sg * a1);
+            }
+        }
+    }
     if (!is_fwd) {
-        float* out = partial + static_cast<int64_t>(blockIdx.x) * (12 * (kN / 2));
+        float* out = slot_out;
         for (int s = 0; s < 12; ++s) {
             const int K = s & 3, P = s >> 2;
             for (int c = 0; c < 2; ++c) {
@@ -946,22 +1010,41 @@ __global__ void __launch_bounds__(256) k_prep_half8192(const double2* __restrict
                           static_cast<float>(sn));
 }
 
-// out[s * out_stride + out_offset + j] = sum over slots of partial[slot][s * width + j], slots in index order
-__global__ void k_reduce_partials_strided(const float* __restrict__ partial, int slots, int stages, int width, int out_stride,
-                                          int out_offset, float* __restrict__ out) {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= stages * width) return;
+// Wide mode: dtheta [13][4096] from the 2 * ctas slots (kSlotFloatsWide floats each; slots 0 .. ctas - 1 hold the lower
+// half's CTAs).  Stage s < 12, angle 2048 h + j = the sum over half h's slots of entry s * 2048 + j; stage 12, angle i =
+// the sum over all slots of entry kSlotFloats + i.  A block = 8 slot lanes x 32 angles: lane y adds slots y, y + 8, ...
+// in order, then the eight sums are added in lane order, so the result does not depend on timing.
+__global__ void __launch_bounds__(256) k_reduce_wide(const float* __restrict__ partial, int ctas, float* __restrict__ out) {
+    __shared__ float sh[8][32];
+    const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + x;  // 13 * 4096 is a multiple of 32
+    const int s = k >> 12, r = k & 4095;
+    int first = 0, count = 2 * ctas, entry = kSlotFloats + r;
+    if (s < 12) first = (r >> 11) * ctas, count = ctas, entry = s * (kN / 2) + (r & 2047);
+    const float* src = partial + static_cast<int64_t>(first) * kSlotFloatsWide + entry;
     float acc = 0.f;
-    for (int s = 0; s < slots; ++s) acc += partial[static_cast<int64_t>(s) * stages * width + k];
-    out[(k / width) * out_stride + out_offset + (k % width)] = acc;
+#pragma unroll 4
+    for (int c = y; c < count; c += 8) acc += src[static_cast<int64_t>(c) * kSlotFloatsWide];
+    sh[y][x] = acc;
+    __syncthreads();
+    if (y == 0) {
+        float a = sh[0][x];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) a += sh[i][x];
+        out[k] = a;
+    }
 }
 }  // namespace b4k
+
+// floats the wide mode needs in the plan's partial-sum buffer
+size_t bwd8192_partial_floats(int sm_count) { return size_t(2) * sm_count * b4k::kSlotFloatsWide; }
 
 size_t bwd8192_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1); }
 
 bool bwd8192_available(const bfq_plan* plan) {
     return plan->n == 2 * f4k::kN && plan->cc_major == 10 && plan->img_b8192[0] != nullptr && plan->img_b8192[1] != nullptr &&
-           plan->prep_half8192 != nullptr && plan->prep8192 != nullptr && plan->partial_slots >= plan->sm_count &&
+           plan->prep_half8192 != nullptr && plan->prep8192 != nullptr &&
+           plan->partial_floats >= bwd8192_partial_floats(plan->sm_count) &&
            encode_tiled() != nullptr;
 }
 
@@ -981,46 +1064,44 @@ cudaError_t bwd8192_build_tables(const bfq_plan* plan, cudaStream_t st) {
     return cudaSuccess;
 }
 
-// Stages 0 .. 11 of an n = 8192 backward (bf16 rows): one launch per half of the rows' elements; dx complete, d-theta rows
-// 0 .. 11.  Row 12 of d-theta is the caller's business.
+// The n = 8192 backward (bf16 rows): both halves of the rows' elements in one launch (2 x grid CTAs), then one reduction;
+// dx and all 13 rows of d-theta.
 cudaError_t bwd8192_launch_halves(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
                                   float* dtheta, cudaStream_t st) {
     static bool attr_set[kMaxDevices] = {false};
     auto kern = b4k::k_bwd4096<false, true>;
     if (!attr_set[plan->device]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(b4k::Smem::kBytes));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(b4k::Smem::kBytesWide));
         if (e != cudaSuccess) return e;
         attr_set[plan->device] = true;
     }
     const int64_t pairs = (rows + 1) / 2;
     const int grid = int(pairs < plan->sm_count ? pairs : plan->sm_count);
-    const int n8 = 2 * f4k::kN;
-    for (int h = 0; h < 2; ++h) {
-        CUtensorMap xmap, gmap;
-        // x: the half's 4096 elements of every row; g: whole rows of 8192 bf16 = 128 lines of 128 bytes
-        if (!encode_row_map(&xmap, static_cast<const uint16_t*>(x) + f4k::kN * h, rows, ld)) return cudaErrorInvalidValue;
-        {
-            const cuuint64_t dims[3] = {64, 128, static_cast<cuuint64_t>(rows)};
-            const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ld) * 2};
-            const cuuint32_t box[3] = {64, 128, 1};
-            const cuuint32_t estr[3] = {1, 1, 1};
-            if (encode_tiled()(&gmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(g), dims, strides, box, estr,
-                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-                return cudaErrorInvalidValue;
-        }
-        kern<<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b8192[h], plan->gsign8192[h],
-                                                              plan->dsign8192[h], dx, ld, plan->partial, int(rows),
-                                                              plan->status_word, plan->tw + 12 * f4k::kN, h);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        const int count = 12 * (f4k::kN / 2);
-        b4k::k_reduce_partials_strided<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid, 12, f4k::kN / 2, n8 / 2,
-                                                                          (f4k::kN / 2) * h, dtheta);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
+    CUtensorMap xmap, gmap;
+    b4k::WideHalf upper{};
+    // x: one half's 4096 elements of every row; g: whole rows of 8192 bf16 = 128 lines of 128 bytes
+    if (!encode_row_map(&xmap, static_cast<const uint16_t*>(x), rows, ld)) return cudaErrorInvalidValue;
+    if (!encode_row_map(&upper.xmap, static_cast<const uint16_t*>(x) + f4k::kN, rows, ld)) return cudaErrorInvalidValue;
+    {
+        const cuuint64_t dims[3] = {64, 128, static_cast<cuuint64_t>(rows)};
+        const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ld) * 2};
+        const cuuint32_t box[3] = {64, 128, 1};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (encode_tiled()(&gmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(g), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
     }
-    plan->last_backward_partials = grid;
+    upper.img = plan->img_b8192[1], upper.gsign = plan->gsign8192[1], upper.dsign = plan->dsign8192[1];
+    kern<<<2 * grid, b4k::kCtaThreads, b4k::Smem::kBytesWide, st>>>(xmap, gmap, plan->img_b8192[0], plan->gsign8192[0],
+                                                                  plan->dsign8192[0], dx, ld, plan->partial, int(rows),
+                                                                  plan->status_word, plan->tw + 12 * f4k::kN, upper);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    b4k::k_reduce_wide<<<13 * f4k::kN / 32, 256, 0, st>>>(plan->partial, grid, dtheta);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    plan->last_backward_partials = 2 * grid;
     return cudaSuccess;
 }
 
@@ -1074,11 +1155,11 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
     if (f32) {
         b4k::k_bwd4096<true><<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
                                                                               plan->dsign4096, dx, ld, plan->partial,
-                                                                              int(rows), plan->status_word, nullptr, 0);
+                                                                              int(rows), plan->status_word, nullptr, b4k::WideHalf{});
     } else {
         b4k::k_bwd4096<false><<<grid, b4k::kCtaThreads, b4k::Smem::kBytes, st>>>(xmap, gmap, plan->img_b4096, plan->gsign4096,
                                                                                plan->dsign4096, dx, ld, plan->partial,
-                                                                               int(rows), plan->status_word, nullptr, 0);
+                                                                               int(rows), plan->status_word, nullptr, b4k::WideHalf{});
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

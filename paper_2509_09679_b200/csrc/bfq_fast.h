@@ -40,10 +40,6 @@ cudaError_t fwdq8192_launch_codes_rows(const bfq_plan* plan, const void* x, int6
                                        uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 cudaError_t fwdq8192_launch_f32(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
                                 uint16_t* scales, void* y_f32, int64_t ldy, cudaStream_t st);
-// d-theta of stage 12 (4096 values) from x and g rows (bf16): the forward transform up to stage 12 and the sums
-// g_hi * y_lo - g_lo * y_hi over all rows, reduced in a fixed order
-cudaError_t fwdq8192_launch_dtheta12(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, float* dtheta12,
-                                     cudaStream_t st);
 cudaError_t fwdq8192_launch_bf16(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, void* y, int64_t ldy,
                                  cudaStream_t st);
 
@@ -53,8 +49,10 @@ size_t inv4096_image_bytes();
 size_t bwd4096_dsign_bytes();
 size_t bwd4096_gsign_bytes();
 bool bwd4096_available(const bfq_plan* plan);
-// n = 8192 bf16 rows: stages 0 .. 11 as two launches of the n = 4096 backward kernel, one per half of the elements
+// n = 8192 bf16 rows: the n = 4096 backward kernel on the two halves of the elements (one launch, twice the CTAs); the
+// stage that joins the halves is folded into the read of g and its sums are taken there too
 size_t bwd8192_prep_bytes();
+size_t bwd8192_partial_floats(int sm_count);
 bool bwd8192_available(const bfq_plan* plan);
 cudaError_t bwd8192_build_tables(const bfq_plan* plan, cudaStream_t st);
 cudaError_t bwd8192_launch_halves(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,

@@ -125,10 +125,6 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
 // (`codes` then points to them, leading dimension ldy); the absmax hand-shake between the two CTAs is kept, since it is
 // also what tells a CTA that its peer has read the exchange box of the row.
 // STEP: token passing between the row groups of a CTA as in the n = 4096 kernel (0: none).
-// BITS = 64: nothing is quantized or stored per row; the kernel accumulates the stage-12 angle gradient instead: with the
-// upstream gradient rows `gup` (bf16, leading dimension ldy), sum over this CTA's rows of g_hi * y_lo - g_lo * y_hi for
-// the 2048 stage-12 pairs whose outputs this rank finishes; one set of sums per row group, written to
-// part12[(CTA * G + group) * 2048 + 256 i + 2 t + e] at the end (fixed ownership: the order of the additions is fixed).
 // ROWS (BITS = 2, 4, 8): the rotated rows are written as well, in bf16, to `yrows` (leading dimension ldy).
 // IN_F32: fp32 rows (a half row is 16 KB): one input slot per group instead of two, re-armed after the second
 // regrouping's barrier.  BITS = 32 (with IN_F32): the rotated rows in fp32 (`codes` then points to them).
@@ -137,7 +133,7 @@ __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
            const float* __restrict__ img, const int* __restrict__ form, uint8_t* __restrict__ codes,
            uint16_t* __restrict__ scales, int64_t ldy, int rows, int* __restrict__ status,
-           __nv_bfloat16* __restrict__ yrows, const __nv_bfloat16* __restrict__ gup, float* __restrict__ part12) {
+           __nv_bfloat16* __restrict__ yrows) {
     using S = Smem<G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -255,9 +251,6 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     uint8_t* const out_t = codes + (t >> 1) + 64 * 8 * rank + ((t & 1) ? 1024 : 0);
 
     // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
-    u64 acc12[8];  // BITS = 64: stage-12 sums of this thread's 16 pairs
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc12[i] = pack2(0.f, 0.f);
     auto row_loop = [&](auto form_tag) {
     constexpr int FORM = decltype(form_tag)::value;
     u64 P[16];
@@ -321,12 +314,6 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
 #pragma unroll
             for (int i = 0; i < 8; ++i) st_async_b64(peer_box + i * 1024u, P[i], peer_bar_swap);
         }
-        uint32_t gl[BITS == 64 ? 8 : 1], gh[BITS == 64 ? 8 : 1];  // upstream gradient words of the outputs this rank finishes
-        if constexpr (BITS == 64) {
-            const uint32_t* grow = reinterpret_cast<const uint32_t*>(gup + static_cast<int64_t>(row) * ldy) + 1024 * rank + t;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) gl[i] = __ldg(grow + 128 * i), gh[i] = __ldg(grow + 2048 + 128 * i);
-        }
         mbar_wait_cluster_bounded(bar_swap, k & 1, status);
         if (rank == 0) {
 #pragma unroll
@@ -367,14 +354,6 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         mbar_wait_cluster_bounded(bar_amax, k & 1, status);
         amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
         float inv;
-        if constexpr (BITS == 64) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const u64 g_lo = pack2u(bf16_lo(gl[i]), gl[i] & 0xFFFF0000u), g_hi = pack2u(bf16_lo(gh[i]), gh[i] & 0xFFFF0000u);
-                acc12[i] = sub2(fma2(g_hi, A[i], acc12[i]), mul2(g_lo, B[i]));
-            }
-            continue;
-        }
         static_assert(!(ROWS && BITS == 16), "BITS = 16 writes the rows already");
         if constexpr (BITS == 16 || ROWS) {
             // A[i] holds elements 2048 rank + 256 i + 2 t (+1), B[i] the same 4096 further on: one 32-bit word each
@@ -400,7 +379,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             }
         }
         if constexpr (BITS == 16 || BITS == 32) continue;
-        constexpr int kQmax = BITS >= 16 ? 1 : (1 << (BITS - 1)) - 1;  // (BITS >= 16 never gets here)
+        constexpr int kQmax = BITS >= 16 ? 1 : (1 << (BITS - 1)) - 1;
         const uint16_t s16 = row_scale_fast<kQmax>(amax, &inv);
         stg16_if(rank == 0 && t == 0, scales + row, s16);
         if constexpr (BITS != 2 && BITS < 16) {
@@ -502,11 +481,6 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         row_loop(std::integral_constant<int, kFormShear>());
     }
 
-    if constexpr (BITS == 64) {
-        u64* out = reinterpret_cast<u64*>(part12 + (static_cast<int64_t>(blockIdx.x) * G + g) * 2048) + t;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) out[128 * i] = acc12[i];
-    }
     tmem_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc512(tmem_base);
@@ -634,8 +608,7 @@ bool fwdq8192_available(const bfq_plan* plan) {
 
 template <int BITS, bool ROWS = false, bool IN_F32 = false>
 static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
-                                        uint16_t* scales, int64_t ldy, cudaStream_t st, void* yrows = nullptr,
-                                        const void* gup = nullptr, float* part12 = nullptr, int* clusters_out = nullptr) {
+                                        uint16_t* scales, int64_t ldy, cudaStream_t st, void* yrows = nullptr) {
     constexpr int G = 4;
     using S = f8k::Smem<G>;
     auto kern = f8k::k_fwdq8192<G, BITS, 2, ROWS, IN_F32>;
@@ -658,7 +631,6 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
     const int64_t want = (rows + G - 1) / G;
     const int max_clusters = plan->sm_count / 2;
     const int clusters = int(want < max_clusters ? want : max_clusters);
-    if (clusters_out != nullptr) *clusters_out = clusters;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.blockDim = dim3(G * f4k::kGroupThreads, 1, 1);
@@ -675,7 +647,7 @@ static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, map_lo, map_hi, static_cast<const float*>(plan->img8192),
                               static_cast<const int*>(plan->form_flag), codes, scales, ldy, int(rows), plan->status_word,
-                              static_cast<__nv_bfloat16*>(yrows), static_cast<const __nv_bfloat16*>(gup), part12);
+                              static_cast<__nv_bfloat16*>(yrows));
 }
 
 cudaError_t fwdq8192_launch(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
@@ -691,28 +663,6 @@ cudaError_t fwdq8192_launch_codes_rows(const bfq_plan* plan, const void* x, int6
     if (bits == 2) return fwdq8192_launch_bits<2, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
     if (bits == 4) return fwdq8192_launch_bits<4, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
     return fwdq8192_launch_bits<8, true>(plan, x, rows, ldx, codes, scales, ldy, st, y);
-}
-
-namespace f8k {
-// dtheta12[2048 rank + p] = sum over clusters and row groups, in index order, of the CTAs' sums
-__global__ void k_reduce_dtheta12(const float* __restrict__ part12, int clusters, int groups, float* __restrict__ out) {
-    const int q = blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= 4096) return;
-    const int rank = q >> 11, p = q & 2047;
-    float acc = 0.f;
-    for (int c = 0; c < clusters; ++c)
-        for (int g = 0; g < groups; ++g) acc += part12[(static_cast<int64_t>(2 * c + rank) * groups + g) * 2048 + p];
-    out[q] = acc;
-}
-}  // namespace f8k
-
-cudaError_t fwdq8192_launch_dtheta12(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, float* dtheta12,
-                                     cudaStream_t st) {
-    int clusters = 0;
-    cudaError_t e = fwdq8192_launch_bits<64>(plan, x, rows, ld, nullptr, nullptr, ld, st, nullptr, g, plan->partial, &clusters);
-    if (e != cudaSuccess) return e;
-    f8k::k_reduce_dtheta12<<<16, 256, 0, st>>>(plan->partial, clusters, 4, dtheta12);
-    return cudaGetLastError();
 }
 
 // fp32 rows in: codes + scales (bits = 2, 4, 8), or the rotated rows in fp32 (bits = 0, y with leading dimension ldy)

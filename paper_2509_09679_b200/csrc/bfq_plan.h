@@ -39,6 +39,7 @@ struct bfq_plan {
     bool comp5120_valid = false;    // they match the current angles
     float* partial = nullptr;    // [partial_slots][log_n][n/2] d-theta partial sums
     int64_t partial_slots = 0;
+    size_t partial_floats = 0;   // floats allocated behind `partial` (at n = 8192 the tuned backward may need more than the above)
     int* status_word = nullptr;  // device: non-zero when a bounded wait gave up
     int* form_flag = nullptr;    // device (status_word + 1): stage form the table build selected for the tuned kernels
     // bfq_forward_quant_host: copy-in and copy-out streams and the events that order them with the caller's stream
