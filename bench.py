@@ -207,7 +207,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (profiler captures of a small case)")
-    ap.add_argument("--n", type=int, default=4096, choices=[4096, 8192], help="row length for --op backward")
+    ap.add_argument("--n", type=int, default=4096, choices=[4096, 8192], help="row length for --op backward / inverse")
     ap.add_argument("--op", default="forward_quant", choices=["forward_quant", "backward", "inverse", "int2_8192", "composite5120", "dequant_gemm", "fma_peak"],
                     help="backward / int2_8192: time only bfq_backward on the learning batch / bfq_forward_quant "
                          "(INT2) on the n = 8192 activations (for profiler captures; prints a short JSON line, "
@@ -366,8 +366,9 @@ def run_backward_only(torch, args, synth, Plan, dev):
 
 
 def run_inverse_only(torch, args, synth, Plan, dev):
-    """bfq_inverse alone on (a prefix of) the learning batch's gradient rows."""
-    wl = synth.WORKLOADS["learn4096"]
+    """bfq_inverse alone on (a prefix of) the learning batch's gradient rows, or with --n 8192 on standard-normal rows of
+    that length (the row count of the n = 8192 activations)."""
+    wl = synth.WORKLOADS["learn4096" if args.n == 4096 else "act8192_int2"]
     rows = args.rows or wl.n_rows
     plan = Plan(wl.n, dev)
     plan.set_angles(wl.theta(device=dev))
@@ -376,7 +377,7 @@ def run_inverse_only(torch, args, synth, Plan, dev):
     for _ in range(args.warmup):
         plan.inverse(g, out=out)
     ms = event_time_ms(torch, lambda: plan.inverse(g, out=out), args.steps)
-    print(json.dumps({"op": "inverse", "workload": "learn4096", "rows": rows, "ms": ms,
+    print(json.dumps({"op": "inverse", "workload": "learn4096" if args.n == 4096 else "act8192_int2", "rows": rows, "ms": ms,
                       "rows_per_s": rows / (ms * 1e-3), "status": plan.device_status()}))
 
 
@@ -587,6 +588,7 @@ def time_others(torch, synth, Plan, dev):
     del x32
     y8 = torch.empty_like(x)
     record("forward_bf16_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan8.forward(x, out=y8), 5)
+    record("inverse_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan8.inverse(x, out=y8), 5)
     # backward at n = 8192 (forward cluster kernel for the last stage's sums + the n = 4096 backward kernel per half): a quarter of the rows
     rows8 = wl.n_rows // 4
     g8 = torch.randn((rows8, wl.n), device=dev, dtype=torch.float32).to(x.dtype)

@@ -223,7 +223,8 @@ int bfq_last_cuda_error(const bfq_plan* plan);
  * cosines it has been through; when such a product leaves [2^-64, 1] (an angle within ~1e-19 .. of an odd multiple of
  * pi/2 along some path, e.g. angles that are exact multiples of pi/2) the table build selects the three-shear form
  * instead, which has no such limit.  Returns bit 0 = forward tables use the fallback, bit 1 = inverse tables (built by
- * the first bfq_inverse / bfq_backward after bfq_set_angles) use the fallback; or a negative bfq_status.  Synchronises
+ * the first bfq_inverse / bfq_backward after bfq_set_angles; at n = 8192 the tables of either half of the row) use the
+ * fallback; or a negative bfq_status.  Synchronises
  * the device.  With the scaled form, inputs must stay below about 2^56 in magnitude (intermediate values are the true
  * values divided by the factor).  (No counterpart in the paper; informational.)
  */

@@ -169,6 +169,7 @@ static void release_plan(bfq_plan* plan) {
     cudaFree(plan->prep8192);
     for (int h = 0; h < 2; ++h) {
         cudaFree(plan->img_b8192[h]);
+        cudaFree(plan->img_i8192[h]);
         cudaFree(plan->dsign8192[h]);
         cudaFree(plan->gsign8192[h]);
     }
@@ -233,6 +234,7 @@ int bfq_plan_create(bfq_plan** out, int n, int64_t max_rows, int device) {
     if (e == cudaSuccess && n == 8192) e = cudaMalloc(&plan->prep8192, fwdq8192_prep_bytes());
     for (int h = 0; h < 2 && n == 8192; ++h) {
         if (e == cudaSuccess) e = cudaMalloc(&plan->img_b8192[h], bwd4096_image_bytes());
+        if (e == cudaSuccess) e = cudaMalloc(&plan->img_i8192[h], inv4096_image_bytes());
         if (e == cudaSuccess) e = cudaMalloc(&plan->dsign8192[h], bwd4096_dsign_bytes());
         if (e == cudaSuccess) e = cudaMalloc(&plan->gsign8192[h], bwd4096_gsign_bytes());
     }
@@ -587,6 +589,16 @@ int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64
         if (e == cudaSuccess) e = inv4096_launch(plan, y, rows, ldy, x, xt == BFQ_BF16, ldx, st);
         return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
     }
+    if (yt == BFQ_BF16 && rows < (int64_t(1) << 31) && x != y && !env_flag("BFQ_GENERIC_ONLY") && bwd8192_available(plan)) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        cudaError_t e = cudaSuccess;
+        if (!plan->bwd_tables_valid) {
+            e = bwd8192_build_tables(plan, st);
+            plan->bwd_tables_valid = (e == cudaSuccess);
+        }
+        if (e == cudaSuccess) e = inv8192_launch(plan, y, rows, ldy, x, xt == BFQ_BF16, ldx, st);
+        return e == cudaSuccess ? BFQ_OK : cuda_fail(plan, e);
+    }
     GenericParams p{};
     p.tw = plan->tw, p.x = y, p.xt = yt, p.ldx = ldy, p.y = x, p.yt = xt, p.ldy = ldx, p.rows = rows;
     cudaError_t e = launch_generic<kModeInverse>(plan, p, static_cast<cudaStream_t>(stream));
@@ -736,10 +748,10 @@ int bfq_stage_form(bfq_plan* plan) {
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(plan, guard.err);
     cudaError_t e = cudaDeviceSynchronize();
-    int words[2] = {0, 0};
+    int words[3] = {0, 0, 0};  // forward; inverse (n = 4096, or the lower half at n = 8192); inverse, upper half at n = 8192
     if (e == cudaSuccess) e = cudaMemcpy(words, plan->form_flag, sizeof(words), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(plan, e);
-    return (words[0] != 0 ? 1 : 0) | (words[1] != 0 ? 2 : 0);
+    return (words[0] != 0 ? 1 : 0) | ((words[1] | words[2]) != 0 ? 2 : 0);
 }
 
 int bfq_backward_partials(const bfq_plan* plan) { return plan == nullptr ? 0 : plan->last_backward_partials; }

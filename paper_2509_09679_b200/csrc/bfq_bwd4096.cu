@@ -790,12 +790,32 @@ __device__ __forceinline__ void inv_stages(u64 (&P)[16], uint32_t (&Tcur)[32], u
     if constexpr (S > 0) inv_stages<FORM, S - 1>(P, Tnext, Tcur, tlane, a, buf2, buf1, after_phase3);
 }
 
+// what the CTAs of the upper half use in the wide mode of the inverse kernel instead of img, img_scaled, form, gsign
+struct InvUpper {
+    const float* img;
+    const float* img_scaled;
+    const int* form;
+    const uint32_t* gsign;
+};
+
 // IN_F32: the rows come in fp32 (16 KB each): one input slot per group instead of two, re-armed after phase 3.
-template <int G, bool OUT_BF16, bool IN_F32 = false>
+// WIDE (bf16 rows in): n = 8192.  x = Q^T y = (Q_lo^T (+) Q_hi^T) B_12^T y: even CTAs produce the lower 4096 elements of x,
+// odd CTAs the upper (CTAs 2i and 2i + 1 work on the same rows at about the same time, so the second read of a row comes
+// from L2).  A y row is 16 KB in one slot; the transposed stage-12 rotation y'_own = c y_own +- s y_other with (cos, sin)
+// from `tw12` is applied as the row is read, then the half's own twelve stages follow from its own tables.
+template <int G, bool OUT_BF16, bool IN_F32 = false, bool WIDE = false>
 __global__ void __launch_bounds__(G * kThreads, 1)
-k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ img, const float* __restrict__ img_scaled,
-          const int* __restrict__ form, const uint32_t* __restrict__ gsign, void* __restrict__ xout, int64_t ldx, int rows,
-          int* __restrict__ status) {
+k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ img_lo, const float* __restrict__ img_scaled_lo,
+          const int* __restrict__ form_lo, const uint32_t* __restrict__ gsign_lo, void* __restrict__ xout, int64_t ldx, int rows,
+          int* __restrict__ status, const float2* __restrict__ tw12, const InvUpper upper) {
+    static_assert(!(IN_F32 && WIDE), "the wide mode takes bf16 rows");
+    const int half = WIDE ? int(blockIdx.x & 1u) : 0;
+    const int cta = WIDE ? int(blockIdx.x >> 1) : int(blockIdx.x);
+    const int ctas = WIDE ? int((gridDim.x + 1u) >> 1) : int(gridDim.x);
+    const float* const img = (WIDE && half) ? upper.img : img_lo;
+    const float* const img_scaled = (WIDE && half) ? upper.img_scaled : img_scaled_lo;
+    const int* const form = (WIDE && half) ? upper.form : form_lo;
+    const uint32_t* const gsign = (WIDE && half) ? upper.gsign : gsign_lo;
     using S = InvSmem<G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -815,14 +835,14 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sbase + S::kTmemOff));
     const uint32_t tlane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 
-    const int first = blockIdx.x * G + g;
-    const int stride = gridDim.x * G;
+    const int first = cta * G + g;
+    const int stride = ctas * G;
     const int count = first < rows ? (rows - first + stride - 1) / stride : 0;
     const uint32_t in_base = sbase + S::kInOff + g * kInSlots * kRowBytes;
     const uint32_t bar_base = sbase + S::kBarOff + 8 * g * kInSlots;
-    constexpr int kSlotsUsed = IN_F32 ? 1 : kInSlots;
-    constexpr uint32_t kSlotBytes = IN_F32 ? 2 * kRowBytes : kRowBytes;
-    static_assert(kInSlots == 2, "an fp32 row takes the group's two bf16 slots");
+    constexpr int kSlotsUsed = (IN_F32 || WIDE) ? 1 : kInSlots;
+    constexpr uint32_t kSlotBytes = (IN_F32 || WIDE) ? 2 * kRowBytes : kRowBytes;
+    static_assert(kInSlots == 2, "an fp32 row, or a bf16 row of 8192, takes the group's two bf16 slots");
     if (t == 0) {
         for (int k = 0; k < kSlotsUsed && k < count; ++k) {
             mbar_expect_tx(bar_base + 8 * k, kSlotBytes);
@@ -902,9 +922,9 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
     uint32_t T0[32], T1[32];
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
-        const int slot = IN_F32 ? 0 : (k & 1);
+        const int slot = kSlotsUsed == 1 ? 0 : (k & 1);
         tmem_ld32(tlane + (FORM == kFormShear ? 32 * 11 : 32 * 10), T0);
-        mbar_wait_bounded(bar_base + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status);
+        mbar_wait_bounded(bar_base + 8 * slot, (kSlotsUsed == 1 ? k : (k >> 1)) & 1, status);
         const uint32_t tile = in_base + slot * kSlotBytes;
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
@@ -933,6 +953,19 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int m = 4 * qq + i;
+                if constexpr (WIDE) {
+                    // elements 2t + 256m, +1 of both halves of the row (the upper half is 8192 bytes further on, the same
+                    // line modulo 8) and (cos, sin) of the two stage-12 pairs they form
+                    const uint32_t at = tile + ((m & 1) ? g_a1 : g_a0) + 512u * m;
+                    const uint32_t wo = lds32(at + 8192u * half), wx = lds32(at + 8192u * (half ^ 1));
+                    const float4 cs = __ldg(reinterpret_cast<const float4*>(tw12 + 2 * t + 256 * m));
+                    const float sg = half ? -1.f : 1.f;
+                    const u64 own = pack2u(bf16_lo(wo), wo & 0xFFFF0000u), oth = pack2u(bf16_lo(wx), wx & 0xFFFF0000u);
+                    uint32_t lo, hi;
+                    unpack2u(fma2(pack2(sg * cs.y, sg * cs.w), oth, mul2(pack2(cs.x, cs.z), own)), lo, hi);
+                    P[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
+                    continue;
+                }
                 const uint32_t w = lds32(tile + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
                 P[m] = pack2u(bf16_lo(w), w & 0xFFFF0000u);
             }
@@ -947,7 +980,7 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
         const uint32_t sa_ = kSigns ? sgn_a : 0u, sb_ = kSigns ? sgn_b : 0u;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int64_t off = static_cast<int64_t>(row) * ldx + 16 * (t & 15) + 512 * (t >> 4) + 256 * h;
+            const int64_t off = static_cast<int64_t>(row) * ldx + (WIDE ? kN * half : 0) + 16 * (t & 15) + 512 * (t >> 4) + 256 * h;
             if constexpr (OUT_BF16) {
                 uint32_t w[8];
 #pragma unroll
@@ -997,11 +1030,12 @@ namespace b4k {
 // One thread per angle of stages 0 .. 11 of half `half` of an n = 8192 transform: the staging entries the table builds
 // above read (three-shear constants, cos, sin; negation flag), from the (cos, sin) in double that bfq_set_angles left.
 __global__ void __launch_bounds__(256) k_prep_half8192(const double2* __restrict__ cs8192, int half, float4* __restrict__ prep,
-                                                        uint8_t* __restrict__ flip) {
+                                                        uint8_t* __restrict__ flip, double2* __restrict__ cs_half) {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= 12 * (kN / 2)) return;
     const int s = k / (kN / 2), j = k % (kN / 2);
     const double2 v = cs8192[s * kN + (kN / 2) * half + j];
+    cs_half[k] = v;  // what the scaled inverse table is built from
     const double c = v.x, sn = v.y;
     const bool f = c < 0.0;
     const double sp = f ? -sn : sn, cp = f ? -c : c;
@@ -1039,11 +1073,11 @@ __global__ void __launch_bounds__(256) k_reduce_wide(const float* __restrict__ p
 // floats the wide mode needs in the plan's partial-sum buffer
 size_t bwd8192_partial_floats(int sm_count) { return size_t(2) * sm_count * b4k::kSlotFloatsWide; }
 
-size_t bwd8192_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1); }
+size_t bwd8192_prep_bytes() { return size_t(12) * (f4k::kN / 2) * (sizeof(float4) + 1 + sizeof(double2)); }
 
 bool bwd8192_available(const bfq_plan* plan) {
     return plan->n == 2 * f4k::kN && plan->cc_major == 10 && plan->img_b8192[0] != nullptr && plan->img_b8192[1] != nullptr &&
-           plan->prep_half8192 != nullptr && plan->prep8192 != nullptr &&
+           plan->prep_half8192 != nullptr && plan->prep8192 != nullptr && plan->img_i8192[0] != nullptr && plan->img_i8192[1] != nullptr &&
            plan->partial_floats >= bwd8192_partial_floats(plan->sm_count) &&
            encode_tiled() != nullptr;
 }
@@ -1054,11 +1088,18 @@ cudaError_t bwd8192_build_tables(const bfq_plan* plan, cudaStream_t st) {
     const double2* cs = reinterpret_cast<const double2*>(reinterpret_cast<const float4*>(plan->prep8192) + count8);
     float4* prep = reinterpret_cast<float4*>(plan->prep_half8192);
     uint8_t* flip = reinterpret_cast<uint8_t*>(prep + count);
+    double2* cs_half = reinterpret_cast<double2*>(flip + count);  // count is a multiple of 16
     for (int h = 0; h < 2; ++h) {
-        b4k::k_prep_half8192<<<(count + 255) / 256, 256, 0, st>>>(cs, h, prep, flip);
+        b4k::k_prep_half8192<<<(count + 255) / 256, 256, 0, st>>>(cs, h, prep, flip, cs_half);
         b4k::k_build_image_bwd4096<<<(count + 255) / 256, 256, 0, st>>>(prep, flip, plan->img_b8192[h], plan->dsign8192[h]);
         b4k::k_build_gsign4096<<<(16 * b4k::kThreads + 255) / 256, 256, 0, st>>>(flip, plan->gsign8192[h]);
-        const cudaError_t e = cudaGetLastError();
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        // the half's scaled reverse walk (inverse kernel) and its range flag: words 1 and 2 of the plan's form flags
+        e = cudaMemsetAsync(plan->form_flag + 1 + h, 0, sizeof(int), st);
+        if (e != cudaSuccess) return e;
+        b4k::k_build_image_inv4096<<<(count + 255) / 256, 256, 0, st>>>(cs_half, plan->img_i8192[h], plan->form_flag + 1 + h);
+        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -1186,7 +1227,8 @@ cudaError_t inv4096_launch_f32(bfq_plan* plan, const void* y, int64_t rows, int6
     const int64_t want = (rows + G - 1) / G;
     const int grid = int(want < plan->sm_count ? want : plan->sm_count);
     kern<<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->img_i4096, plan->form_flag + 1,
-                                                    plan->gsign4096, x, ldx, int(rows), plan->status_word);
+                                                    plan->gsign4096, x, ldx, int(rows), plan->status_word, nullptr,
+                                                    b4k::InvUpper{});
     return cudaGetLastError();
 }
 
@@ -1210,11 +1252,57 @@ cudaError_t inv4096_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t 
     if (x_bf16) {
         b4k::k_inv4096<G, true><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->img_i4096,
                                                                             plan->form_flag + 1, plan->gsign4096, x, ldx,
-                                                                            int(rows), plan->status_word);
+                                                                            int(rows), plan->status_word, nullptr,
+                                                                            b4k::InvUpper{});
     } else {
         b4k::k_inv4096<G, false><<<grid, G * b4k::kThreads, S::kBytes, st>>>(ymap, plan->img_b4096, plan->img_i4096,
                                                                              plan->form_flag + 1, plan->gsign4096, x, ldx,
-                                                                             int(rows), plan->status_word);
+                                                                             int(rows), plan->status_word, nullptr,
+                                                                             b4k::InvUpper{});
+    }
+    return cudaGetLastError();
+}
+
+// n = 8192, bf16 rows in, bf16 or fp32 rows out: the inverse kernel's wide mode, even CTAs on the lower halves of x, odd
+// CTAs on the upper halves
+cudaError_t inv8192_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, bool x_bf16, int64_t ldx,
+                           cudaStream_t st) {
+    constexpr int G = 4;
+    using S = b4k::InvSmem<G>;
+    static bool attr_set[kMaxDevices] = {false};
+    if (!attr_set[plan->device]) {
+        cudaError_t e = cudaFuncSetAttribute(b4k::k_inv4096<G, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             int(S::kBytes));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(b4k::k_inv4096<G, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     int(S::kBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[plan->device] = true;
+    }
+    CUtensorMap ymap;  // whole rows of 8192 bf16 = 128 lines of 128 bytes
+    {
+        const cuuint64_t dims[3] = {64, 128, static_cast<cuuint64_t>(rows)};
+        const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(ldy) * 2};
+        const cuuint32_t box[3] = {64, 128, 1};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (encode_tiled()(&ymap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(y), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    const int64_t want = (rows + G - 1) / G;
+    const int per_half = plan->sm_count / 2 > 0 ? plan->sm_count / 2 : 1;
+    const int grid = 2 * int(want < per_half ? want : per_half);
+    const b4k::InvUpper upper{plan->img_b8192[1], plan->img_i8192[1], plan->form_flag + 2, plan->gsign8192[1]};
+    const float2* tw12 = plan->tw + 12 * f4k::kN;
+    if (x_bf16) {
+        b4k::k_inv4096<G, true, false, true><<<grid, G * b4k::kThreads, S::kBytes, st>>>(
+            ymap, plan->img_b8192[0], plan->img_i8192[0], plan->form_flag + 1, plan->gsign8192[0], x, ldx, int(rows),
+            plan->status_word, tw12, upper);
+    } else {
+        b4k::k_inv4096<G, false, false, true><<<grid, G * b4k::kThreads, S::kBytes, st>>>(
+            ymap, plan->img_b8192[0], plan->img_i8192[0], plan->form_flag + 1, plan->gsign8192[0], x, ldx, int(rows),
+            plan->status_word, tw12, upper);
     }
     return cudaGetLastError();
 }

@@ -55,6 +55,8 @@ size_t bwd8192_prep_bytes();
 size_t bwd8192_partial_floats(int sm_count);
 bool bwd8192_available(const bfq_plan* plan);
 cudaError_t bwd8192_build_tables(const bfq_plan* plan, cudaStream_t st);
+cudaError_t inv8192_launch(bfq_plan* plan, const void* y, int64_t rows, int64_t ldy, void* x, bool x_bf16, int64_t ldx,
+                           cudaStream_t st);
 cudaError_t bwd8192_launch_halves(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
                                   float* dtheta, cudaStream_t st);
 cudaError_t bwd4096_build_tables(const bfq_plan* plan, cudaStream_t st);

@@ -25,6 +25,7 @@ struct bfq_plan {
     bool bwd_tables_valid = false;  // the three above match the current angles
     // n = 8192: backward tables of the two 4096-element halves (stages 0 .. 11), built on first use like the above
     float* img_b8192[2] = {nullptr, nullptr};
+    float* img_i8192[2] = {nullptr, nullptr};  // scaled-form constants of the inverse kernel, per half
     int8_t* dsign8192[2] = {nullptr, nullptr};
     uint32_t* gsign8192[2] = {nullptr, nullptr};
     void* prep_half8192 = nullptr;  // staging of one half: three-shear constants and negation flags

@@ -417,11 +417,11 @@ def test_full_size_int2_n8192_and_fold_sampled():
         del x, codes, scales
 
 
-# ---- tuned inverse for n = 4096 bf16 rows ------------------------------------------------------------------------
+# ---- tuned inverse for n = 4096 and n = 8192 bf16 rows -------------------------------------------------------------
 @pytest.mark.parametrize("rows", [1, 3, 147, 148 * 4 + 1, 1000])
 @pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
-def test_tuned_inverse_n4096(rows, out_dtype):
-    n = 4096
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_tuned_inverse(n, rows, out_dtype):
     theta = synth.angles(n, "uniform", 90 + rows)
     theta[:, ::7] = math.pi / 2
     theta[:, 1::7] = -math.pi
@@ -445,6 +445,20 @@ def test_tuned_inverse_n4096(rows, out_dtype):
     # round trip through the tuned-path forward of the generic kernels
     back = p.forward(x2.float(), out_dtype=torch.float32)
     check_rows_close(back, to_f64(y), 64 * absmax_rows(y), "round trip") if out_dtype == torch.float32 else None
+    if n == 8192:
+        # one half of the row on the three-shear tables, the other on the scaled ones
+        assert p.stage_form() & 2 == 0
+        theta3 = theta2.clone()
+        theta3[3:7, :2048] = math.pi / 2  # four stages of the lower half: cosines of 4e-8 multiply up along every path
+        p.set_angles(theta3.to(DEV))
+        x3 = p.inverse(y.to(DEV), out_dtype=out_dtype)
+        assert p.stage_form() & 2 == 2
+        check_rows_close(x3, oracle.inverse(to_f64(theta3), to_f64(y)), absmax_rows(y), "tuned inverse, mixed forms")
+        theta3[3:7, :2048], theta3[3:7, 2048:] = theta2[3:7, :2048], -math.pi / 2  # now only the upper half
+        p.set_angles(theta3.to(DEV))
+        x3 = p.inverse(y.to(DEV), out_dtype=out_dtype)
+        assert p.stage_form() & 2 == 2
+        check_rows_close(x3, oracle.inverse(to_f64(theta3), to_f64(y)), absmax_rows(y), "tuned inverse, mixed forms (upper)")
 
 
 # ---- Walsh-Hadamard transform (the fixed rotation the paper compares with) and unquantized bf16 rows ---------------
