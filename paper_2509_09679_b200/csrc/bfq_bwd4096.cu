@@ -253,10 +253,10 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
           void* __restrict__ dx_out, int64_t ld, float* __restrict__ partial, int rows, int* __restrict__ status,
           const float2* __restrict__ tw12, const __grid_constant__ WideHalf upper) {
     static_assert(!(IN_F32 && WIDE), "the wide mode takes bf16 rows");
-    // wide mode: the first half of the grid works on the lower halves of the rows, the second on the upper halves (the
-    // hardware hands out CTAs in index order, so the second set fills the SMs as the first set's CTAs finish)
+    // wide mode: even CTAs work on the lower halves of the rows, odd CTAs on the upper halves (CTAs 2i and 2i + 1 take
+    // the same row pairs at about the same time, so the second read of a g row comes from L2)
     const int ctas = WIDE ? int(gridDim.x >> 1) : int(gridDim.x);
-    const int half = WIDE ? int(blockIdx.x >= unsigned(ctas)) : 0;
+    const int half = WIDE ? int(blockIdx.x & 1u) : 0;
     const CUtensorMap* const xm = (WIDE && half) ? &upper.xmap : &xmap;
     const float* const img = (WIDE && half) ? upper.img : img_lo;
     const uint32_t* const gsign = (WIDE && half) ? upper.gsign : gsign_lo;
@@ -296,7 +296,7 @@ k_bwd4096(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUte
     }
 
     const int pairs = (rows + 1) / 2;
-    const int first = int(blockIdx.x) - half * ctas;
+    const int first = WIDE ? int(blockIdx.x >> 1) : int(blockIdx.x);
     const int stride = ctas;
     const int count = first < pairs ? (pairs - first + stride - 1) / stride : 0;
     // both input rings belong to the upper group: one mbarrier per slot counts the x pair and the g pair
@@ -1044,8 +1044,8 @@ __global__ void __launch_bounds__(256) k_prep_half8192(const double2* __restrict
                           static_cast<float>(sn));
 }
 
-// Wide mode: dtheta [13][4096] from the 2 * ctas slots (kSlotFloatsWide floats each; slots 0 .. ctas - 1 hold the lower
-// half's CTAs).  Stage s < 12, angle 2048 h + j = the sum over half h's slots of entry s * 2048 + j; stage 12, angle i =
+// Wide mode: dtheta [13][4096] from the 2 * ctas slots (kSlotFloatsWide floats each; even slots hold the lower half's
+// CTAs).  Stage s < 12, angle 2048 h + j = the sum over half h's slots of entry s * 2048 + j; stage 12, angle i =
 // the sum over all slots of entry kSlotFloats + i.  A block = 8 slot lanes x 32 angles: lane y adds slots y, y + 8, ...
 // in order, then the eight sums are added in lane order, so the result does not depend on timing.
 __global__ void __launch_bounds__(256) k_reduce_wide(const float* __restrict__ partial, int ctas, float* __restrict__ out) {
@@ -1053,12 +1053,12 @@ __global__ void __launch_bounds__(256) k_reduce_wide(const float* __restrict__ p
     const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
     const int k = blockIdx.x * 32 + x;  // 13 * 4096 is a multiple of 32
     const int s = k >> 12, r = k & 4095;
-    int first = 0, count = 2 * ctas, entry = kSlotFloats + r;
-    if (s < 12) first = (r >> 11) * ctas, count = ctas, entry = s * (kN / 2) + (r & 2047);
+    int first = 0, step = 1, count = 2 * ctas, entry = kSlotFloats + r;
+    if (s < 12) first = r >> 11, step = 2, count = ctas, entry = s * (kN / 2) + (r & 2047);
     const float* src = partial + static_cast<int64_t>(first) * kSlotFloatsWide + entry;
     float acc = 0.f;
 #pragma unroll 4
-    for (int c = y; c < count; c += 8) acc += src[static_cast<int64_t>(c) * kSlotFloatsWide];
+    for (int c = y; c < count; c += 8) acc += src[static_cast<int64_t>(c) * step * kSlotFloatsWide];
     sh[y][x] = acc;
     __syncthreads();
     if (y == 0) {
@@ -1105,7 +1105,7 @@ cudaError_t bwd8192_build_tables(const bfq_plan* plan, cudaStream_t st) {
     return cudaSuccess;
 }
 
-// The n = 8192 backward (bf16 rows): both halves of the rows' elements in one launch (2 x grid CTAs), then one reduction;
+// The n = 8192 backward (bf16 rows): both halves of the rows' elements in one launch (grid CTAs each), then one reduction;
 // dx and all 13 rows of d-theta.
 cudaError_t bwd8192_launch_halves(bfq_plan* plan, const void* x, const void* g, int64_t rows, int64_t ld, void* dx,
                                   float* dtheta, cudaStream_t st) {
@@ -1117,7 +1117,8 @@ cudaError_t bwd8192_launch_halves(bfq_plan* plan, const void* x, const void* g, 
         attr_set[plan->device] = true;
     }
     const int64_t pairs = (rows + 1) / 2;
-    const int grid = int(pairs < plan->sm_count ? pairs : plan->sm_count);
+    const int per_half = plan->sm_count / 2 > 0 ? plan->sm_count / 2 : 1;  // one CTA per SM: both halves in one wave
+    const int grid = int(pairs < per_half ? pairs : per_half);
     CUtensorMap xmap, gmap;
     b4k::WideHalf upper{};
     // x: one half's 4096 elements of every row; g: whole rows of 8192 bf16 = 128 lines of 128 bytes

@@ -49,7 +49,7 @@ size_t inv4096_image_bytes();
 size_t bwd4096_dsign_bytes();
 size_t bwd4096_gsign_bytes();
 bool bwd4096_available(const bfq_plan* plan);
-// n = 8192 bf16 rows: the n = 4096 backward kernel on the two halves of the elements (one launch, twice the CTAs); the
+// n = 8192 bf16 rows: the n = 4096 backward kernel on the two halves of the elements (one launch, even CTAs on the lower half, odd CTAs on the upper); the
 // stage that joins the halves is folded into the read of g and its sums are taken there too
 size_t bwd8192_prep_bytes();
 size_t bwd8192_partial_floats(int sm_count);
