@@ -37,6 +37,7 @@ constexpr int kConstCols = 384;              // 12 stages x 32 words
 constexpr int kAccCol = 384;                 // accumulators of stages 0..7: 16 columns each
 constexpr int kUpperSteps = 8;               // half-stage steps of the reverse walk done by the upper group: stages 11 .. 8
 constexpr uint32_t kPairBytes = 2 * kRowBytes;  // two bf16 rows
+constexpr int kWideCol = 416;  // wide inverse: (cos, +-sin) of the stage that joins the halves, 64 columns behind either table
 constexpr int kInvCols = 416;  // scaled inverse: stages 11..1 (32 columns each, stage s at 32 (s - 1)), then stage 0 (64)
 enum : int { kFormScaled = 0, kFormShear = 1 };
 
@@ -892,6 +893,26 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
         }
         tmem_wait_st();
     }
+    if constexpr (WIDE) {
+        // (cos, sin) of the stage-12 pairs 2t + 256m, +1 for m = 0 .. 15, sin with the sign this half applies it with:
+        // 64 columns of the thread's lane, written once by the first group
+        static_assert(kWideCol >= kInvCols && kWideCol >= kConstCols && kWideCol + 64 <= 512, "tensor-memory columns");
+        if (g == 0) {
+            const float sg = half ? -1.f : 1.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint32_t v[16];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float4 cs = __ldg(reinterpret_cast<const float4*>(tw12 + 2 * t + 256 * (4 * j + i)));
+                    v[4 * i + 0] = __float_as_uint(cs.x), v[4 * i + 1] = __float_as_uint(sg * cs.y);
+                    v[4 * i + 2] = __float_as_uint(cs.z), v[4 * i + 3] = __float_as_uint(sg * cs.w);
+                }
+                tmem_st16(tlane + kWideCol + 16 * j, v);
+            }
+            tmem_wait_st();
+        }
+    }
     tmem_fence_before();
     __syncthreads();
     tmem_fence_after();
@@ -926,8 +947,38 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
         tmem_ld32(tlane + (FORM == kFormShear ? 32 * 11 : 32 * 10), T0);
         mbar_wait_bounded(bar_base + 8 * slot, (kSlotsUsed == 1 ? k : (k >> 1)) & 1, status);
         const uint32_t tile = in_base + slot * kSlotBytes;
+        if constexpr (WIDE) {
+            // elements 2t + 256m, +1 of both halves of the row (the upper half is 8192 bytes further on, the same line
+            // modulo 8) and (cos, +-sin) of the two stage-12 pairs they form, eight registers m per tensor-memory load
 #pragma unroll
-        for (int qq = 0; qq < 4; ++qq) {
+            for (int hh = 0; hh < 2; ++hh) {
+                tmem_ld32(tlane + kWideCol + 32 * hh, T1);
+                uint32_t s8[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+                if constexpr (kSigns) {
+                    const uint4 sw0 = __ldg(gsv + (2 * hh) * kThreads + t), sw1 = __ldg(gsv + (2 * hh + 1) * kThreads + t);
+                    s8[0] = sw0.x, s8[1] = sw0.y, s8[2] = sw0.z, s8[3] = sw0.w;
+                    s8[4] = sw1.x, s8[5] = sw1.y, s8[6] = sw1.z, s8[7] = sw1.w;
+                }
+                uint32_t wo[8], wx[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int m = 8 * hh + i;
+                    const uint32_t at = tile + ((m & 1) ? g_a1 : g_a0) + 512u * m;
+                    wo[i] = lds32(at + 8192u * half), wx[i] = lds32(at + 8192u * (half ^ 1));
+                }
+                tmem_wait_ld32(T1);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const u64 own = pack2u(bf16_lo(wo[i]), wo[i] & 0xFFFF0000u), oth = pack2u(bf16_lo(wx[i]), wx[i] & 0xFFFF0000u);
+                    const u64 c2 = pack2u(T1[4 * i], T1[4 * i + 2]), s2 = pack2u(T1[4 * i + 1], T1[4 * i + 3]);
+                    uint32_t lo, hi;
+                    unpack2u(fma2(s2, oth, mul2(c2, own)), lo, hi);
+                    P[8 * hh + i] = pack2u(lo ^ ((s8[i] & 0x8000u) << 16), hi ^ (s8[i] & 0x80000000u));
+                }
+            }
+        }
+#pragma unroll
+        for (int qq = 0; qq < (WIDE ? 0 : 4); ++qq) {
             if constexpr (IN_F32) {
                 // elements 2t + 256m, +1 are the 8-byte word t & 1 of 16-byte chunk (t & 15) >> 1 of 128-byte line
                 // (t >> 4) + 8m; the swizzle moves the chunk to chunk ^ (line & 7)
@@ -953,19 +1004,6 @@ k_inv4096(const __grid_constant__ CUtensorMap ymap, const float* __restrict__ im
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int m = 4 * qq + i;
-                if constexpr (WIDE) {
-                    // elements 2t + 256m, +1 of both halves of the row (the upper half is 8192 bytes further on, the same
-                    // line modulo 8) and (cos, sin) of the two stage-12 pairs they form
-                    const uint32_t at = tile + ((m & 1) ? g_a1 : g_a0) + 512u * m;
-                    const uint32_t wo = lds32(at + 8192u * half), wx = lds32(at + 8192u * (half ^ 1));
-                    const float4 cs = __ldg(reinterpret_cast<const float4*>(tw12 + 2 * t + 256 * m));
-                    const float sg = half ? -1.f : 1.f;
-                    const u64 own = pack2u(bf16_lo(wo), wo & 0xFFFF0000u), oth = pack2u(bf16_lo(wx), wx & 0xFFFF0000u);
-                    uint32_t lo, hi;
-                    unpack2u(fma2(pack2(sg * cs.y, sg * cs.w), oth, mul2(pack2(cs.x, cs.z), own)), lo, hi);
-                    P[m] = pack2u(lo ^ ((s4[i] & 0x8000u) << 16), hi ^ (s4[i] & 0x80000000u));
-                    continue;
-                }
                 const uint32_t w = lds32(tile + ((m & 1) ? g_a1 : g_a0) + 512u * m) ^ s4[i];
                 P[m] = pack2u(bf16_lo(w), w & 0xFFFF0000u);
             }
