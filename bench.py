@@ -38,7 +38,7 @@ EXECUTED_SLOTS_PER_ROW = 2 * (4096 // 2) * 11 + 4 * (4096 // 2) + 4096
 FP32_LANES_PER_SM = 128
 # dram bytes (read + write) per row of the forward+quant kernel, from the committed ncu capture of the
 # current kernel on this workload; set back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES_PER_ROW = (268688128 + 51416576) / 32768  # dram read + write of one k_fwdq4096 launch (profiles/)
+NCU_TRAFFIC_BYTES_PER_ROW = (268692736 + 50886656) / 32768  # dram read + write of one k_fwdq4096 launch (profiles/)
 
 
 def measured_peaks():
