@@ -186,6 +186,40 @@ def test_learn4096_backward_all_rows():
     check_rows_close(dx[ti], dx_ref, absmax_rows(g[ti]), "learn4096 dx")
 
 
+@pytest.mark.slow
+def test_act8192_backward_and_inverse_at_the_timed_sizes():
+    """The two n = 8192 legs the benchmark times, in its launch configuration: backward on a quarter of the activation
+    rows (d-theta over every row against the oracle summed over row blocks, dL/dx on sampled rows), inverse on all of
+    them (sampled rows)."""
+    wl = synth.WORKLOADS["act8192_int2"]
+    theta = wl.theta(device=DEV)
+    x = wl.x(device=DEV)
+    p = Plan(wl.n, DEV)
+    p.set_angles(theta)
+    th64 = to_f64(theta)
+    rows = wl.n_rows // 4
+    g = wl.g(device=DEV, n_rows=rows)
+    dx = torch.empty_like(g)
+    dth = Guarded((wl.L, wl.n // 2), torch.float32, DEV)
+    p.backward(x[:rows], g, dx=dx, dtheta=dth.view)
+    assert p.device_status() == 0 and dth.intact()
+    acc = np.zeros((wl.L, wl.n // 2))
+    for r0 in range(0, rows, 2048):
+        acc += oracle.backward(th64, to_f64(x[r0:r0 + 2048]), to_f64(g[r0:r0 + 2048]))[1]
+    check_dtheta(dth.view, acc, "act8192 dtheta, all rows of the timed batch")
+    ti = torch.from_numpy(np.arange(0, rows, rows // 256)).to(DEV)
+    dx_ref, _ = oracle.backward(th64, to_f64(x[ti]), to_f64(g[ti]))
+    check_rows_close(dx[ti], dx_ref, absmax_rows(g[ti]), "act8192 dx")
+    del g, dx
+    out = torch.empty_like(x)
+    p.inverse(x, out=out)
+    assert p.device_status() == 0
+    ti = torch.from_numpy(np.arange(0, wl.n_rows, wl.n_rows // 256)).to(DEV)
+    check_rows_close(out[ti], oracle.inverse(th64, to_f64(x[ti])), absmax_rows(x[ti]), "act8192 inverse")
+    ti = torch.tensor([0, 1, 2, 3, wl.n_rows - 4, wl.n_rows - 3, wl.n_rows - 2, wl.n_rows - 1], device=DEV)  # first and last CTA
+    check_rows_close(out[ti], oracle.inverse(th64, to_f64(x[ti])), absmax_rows(x[ti]), "act8192 inverse, ends")
+
+
 def test_bounded_wait_runs_out_and_the_plan_recovers():
     """A device-side wait that cannot be satisfied (the kernel is told to expect 16 bytes more per row load than
     arrive) gives up after its poll limit: the kernel returns, the status word reports it once, nothing is written
