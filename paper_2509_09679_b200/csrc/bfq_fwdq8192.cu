@@ -314,7 +314,8 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
 #pragma unroll
             for (int i = 0; i < 8; ++i) st_async_b64(peer_box + i * 1024u, P[i], peer_bar_swap);
         }
-        mbar_wait_cluster_bounded(bar_swap, k & 1, status);
+        if (q == 0) mbar_wait_cluster_bounded(bar_swap, k & 1, status);  // one warp polls, the others sleep at the barrier
+        bar_sync(ex.bar, kGroupThreads);
         if (rank == 0) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) A[i] = P[i], B[i] = lds64(my_box + i * 1024u);
@@ -351,7 +352,8 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         if (t == 0) {
             st_async_b32(peer_amax + (k & 1) * 32 + 16, __float_as_uint(amax), peer_bar_amax);
         }
-        mbar_wait_cluster_bounded(bar_amax, k & 1, status);
+        if (q == 0) mbar_wait_cluster_bounded(bar_amax, k & 1, status);
+        bar_sync(ex.bar, kGroupThreads);
         amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
         float inv;
         static_assert(!(ROWS && BITS == 16), "BITS = 16 writes the rows already");
