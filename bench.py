@@ -582,6 +582,10 @@ def time_others(torch, synth, Plan, dev):
     scales = torch.empty((wl.n_rows,), dtype=torch.float16, device=dev)
     record("forward_int2_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 4 + 2,
            lambda: plan8.forward_quant(x, 2, codes=codes, scales=scales), 5)
+    codes4 = torch.empty((wl.n_rows, wl.n // 2), dtype=torch.uint8, device=dev)
+    record("forward_int4_n8192", wl.n_rows, wl.n, wl.L, 4, 2 * wl.n + wl.n // 2 + 2,
+           lambda: plan8.forward_quant(x, 4, codes=codes4, scales=scales), 5)
+    del codes4
     x32 = x.float()
     record("forward_int2_fp32_rows_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n + wl.n // 4 + 2,
            lambda: plan8.forward_quant(x32, 2, codes=codes, scales=scales), 5)
@@ -589,6 +593,9 @@ def time_others(torch, synth, Plan, dev):
     y8 = torch.empty_like(x)
     record("forward_bf16_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan8.forward(x, out=y8), 5)
     record("inverse_n8192", wl.n_rows, wl.n, wl.L, 4, 4 * wl.n, lambda: plan8.inverse(x, out=y8), 5)
+    record("hadamard_int2_n8192", wl.n_rows, wl.n, wl.L, 1, 2 * wl.n + wl.n // 4 + 2,
+           lambda: plan8.hadamard_quant(x, 2, codes=codes, scales=scales), 5)
+    record("hadamard_bf16_n8192", wl.n_rows, wl.n, wl.L, 1, 4 * wl.n, lambda: plan8.hadamard(x, out=y8), 5)
     # backward at n = 8192 (forward cluster kernel for the last stage's sums + the n = 4096 backward kernel per half): a quarter of the rows
     rows8 = wl.n_rows // 4
     g8 = torch.randn((rows8, wl.n), device=dev, dtype=torch.float32).to(x.dtype)

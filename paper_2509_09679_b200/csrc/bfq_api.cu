@@ -525,6 +525,9 @@ int bfq_hadamard(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows, int6
     if (xt == BFQ_BF16 && yt == BFQ_BF16 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
         fwdq4096_available(plan)) {
         e = fwdq4096_launch(plan, x, rows, ldx, true, nullptr, nullptr, y, ldy, st);
+    } else if (xt == BFQ_BF16 && yt == BFQ_BF16 && x != y && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") &&
+               fwdq8192_available(plan)) {
+        e = fwdq8192_launch_hadamard(plan, x, rows, ldx, 0, nullptr, nullptr, y, ldy, st);
     } else {
         GenericParams p{};
         p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = y, p.yt = yt, p.ldy = ldy, p.rows = rows;
@@ -549,6 +552,8 @@ int bfq_hadamard_quant(bfq_plan* plan, const void* x, bfq_dtype xt, int64_t rows
     if (xt == BFQ_BF16 && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") && fwdq4096_available(plan)) {
         e = bits == 4 ? fwdq4096_launch(plan, x, rows, ldx, true, codes, scales_f16, nullptr, 0, st)
                       : fwdq4096_launch_bits(plan, x, rows, ldx, true, bits, codes, scales_f16, st);
+    } else if (xt == BFQ_BF16 && rows < (int64_t(1) << 31) && !env_flag("BFQ_GENERIC_ONLY") && fwdq8192_available(plan)) {
+        e = fwdq8192_launch_hadamard(plan, x, rows, ldx, bits, codes, scales_f16, nullptr, 0, st);
     } else {
         GenericParams p{};
         p.tw = plan->tw, p.x = x, p.xt = xt, p.ldx = ldx, p.y = nullptr, p.yt = BFQ_F32, p.ldy = plan->n;

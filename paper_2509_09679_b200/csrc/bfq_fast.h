@@ -40,6 +40,8 @@ cudaError_t fwdq8192_launch_codes_rows(const bfq_plan* plan, const void* x, int6
                                        uint8_t* codes, uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 cudaError_t fwdq8192_launch_f32(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
                                 uint16_t* scales, void* y_f32, int64_t ldy, cudaStream_t st);
+cudaError_t fwdq8192_launch_hadamard(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                                     uint16_t* scales, void* y_bf16, int64_t ldy, cudaStream_t st);
 cudaError_t fwdq8192_launch_bf16(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, void* y, int64_t ldy,
                                  cudaStream_t st);
 

@@ -148,18 +148,6 @@ __device__ __forceinline__ void run_chunks(u64 (&P)[16], uint32_t (&Tcur)[CW], u
     if constexpr (C + 1 < CH::kCount) run_chunks<FORM, C + 1, CW, XB>(P, Tnext, Tcur, tbase, ex, turn, issue_next);
 }
 
-// Walsh-Hadamard stages 4*PH .. 4*PH+3 of a phase: (a, b) -> (a + b, a - b), no constants; the 1/sqrt(n) is
-// applied by the epilogue
-template <int K>
-__device__ __forceinline__ void stage_hadamard(u64 (&P)[16]) {
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        const int m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
-        const u64 a = P[m_lo], b = P[m_hi];
-        P[m_lo] = add2(a, b);
-        P[m_hi] = sub2(a, b);
-    }
-}
 template <int XB, class F>
 __device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&& issue_next) {
     stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);

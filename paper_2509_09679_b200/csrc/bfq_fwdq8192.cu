@@ -28,7 +28,7 @@ using namespace f4k;
 
 constexpr int kN8 = 8192;
 constexpr int kCols8 = 384 + 64;  // 12 stages of this half + this rank's share of stage 12
-enum : int { kFormScaled = 0, kFormShear = 1 };  // how stages 0..11 rotate (the image must match)
+enum : int { kFormScaled = 0, kFormShear = 1, kFormHadamard = 2 };  // how stages 0..11 rotate (the image must match)
 
 template <int G>
 struct Smem {
@@ -106,6 +106,28 @@ __device__ __forceinline__ void stage12_quad(u64 (&A)[8], u64 (&B)[8], const uin
     }
 }
 
+// the fixed Hadamard rotation: twelve constant-free stages with the same two regroupings, no tokens
+template <class F>
+__device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&& issue_next) {
+    stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);
+    regroup1(P, ex);
+    stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);
+    regroup2(P, ex);
+    issue_next();
+    stage_hadamard<0>(P), stage_hadamard<1>(P), stage_hadamard<2>(P), stage_hadamard<3>(P);
+}
+// ... and its last stage with the 1/sqrt(8192) of all thirteen
+__device__ __forceinline__ void stage12_hadamard(u64 (&A)[8], u64 (&B)[8]) {
+    const float k = 0.011048543456039806f;  // 2^-6.5
+    const u64 kk = pack2(k, k), nk = pack2(-k, -k);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const u64 ka = mul2(kk, A[i]), b = B[i];
+        A[i] = fma2(kk, b, ka);
+        B[i] = fma2(nk, b, ka);
+    }
+}
+
 // two INT2 codes of a packed pair (elements e, e+1) as a nibble: bits 0-1 = code(e), bits 2-3 = code(e+1)
 __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool plain) {
     if (plain) {
@@ -128,7 +150,8 @@ __device__ __forceinline__ uint32_t nibble_int2(u64 v, u64 inv2, float inv, bool
 // ROWS (BITS = 2, 4, 8): the rotated rows are written as well, in bf16, to `yrows` (leading dimension ldy).
 // IN_F32: fp32 rows (a half row is 16 KB): one input slot per group instead of two, re-armed after the second
 // regrouping's barrier.  BITS = 32 (with IN_F32): the rotated rows in fp32 (`codes` then points to them).
-template <int G, int BITS, int STEP = 2, bool ROWS = false, bool IN_F32 = false>
+// HADAMARD: y = H x instead of the butterfly (no constants: `img` and `form` are not read, tensor memory stays empty).
+template <int G, int BITS, int STEP = 2, bool ROWS = false, bool IN_F32 = false, bool HADAMARD = false>
 __global__ void __launch_bounds__(G * kGroupThreads, 1)
 k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ CUtensorMap map_hi,
            const float* __restrict__ img, const int* __restrict__ form, uint8_t* __restrict__ codes,
@@ -172,7 +195,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     static_assert(STEP >= 0 && (STEP == 0 || G % STEP == 0), "the rings must have equal length");
     constexpr int kRings = STEP == 0 ? 1 : STEP;
     Turn turn;
-    turn.on = STEP > 0;
+    turn.on = STEP > 0 && !HADAMARD;
     turn.wait_id = kTurnBar0 + g;
     turn.pass_id = kTurnBar0 + (g + STEP) % G;
     const bool seeds_ring = (g + STEP) % G < kRings;  // this group's successor starts with the token
@@ -191,8 +214,8 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     // constants of this thread's role: image [form][rank][column quad][role][4], all loads in flight together; the
     // scaled-form image is fetched on the assumption that the table build selected it
     constexpr int kFillBlocks = (kCols8 / 16 + G - 1) / G;
-    bool shear;
-    {
+    bool shear = false;
+    if constexpr (!HADAMARD) {
         float4 fill[kFillBlocks][4];
         auto fetch_image = [&](int which) {
             const float4* base = reinterpret_cast<const float4*>(img) + (static_cast<size_t>(which) * 2 + rank) * (kCols8 / 4) * 128;
@@ -260,7 +283,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     for (int k = 0; k < count; ++k) {
         const int row = first + k * stride;
         const int slot = IN_F32 ? 0 : (k & 1);
-        tmem_ld32(tlane, T0);
+        if constexpr (FORM != kFormHadamard) tmem_ld32(tlane, T0);
         mbar_wait_bounded(bar_in + 8 * slot, (IN_F32 ? k : (k >> 1)) & 1, status);
         const uint32_t src = in_base + slot * kSlotBytes + in_line;
         if constexpr (IN_F32) {
@@ -294,12 +317,17 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
                 }
             }
         }
-        run_chunks<FORM, 0>(P, T0, T1, tlane, ex, turn, [&]() {
+        auto issue_next = [&]() {
             if (t == 0 && k + kSlotsUsed < count) {
                 mbar_expect_tx(bar_in + 8 * slot, kSlotBytes);
                 tma_load_3d(in_base + slot * kSlotBytes, tmap, 0, 0, first + (k + kSlotsUsed) * stride, bar_in + 8 * slot);
             }
-        });  // the first 32 of this rank's stage-12 constants are now requested in T0
+        };
+        if constexpr (FORM == kFormHadamard) {
+            run_hadamard(P, ex, issue_next);
+        } else {
+            run_chunks<FORM, 0>(P, T0, T1, tlane, ex, turn, issue_next);  // the first 32 of this rank's stage-12 constants are now requested in T0
+        }
 
         // ---- stage 12: rank 0 finishes registers 0-7 of both halves, rank 1 registers 8-15 ----
         u64 A[8], B[8];  // lower-half / upper-half values of the registers this rank finishes
@@ -323,11 +351,15 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
 #pragma unroll
             for (int i = 0; i < 8; ++i) A[i] = lds64(my_box + i * 1024u), B[i] = P[8 + i];
         }
-        tmem_wait_ld32(T0);
-        tmem_ld32(tlane + 416, T1);
-        stage12_quad<0>(A, B, T0);
-        tmem_wait_ld32(T1);
-        stage12_quad<4>(A, B, T1);
+        if constexpr (FORM == kFormHadamard) {
+            stage12_hadamard(A, B);
+        } else {
+            tmem_wait_ld32(T0);
+            tmem_ld32(tlane + 416, T1);
+            stage12_quad<0>(A, B, T0);
+            tmem_wait_ld32(T1);
+            stage12_quad<4>(A, B, T1);
+        }
 
         // ---- absmax of the whole row: thread, warp, group, then the peer's half ----
         float m0 = 0.f, m1 = 0.f;
@@ -477,7 +509,9 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     }
     if (g < kRings) turn.acquire();  // each ring's first group takes its token back: no arrival stays pending
     };
-    if (!shear) {
+    if constexpr (HADAMARD) {
+        row_loop(std::integral_constant<int, kFormHadamard>());
+    } else if (!shear) {
         row_loop(std::integral_constant<int, kFormScaled>());
     } else {
         row_loop(std::integral_constant<int, kFormShear>());
@@ -608,12 +642,12 @@ bool fwdq8192_available(const bfq_plan* plan) {
            encode_tiled() != nullptr;
 }
 
-template <int BITS, bool ROWS = false, bool IN_F32 = false>
+template <int BITS, bool ROWS = false, bool IN_F32 = false, bool HADAMARD = false>
 static cudaError_t fwdq8192_launch_bits(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, uint8_t* codes,
                                         uint16_t* scales, int64_t ldy, cudaStream_t st, void* yrows = nullptr) {
     constexpr int G = 4;
     using S = f8k::Smem<G>;
-    auto kern = f8k::k_fwdq8192<G, BITS, 2, ROWS, IN_F32>;
+    auto kern = f8k::k_fwdq8192<G, BITS, 2, ROWS, IN_F32, HADAMARD>;
     static bool attr_set[kMaxDevices] = {false};
     if (!attr_set[plan->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(S::kBytes));
@@ -674,6 +708,16 @@ cudaError_t fwdq8192_launch_f32(const bfq_plan* plan, const void* x, int64_t row
     if (bits == 2) return fwdq8192_launch_bits<2, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
     if (bits == 4) return fwdq8192_launch_bits<4, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
     return fwdq8192_launch_bits<8, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
+}
+
+// y = H x (the fixed Hadamard rotation) on bf16 rows: codes + scales (bits = 2, 4, 8) or the rotated rows in bf16 (bits = 0)
+cudaError_t fwdq8192_launch_hadamard(const bfq_plan* plan, const void* x, int64_t rows, int64_t ldx, int bits, uint8_t* codes,
+                                     uint16_t* scales, void* y, int64_t ldy, cudaStream_t st) {
+    if (bits == 0)
+        return fwdq8192_launch_bits<16, false, false, true>(plan, x, rows, ldx, static_cast<uint8_t*>(y), nullptr, ldy, st);
+    if (bits == 2) return fwdq8192_launch_bits<2, false, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
+    if (bits == 4) return fwdq8192_launch_bits<4, false, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
+    return fwdq8192_launch_bits<8, false, false, true>(plan, x, rows, ldx, codes, scales, 0, st);
 }
 
 // y = Q x in bf16 (the weight-only setting: activations stay 16-bit)

@@ -179,6 +179,19 @@ __device__ __forceinline__ int sign_before(const uint8_t* __restrict__ flip, int
     return f ? -1 : 1;
 }
 
+// Walsh-Hadamard local stage K: (a, b) -> (a + b, a - b) on packed registers m and m | 2^K, no constants; the
+// 1/sqrt(n) is applied later, once
+template <int K>
+__device__ __forceinline__ void stage_hadamard(u64 (&P)[16]) {
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int m_lo = ((u >> K) << (K + 1)) | (u & ((1 << K) - 1)), m_hi = m_lo | (1 << K);
+        const u64 a = P[m_lo], b = P[m_hi];
+        P[m_lo] = add2(a, b);
+        P[m_hi] = sub2(a, b);
+    }
+}
+
 }  // namespace f4k
 
 // ---- host side: launch that lets the kernel's set-up overlap the tail of the kernel before it in the stream ----

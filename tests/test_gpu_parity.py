@@ -481,8 +481,8 @@ def test_hadamard_every_n(n, dtype):
 
 
 @pytest.mark.parametrize("rows", [1, 5, 593, 1000])
-def test_tuned_n4096_hadamard_and_bf16_rows(rows):
-    n = 4096
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_tuned_hadamard_and_bf16_rows(n, rows):
     theta = synth.angles(n, "uniform", 110 + rows)
     x = synth.rows(rows, n, "student_t3", 111 + rows, outliers=8, outlier_scale=50.0, dtype=torch.bfloat16)
     p = plan_for(n, theta)
@@ -505,6 +505,10 @@ def test_tuned_n4096_hadamard_and_bf16_rows(rows):
     scales = Guarded((rows,), torch.float16, DEV)
     p.hadamard_quant(xv, 4, codes=codes.view, scales=scales.view)
     check_quant(codes.view, scales.view, h_ref, 4, "tuned hadamard INT4")
+    assert codes.intact() and scales.intact() and p.device_status() == 0
+    codes = Guarded((rows, n // 4), torch.uint8, DEV)
+    p.hadamard_quant(xv, 2, codes=codes.view, scales=scales.view)
+    check_quant(codes.view, scales.view, h_ref, 2, "tuned hadamard INT2")
     assert codes.intact() and scales.intact() and p.device_status() == 0
 
 
