@@ -273,6 +273,18 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     // even lane stores the bytes of the lower half of the row, the odd lane those of the upper half.
     uint8_t* const out_t = codes + (t >> 1) + 64 * 8 * rank + ((t & 1) ? 1024 : 0);
 
+    // Waiting for the peer CTA: with bf16 rows and the butterfly one warp of the row group polls and the other three
+    // sleep at the group's named barrier (1.4 % faster than all four polling); with fp32 rows or the Hadamard stages
+    // the extra barrier costs more than the polling (4.8 % / 3.5 % slower), so there every warp polls
+    constexpr bool kOnePoller = !IN_F32 && !HADAMARD;
+    auto wait_peer = [&](uint32_t bar, uint32_t parity) {
+        if constexpr (kOnePoller) {
+            if (q == 0) mbar_wait_cluster_bounded(bar, parity, status);
+            bar_sync(ex.bar, kGroupThreads);
+        } else {
+            mbar_wait_cluster_bounded(bar, parity, status);
+        }
+    };
     // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
     auto row_loop = [&](auto form_tag) {
     constexpr int FORM = decltype(form_tag)::value;
@@ -342,8 +354,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
 #pragma unroll
             for (int i = 0; i < 8; ++i) st_async_b64(peer_box + i * 1024u, P[i], peer_bar_swap);
         }
-        if (q == 0) mbar_wait_cluster_bounded(bar_swap, k & 1, status);  // one warp polls, the others sleep at the barrier
-        bar_sync(ex.bar, kGroupThreads);
+        wait_peer(bar_swap, k & 1);
         if (rank == 0) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) A[i] = P[i], B[i] = lds64(my_box + i * 1024u);
@@ -384,8 +395,7 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         if (t == 0) {
             st_async_b32(peer_amax + (k & 1) * 32 + 16, __float_as_uint(amax), peer_bar_amax);
         }
-        if (q == 0) mbar_wait_cluster_bounded(bar_amax, k & 1, status);
-        bar_sync(ex.bar, kGroupThreads);
+        wait_peer(bar_amax, k & 1);
         amax = fmaxf(amax, __uint_as_float(lds32(aslot + 16)));
         float inv;
         static_assert(!(ROWS && BITS == 16), "BITS = 16 writes the rows already");
