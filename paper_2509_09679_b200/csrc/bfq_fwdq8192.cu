@@ -432,36 +432,42 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
             // scale, so v * inv + 1.5 * 2^23 carries the two's complement code in its low mantissa bits.
             const bool plain = (((s16 >> 10) & 31u) != 0u) && (s16 != 0x7BFFu);
             const u64 inv2 = pack2(inv, inv);
-            auto code2 = [&](u64 v) -> uint32_t {
+            // u = code + 2^(BITS-1) in the low BITS bits of v * inv + (1.5 * 2^23 + 2^(BITS-1)), the bits above them up to
+            // bit 22 zero: (hi << BITS) + lo has both fields in place; the XOR turns offset binary into two's complement
+            constexpr float kMagic = 12582912.0f + float(1 << (BITS - 1));
+            const u64 magic2 = pack2(kMagic, kMagic);
+            auto code_fast = [&](u64 v) -> uint32_t {
                 uint32_t lo, hi;
-                if (plain) {
-                    // u = code + 2^(BITS-1) in the low BITS bits of v * inv + (1.5 * 2^23 + 2^(BITS-1)), the bits above
-                    // them up to bit 22 zero: (hi << BITS) + lo has both fields in place; the XOR turns offset binary
-                    // into two's complement
-                    constexpr float kMagic = 12582912.0f + float(1 << (BITS - 1));
-                    unpack2u(fma2(v, inv2, pack2(kMagic, kMagic)), lo, hi);
-                    return ((hi << BITS) + lo) ^ ((1u << (BITS - 1)) | (1u << (2 * BITS - 1)));
-                } else {
-                    float a, b;
-                    unpack2(v, a, b);
-                    lo = static_cast<uint32_t>(static_cast<int>(fminf(fmaxf(rintf(a * inv), float(-kQmax - 1)), float(kQmax))));
-                    hi = static_cast<uint32_t>(static_cast<int>(fminf(fmaxf(rintf(b * inv), float(-kQmax - 1)), float(kQmax))));
-                }
+                unpack2u(fma2(v, inv2, magic2), lo, hi);
+                return ((hi << BITS) + lo) ^ ((1u << (BITS - 1)) | (1u << (2 * BITS - 1)));
+            };
+            auto code_slow = [&](u64 v) -> uint32_t {
+                float a, b;
+                unpack2(v, a, b);
+                const uint32_t lo = static_cast<uint32_t>(static_cast<int>(fminf(fmaxf(rintf(a * inv), float(-kQmax - 1)), float(kQmax))));
+                const uint32_t hi = static_cast<uint32_t>(static_cast<int>(fminf(fmaxf(rintf(b * inv), float(-kQmax - 1)), float(kQmax))));
                 constexpr uint32_t kMask = (1u << BITS) - 1u;
                 return (lo & kMask) | ((hi & kMask) << BITS);
             };
             const size_t base = static_cast<size_t>(row) * (kN8 * BITS / 8);
+            auto store_all = [&](auto&& code2) {  // the scale decides once per row which of the two bodies runs
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t ca = code2(A[i]), cb = code2(B[i]);
-                if constexpr (BITS == 4) {
-                    codes[base + 1024 * rank + 128 * i + t] = static_cast<uint8_t>(ca);
-                    codes[base + 2048 + 1024 * rank + 128 * i + t] = static_cast<uint8_t>(cb);
-                } else {
-                    uint16_t* c16 = reinterpret_cast<uint16_t*>(codes + base);
-                    c16[1024 * rank + 128 * i + t] = static_cast<uint16_t>(ca);
-                    c16[2048 + 1024 * rank + 128 * i + t] = static_cast<uint16_t>(cb);
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t ca = code2(A[i]), cb = code2(B[i]);
+                    if constexpr (BITS == 4) {
+                        codes[base + 1024 * rank + 128 * i + t] = static_cast<uint8_t>(ca);
+                        codes[base + 2048 + 1024 * rank + 128 * i + t] = static_cast<uint8_t>(cb);
+                    } else {
+                        uint16_t* c16 = reinterpret_cast<uint16_t*>(codes + base);
+                        c16[1024 * rank + 128 * i + t] = static_cast<uint16_t>(ca);
+                        c16[2048 + 1024 * rank + 128 * i + t] = static_cast<uint16_t>(cb);
+                    }
                 }
+            };
+            if (plain) {
+                store_all(code_fast);
+            } else {
+                store_all(code_slow);
             }
             continue;
         }
