@@ -106,6 +106,10 @@ __device__ __forceinline__ void stage12_quad(u64 (&A)[8], u64 (&B)[8], const uin
     }
 }
 
+struct RuntimeRank {
+    uint32_t value;
+};
+
 // the fixed Hadamard rotation: twelve constant-free stages with the same two regroupings, no tokens
 template <class F>
 __device__ __forceinline__ void run_hadamard(u64 (&P)[16], const ExAddr& ex, F&& issue_next) {
@@ -286,8 +290,13 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         }
     };
     // the whole row loop exists once per stage form: the choice is made once per launch, outside the loop
-    auto row_loop = [&](auto form_tag) {
+    // ... and, where rows are the output (BITS >= 16), once per CTA rank, so that "registers 0-7 are mine, 8-15 the peer's"
+    // (or the reverse) is a renaming at compile time instead of register moves per row; a CTA only ever runs its own
+    // copy.  Measured on 65536 rows: bf16 rows out 0.614 -> 0.596 ms; the code variants got slower with it (INT2 0.658 ->
+    // 0.681 ms, INT4 0.633 -> 0.666 ms), so they keep the rank as a run-time value.
+    auto row_loop = [&](auto form_tag, auto rank_tag) {
     constexpr int FORM = decltype(form_tag)::value;
+    const uint32_t rank = rank_tag.value;
     u64 P[16];
     uint32_t T0[32], T1[32];
 
@@ -525,12 +534,23 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
     }
     if (g < kRings) turn.acquire();  // each ring's first group takes its token back: no arrival stays pending
     };
+    auto for_rank = [&](auto form_tag) {
+        if constexpr (BITS >= 16) {
+            if (rank == 0) {
+                row_loop(form_tag, std::integral_constant<uint32_t, 0>());
+            } else {
+                row_loop(form_tag, std::integral_constant<uint32_t, 1>());
+            }
+        } else {
+            row_loop(form_tag, RuntimeRank{rank});
+        }
+    };
     if constexpr (HADAMARD) {
-        row_loop(std::integral_constant<int, kFormHadamard>());
+        for_rank(std::integral_constant<int, kFormHadamard>());
     } else if (!shear) {
-        row_loop(std::integral_constant<int, kFormScaled>());
+        for_rank(std::integral_constant<int, kFormScaled>());
     } else {
-        row_loop(std::integral_constant<int, kFormShear>());
+        for_rank(std::integral_constant<int, kFormShear>());
     }
 
     tmem_fence_before();
