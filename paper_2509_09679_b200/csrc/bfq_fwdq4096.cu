@@ -472,26 +472,27 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
         }
         if constexpr (OUT == kOutInt2) {
             // elements 2t + 256m, +1 are half of byte t/2 + 64m: the low half for even t, the high half for odd t.
-            // The sixteen 4-bit halves (two codes each) travel in two words, registers 0..7 and 8..15.
+            // The sixteen 4-bit halves (two codes each) travel in the low halves of the bytes of four words, registers
+            // 4w .. 4w+3 in word w.
             const bool plain2 = (((s16 >> 10) & 31u) != 0u) && (s16 != 0x7BFFu);
-            uint32_t w0 = 0u, w1 = 0u;
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
             if (plain2) {
                 // |v * inv| <= 1.0005: v * inv + (1.5 * 2^23 + 2) has u = code + 2 in {1, 2, 3} in its low bits above
-                // the constant pattern C = 0x4B400000, so hi * 4 + lo = 5 C + (4 u_hi + u_lo); a Horner chain over the
-                // registers gives the nibbles times 16^m plus a constant, one subtraction removes it and one XOR turns
+                // the constant pattern C = 0x4B400000, so hi * 4 + lo = 5 C + (4 u_hi + u_lo); a Horner chain over four
+                // registers gives the nibbles times 256^i plus a constant, one subtraction removes it and one XOR turns
                 // every u into the two's complement code
                 const u64 inv2 = pack2(inv, inv), magic2 = pack2(12582914.0f, 12582914.0f);
+                constexpr uint32_t kBias = static_cast<uint32_t>((5ull * 0x4B400000ull * 0x01010101ull) & 0xFFFFFFFFull);
 #pragma unroll
-                for (int m = 7; m >= 0; --m) {
-                    uint32_t lo, hi;
-                    unpack2u(fma2(P[m], inv2, magic2), lo, hi);
-                    w0 = w0 * 16u + (hi * 4u + lo);
-                    unpack2u(fma2(P[8 + m], inv2, magic2), lo, hi);
-                    w1 = w1 * 16u + (hi * 4u + lo);
+                for (int q4 = 0; q4 < 4; ++q4) {
+#pragma unroll
+                    for (int i = 3; i >= 0; --i) {
+                        uint32_t lo, hi;
+                        unpack2u(fma2(P[4 * q4 + i], inv2, magic2), lo, hi);
+                        w[q4] = w[q4] * 256u + (hi * 4u + lo);
+                    }
+                    w[q4] = (w[q4] - kBias) ^ 0x0A0A0A0Au;
                 }
-                constexpr uint32_t kBias = static_cast<uint32_t>((5ull * 0x4B400000ull * 0x11111111ull) & 0xFFFFFFFFull);
-                w0 = (w0 - kBias) ^ 0xAAAAAAAAu;
-                w1 = (w1 - kBias) ^ 0xAAAAAAAAu;
             } else {
 #pragma unroll
                 for (int m = 0; m < 16; ++m) {
@@ -499,23 +500,17 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                     unpack2(P[m], a, b);
                     const uint32_t c = (static_cast<uint32_t>(quant1(a, inv, -2, 1)) & 3u) |
                                        ((static_cast<uint32_t>(quant1(b, inv, -2, 1)) & 3u) << 2);
-                    if (m < 8) w0 |= c << (4 * m); else w1 |= c << (4 * (m - 8));
+                    w[m >> 2] |= c << (8 * (m & 3));
                 }
             }
             // the even thread writes bytes m = 0..7 (its nibbles + the odd thread's), the odd one 8..15 (the even
-            // thread's nibbles + its own): one exchange of a word, then nibble m of the two words side by side in byte m
+            // thread's nibbles + its own): one exchange per word, then the two nibbles of a byte side by side
             const bool odd = t & 1;
-            const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, odd ? w0 : w1, 1);
-            const uint32_t low = odd ? other : w0, high = odd ? w1 : other;
-            auto spread4 = [](uint32_t x) {  // nibbles 0..3 of x into the low halves of bytes 0..3
-                x &= 0xFFFFu;
-                x = (x | (x << 8)) & 0x00FF00FFu;
-                return (x | (x << 4)) & 0x0F0F0F0Fu;
-            };
             uint8_t* out2 = codes + static_cast<size_t>(row) * (kN / 4) + (t >> 1) + (odd ? 64 * 8 : 0);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const uint32_t bytes = spread4(low >> (16 * h)) | (spread4(high >> (16 * h)) << 4);
+                const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, odd ? w[h] : w[2 + h], 1);
+                const uint32_t bytes = (odd ? other : w[h]) + ((odd ? w[2 + h] : other) << 4);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) out2[64 * (4 * h + j)] = static_cast<uint8_t>(bytes >> (8 * j));
             }

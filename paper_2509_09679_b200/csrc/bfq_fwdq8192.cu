@@ -485,44 +485,42 @@ k_fwdq8192(const __grid_constant__ CUtensorMap map_lo, const __grid_constant__ C
         const bool plain = (e16 != 0u) && (s16 != 0x7BFFu);  // normal fp16 scale: |v*inv| <= 1.0005, no clipping
         const u64 inv2 = pack2(inv, inv);
         uint8_t* out = out_t + static_cast<size_t>(row) * (kN8 / 4);
-        // the eight nibbles (two codes each) of the lower-half registers in one word, those of the upper half in another
-        uint32_t wa = 0u, wb = 0u;
+        // the nibbles (two codes each) of the lower-half registers in the low halves of the bytes of two words (registers
+        // 0-3, 4-7), those of the upper half in two more
+        uint32_t wa[2] = {0u, 0u}, wb[2] = {0u, 0u};
         if (plain) {
             // v * inv + (1.5 * 2^23 + 2) has u = code + 2 in {1, 2, 3} in its low bits above the constant pattern
-            // C = 0x4B400000, so hi * 4 + lo = 5 C + (4 u_hi + u_lo) and a Horner chain over the registers yields the sum
-            // of the nibbles times 16^i plus a constant; one subtraction removes it, one XOR turns u into the code
+            // C = 0x4B400000, so hi * 4 + lo = 5 C + (4 u_hi + u_lo) and a Horner chain over four registers yields the sum
+            // of the nibbles times 256^i plus a constant; one subtraction removes it, one XOR turns u into the code
             const u64 magic2 = pack2(12582914.0f, 12582914.0f);
 #pragma unroll
-            for (int i = 7; i >= 0; --i) {
-                uint32_t lo, hi;
-                unpack2u(fma2(A[i], inv2, magic2), lo, hi);
-                wa = wa * 16u + (hi * 4u + lo);
-                unpack2u(fma2(B[i], inv2, magic2), lo, hi);
-                wb = wb * 16u + (hi * 4u + lo);
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                for (int i = 3; i >= 0; --i) {
+                    uint32_t lo, hi;
+                    unpack2u(fma2(A[4 * h + i], inv2, magic2), lo, hi);
+                    wa[h] = wa[h] * 256u + (hi * 4u + lo);
+                    unpack2u(fma2(B[4 * h + i], inv2, magic2), lo, hi);
+                    wb[h] = wb[h] * 256u + (hi * 4u + lo);
+                }
+                constexpr uint32_t kBias = static_cast<uint32_t>((5ull * 0x4B400000ull * 0x01010101ull) & 0xFFFFFFFFull);
+                wa[h] = (wa[h] - kBias) ^ 0x0A0A0A0Au;
+                wb[h] = (wb[h] - kBias) ^ 0x0A0A0A0Au;
             }
-            constexpr uint32_t kBias = static_cast<uint32_t>((5ull * 0x4B400000ull * 0x11111111ull) & 0xFFFFFFFFull);
-            wa = (wa - kBias) ^ 0xAAAAAAAAu;
-            wb = (wb - kBias) ^ 0xAAAAAAAAu;
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                wa |= nibble_int2(A[i], inv2, inv, false) << (4 * i);
-                wb |= nibble_int2(B[i], inv2, inv, false) << (4 * i);
+                wa[i >> 2] |= nibble_int2(A[i], inv2, inv, false) << (8 * (i & 3));
+                wb[i >> 2] |= nibble_int2(B[i], inv2, inv, false) << (8 * (i & 3));
             }
         }
         // even lane: bytes of the lower half = its nibbles + the odd lane's; odd lane: bytes of the upper half = the even
-        // lane's nibbles + its own.  One exchange of a word, then nibble i of the two words side by side in byte i.
+        // lane's nibbles + its own.  One exchange per word, then the two nibbles of a byte side by side.
         const bool odd = t & 1;
-        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, odd ? wa : wb, 1);
-        const uint32_t low = odd ? got : wa, high = odd ? wb : got;
-        auto spread4 = [](uint32_t x) {  // nibbles 0..3 of x into the low halves of bytes 0..3
-            x &= 0xFFFFu;
-            x = (x | (x << 8)) & 0x00FF00FFu;
-            return (x | (x << 4)) & 0x0F0F0F0Fu;
-        };
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const uint32_t bytes = spread4(low >> (16 * h)) | (spread4(high >> (16 * h)) << 4);
+            const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, odd ? wa[h] : wb[h], 1);
+            const uint32_t bytes = (odd ? got : wa[h]) + ((odd ? wb[h] : got) << 4);
 #pragma unroll
             for (int j = 0; j < 4; ++j) out[64 * (4 * h + j)] = static_cast<uint8_t>(bytes >> (8 * j));
         }
