@@ -530,9 +530,10 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
             for (int m = 0; m < 16; ++m) {
                 uint32_t lo, hi;
                 unpack2u(fma2(P[m], inv2, magic2), lo, hi);
-                const uint32_t byte = (hi * 16u + lo) ^ 0x88u;  // offset-binary -> two's complement
-                out[128 * m] = static_cast<uint8_t>(byte);
-                if constexpr (kCount) red_shared_inc(hist_g + 4u * (byte & 0xFFu));
+                const uint32_t ob = hi * 16u + lo;  // 17 * 0x4B400000 + the offset-binary byte
+                out[128 * m] = static_cast<uint8_t>(ob ^ 0x88u);  // offset binary -> two's complement
+                // counted by its offset-binary value; the constant is taken off the base address instead of the index
+                if constexpr (kCount) red_shared_inc(hist_g - 4u * (17u * 0x4B400000u) + 4u * ob);
             }
         } else {
 #pragma unroll
@@ -543,7 +544,7 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
                 const int qb = static_cast<int>(fminf(fmaxf(rintf(b * inv), -8.f), 7.f));
                 const uint32_t byte = static_cast<uint32_t>((qa & 0xF) | ((qb & 0xF) << 4));
                 out[128 * m] = static_cast<uint8_t>(byte);
-                if constexpr (kCount) red_shared_inc(hist_g + 4u * byte);
+                if constexpr (kCount) red_shared_inc(hist_g + 4u * (byte ^ 0x88u));
             }
         }
     }
@@ -561,16 +562,16 @@ k_fwdq4096(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ i
     }
 
     if constexpr (kCount) {
-        // byte counts of the G groups -> the CTA's 16 code counts (a byte holds two codes) -> the caller's histogram,
-        // indexed by code + 8.  Integer additions: the result does not depend on their order.
+        // counts of the G groups per offset-binary byte (two nibbles code + 8) -> the CTA's 16 code counts -> the caller's
+        // histogram, indexed by code + 8.  Integer additions: the result does not depend on their order.
         __syncthreads();
         if (threadIdx.x < 256) {
             uint32_t n = 0;
 #pragma unroll
             for (int gg = 0; gg < G; ++gg) n += lds32(sbase + S::kHistOff + 1024u * gg + 4u * threadIdx.x);
             if (n != 0u) {
-                red_shared_add64(sbase + S::kBinsOff + 8u * ((threadIdx.x & 15u) ^ 8u), n);
-                red_shared_add64(sbase + S::kBinsOff + 8u * ((threadIdx.x >> 4) ^ 8u), n);
+                red_shared_add64(sbase + S::kBinsOff + 8u * (threadIdx.x & 15u), n);
+                red_shared_add64(sbase + S::kBinsOff + 8u * (threadIdx.x >> 4), n);
             }
         }
         __syncthreads();
