@@ -129,7 +129,7 @@ static cudaError_t launch_backward_t(bfq_plan* plan, BackwardParams p, float* dt
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int count = LOG_N * G::kHalf;
-    k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid * G::kGroups, count, dtheta);
+    k_reduce_partials<<<(count + 31) / 32, 256, 0, st>>>(plan->partial, grid * G::kGroups, count, dtheta);
     plan->last_backward_partials = grid * G::kGroups;
     return cudaGetLastError();
 }

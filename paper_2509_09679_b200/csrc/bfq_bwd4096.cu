@@ -1244,7 +1244,7 @@ cudaError_t bwd4096_launch(bfq_plan* plan, const void* x, const void* g, int64_t
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int count = 12 * (f4k::kN / 2);
-    k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(plan->partial, grid, count, dtheta);
+    k_reduce_partials<<<(count + 31) / 32, 256, 0, st>>>(plan->partial, grid, count, dtheta);
     plan->last_backward_partials = grid;
     return cudaGetLastError();
 }

@@ -85,7 +85,7 @@ static cudaError_t launch(int device, const PerDevice& d, BackwardParams p, cons
     kern<<<grid, G::kThreads, smem, st>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    k_reduce_partials<<<(count + 255) / 256, 256, 0, st>>>(partial, grid * G::kGroups, count, dtheta);
+    k_reduce_partials<<<(count + 31) / 32, 256, 0, st>>>(partial, grid * G::kGroups, count, dtheta);
     return cudaGetLastError();
 }
 
