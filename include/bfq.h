@@ -136,7 +136,7 @@ int bfq_inverse(bfq_plan* plan, const void* y, bfq_dtype yt, int64_t rows, int64
  *     stage s, z the stage input and gbar the gradient at the stage output.
  * x, g: [rows][ld]; dx: [rows][ld] of dxt (may be NULL to skip); dtheta: device fp32
  * [log2 n][n/2], overwritten.  The sum over rows has a fixed order (per-CTA partial sums over a
- * static row assignment, then CTAs in index order): results are bit-identical run to run on the
+ * static row assignment, then the CTAs' sums added in a fixed order): results are bit-identical run to run on the
  * same device.  The quantizer is not differentiated here; g is the caller's.
  */
 int bfq_backward(bfq_plan* plan, const void* x, bfq_dtype xt, const void* g, bfq_dtype gt,

@@ -17,7 +17,7 @@
 //      are written out), then y and g are both un-rotated.  After stage 0, g is dx up to the parity sign.
 // d-theta accumulators are owned by thread role (no atomics): stages 0-7 in the tensor-memory columns the
 // constants leave free, stages 8-11 in shared memory (stage 8 the lower group's, 9-11 the upper group's).  Each CTA walks its row pairs in a fixed order and
-// writes its sums to its own slot; a second kernel adds the slots in index order: bit-reproducible.
+// writes its sums to its own slot; a second kernel adds the slots in a fixed order: bit-reproducible.
 #include <type_traits>
 
 #include "bfq_fast.h"
