@@ -274,7 +274,12 @@ def main():
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-        time.sleep(0.25)
+    # the clock sampler needs a moment to start: spend it on further untimed steps, so that the timed region does not
+    # begin on a GPU that has just idled for a quarter of a second
+    t_ready = time.time() + 0.25
+    while time.time() < t_ready:
+        step()
+        torch.cuda.synchronize()
     # The timed region: exactly `steps` steps between two events, nothing else on the stream.  (An event recorded between
     # the table build and the forward kernel keeps that kernel from being launched programmatically ahead of the build's
     # end: with a pair of events around every forward launch the step reads 5 % longer and the kernel 4 % longer than
